@@ -1,0 +1,178 @@
+"""CPU oracle for the Sparrow speculative-step attention -- TEST INFRASTRUCTURE ONLY.
+
+Thin ctypes marshalling around ``sparrow_oracle.c`` (plain C, fp64).  Only the tests, the smoke
+check and the benchmark's CPU-baseline leg may import this package; the product never does.
+Arrays are numpy: bf16 tensors travel as ``uint16`` bit patterns, results come back as float64.
+"""
+import ctypes
+import os
+
+import numpy as np
+
+from . import build as _build
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = ctypes.CDLL(_build.build())
+        i32, i64, f64, vp = ctypes.c_int32, ctypes.c_int64, ctypes.c_double, ctypes.c_void_p
+        L.oracle_ancestor_masks.argtypes = [vp, i32, vp]
+        L.oracle_verify_visibility.argtypes = [i32, i32, vp, vp, i64]
+        L.oracle_anchor_idx.argtypes = [i32, vp, i32, i32, i32, vp, vp]
+        L.oracle_anchor_visibility.argtypes = [vp, i32, i32, i32, vp, i64]
+        L.oracle_attention.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32,
+                                       i64, i64, f64, vp, i64, i32, vp, vp]
+        L.oracle_verify_attn.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32,
+                                         i64, i64, f64, vp, i64, i32, vp, vp]
+        L.oracle_anchor_attn.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32,
+                                         i64, i64, f64, vp, i64, i32, vp, vp]
+        for f in ("oracle_ancestor_masks", "oracle_verify_visibility", "oracle_anchor_idx",
+                  "oracle_anchor_visibility", "oracle_attention", "oracle_verify_attn",
+                  "oracle_anchor_attn"):
+            getattr(L, f).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+class OracleError(RuntimeError):
+    pass
+
+
+def _chk(rc, what):
+    if rc != 0:
+        raise OracleError(f"{what} failed with oracle status {rc}")
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _c(a, dtype):
+    a = np.ascontiguousarray(a, dtype=dtype)
+    return a
+
+
+def host_threads() -> int:
+    try:
+        return max(1, len(os.sched_getaffinity(0)))
+    except AttributeError:
+        return max(1, os.cpu_count() or 1)
+
+
+def ancestor_masks(parents) -> np.ndarray:
+    """parents: int32 [T] -> uint64 [T]; bit a of entry i set iff a == i or a is an ancestor of i."""
+    parents = _c(parents, np.int32)
+    T = parents.shape[0]
+    anc = np.zeros(max(T, 1), dtype=np.uint64)
+    _chk(lib().oracle_ancestor_masks(_p(parents), T, _p(anc)), "oracle_ancestor_masks")
+    return anc[:T]
+
+
+def verify_visibility(kv_len: int, anc) -> np.ndarray:
+    anc = _c(anc, np.uint64)
+    T = anc.shape[0]
+    vis = np.zeros((T, kv_len + T), dtype=np.uint8)
+    _chk(lib().oracle_verify_visibility(kv_len, T, _p(anc), _p(vis), vis.shape[1]),
+         "oracle_verify_visibility")
+    return vis
+
+
+def anchor_idx(seq_len: int, vis_spans, window: int, T: int) -> np.ndarray:
+    spans = _c(np.asarray(vis_spans, dtype=np.int32).reshape(-1, 2), np.int32)
+    idx = np.zeros(seq_len + T + 1, dtype=np.int32)
+    n = ctypes.c_int32(0)
+    _chk(lib().oracle_anchor_idx(seq_len, _p(spans) if spans.size else None, spans.shape[0],
+                                 window, T, _p(idx), ctypes.byref(n)), "oracle_anchor_idx")
+    return idx[: n.value].copy()
+
+
+def anchor_visibility(idx, window: int, T: int) -> np.ndarray:
+    idx = _c(idx, np.int32)
+    n = idx.shape[0]
+    vis = np.zeros((T, n), dtype=np.uint8)
+    _chk(lib().oracle_anchor_visibility(_p(idx), n, window, T, _p(vis), n),
+         "oracle_anchor_visibility")
+    return vis
+
+
+def _rows_arg(rows):
+    if rows is None:
+        return None, 0
+    rows = _c(np.asarray(rows).reshape(-1, 3), np.int32)
+    return rows, rows.shape[0]
+
+
+def _outs(rows, n_rows, B, T, Hq, D):
+    if rows is None:
+        return np.zeros((B, T, Hq, D)), np.zeros((B, Hq, T))
+    return np.zeros((n_rows, D)), np.zeros((n_rows,))
+
+
+def _kv_strides(k, B, Hkv, D):
+    assert k.ndim == 4 and k.shape[0] == B and k.shape[1] == Hkv and k.shape[3] == D
+    assert k.flags.c_contiguous
+    return k.shape[1] * k.shape[2] * D, k.shape[2] * D
+
+
+def attention(q, k, v, vis, n_keys_b, scale, key_rows=None, rows=None, n_threads=None):
+    """Core: q uint16 [B,T,Hq,D]; k,v uint16 [B,Hkv,cap,D]; vis uint8 [B,T,n_keys]."""
+    q, k, v = _c(q, np.uint16), _c(k, np.uint16), _c(v, np.uint16)
+    vis = _c(vis, np.uint8)
+    B, T, Hq, D = q.shape
+    Hkv = k.shape[1]
+    n_keys = vis.shape[2]
+    nk = _c(n_keys_b, np.int32)
+    sb, sh = _kv_strides(k, B, Hkv, D)
+    assert v.shape == k.shape
+    if key_rows is not None:
+        key_rows = _c(key_rows, np.int32)
+        assert key_rows.shape == (B, n_keys)
+        assert key_rows.size == 0 or (key_rows.min() >= 0 and key_rows.max() < k.shape[2])
+    else:
+        assert n_keys <= k.shape[2]
+    rows_a, n_rows = _rows_arg(rows)
+    out, lse = _outs(rows_a, n_rows, B, T, Hq, D)
+    _chk(lib().oracle_attention(_p(q), _p(k), _p(v), _p(key_rows), _p(vis), _p(nk), B, T, Hq, Hkv,
+                                D, n_keys, sb, sh, float(scale), _p(rows_a), n_rows,
+                                n_threads or host_threads(), _p(out), _p(lse)), "oracle_attention")
+    return out, lse
+
+
+def verify_attn(q, k_cache, v_cache, kv_len, parents, scale, rows=None, n_threads=None):
+    """Verification mode. parents int32 [B,T]; kv_len int32 [B]. Returns (out f64, lse f64)."""
+    q, k, v = _c(q, np.uint16), _c(k_cache, np.uint16), _c(v_cache, np.uint16)
+    B, T, Hq, D = q.shape
+    Hkv = k.shape[1]
+    kv_len = _c(kv_len, np.int32)
+    parents = _c(parents, np.int32)
+    assert kv_len.shape == (B,) and parents.shape == (B, T)
+    assert int(kv_len.max()) + T <= k.shape[2]
+    sb, sh = _kv_strides(k, B, Hkv, D)
+    rows_a, n_rows = _rows_arg(rows)
+    out, lse = _outs(rows_a, n_rows, B, T, Hq, D)
+    _chk(lib().oracle_verify_attn(_p(q), _p(k), _p(v), _p(kv_len), _p(parents), B, T, Hq, Hkv, D,
+                                  sb, sh, float(scale), _p(rows_a), n_rows,
+                                  n_threads or host_threads(), _p(out), _p(lse)),
+         "oracle_verify_attn")
+    return out, lse
+
+
+def anchor_attn(q, k, v, idx, window, scale, rows=None, n_threads=None):
+    """Text-anchored window mode. idx int32 [B,n_anchor]; T = q.shape[1]."""
+    q, k, v = _c(q, np.uint16), _c(k, np.uint16), _c(v, np.uint16)
+    B, T, Hq, D = q.shape
+    Hkv = k.shape[1]
+    idx = _c(idx, np.int32)
+    assert idx.ndim == 2 and idx.shape[0] == B
+    assert idx.size == 0 or (idx.min() >= 0 and idx.max() < k.shape[2])
+    sb, sh = _kv_strides(k, B, Hkv, D)
+    rows_a, n_rows = _rows_arg(rows)
+    out, lse = _outs(rows_a, n_rows, B, T, Hq, D)
+    _chk(lib().oracle_anchor_attn(_p(q), _p(k), _p(v), _p(idx), idx.shape[1], window, B, T, Hq,
+                                  Hkv, D, sb, sh, float(scale), _p(rows_a), n_rows,
+                                  n_threads or host_threads(), _p(out), _p(lse)),
+         "oracle_anchor_attn")
+    return out, lse

@@ -1,0 +1,388 @@
+"""Pins for the CPU oracle: closed forms, invariants, library routines, brute force.
+
+Nothing here touches the CUDA path.  Each block is chosen so that a plausible slip in the oracle
+(a dropped scale, a sign, a transposed operand, an off-by-one in a mask, a wrong GQA head map)
+breaks at least one assertion; the ``test_pins_detect_*`` cases check that claim by feeding the
+oracle deliberately wrong arguments and requiring the pin to notice.
+"""
+import itertools
+import json
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2602_15318_b200 import workloads as W
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def bf16_bits(a):
+    """float array (values exactly representable or to be rounded) -> bf16 bit patterns."""
+    t = torch.as_tensor(np.asarray(a, dtype=np.float32)).to(torch.bfloat16)
+    return t.view(torch.int16).numpy().view(np.uint16)
+
+
+def bits_to_f64(bits):
+    return torch.from_numpy(bits.view(np.int16).copy()).view(torch.bfloat16).double().numpy()
+
+
+def rand_bits(rng, shape):
+    return bf16_bits(rng.standard_normal(shape))
+
+
+def core(q, k, v, vis, scale, **kw):
+    """q [T,Hq,D], k/v [Hkv,n,D], vis [T,n] -> out [T,Hq,D], lse [Hq,T] (batch of one)."""
+    out, lse = oracle.attention(q[None], k[None], v[None], vis[None], [vis.shape[1]], scale, **kw)
+    return out[0], lse[0]
+
+
+# ---------------------------------------------------------------- closed forms ---------------
+
+def test_hand_worked_example_eq2():
+    g = json.load(open(os.path.join(GOLD, "hand_softmax_d4.json")))
+    q = bf16_bits(g["q"]).reshape(1, 1, 4)
+    k = bf16_bits(g["k"]).reshape(1, 3, 4)
+    v = bf16_bits(g["v"]).reshape(1, 3, 4)
+    out, lse = core(q, k, v, np.ones((1, 3), np.uint8), math.log(2.0))
+    np.testing.assert_allclose(out[0, 0], g["out"], rtol=0, atol=1e-14)
+    assert abs(lse[0, 0] - g["lse"]) < 1e-14
+
+
+@pytest.mark.parametrize("D,n", [(4, 5), (128, 37)])
+def test_equal_keys_give_mean_of_values(D, n):
+    rng = np.random.default_rng(1)
+    q = rand_bits(rng, (3, 2, D))
+    krow = rand_bits(rng, (1, 1, D))
+    k = np.repeat(krow, n, axis=1)
+    v = rand_bits(rng, (1, n, D))
+    vis = np.ones((3, n), np.uint8)
+    vis[1, ::2] = 0                       # a masked row: mean over the visible subset only
+    scale = 0.37
+    out, lse = core(q, k, v, vis, scale)
+    qf, kf, vf = bits_to_f64(q), bits_to_f64(krow)[0, 0], bits_to_f64(v)[0]
+    for t in range(3):
+        sel = vis[t].astype(bool)
+        for h in range(2):
+            s = scale * float(qf[t, h] @ kf)
+            np.testing.assert_allclose(out[t, h], vf[sel].mean(axis=0), atol=1e-13)
+            assert abs(lse[h, t] - (s + math.log(sel.sum()))) < 1e-12
+
+
+def test_two_keys_logistic_weights():
+    rng = np.random.default_rng(2)
+    D = 128
+    q = rand_bits(rng, (1, 1, D)); k = rand_bits(rng, (1, 2, D)); v = rand_bits(rng, (1, 2, D))
+    scale = 1 / math.sqrt(D)
+    out, lse = core(q, k, v, np.ones((1, 2), np.uint8), scale)
+    qf, kf, vf = bits_to_f64(q)[0, 0], bits_to_f64(k)[0], bits_to_f64(v)[0]
+    s = scale * (kf @ qf)
+    w0 = 1.0 / (1.0 + math.exp(s[1] - s[0]))
+    np.testing.assert_allclose(out[0, 0], w0 * vf[0] + (1 - w0) * vf[1], atol=1e-14)
+    assert abs(lse[0, 0] - (s[0] + math.log1p(math.exp(s[1] - s[0])))) < 1e-13
+
+
+def test_empty_visibility_row():
+    rng = np.random.default_rng(3)
+    q = rand_bits(rng, (2, 1, 8)); k = rand_bits(rng, (1, 4, 8)); v = rand_bits(rng, (1, 4, 8))
+    vis = np.ones((2, 4), np.uint8); vis[1] = 0
+    out, lse = core(q, k, v, vis, 1.0)
+    assert np.all(out[1] == 0) and lse[0, 1] == -np.inf and np.isfinite(lse[0, 0])
+
+
+# ---------------------------------------------------------------- invariants -----------------
+
+def _case(seed, T=4, Hq=4, Hkv=2, D=16, n=24):
+    rng = np.random.default_rng(seed)
+    return (rand_bits(rng, (T, Hq, D)), rand_bits(rng, (Hkv, n, D)), rand_bits(rng, (Hkv, n, D)),
+            (rng.random((T, n)) < 0.7).astype(np.uint8))
+
+
+def test_score_shift_moves_lse_only():
+    q, k, v, vis = _case(4)
+    vis[:, 0] = 1
+    T, Hq, D = q.shape
+    c = 3.0
+    q2 = np.concatenate([q, np.broadcast_to(bf16_bits([1.0]), (T, Hq, 1))], axis=2)
+    k2 = np.concatenate([k, np.broadcast_to(bf16_bits([c]), k.shape[:2] + (1,))], axis=2)
+    k0 = np.concatenate([k, np.broadcast_to(bf16_bits([0.0]), k.shape[:2] + (1,))], axis=2)
+    v2 = np.concatenate([v, v[:, :, :1]], axis=2)
+    scale = 0.25
+    o_a, l_a = core(q2, k0, v2, vis, scale)
+    o_b, l_b = core(q2, k2, v2, vis, scale)
+    np.testing.assert_allclose(o_a, o_b, atol=1e-13)
+    np.testing.assert_allclose(l_b - l_a, scale * c, atol=1e-12)
+
+
+def test_key_permutation_invariance():
+    q, k, v, vis = _case(5)
+    vis[:, 0] = 1
+    perm = np.random.default_rng(6).permutation(k.shape[1])
+    o_a, l_a = core(q, k, v, vis, 0.3)
+    o_b, l_b = core(q, k[:, perm], v[:, perm], vis[:, perm], 0.3)
+    np.testing.assert_allclose(o_a, o_b, atol=1e-13)
+    np.testing.assert_allclose(l_a, l_b, atol=1e-13)
+
+
+def test_split_and_merge_by_logsumexp():
+    """Two calls over disjoint key sets, merged by log-sum-exp, equal one call (the identity the
+    split-combine step of the CUDA path relies on)."""
+    q, k, v, vis = _case(7, n=30)
+    vis[:, 0] = 1; vis[:, 29] = 1
+    va, vb = vis.copy(), vis.copy()
+    va[:, 13:] = 0; vb[:, :13] = 0
+    o, l = core(q, k, v, vis, 0.3)
+    oa, la = core(q, k, v, va, 0.3)
+    ob, lb = core(q, k, v, vb, 0.3)
+    lm = np.logaddexp(la, lb)
+    wa, wb = np.exp(la - lm).T[..., None], np.exp(lb - lm).T[..., None]
+    np.testing.assert_allclose(lm, l, atol=1e-12)
+    np.testing.assert_allclose(wa * oa + wb * ob, o, atol=1e-12)
+
+
+def test_softmax_weights_sum_to_one():
+    """V = all ones (any column) -> out is exactly the sum of the weights."""
+    q, k, v, vis = _case(8)
+    vis[:, 3] = 1
+    ones = np.broadcast_to(bf16_bits([1.0]), v.shape).copy()
+    out, _ = core(q, k, ones, vis, 0.5)
+    np.testing.assert_allclose(out, 1.0, atol=1e-13)
+
+
+# ---------------------------------------------------------------- library routines -----------
+
+def sdpa(q, k, v, mask, scale, G):
+    """torch's float64 scaled_dot_product_attention with the KV heads repeated G times (the
+    repeat_kv convention: query head h reads KV head h // G)."""
+    qt = torch.from_numpy(bits_to_f64(q)).permute(1, 0, 2)[None]            # [1,Hq,T,D]
+    kt = torch.from_numpy(bits_to_f64(k))[None].repeat_interleave(G, dim=1)
+    vt = torch.from_numpy(bits_to_f64(v))[None].repeat_interleave(G, dim=1)
+    o = torch.nn.functional.scaled_dot_product_attention(qt, kt, vt, attn_mask=mask, scale=scale)
+    return o[0].permute(1, 0, 2).numpy()
+
+
+def lse_lib(q, k, mask, scale, G):
+    from scipy.special import logsumexp
+    qf, kf = bits_to_f64(q), np.repeat(bits_to_f64(k), G, axis=0)
+    s = scale * np.einsum("thd,hjd->htj", qf, kf)
+    s = np.where(mask[None], s, -np.inf)
+    return logsumexp(s, axis=2)
+
+
+def test_unmasked_equals_sdpa():
+    rng = np.random.default_rng(10)
+    T, Hq, Hkv, D, n = 5, 28, 4, 128, 300
+    q, k, v = rand_bits(rng, (T, Hq, D)), rand_bits(rng, (Hkv, n, D)), rand_bits(rng, (Hkv, n, D))
+    scale = 1 / math.sqrt(D)
+    out, lse = core(q, k, v, np.ones((T, n), np.uint8), scale)
+    np.testing.assert_allclose(out, sdpa(q, k, v, None, scale, 7), atol=1e-12)
+    np.testing.assert_allclose(lse, lse_lib(q, k, np.ones((T, n), bool), scale, 7), atol=1e-12)
+
+
+def test_chain_equals_causal_attention():
+    """Chain parents [-1,0,1,..] = causal attention over kv_len+T keys, last T query rows."""
+    rng = np.random.default_rng(11)
+    T, Hq, Hkv, D, kv_len = 8, 28, 4, 128, 200
+    n = kv_len + T
+    q, k, v = rand_bits(rng, (T, Hq, D)), rand_bits(rng, (Hkv, n, D)), rand_bits(rng, (Hkv, n, D))
+    scale = 1 / math.sqrt(D)
+    parents = np.array([W.chain_parents(T)], np.int32)
+    out, lse = oracle.verify_attn(q[None], k[None], v[None], [kv_len], parents, scale)
+    causal = torch.ones(T, n, dtype=torch.bool).tril(diagonal=kv_len)     # bottom-right aligned
+    np.testing.assert_allclose(out[0], sdpa(q, k, v, causal, scale, 7), atol=1e-12)
+    np.testing.assert_allclose(lse[0], lse_lib(q, k, causal.numpy(), scale, 7), atol=1e-12)
+    # square causal via the library flag: the last T rows of full causal self-attention
+    qfull = np.concatenate([rand_bits(rng, (kv_len, Hq, D)), q], axis=0)
+    qt = torch.from_numpy(bits_to_f64(qfull)).permute(1, 0, 2)[None]
+    kt = torch.from_numpy(bits_to_f64(k))[None].repeat_interleave(7, dim=1)
+    vt = torch.from_numpy(bits_to_f64(v))[None].repeat_interleave(7, dim=1)
+    o = torch.nn.functional.scaled_dot_product_attention(qt, kt, vt, is_causal=True, scale=scale)
+    np.testing.assert_allclose(out[0], o[0, :, kv_len:].permute(1, 0, 2).numpy(), atol=1e-12)
+
+
+def test_last_chain_node_and_forest_visibility():
+    """Full-visibility readings: the last node of a chain sees every key; an all-roots forest sees
+    the prefix plus itself only."""
+    rng = np.random.default_rng(12)
+    T, Hq, Hkv, D, kv_len = 6, 14, 2, 32, 50
+    n = kv_len + T
+    q, k, v = rand_bits(rng, (T, Hq, D)), rand_bits(rng, (Hkv, n, D)), rand_bits(rng, (Hkv, n, D))
+    scale = 0.2
+    out, lse = oracle.verify_attn(q[None], k[None], v[None], [kv_len],
+                                  np.array([W.chain_parents(T)], np.int32), scale)
+    full = sdpa(q, k, v, None, scale, 7)
+    np.testing.assert_allclose(out[0, T - 1], full[T - 1], atol=1e-12)
+    out_f, lse_f = oracle.verify_attn(q[None], k[None], v[None], [kv_len],
+                                      np.full((1, T), -1, np.int32), scale)
+    m = torch.zeros(T, n, dtype=torch.bool); m[:, :kv_len] = True
+    m[torch.arange(T), kv_len + torch.arange(T)] = True
+    np.testing.assert_allclose(out_f[0], sdpa(q, k, v, m, scale, 7), atol=1e-12)
+    np.testing.assert_allclose(lse_f[0], lse_lib(q, k, m.numpy(), scale, 7), atol=1e-12)
+
+
+def test_random_tree_equals_masked_sdpa():
+    rng = np.random.default_rng(13)
+    T, Hq, Hkv, D, kv_len = 12, 28, 4, 128, 77
+    n = kv_len + T
+    q, k, v = rand_bits(rng, (T, Hq, D)), rand_bits(rng, (Hkv, n, D)), rand_bits(rng, (Hkv, n, D))
+    parents = W.random_tree_parents(99, 4, T, max_depth=4, max_children=3)
+    mask = torch.zeros(T, n, dtype=torch.bool); mask[:, :kv_len] = True
+    for t in range(T):                     # walk to the root
+        a = t
+        while a >= 0:
+            mask[t, kv_len + a] = True
+            a = parents[a]
+    scale = 1 / math.sqrt(D)
+    out, lse = oracle.verify_attn(q[None], k[None], v[None], [kv_len],
+                                  np.array([parents], np.int32), scale)
+    np.testing.assert_allclose(out[0], sdpa(q, k, v, mask, scale, 7), atol=1e-12)
+    np.testing.assert_allclose(lse[0], lse_lib(q, k, mask.numpy(), scale, 7), atol=1e-12)
+
+
+def test_anchored_equals_dense_on_gathered_subset():
+    """Eq. 2: attention restricted to the text-anchored rows = dense attention on those rows
+    copied into a compact buffer (causal among the T draft rows)."""
+    rng = np.random.default_rng(14)
+    T, Hq, Hkv, D = 4, 28, 4, 128
+    seq_len, spans, window = 300, [[10, 250]], 0
+    cap = seq_len + T
+    q, k, v = rand_bits(rng, (T, Hq, D)), rand_bits(rng, (Hkv, cap, D)), rand_bits(rng, (Hkv, cap, D))
+    idx = oracle.anchor_idx(seq_len, spans, window, T)
+    assert len(idx) == 10 + 50 + T
+    scale = 1 / math.sqrt(D)
+    out, lse = oracle.anchor_attn(q[None], k[None], v[None], idx[None], window, scale)
+    kg, vg = k[:, idx], v[:, idx]
+    n = len(idx)
+    causal = torch.ones(T, n, dtype=torch.bool).tril(diagonal=n - T)
+    np.testing.assert_allclose(out[0], sdpa(q, kg, vg, causal, scale, 7), atol=1e-12)
+    np.testing.assert_allclose(lse[0], lse_lib(q, kg, causal.numpy(), scale, 7), atol=1e-12)
+
+
+def test_anchored_window_lower_bound():
+    rng = np.random.default_rng(15)
+    T, Hq, Hkv, D = 3, 7, 1, 16
+    idx = np.array([2, 5, 9, 30, 31, 40, 41, 42], np.int32)   # last 3 = draft rows
+    cap = 43
+    q, k, v = rand_bits(rng, (T, Hq, D)), rand_bits(rng, (Hkv, cap, D)), rand_bits(rng, (Hkv, cap, D))
+    window = 12
+    vis = oracle.anchor_visibility(idx, window, T)
+    want = np.array([[(p <= qp) and (qp - window < p) for p in idx] for qp in idx[-T:]], np.uint8)
+    assert np.array_equal(vis, want)
+    assert vis[0].tolist() == [0, 0, 0, 1, 1, 1, 0, 0]      # qpos 40: window covers 29..40
+    out, lse = oracle.anchor_attn(q[None], k[None], v[None], idx[None], window, 0.3)
+    np.testing.assert_allclose(out[0], sdpa(q, k[:, idx], v[:, idx], torch.from_numpy(want.astype(bool)), 0.3, 7), atol=1e-12)
+
+
+def test_sampled_rows_match_full():
+    case = W.make_verify_case(5, [100, 64], 5, "random")
+    qb, kb, vb = W.bf16_bits(case.q), W.bf16_bits(case.k), W.bf16_bits(case.v)
+    par = case.parents.numpy()
+    out, lse = oracle.verify_attn(qb, kb, vb, case.kv_len, par, W.SCALE)
+    rows = [(0, 0, 0), (1, 4, 27), (0, 3, 13), (1, 2, 6)]
+    o2, l2 = oracle.verify_attn(qb, kb, vb, case.kv_len, par, W.SCALE, rows=rows)
+    for i, (b, t, h) in enumerate(rows):
+        assert np.array_equal(o2[i], out[b, t, h]) and l2[i] == lse[b, h, t]
+
+
+# ---------------------------------------------------------------- masks and indices ----------
+
+def walk_mask(parents, i):
+    m, a = 0, i
+    while a >= 0:
+        m |= 1 << a
+        a = parents[a]
+    return m
+
+
+def test_ancestor_masks_all_small_trees():
+    for T in range(1, 7):
+        for par in itertools.product(*[range(-1, i) for i in range(T)]):
+            got = oracle.ancestor_masks(np.array(par, np.int32))
+            assert [int(x) for x in got] == [walk_mask(par, i) for i in range(T)]
+
+
+def test_ancestor_masks_closed_forms():
+    T = 64
+    chain = oracle.ancestor_masks(np.array(W.chain_parents(T), np.int32))
+    assert [int(x) for x in chain] == [(1 << (t + 1)) - 1 for t in range(T)]
+    forest = oracle.ancestor_masks(np.full(T, -1, np.int32))
+    assert [int(x) for x in forest] == [1 << t for t in range(T)]
+    par = W.random_tree_parents(W.config_seed(2), 4, T)
+    anc = oracle.ancestor_masks(np.array(par, np.int32))
+    depth = [0] * T
+    for i in range(T):
+        depth[i] = 1 if par[i] < 0 else depth[par[i]] + 1
+    assert [bin(int(x)).count("1") for x in anc] == depth
+    assert max(depth) <= 8
+    assert max(par.count(j) for j in range(T)) <= 4
+
+
+def test_ancestor_masks_reject_bad_trees():
+    for bad in ([0], [-1, 1], [-1, 2, 0], [-2]):
+        with pytest.raises(oracle.OracleError):
+            oracle.ancestor_masks(np.array(bad, np.int32))
+
+
+def test_verify_visibility_layout():
+    anc = oracle.ancestor_masks(np.array([-1, 0, 0, 2], np.int32))
+    vis = oracle.verify_visibility(3, anc)
+    assert vis.shape == (4, 7)
+    assert vis.tolist() == [[1, 1, 1, 1, 0, 0, 0], [1, 1, 1, 1, 1, 0, 0],
+                            [1, 1, 1, 1, 0, 1, 0], [1, 1, 1, 1, 0, 1, 1]]
+
+
+def test_anchor_idx_brute_force_and_c4_closed_form():
+    rng = np.random.default_rng(20)
+    for _ in range(30):
+        L = int(rng.integers(1, 200))
+        cuts = sorted(rng.integers(0, L + 1, size=4).tolist())
+        spans = [[cuts[0], cuts[1]], [cuts[2], cuts[3]]]
+        Wn = int(rng.integers(0, 80)); T = int(rng.integers(0, 9))
+        want = W.text_anchor_list(L, spans, Wn, T)
+        assert oracle.anchor_idx(L, spans, Wn, T).tolist() == want
+    got = oracle.anchor_idx(26112, [[64, 25664]], 1024, 8)
+    assert got.tolist() == list(range(25664, 26112)) + list(range(26112, 26120))
+    assert len(got) == 456
+    assert oracle.anchor_idx(100, [], 0, 2).tolist() == list(range(102))
+
+
+# ---------------------------------------------------------------- the pins bite --------------
+
+def _pin_case():
+    rng = np.random.default_rng(30)
+    T, Hq, Hkv, D, kv_len = 6, 28, 4, 128, 90
+    n = kv_len + T
+    q, k, v = rand_bits(rng, (T, Hq, D)), rand_bits(rng, (Hkv, n, D)), rand_bits(rng, (Hkv, n, D))
+    causal = torch.ones(T, n, dtype=torch.bool).tril(diagonal=kv_len)
+    scale = 1 / math.sqrt(D)
+    return q, k, v, kv_len, causal, scale, sdpa(q, k, v, causal, scale, 7), lse_lib(q, k, causal.numpy(), scale, 7)
+
+
+def _differs(a, b, tol=1e-6):
+    return float(np.max(np.abs(a - b))) > tol
+
+
+def test_pins_detect_planted_mistakes():
+    q, k, v, kv_len, causal, scale, ref_o, ref_l = _pin_case()
+    T = q.shape[0]
+    chain = np.array([W.chain_parents(T)], np.int32)
+    run = lambda q_, k_, v_, kl, sc, par=chain: oracle.verify_attn(q_[None], k_[None], v_[None], [kl], par, sc)
+    o, l = run(q, k, v, kv_len, scale)
+    assert not _differs(o[0], ref_o, 1e-12) and not _differs(l[0], ref_l, 1e-12)
+    o, l = run(q, v, k, kv_len, scale)                       # K and V exchanged
+    assert _differs(o[0], ref_o) and _differs(l[0], ref_l)
+    o, l = run(q, k, v, kv_len, 1.0)                         # scale dropped
+    assert _differs(o[0], ref_o) and _differs(l[0], ref_l)
+    o, l = run(q, k, v, kv_len, -scale)                      # sign of the scores
+    assert _differs(o[0], ref_o) and _differs(l[0], ref_l)
+    o, l = run(q, k, v, kv_len - 1, scale)                   # off-by-one prefix
+    assert _differs(o[0], ref_o) and _differs(l[0], ref_l)
+    o, l = run(q[:, ::-1].copy(), k, v, kv_len, scale)       # wrong query-head -> KV-head map
+    assert _differs(o[0], ref_o) and _differs(l[0], ref_l)
+    o, l = run(q, k, v, kv_len, scale, np.full((1, T), -1, np.int32))   # tree mask ignored
+    assert _differs(o[0], ref_o) and _differs(l[0], ref_l)
+    o, l = run(q[::-1].copy(), k, v, kv_len, scale)          # token order reversed
+    assert _differs(o[0], ref_o) and _differs(l[0], ref_l)
