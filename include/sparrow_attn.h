@@ -1,0 +1,172 @@
+/*
+ * sparrow_attn.h -- C ABI of libsparrow_attn: the attention of one speculative decoding step of
+ * Sparrow (video-LLM speculative decoding) on one NVIDIA B200 (sm_100a).
+ *
+ * Two modes:
+ *   (a) verification -- T draft tokens arranged as a chain or tree attend over the target model's
+ *       whole KV cache (visual + text prefix) plus their own ancestors.  The paper's Appendix A
+ *       ("Speculative Decoding") and Section 4 ("Metrics") state that the target verifies all
+ *       candidates of a (dynamic) draft tree in a single parallel forward pass and that the method
+ *       is lossless, i.e. this is the target's ordinary softmax attention under the tree mask.
+ *   (b) text-anchored window attention -- Eq. 2 (Section 3.1, VATA): Softmax(Q_t K_T^T/sqrt(d)) V_T
+ *       with K_T, V_T restricted to the text-anchored positions T; the visual KV rows are never
+ *       touched.
+ *
+ * For every batch entry b, query head h (KV head h / 7), draft token t and visible key set Vis:
+ *     s_j = softmax_scale * <q[b,t,h,:], k[b,h/7,j,:]>,   lse = log sum_{j in Vis} exp(s_j),
+ *     out = sum_{j in Vis} exp(s_j - lse) * v[b,h/7,j,:].
+ *
+ * Conventions
+ *   - Every function returns a sparrow_status; nothing aborts or throws.  Argument errors are
+ *     detected on the host before anything is launched.  Problems only the device can see (a
+ *     malformed device-side parent array, an anchor index outside the buffer) set a sticky status
+ *     word, read by sparrow_last_device_status(); the kernels always terminate, never read out of
+ *     bounds, and treat a bad parent as "root" and a bad anchor row as "not visible".
+ *   - "DEV" pointers are device memory of the context's GPU, "HOST" pointers are host memory.
+ *   - The caller owns every buffer including the workspace; the library owns only the context.
+ *   - The two attention calls allocate nothing, copy nothing from the host and do not
+ *     synchronise: they enqueue kernels on `stream` and return.
+ *   - bf16 tensors are passed as void*; element strides are in elements, not bytes.
+ */
+#ifndef SPARROW_ATTN_H_
+#define SPARROW_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SPARROW_OK            = 0,
+    SPARROW_ERR_NULL      = 1,  /* a required pointer is NULL */
+    SPARROW_ERR_SHAPE     = 2,  /* unsupported head geometry, T, batch, lengths, alignment */
+    SPARROW_ERR_TREE      = 3,  /* parents[] is not a topologically ordered forest */
+    SPARROW_ERR_ANCHOR    = 4,  /* anchor list not strictly increasing / out of range */
+    SPARROW_ERR_WORKSPACE = 5,  /* workspace missing, misaligned or too small */
+    SPARROW_ERR_CUDA      = 6,  /* a CUDA runtime / driver call failed */
+    SPARROW_ERR_TIMEOUT   = 7,  /* a bounded device-side wait gave up */
+    SPARROW_ERR_ARCH      = 8   /* the device is not compute capability 10.x */
+} sparrow_status;
+
+#define SPARROW_MAX_T      64   /* draft tokens per sequence (one 64-bit ancestor word per token) */
+#define SPARROW_MAX_BATCH  64   /* sequences per call */
+#define SPARROW_HEAD_DIM   128  /* only value accepted */
+#define SPARROW_GQA_GROUP  7    /* query heads per KV head; only value accepted */
+
+/* Fixed per context.  K/V buffers hold, for batch b and KV head g, `kv_capacity` rows of 128 bf16:
+ * element offset of (b, g, row, d) = b*kv_stride_batch + g*kv_stride_head + row*128 + d.
+ * Both strides must be multiples of 8 elements and the base pointers 16-byte aligned. */
+typedef struct {
+    int32_t batch;           /* 1 .. SPARROW_MAX_BATCH */
+    int32_t n_q_heads;       /* must equal 7 * n_kv_heads */
+    int32_t n_kv_heads;
+    int32_t head_dim;        /* must be 128 */
+    int32_t kv_capacity;     /* rows per (batch, KV head) */
+    float   softmax_scale;   /* e.g. 1/sqrt(128); applied in fp32 to the fp32 scores */
+    int64_t kv_stride_batch;
+    int64_t kv_stride_head;
+} sparrow_layout;
+
+typedef struct sparrow_ctx sparrow_ctx;
+
+/* Creates a context on CUDA device `device` (queries the SM count, loads the kernels).
+ * SPARROW_ERR_ARCH unless the device is sm_100; SPARROW_ERR_CUDA when no usable device exists. */
+sparrow_status sparrow_create(sparrow_ctx** ctx, const sparrow_layout* layout, int device);
+sparrow_status sparrow_destroy(sparrow_ctx* ctx);
+
+/* Bytes of device scratch the calls need for draft blocks of up to max_T tokens (split-KV partial
+ * outputs, the device status word, staging for the host-buffer entry point).  0 on bad arguments. */
+size_t sparrow_workspace_bytes(const sparrow_ctx* ctx, int32_t max_T);
+/* Registers caller-owned scratch (256-byte aligned, >= sparrow_workspace_bytes(max_T) for the
+ * largest T that will be used).  Clears the device status word with a cudaMemset (synchronising).
+ * Calls that share one workspace must be ordered on the GPU (same stream, or event dependencies). */
+sparrow_status sparrow_set_workspace(sparrow_ctx* ctx, void* dev_ptr, size_t bytes);
+
+/* (a) Verification attention (Appendix A; Section 4 "Metrics": tree-structured, lossless).
+ *   q        DEV bf16 [batch][T][n_q_heads][128], dense
+ *   k_cache,
+ *   v_cache  DEV bf16, layout above; rows [0, kv_len[b]) are the committed prefix, rows
+ *            [kv_len[b], kv_len[b]+T) already hold the T draft tokens' keys / values; rows past
+ *            that may hold anything (including NaN patterns) and are ignored
+ *   kv_len   HOST int32 [batch]; 0 <= kv_len[b], kv_len[b] + T <= kv_capacity
+ *   parents  DEV int32 [batch][T]; parents[i] = parent node of draft token i, -1 for a root,
+ *            parents[i] < i.  Token t sees the prefix, itself and its ancestors.
+ *   T        1 .. SPARROW_MAX_T
+ *   out      DEV bf16 [batch][T][n_q_heads][128]
+ *   lse      DEV fp32 [batch][n_q_heads][T], natural log of the softmax normaliser
+ *   stream   cudaStream_t (NULL = default stream)
+ * Split-KV pass over ~one work item per SM followed by a log-sum-exp combine, both enqueued on
+ * `stream`.  Results are deterministic for fixed arguments. */
+sparrow_status sparrow_verify_attn(sparrow_ctx* ctx, const void* q, const void* k_cache,
+                                   const void* v_cache, const int32_t* kv_len,
+                                   const int32_t* parents, int32_t T, void* out, float* lse,
+                                   void* stream);
+
+/* (b) Text-anchored window attention (Eq. 2, Section 3.1).
+ *   k, v        DEV bf16 full-length buffers (layout above); only rows named by anchor_idx are read
+ *   anchor_idx  DEV int32 [batch][n_anchor], strictly increasing per sequence, every entry in
+ *               [0, kv_capacity); the last T entries are the T query tokens' own rows
+ *   n_anchor    T .. kv_capacity
+ *   window      query t, at position qpos = anchor_idx[n_anchor-T+t], sees anchor p iff
+ *               qpos - window < p <= qpos; window <= 0 removes the lower bound.  (The paper names
+ *               a window but does not define it; this is the library's rule.)
+ *   T           1 .. SPARROW_MAX_T query tokens
+ *   q, out, lse as in (a). */
+sparrow_status sparrow_anchor_attn(sparrow_ctx* ctx, const void* q, const void* k, const void* v,
+                                   const int32_t* anchor_idx, int32_t n_anchor, int32_t window,
+                                   int32_t T, void* out, float* lse, void* stream);
+
+/* Verification step with HOST buffers (what a caller without device-side glue uses): copies q,
+ * the T new K/V rows per (batch, KV head) and parents to the device, writes the new rows into
+ * cache rows [kv_len[b], kv_len[b]+T), runs (a), copies out / lse back and synchronises `stream`.
+ *   q_host       HOST bf16 [batch][T][n_q_heads][128]      (pinned memory recommended)
+ *   k_new_host,
+ *   v_new_host   HOST bf16 [batch][n_kv_heads][T][128]
+ *   parents_host HOST int32 [batch][T]  (validated on the host: SPARROW_ERR_TREE)
+ *   out_host     HOST bf16 [batch][T][n_q_heads][128];  lse_host HOST fp32 [batch][n_q_heads][T]
+ * Device staging comes from the registered workspace; nothing is allocated. */
+sparrow_status sparrow_verify_step_host(sparrow_ctx* ctx, const void* q_host,
+                                        const void* k_new_host, const void* v_new_host,
+                                        void* k_cache, void* v_cache, const int32_t* kv_len,
+                                        const int32_t* parents_host, int32_t T, void* out_host,
+                                        float* lse_host, void* stream);
+
+/* Host helpers, exported so mask / index construction can be checked bit for bit.
+ * Ancestor words of a draft tree (Section 4: dynamic draft trees): masks[i] has bit a set iff
+ * a == i or a is an ancestor of i.  SPARROW_ERR_TREE unless -1 <= parents[i] < i. */
+sparrow_status sparrow_build_ancestor_masks(const int32_t* parents_host, int32_t T,
+                                            uint64_t* masks_host);
+/* Anchor list for Eq. 2's index set T: positions p of [0, seq_len) outside every visual span
+ * [begin, end) with p >= seq_len - window (window <= 0: all), increasing, then the T draft rows
+ * seq_len .. seq_len+T-1.  idx_host must hold seq_len + T entries. */
+sparrow_status sparrow_build_anchor_idx(int32_t seq_len, const int32_t* vis_spans, int32_t n_spans,
+                                        int32_t window, int32_t T, int32_t* idx_host,
+                                        int32_t* n_anchor_out);
+/* Runs the kernels' own device-side mask construction: parents_dev DEV int32 [T] ->
+ * masks_dev DEV uint64 [T]. */
+sparrow_status sparrow_debug_ancestor_masks_device(sparrow_ctx* ctx, const int32_t* parents_dev,
+                                                   int32_t T, uint64_t* masks_dev, void* stream);
+
+/* Host-side split schedule, exported for inspection (pure host code, needs no GPU): for `batch`
+ * sequences of n_keys[b] keys, draft blocks of T tokens and a device with n_sm SMs, writes
+ * splits_out[b] = key-range pieces per (sequence, KV head, row group) and the total number of
+ * work items.  Piece s of n covers keys [n_keys*s/n, n_keys*(s+1)/n). */
+sparrow_status sparrow_plan_splits(int32_t n_sm, int32_t batch, int32_t n_kv_heads,
+                                   const int32_t* n_keys, int32_t T, int32_t* splits_out,
+                                   int32_t* n_items_out);
+
+/* Synchronises `stream`, returns the sticky device status (SPARROW_OK, SPARROW_ERR_TREE,
+ * SPARROW_ERR_ANCHOR or SPARROW_ERR_TIMEOUT) and clears it.  Not for the hot path. */
+sparrow_status sparrow_last_device_status(sparrow_ctx* ctx, void* stream);
+
+/* Number of kernels the library has launched through this context (for launch accounting). */
+int64_t sparrow_launch_count(const sparrow_ctx* ctx);
+
+const char* sparrow_status_string(sparrow_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPARROW_ATTN_H_ */

@@ -1,0 +1,213 @@
+"""ctypes binding of libsparrow_attn: argument marshalling only.
+
+Every step of the attention path runs in the library's CUDA kernels; torch is used here for device
+memory and streams.  The functions carry the C ABI's names and argument order.  There is no CPU
+fallback: if the shared library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsparrow_attn.so")
+
+STATUS_NAMES = {0: "SPARROW_OK", 1: "SPARROW_ERR_NULL", 2: "SPARROW_ERR_SHAPE", 3: "SPARROW_ERR_TREE",
+                4: "SPARROW_ERR_ANCHOR", 5: "SPARROW_ERR_WORKSPACE", 6: "SPARROW_ERR_CUDA",
+                7: "SPARROW_ERR_TIMEOUT", 8: "SPARROW_ERR_ARCH"}
+
+EXPORTS = ["sparrow_create", "sparrow_destroy", "sparrow_workspace_bytes", "sparrow_set_workspace",
+           "sparrow_verify_attn", "sparrow_anchor_attn", "sparrow_verify_step_host",
+           "sparrow_build_ancestor_masks", "sparrow_build_anchor_idx",
+           "sparrow_debug_ancestor_masks_device", "sparrow_plan_splits",
+           "sparrow_last_device_status", "sparrow_launch_count", "sparrow_status_string"]
+
+
+class SparrowError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: {STATUS_NAMES.get(status, status)}")
+
+
+class Layout(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32), ("kv_capacity", ctypes.c_int32),
+                ("softmax_scale", ctypes.c_float), ("kv_stride_batch", ctypes.c_int64),
+                ("kv_stride_head", ctypes.c_int64)]
+
+
+_lib = None
+
+
+def lib():
+    """Loads the shared library (raises if it has not been built)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} not found: build it with "
+                               "`python -m paper_2602_15318_b200.build` (there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+        L.sparrow_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(Layout), ctypes.c_int]
+        L.sparrow_destroy.argtypes = [vp]
+        L.sparrow_workspace_bytes.argtypes = [vp, i32]
+        L.sparrow_workspace_bytes.restype = ctypes.c_size_t
+        L.sparrow_set_workspace.argtypes = [vp, vp, ctypes.c_size_t]
+        L.sparrow_verify_attn.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp, vp, vp]
+        L.sparrow_anchor_attn.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp]
+        L.sparrow_verify_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp]
+        L.sparrow_build_ancestor_masks.argtypes = [vp, i32, vp]
+        L.sparrow_build_anchor_idx.argtypes = [i32, vp, i32, i32, i32, vp, vp]
+        L.sparrow_debug_ancestor_masks_device.argtypes = [vp, vp, i32, vp, vp]
+        L.sparrow_plan_splits.argtypes = [i32, i32, i32, vp, i32, vp, vp]
+        L.sparrow_last_device_status.argtypes = [vp, vp]
+        L.sparrow_launch_count.argtypes = [vp]
+        L.sparrow_launch_count.restype = i64
+        L.sparrow_status_string.argtypes = [ctypes.c_int]
+        L.sparrow_status_string.restype = ctypes.c_char_p
+        for name in EXPORTS:
+            if name not in ("sparrow_workspace_bytes", "sparrow_launch_count", "sparrow_status_string"):
+                getattr(L, name).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def _chk(status: int, what: str):
+    if status != 0:
+        raise SparrowError(status, what)
+
+
+def _ptr(t) -> Optional[int]:
+    if t is None:
+        return None
+    return t.data_ptr()
+
+
+def _stream_handle(stream) -> Optional[int]:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream or None
+    if isinstance(stream, torch.cuda.Stream):
+        return stream.cuda_stream or None
+    return stream or None
+
+
+def _i32_array(values: Sequence[int]):
+    return (ctypes.c_int32 * len(values))(*[int(x) for x in values])
+
+
+class Context:
+    """Owns a sparrow_ctx and (by default) a torch-allocated workspace registered with it."""
+
+    def __init__(self, batch: int, kv_capacity: int, kv_stride_batch: int, kv_stride_head: int,
+                 softmax_scale: float, n_q_heads: int = 28, n_kv_heads: int = 4, head_dim: int = 128,
+                 device: int = 0, max_T: int = 64, allocate_workspace: bool = True):
+        self.layout = Layout(batch, n_q_heads, n_kv_heads, head_dim, kv_capacity, softmax_scale,
+                             kv_stride_batch, kv_stride_head)
+        self.device = device
+        self.handle = ctypes.c_void_p()
+        _chk(lib().sparrow_create(ctypes.byref(self.handle), ctypes.byref(self.layout), device),
+             "sparrow_create")
+        self.workspace = None
+        if allocate_workspace:
+            n = self.workspace_bytes(max_T)
+            self.workspace = torch.empty(n, dtype=torch.uint8, device=f"cuda:{device}")
+            self.set_workspace(self.workspace.data_ptr(), n)
+
+    @classmethod
+    def for_cache(cls, k_cache: torch.Tensor, softmax_scale: float, n_q_heads: int = 28, **kw):
+        """Context matching a [B, Hkv, capacity, 128] bf16 cache tensor's strides."""
+        assert k_cache.dim() == 4 and k_cache.stride(3) == 1 and k_cache.stride(2) == k_cache.shape[3]
+        return cls(k_cache.shape[0], k_cache.shape[2], k_cache.stride(0), k_cache.stride(1),
+                   softmax_scale, n_q_heads=n_q_heads, n_kv_heads=k_cache.shape[1],
+                   head_dim=k_cache.shape[3], device=k_cache.device.index or 0, **kw)
+
+    def workspace_bytes(self, max_T: int) -> int:
+        return int(lib().sparrow_workspace_bytes(self.handle, max_T))
+
+    def set_workspace(self, ptr: int, nbytes: int):
+        _chk(lib().sparrow_set_workspace(self.handle, ptr, nbytes), "sparrow_set_workspace")
+
+    def launch_count(self) -> int:
+        return int(lib().sparrow_launch_count(self.handle))
+
+    def last_device_status(self, stream=None) -> int:
+        return int(lib().sparrow_last_device_status(self.handle, _stream_handle(stream)))
+
+    def close(self):
+        if self.handle:
+            lib().sparrow_destroy(self.handle)
+            self.handle = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def sparrow_verify_attn(ctx: Context, q, k_cache, v_cache, kv_len: Sequence[int], parents, T: int,
+                        out, lse, stream=None):
+    """q/out: CUDA bf16 [B,T,Hq,128]; caches: CUDA bf16; kv_len: host ints; parents: CUDA int32
+    [B,T]; lse: CUDA fp32 [B,Hq,T]."""
+    kl = _i32_array(kv_len)
+    _chk(lib().sparrow_verify_attn(ctx.handle, _ptr(q), _ptr(k_cache), _ptr(v_cache), kl, _ptr(parents),
+                                   T, _ptr(out), _ptr(lse), _stream_handle(stream)), "sparrow_verify_attn")
+
+
+def sparrow_anchor_attn(ctx: Context, q, k, v, anchor_idx, n_anchor: int, window: int, T: int, out, lse,
+                        stream=None):
+    _chk(lib().sparrow_anchor_attn(ctx.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(anchor_idx), n_anchor,
+                                   window, T, _ptr(out), _ptr(lse), _stream_handle(stream)),
+         "sparrow_anchor_attn")
+
+
+def sparrow_verify_step_host(ctx: Context, q_host, k_new_host, v_new_host, k_cache, v_cache,
+                             kv_len: Sequence[int], parents_host, T: int, out_host, lse_host, stream=None):
+    """Host tensors (ideally pinned) in and out; the caches stay on the device."""
+    kl = _i32_array(kv_len)
+    _chk(lib().sparrow_verify_step_host(ctx.handle, _ptr(q_host), _ptr(k_new_host), _ptr(v_new_host),
+                                        _ptr(k_cache), _ptr(v_cache), kl, _ptr(parents_host), T,
+                                        _ptr(out_host), _ptr(lse_host), _stream_handle(stream)),
+         "sparrow_verify_step_host")
+
+
+def sparrow_build_ancestor_masks(parents: Sequence[int]):
+    T = len(parents)
+    par = _i32_array(parents)
+    masks = (ctypes.c_uint64 * max(T, 1))()
+    _chk(lib().sparrow_build_ancestor_masks(par, T, masks), "sparrow_build_ancestor_masks")
+    return [int(masks[i]) for i in range(T)]
+
+
+def sparrow_build_anchor_idx(seq_len: int, vis_spans, window: int, T: int):
+    flat = [int(x) for s in vis_spans for x in s]
+    spans = _i32_array(flat) if flat else None
+    idx = (ctypes.c_int32 * (max(seq_len, 0) + max(T, 0) + 1))()
+    n = ctypes.c_int32(0)
+    _chk(lib().sparrow_build_anchor_idx(seq_len, spans, len(flat) // 2, window, T, idx, ctypes.byref(n)),
+         "sparrow_build_anchor_idx")
+    return [int(idx[i]) for i in range(n.value)]
+
+
+def sparrow_debug_ancestor_masks_device(ctx: Context, parents_dev: torch.Tensor, T: int, stream=None):
+    masks = torch.zeros(T, dtype=torch.int64, device=parents_dev.device)
+    _chk(lib().sparrow_debug_ancestor_masks_device(ctx.handle, _ptr(parents_dev), T, _ptr(masks),
+                                                   _stream_handle(stream)),
+         "sparrow_debug_ancestor_masks_device")
+    return masks
+
+
+def sparrow_plan_splits(n_sm: int, n_kv_heads: int, n_keys: Sequence[int], T: int):
+    nk = _i32_array(n_keys)
+    splits = (ctypes.c_int32 * len(n_keys))()
+    n_items = ctypes.c_int32(0)
+    _chk(lib().sparrow_plan_splits(n_sm, len(n_keys), n_kv_heads, nk, T, splits, ctypes.byref(n_items)),
+         "sparrow_plan_splits")
+    return [int(x) for x in splits], int(n_items.value)
+
+
+def sparrow_status_string(status: int) -> str:
+    return lib().sparrow_status_string(status).decode()

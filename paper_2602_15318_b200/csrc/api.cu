@@ -1,0 +1,459 @@
+// Host side of libsparrow_attn: context, argument validation, split planning and kernel launches
+// behind the C ABI declared in include/sparrow_attn.h.  No torch types, no allocation on the hot
+// calls, no host synchronisation on the hot calls.
+#include "sparrow_attn.h"
+
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "combine.cuh"
+#include "common.cuh"
+#include "split_gather.cuh"
+
+using namespace sparrow;
+
+struct sparrow_ctx {
+    sparrow_layout layout;
+    int device;
+    int n_sm;
+    unsigned char* ws;
+    size_t ws_bytes;
+    std::atomic<long long> launches;
+    bool use_pdl;
+};
+
+namespace {
+
+constexpr size_t kStatusBytes = 256;
+constexpr int kMinPieceKeys = 128;
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Staging {
+    size_t q, out, lse, parents, total;
+};
+
+Staging staging_layout(const sparrow_layout& L)
+{
+    Staging s;
+    const size_t B = (size_t)L.batch;
+    s.q = 0;
+    s.out = s.q + align_up(B * kMaxT * L.n_q_heads * kD * 2, 256);
+    s.lse = s.out + align_up(B * kMaxT * L.n_q_heads * kD * 2, 256);
+    s.parents = s.lse + align_up(B * kMaxT * L.n_q_heads * 4, 256);
+    s.total = s.parents + align_up(B * kMaxT * 4, 256);
+    return s;
+}
+
+int rows_per_group_for(int /*M*/) { return gather::kRows; }
+
+int max_items(int n_sm, int batch, int n_kv_heads, int n_groups)
+{
+    return n_sm + batch * n_kv_heads * n_groups;
+}
+
+// Chooses the number of key-range pieces per sequence so that the total number of work items is
+// close to (and not above) the SM count while every item streams about the same number of keys.
+sparrow_status make_plan(int n_sm, int batch, int n_kv_heads, const int32_t* n_keys, int T, SplitPlan* p)
+{
+    if (batch < 1 || batch > kMaxBatch || T < 1 || T > kMaxT || n_kv_heads < 1 || n_sm < 1) return SPARROW_ERR_SHAPE;
+    std::memset(p, 0, sizeof(*p));
+    p->batch = batch;
+    p->T = T;
+    p->M = kGroup * T;
+    p->rows_per_group = rows_per_group_for(p->M);
+    p->n_groups = (p->M + p->rows_per_group - 1) / p->rows_per_group;
+    p->n_kv_heads = n_kv_heads;
+    p->part_rows = p->rows_per_group;
+    const int units = n_kv_heads * p->n_groups;
+    int max_keys = 1;
+    for (int b = 0; b < batch; ++b) {
+        if (n_keys[b] < 1) return SPARROW_ERR_SHAPE;
+        if (n_keys[b] > max_keys) max_keys = n_keys[b];
+    }
+    auto items_for = [&](long long L) {
+        long long n = 0;
+        for (int b = 0; b < batch; ++b) n += (long long)units * ((n_keys[b] + L - 1) / L);
+        return n;
+    };
+    long long lo = kMinPieceKeys, hi = max_keys > kMinPieceKeys ? max_keys : kMinPieceKeys;
+    if (items_for(lo) > n_sm) {                 // smallest piece length that fits the SM count
+        while (lo < hi) {
+            const long long mid = (lo + hi) / 2;
+            if (items_for(mid) <= n_sm) hi = mid; else lo = mid + 1;
+        }
+    }
+    int total = 0;
+    for (int b = 0; b < batch; ++b) {
+        p->n_keys[b] = n_keys[b];
+        p->n_splits[b] = (int)((n_keys[b] + lo - 1) / lo);
+        p->item_begin[b] = total;
+        total += units * p->n_splits[b];
+    }
+    p->item_begin[batch] = total;
+    p->n_items = total;
+    return SPARROW_OK;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+sparrow_status check_ws(const sparrow_ctx* c, const SplitPlan& p)
+{
+    if (!c->ws) return SPARROW_ERR_WORKSPACE;
+    const Staging st = staging_layout(c->layout);
+    const size_t rows = (size_t)p.n_items * p.part_rows;
+    const size_t need = kStatusBytes + st.total + (align_up(rows, 64) + rows * kD) * sizeof(float);
+    return need <= c->ws_bytes ? SPARROW_OK : SPARROW_ERR_WORKSPACE;
+}
+
+float* lse_part_ptr(const sparrow_ctx* c) { return reinterpret_cast<float*>(c->ws + kStatusBytes + staging_layout(c->layout).total); }
+float* o_part_ptr(const sparrow_ctx* c, const SplitPlan& p)
+{
+    return lse_part_ptr(c) + align_up((size_t)p.n_items * p.part_rows, 64);
+}
+
+sparrow_status launch_combine(sparrow_ctx* c, const SplitPlan& plan, void* out, float* lse, cudaStream_t st)
+{
+    CombineArgs ca;
+    ca.o_part = o_part_ptr(c, plan);
+    ca.lse_part = lse_part_ptr(c);
+    ca.out = static_cast<__nv_bfloat16*>(out);
+    ca.lse = lse;
+    ca.n_q_heads = c->layout.n_q_heads;
+    ca.use_pdl = c->use_pdl ? 1 : 0;
+    const int rows = plan.batch * plan.n_kv_heads * plan.M;
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3((rows + combine::kWarps - 1) / combine::kWarps);
+    cfg.blockDim = dim3(combine::kWarps * 32);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = c->use_pdl ? 1 : 0;
+    if (cudaLaunchKernelEx(&cfg, combine::combine_kernel, plan, ca) != cudaSuccess) return SPARROW_ERR_CUDA;
+    c->launches.fetch_add(1);
+    return SPARROW_OK;
+}
+
+sparrow_status launch_split_gather(sparrow_ctx* c, const SplitPlan& plan, const void* q, const void* k, const void* v,
+                                   const int32_t* parents, const int32_t* anchor_idx, int n_anchor, int window,
+                                   cudaStream_t st)
+{
+    SplitArgs a;
+    a.q = static_cast<const __nv_bfloat16*>(q);
+    a.k = static_cast<const __nv_bfloat16*>(k);
+    a.v = static_cast<const __nv_bfloat16*>(v);
+    a.parents = parents;
+    a.anchor_idx = anchor_idx;
+    a.n_anchor = n_anchor;
+    a.window = window;
+    a.n_q_heads = c->layout.n_q_heads;
+    a.kv_capacity = c->layout.kv_capacity;
+    a.kv_stride_batch = c->layout.kv_stride_batch;
+    a.kv_stride_head = c->layout.kv_stride_head;
+    a.scale_log2e = c->layout.softmax_scale * 1.4426950408889634f;
+    a.o_part = o_part_ptr(c, plan);
+    a.lse_part = lse_part_ptr(c);
+    a.status = reinterpret_cast<unsigned*>(c->ws);
+    gather::split_gather_kernel<<<plan.n_items, gather::kThreads, gather::kSmemBytes, st>>>(plan, a);
+    if (cudaGetLastError() != cudaSuccess) return SPARROW_ERR_CUDA;
+    c->launches.fetch_add(1);
+    return SPARROW_OK;
+}
+
+__global__ void ancestor_masks_kernel(const int32_t* parents, int T, unsigned long long* masks, unsigned* status)
+{
+    const int i = threadIdx.x;
+    if (i < T) masks[i] = ancestor_word(parents, T, i, status);
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+        want = dev;
+    }
+    ~DeviceGuard() { if (ok && prev != want) cudaSetDevice(prev); }
+    int want = -1;
+};
+
+sparrow_status check_tree_host(const int32_t* parents, int T)
+{
+    for (int i = 0; i < T; ++i)
+        if (parents[i] < -1 || parents[i] >= i) return SPARROW_ERR_TREE;
+    return SPARROW_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* sparrow_status_string(sparrow_status s)
+{
+    switch (s) {
+        case SPARROW_OK: return "ok";
+        case SPARROW_ERR_NULL: return "null pointer";
+        case SPARROW_ERR_SHAPE: return "unsupported shape or size";
+        case SPARROW_ERR_TREE: return "parents[] is not a topologically ordered forest";
+        case SPARROW_ERR_ANCHOR: return "bad anchor list";
+        case SPARROW_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case SPARROW_ERR_CUDA: return "CUDA call failed";
+        case SPARROW_ERR_TIMEOUT: return "device-side wait timed out";
+        case SPARROW_ERR_ARCH: return "device is not sm_100";
+    }
+    return "unknown status";
+}
+
+sparrow_status sparrow_create(sparrow_ctx** out, const sparrow_layout* L, int device)
+{
+    if (!out || !L) return SPARROW_ERR_NULL;
+    *out = nullptr;
+    if (L->batch < 1 || L->batch > kMaxBatch || L->head_dim != kD || L->n_kv_heads < 1 ||
+        L->n_q_heads != kGroup * L->n_kv_heads || L->kv_capacity < 1 ||
+        !(L->softmax_scale > 0.f) || !std::isfinite(L->softmax_scale) ||
+        L->kv_stride_head < (int64_t)L->kv_capacity * kD || (L->kv_stride_head % 8) != 0 ||
+        (L->kv_stride_batch % 8) != 0 ||
+        (L->batch > 1 && L->kv_stride_batch < L->kv_stride_head * (int64_t)L->n_kv_heads))
+        return SPARROW_ERR_SHAPE;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) { cudaGetLastError(); return SPARROW_ERR_CUDA; }
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return SPARROW_ERR_CUDA;
+    if (prop.major != 10) return SPARROW_ERR_ARCH;
+    DeviceGuard guard(device);
+    if (!guard.ok) return SPARROW_ERR_CUDA;
+    if (cudaFuncSetAttribute(gather::split_gather_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             gather::kSmemBytes) != cudaSuccess)
+        return SPARROW_ERR_CUDA;
+    sparrow_ctx* c = new (std::nothrow) sparrow_ctx();
+    if (!c) return SPARROW_ERR_CUDA;
+    c->layout = *L;
+    c->device = device;
+    c->n_sm = prop.multiProcessorCount;
+    c->ws = nullptr;
+    c->ws_bytes = 0;
+    c->launches.store(0);
+    const char* e = std::getenv("SPARROW_NO_PDL");
+    c->use_pdl = !(e && e[0] == '1');
+    *out = c;
+    return SPARROW_OK;
+}
+
+sparrow_status sparrow_destroy(sparrow_ctx* c)
+{
+    if (!c) return SPARROW_ERR_NULL;
+    delete c;
+    return SPARROW_OK;
+}
+
+size_t sparrow_workspace_bytes(const sparrow_ctx* c, int32_t max_T)
+{
+    if (!c || max_T < 1 || max_T > kMaxT) return 0;
+    const int M = kGroup * max_T;
+    const int rpg = rows_per_group_for(M);
+    const int groups = (M + rpg - 1) / rpg;
+    const size_t items = (size_t)max_items(c->n_sm, c->layout.batch, c->layout.n_kv_heads, groups);
+    return kStatusBytes + staging_layout(c->layout).total + align_up(items * rpg * sizeof(float), 256) +
+           items * rpg * kD * sizeof(float) + 256;
+}
+
+sparrow_status sparrow_set_workspace(sparrow_ctx* c, void* p, size_t bytes)
+{
+    if (!c || !p) return SPARROW_ERR_NULL;
+    if ((reinterpret_cast<uintptr_t>(p) & 255u) != 0 || bytes < kStatusBytes + staging_layout(c->layout).total)
+        return SPARROW_ERR_WORKSPACE;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return SPARROW_ERR_CUDA;
+    if (cudaMemset(p, 0, kStatusBytes) != cudaSuccess) return SPARROW_ERR_CUDA;
+    c->ws = static_cast<unsigned char*>(p);
+    c->ws_bytes = bytes;
+    return SPARROW_OK;
+}
+
+sparrow_status sparrow_plan_splits(int32_t n_sm, int32_t batch, int32_t n_kv_heads, const int32_t* n_keys,
+                                   int32_t T, int32_t* splits_out, int32_t* n_items_out)
+{
+    if (!n_keys || !splits_out || !n_items_out) return SPARROW_ERR_NULL;
+    SplitPlan p;
+    const sparrow_status s = make_plan(n_sm, batch, n_kv_heads, n_keys, T, &p);
+    if (s != SPARROW_OK) return s;
+    for (int b = 0; b < batch; ++b) splits_out[b] = p.n_splits[b];
+    *n_items_out = p.n_items;
+    return SPARROW_OK;
+}
+
+sparrow_status sparrow_verify_attn(sparrow_ctx* c, const void* q, const void* k, const void* v,
+                                   const int32_t* kv_len, const int32_t* parents, int32_t T, void* out,
+                                   float* lse, void* stream)
+{
+    if (!c || !q || !k || !v || !kv_len || !parents || !out || !lse) return SPARROW_ERR_NULL;
+    if (T < 1 || T > kMaxT) return SPARROW_ERR_SHAPE;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return SPARROW_ERR_SHAPE;
+    int32_t n_keys[kMaxBatch];
+    for (int b = 0; b < c->layout.batch; ++b) {
+        if (kv_len[b] < 0 || (int64_t)kv_len[b] + T > c->layout.kv_capacity) return SPARROW_ERR_SHAPE;
+        n_keys[b] = kv_len[b] + T;
+    }
+    SplitPlan plan;
+    sparrow_status s = make_plan(c->n_sm, c->layout.batch, c->layout.n_kv_heads, n_keys, T, &plan);
+    if (s != SPARROW_OK) return s;
+    for (int b = 0; b < c->layout.batch; ++b) plan.kv_len[b] = kv_len[b];
+    if ((s = check_ws(c, plan)) != SPARROW_OK) return s;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return SPARROW_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if ((s = launch_split_gather(c, plan, q, k, v, parents, nullptr, 0, 0, st)) != SPARROW_OK) return s;
+    return launch_combine(c, plan, out, lse, st);
+}
+
+sparrow_status sparrow_anchor_attn(sparrow_ctx* c, const void* q, const void* k, const void* v,
+                                   const int32_t* anchor_idx, int32_t n_anchor, int32_t window, int32_t T,
+                                   void* out, float* lse, void* stream)
+{
+    if (!c || !q || !k || !v || !anchor_idx || !out || !lse) return SPARROW_ERR_NULL;
+    if (T < 1 || T > kMaxT) return SPARROW_ERR_SHAPE;
+    if (n_anchor < T || n_anchor > c->layout.kv_capacity) return SPARROW_ERR_ANCHOR;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return SPARROW_ERR_SHAPE;
+    int32_t n_keys[kMaxBatch];
+    for (int b = 0; b < c->layout.batch; ++b) n_keys[b] = n_anchor;
+    SplitPlan plan;
+    sparrow_status s = make_plan(c->n_sm, c->layout.batch, c->layout.n_kv_heads, n_keys, T, &plan);
+    if (s != SPARROW_OK) return s;
+    if ((s = check_ws(c, plan)) != SPARROW_OK) return s;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return SPARROW_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if ((s = launch_split_gather(c, plan, q, k, v, nullptr, anchor_idx, n_anchor, window, st)) != SPARROW_OK) return s;
+    return launch_combine(c, plan, out, lse, st);
+}
+
+sparrow_status sparrow_verify_step_host(sparrow_ctx* c, const void* q_host, const void* k_new_host,
+                                        const void* v_new_host, void* k_cache, void* v_cache,
+                                        const int32_t* kv_len, const int32_t* parents_host, int32_t T,
+                                        void* out_host, float* lse_host, void* stream)
+{
+    if (!c || !q_host || !k_new_host || !v_new_host || !k_cache || !v_cache || !kv_len || !parents_host ||
+        !out_host || !lse_host)
+        return SPARROW_ERR_NULL;
+    if (T < 1 || T > kMaxT) return SPARROW_ERR_SHAPE;
+    if (!c->ws) return SPARROW_ERR_WORKSPACE;
+    const sparrow_layout& L = c->layout;
+    for (int b = 0; b < L.batch; ++b) {
+        if (kv_len[b] < 0 || (int64_t)kv_len[b] + T > L.kv_capacity) return SPARROW_ERR_SHAPE;
+        const sparrow_status ts = check_tree_host(parents_host + (size_t)b * T, T);
+        if (ts != SPARROW_OK) return ts;
+    }
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return SPARROW_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const Staging sl = staging_layout(L);
+    unsigned char* base = c->ws + kStatusBytes;
+    void* q_dev = base + sl.q;
+    void* out_dev = base + sl.out;
+    float* lse_dev = reinterpret_cast<float*>(base + sl.lse);
+    int32_t* par_dev = reinterpret_cast<int32_t*>(base + sl.parents);
+    const size_t q_bytes = (size_t)L.batch * T * L.n_q_heads * kD * 2;
+    const size_t lse_bytes = (size_t)L.batch * L.n_q_heads * T * 4;
+    if (cudaMemcpyAsync(q_dev, q_host, q_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return SPARROW_ERR_CUDA;
+    if (cudaMemcpyAsync(par_dev, parents_host, (size_t)L.batch * T * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return SPARROW_ERR_CUDA;
+    const size_t row_block = (size_t)T * kD * 2;             // T new rows of one (batch, KV head)
+    for (int b = 0; b < L.batch; ++b) {
+        const size_t dst_off = ((size_t)b * L.kv_stride_batch + (size_t)kv_len[b] * kD) * 2;
+        const size_t src_off = (size_t)b * L.n_kv_heads * row_block;
+        if (cudaMemcpy2DAsync(static_cast<unsigned char*>(k_cache) + dst_off, (size_t)L.kv_stride_head * 2,
+                              static_cast<const unsigned char*>(k_new_host) + src_off, row_block, row_block,
+                              L.n_kv_heads, cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return SPARROW_ERR_CUDA;
+        if (cudaMemcpy2DAsync(static_cast<unsigned char*>(v_cache) + dst_off, (size_t)L.kv_stride_head * 2,
+                              static_cast<const unsigned char*>(v_new_host) + src_off, row_block, row_block,
+                              L.n_kv_heads, cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return SPARROW_ERR_CUDA;
+    }
+    const sparrow_status s = sparrow_verify_attn(c, q_dev, k_cache, v_cache, kv_len, par_dev, T, out_dev, lse_dev, stream);
+    if (s != SPARROW_OK) return s;
+    if (cudaMemcpyAsync(out_host, out_dev, q_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return SPARROW_ERR_CUDA;
+    if (cudaMemcpyAsync(lse_host, lse_dev, lse_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return SPARROW_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return SPARROW_ERR_CUDA;
+    return SPARROW_OK;
+}
+
+sparrow_status sparrow_build_ancestor_masks(const int32_t* parents, int32_t T, uint64_t* masks)
+{
+    if (!parents || !masks) return SPARROW_ERR_NULL;
+    if (T < 1 || T > kMaxT) return SPARROW_ERR_SHAPE;
+    const sparrow_status s = check_tree_host(parents, T);
+    if (s != SPARROW_OK) return s;
+    for (int i = 0; i < T; ++i) {                  // walk each node up to its root
+        uint64_t m = 0;
+        for (int a = i; a >= 0; a = parents[a]) m |= (uint64_t)1 << a;
+        masks[i] = m;
+    }
+    return SPARROW_OK;
+}
+
+sparrow_status sparrow_build_anchor_idx(int32_t seq_len, const int32_t* spans, int32_t n_spans, int32_t window,
+                                        int32_t T, int32_t* idx, int32_t* n_out)
+{
+    if (!idx || !n_out || (n_spans > 0 && !spans)) return SPARROW_ERR_NULL;
+    if (seq_len < 0 || T < 0 || n_spans < 0) return SPARROW_ERR_SHAPE;
+    for (int s = 0; s < n_spans; ++s)
+        if (spans[2 * s] > spans[2 * s + 1]) return SPARROW_ERR_ANCHOR;
+    const int32_t first = window > 0 && seq_len > window ? seq_len - window : 0;
+    int32_t n = 0;
+    for (int32_t p = first; p < seq_len; ++p) {
+        bool text = true;
+        for (int s = 0; s < n_spans && text; ++s) text = !(spans[2 * s] <= p && p < spans[2 * s + 1]);
+        if (text) idx[n++] = p;
+    }
+    for (int32_t t = 0; t < T; ++t) idx[n++] = seq_len + t;
+    *n_out = n;
+    return SPARROW_OK;
+}
+
+sparrow_status sparrow_debug_ancestor_masks_device(sparrow_ctx* c, const int32_t* parents_dev, int32_t T,
+                                                   uint64_t* masks_dev, void* stream)
+{
+    if (!c || !parents_dev || !masks_dev) return SPARROW_ERR_NULL;
+    if (T < 1 || T > kMaxT) return SPARROW_ERR_SHAPE;
+    if (!c->ws) return SPARROW_ERR_WORKSPACE;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return SPARROW_ERR_CUDA;
+    ancestor_masks_kernel<<<1, kMaxT, 0, static_cast<cudaStream_t>(stream)>>>(
+        parents_dev, T, reinterpret_cast<unsigned long long*>(masks_dev), reinterpret_cast<unsigned*>(c->ws));
+    if (cudaGetLastError() != cudaSuccess) return SPARROW_ERR_CUDA;
+    c->launches.fetch_add(1);
+    return SPARROW_OK;
+}
+
+sparrow_status sparrow_last_device_status(sparrow_ctx* c, void* stream)
+{
+    if (!c) return SPARROW_ERR_NULL;
+    if (!c->ws) return SPARROW_ERR_WORKSPACE;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return SPARROW_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned word = 0;
+    if (cudaMemcpyAsync(&word, c->ws, sizeof word, cudaMemcpyDeviceToHost, st) != cudaSuccess) return SPARROW_ERR_CUDA;
+    if (cudaMemsetAsync(c->ws, 0, sizeof word, st) != cudaSuccess) return SPARROW_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return SPARROW_ERR_CUDA;
+    if (word & kStatTimeout) return SPARROW_ERR_TIMEOUT;
+    if (word & kStatTree) return SPARROW_ERR_TREE;
+    if (word & kStatAnchor) return SPARROW_ERR_ANCHOR;
+    return SPARROW_OK;
+}
+
+int64_t sparrow_launch_count(const sparrow_ctx* c) { return c ? (int64_t)c->launches.load() : 0; }
+
+}  // extern "C"

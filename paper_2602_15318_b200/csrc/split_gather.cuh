@@ -1,0 +1,297 @@
+// Split-KV pass with row-gathered K/V loads: the kernel behind the text-anchored window mode
+// (Eq. 2: keys/values restricted to the anchor list) and a general path for any key layout.
+//
+// One CTA = one work item (sequence, KV head, group of up to 128 packed query rows, key-range
+// piece).  The 7 query heads of the GQA group times the T draft tokens form one packed block
+// (row r = t*7 + g), so every gathered K/V row is loaded once per KV head.  K/V rows are fetched
+// with 16-byte cp.async (row index = key index, or anchor_idx[key] when gathering) into a
+// two-stage XOR-swizzled shared-memory ring; S = QK^T and O += PV run on mma.sync m16n8k16 bf16
+// with fp32 accumulation; the online softmax is fp32 with quad shuffles.  Per item the kernel
+// writes a normalised fp32 partial output and a natural-log LSE for the combine step.
+#pragma once
+#include "common.cuh"
+
+namespace sparrow {
+
+struct SplitArgs {
+    const __nv_bfloat16* q;
+    const __nv_bfloat16* k;
+    const __nv_bfloat16* v;
+    const int32_t* parents;      // verification: DEV [B][T]; nullptr in anchored mode
+    const int32_t* anchor_idx;   // anchored: DEV [B][n_anchor]; nullptr in verification mode
+    int32_t n_anchor;
+    int32_t window;
+    int32_t n_q_heads;
+    int32_t kv_capacity;
+    int64_t kv_stride_batch;
+    int64_t kv_stride_head;
+    float scale_log2e;           // softmax_scale * log2(e)
+    float* o_part;               // [n_items][part_rows][128]
+    float* lse_part;             // [n_items][part_rows]
+    unsigned* status;
+};
+
+namespace gather {
+
+constexpr int kThreads = 256;
+constexpr int kRows = 128;        // packed query rows per CTA (8 warps x 16)
+constexpr int kTile = 64;         // keys per stage
+constexpr int kStageBytes = kTile * kD * 2;            // one K or V tile: 16 KB
+constexpr int kSmemBytes = 4 * kStageBytes + kMaxT * 8 + kMaxT * 4 + 2 * kTile * 4;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p)
+{
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
+
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&h);
+}
+// byte offset of 16-byte chunk c of row r inside a [rows][128] bf16 tile (XOR swizzle)
+__device__ __forceinline__ uint32_t swz(int r, int c) { return (uint32_t)(r * 256 + ((c ^ (r & 7)) << 4)); }
+
+__global__ void __launch_bounds__(kThreads, 1)
+split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constant__ SplitArgs args)
+{
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char* kv_smem = smem;                                   // [2 stages][K 16K | V 16K]
+    unsigned long long* anc_s = reinterpret_cast<unsigned long long*>(smem + 4 * kStageBytes);
+    int32_t* qpos_s = reinterpret_cast<int32_t*>(smem + 4 * kStageBytes + kMaxT * 8);
+    int32_t* apos_s = qpos_s + kMaxT;                                // [2][kTile] gathered row ids
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int g4 = lane >> 2, c4 = lane & 3;
+    const Item it = decode_item(plan, blockIdx.x);
+    const int T = plan.T, M = plan.M;
+    const bool anchored = args.anchor_idx != nullptr;
+    const int kv_len = anchored ? 0 : plan.kv_len[it.b];
+    const int32_t* aidx = anchored ? args.anchor_idx + (size_t)it.b * args.n_anchor : nullptr;
+
+    // ---- prologue: masks / query positions, packed Q block -> registers --------------------
+    if (tid < T) {
+        if (anchored) {
+            int p = aidx[args.n_anchor - T + tid];
+            if (p < 0 || p >= args.kv_capacity) { atomicOr(args.status, kStatAnchor); p = -1; }
+            qpos_s[tid] = p;
+        } else {
+            anc_s[tid] = ancestor_word(args.parents + (size_t)it.b * T, T, tid, args.status);
+        }
+    }
+    for (int i = tid; i < kRows * 16; i += kThreads) {
+        const int r = i >> 4, c = i & 15;
+        const int R = it.group * plan.rows_per_group + r;
+        uint4 val = make_uint4(0, 0, 0, 0);
+        if (R < M && r < plan.rows_per_group) {
+            const int t = R / kGroup, g = R % kGroup;
+            const __nv_bfloat16* src = args.q + (((size_t)it.b * T + t) * args.n_q_heads + it.kvh * kGroup + g) * kD + c * 8;
+            val = *reinterpret_cast<const uint4*>(src);
+        }
+        *reinterpret_cast<uint4*>(kv_smem + swz(r, c)) = val;
+    }
+    __syncthreads();
+    uint32_t qf[8][4];
+    {
+        const int r = warp * 16 + (lane & 15);
+        #pragma unroll
+        for (int ks = 0; ks < 8; ++ks)
+            ldsm_x4(smem_u32(kv_smem + swz(r, ks * 2 + (lane >> 4))), qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
+    }
+    // per-thread row state: rows lr0 = warp*16+g4 and lr0+8
+    int rowR[2]; bool row_ok[2]; unsigned long long row_anc[2]; int row_qpos[2];
+    #pragma unroll
+    for (int rr = 0; rr < 2; ++rr) {
+        const int lr = warp * 16 + g4 + rr * 8;
+        rowR[rr] = it.group * plan.rows_per_group + lr;
+        row_ok[rr] = rowR[rr] < M && lr < plan.rows_per_group;
+        const int t = row_ok[rr] ? rowR[rr] / kGroup : 0;
+        row_anc[rr] = anchored ? 0ull : anc_s[t];
+        row_qpos[rr] = anchored ? qpos_s[t] : 0;
+    }
+    __syncthreads();                      // Q staging area is reused by the K/V ring from here on
+
+    const __nv_bfloat16* kbase = args.k + (size_t)it.b * args.kv_stride_batch + (size_t)it.kvh * args.kv_stride_head;
+    const __nv_bfloat16* vbase = args.v + (size_t)it.b * args.kv_stride_batch + (size_t)it.kvh * args.kv_stride_head;
+    const int n_tiles = (it.key_end - it.key_begin + kTile - 1) / kTile;
+
+    auto load_tile = [&](int stage, int tile) {
+        unsigned char* ks = kv_smem + stage * 2 * kStageBytes;
+        unsigned char* vs = ks + kStageBytes;
+        #pragma unroll
+        for (int i = 0; i < (kTile * 16) / kThreads; ++i) {
+            const int idx = tid + i * kThreads;
+            const int r = idx >> 4, c = idx & 15;
+            const int j = it.key_begin + tile * kTile + r;
+            int row = -1;
+            if (j < it.key_end) {
+                if (anchored) {
+                    row = __ldg(aidx + j);
+                    if (row < 0 || row >= args.kv_capacity) { atomicOr(args.status, kStatAnchor); row = -1; }
+                } else {
+                    row = j;
+                }
+            }
+            if (anchored && c == 0) apos_s[stage * kTile + r] = row;
+            const size_t off = (size_t)(row < 0 ? 0 : row) * kD + c * 8;
+            const int bytes = row < 0 ? 0 : 16;          // 0 -> the 16 bytes are zero-filled
+            cp_async16(smem_u32(ks + swz(r, c)), kbase + off, bytes);
+            cp_async16(smem_u32(vs + swz(r, c)), vbase + off, bytes);
+        }
+    };
+
+    float o[16][4];
+    #pragma unroll
+    for (int i = 0; i < 16; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+    float m_run[2] = {-INFINITY, -INFINITY};
+    float l_run[2] = {0.f, 0.f};
+    const float c2 = args.scale_log2e;
+
+    if (n_tiles > 0) { load_tile(0, 0); }
+    cp_async_commit();
+    for (int tile = 0; tile < n_tiles; ++tile) {
+        const int stage = tile & 1;
+        if (tile + 1 < n_tiles) load_tile(stage ^ 1, tile + 1);
+        cp_async_commit();
+        cp_async_wait<1>();
+        __syncthreads();
+        const unsigned char* ks = kv_smem + stage * 2 * kStageBytes;
+        const unsigned char* vs = ks + kStageBytes;
+
+        // S = Q K^T for 16 rows x 64 keys
+        float s[8][4];
+        #pragma unroll
+        for (int i = 0; i < 8; ++i) { s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f; }
+        #pragma unroll
+        for (int kstep = 0; kstep < 8; ++kstep) {
+            #pragma unroll
+            for (int np = 0; np < 4; ++np) {
+                const int mi = lane >> 3;
+                const int key = np * 16 + (mi >> 1) * 8 + (lane & 7);
+                uint32_t b0, b1, b2, b3;
+                ldsm_x4(smem_u32(ks + swz(key, kstep * 2 + (mi & 1))), b0, b1, b2, b3);
+                mma_bf16(s[2 * np], qf[kstep], b0, b1);
+                mma_bf16(s[2 * np + 1], qf[kstep], b2, b3);
+            }
+        }
+        // visibility
+        const int j0 = it.key_begin + tile * kTile;
+        const bool need_mask = anchored || (j0 + kTile > it.key_end) || (j0 + kTile > kv_len);
+        if (need_mask) {
+            #pragma unroll
+            for (int nt = 0; nt < 8; ++nt) {
+                #pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int rr = e >> 1;
+                    const int col = nt * 8 + 2 * c4 + (e & 1);
+                    const int j = j0 + col;
+                    bool vis = j < it.key_end;
+                    if (vis) {
+                        if (anchored) {
+                            const int p = apos_s[stage * kTile + col];
+                            const int qp = row_qpos[rr];
+                            vis = p >= 0 && qp >= 0 && p <= qp && (args.window <= 0 || qp - args.window < p);
+                        } else if (j >= kv_len) {
+                            vis = (row_anc[rr] >> (j - kv_len)) & 1ull;
+                        }
+                    }
+                    if (!vis) s[nt][e] = -INFINITY;
+                }
+            }
+        }
+        // online softmax (fp32); the row sum uses the unrounded probabilities
+        float alpha[2];
+        #pragma unroll
+        for (int rr = 0; rr < 2; ++rr) {
+            float mx = -INFINITY;
+            #pragma unroll
+            for (int nt = 0; nt < 8; ++nt) mx = fmaxf(mx, fmaxf(s[nt][2 * rr], s[nt][2 * rr + 1]));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            const float m_new = fmaxf(m_run[rr], mx);
+            const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+            alpha[rr] = exp2f((m_run[rr] - m_use) * c2);
+            m_run[rr] = m_new;
+            const float mc = m_use * c2;
+            float sum = 0.f;
+            #pragma unroll
+            for (int nt = 0; nt < 8; ++nt) {
+                s[nt][2 * rr] = exp2f(fmaf(s[nt][2 * rr], c2, -mc));
+                s[nt][2 * rr + 1] = exp2f(fmaf(s[nt][2 * rr + 1], c2, -mc));
+                sum += s[nt][2 * rr] + s[nt][2 * rr + 1];
+            }
+            l_run[rr] = l_run[rr] * alpha[rr] + sum;
+        }
+        #pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            o[i][0] *= alpha[0]; o[i][1] *= alpha[0];
+            o[i][2] *= alpha[1]; o[i][3] *= alpha[1];
+        }
+        // O += P V
+        #pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+            uint32_t a[4];
+            a[0] = pack_bf16(s[2 * kk][0], s[2 * kk][1]);
+            a[1] = pack_bf16(s[2 * kk][2], s[2 * kk][3]);
+            a[2] = pack_bf16(s[2 * kk + 1][0], s[2 * kk + 1][1]);
+            a[3] = pack_bf16(s[2 * kk + 1][2], s[2 * kk + 1][3]);
+            #pragma unroll
+            for (int dn = 0; dn < 8; ++dn) {
+                const int mi = lane >> 3;
+                const int key = kk * 16 + (mi & 1) * 8 + (lane & 7);
+                uint32_t b0, b1, b2, b3;
+                ldsm_x4_t(smem_u32(vs + swz(key, dn * 2 + (mi >> 1))), b0, b1, b2, b3);
+                mma_bf16(o[2 * dn], a, b0, b1);
+                mma_bf16(o[2 * dn + 1], a, b2, b3);
+            }
+        }
+        __syncthreads();                  // this stage is refilled by the next iteration's loads
+    }
+    cp_async_wait<0>();
+
+    // ---- epilogue: normalised partial output + natural-log LSE ------------------------------
+    #pragma unroll
+    for (int rr = 0; rr < 2; ++rr) {
+        float l = l_run[rr];
+        l += __shfl_xor_sync(0xffffffffu, l, 1);
+        l += __shfl_xor_sync(0xffffffffu, l, 2);
+        if (!row_ok[rr]) continue;
+        const int lr = warp * 16 + g4 + rr * 8;
+        const float inv = l > 0.f ? 1.f / l : 0.f;
+        const size_t prow = (size_t)blockIdx.x * plan.part_rows + lr;
+        float* dst = args.o_part + prow * kD;
+        #pragma unroll
+        for (int nt = 0; nt < 16; ++nt) {
+            float2 val = make_float2(o[nt][2 * rr] * inv, o[nt][2 * rr + 1] * inv);
+            *reinterpret_cast<float2*>(dst + nt * 8 + 2 * c4) = val;
+        }
+        if (c4 == 0)
+            args.lse_part[prow] = l > 0.f ? (m_run[rr] * c2 + log2f(l)) * 0.6931471805599453f : -INFINITY;
+    }
+}
+
+}  // namespace gather
+}  // namespace sparrow

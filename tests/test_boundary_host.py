@@ -1,0 +1,93 @@
+"""Host-side checks of the C-ABI library that need no GPU: it loads, exports every symbol the
+header declares, and its pure-host helpers agree bit for bit with the oracle."""
+import itertools
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2602_15318_b200 import binding as B
+from paper_2602_15318_b200 import build, workloads as W
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    build.build()
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "sparrow_attn.h")).read()
+    declared = set(re.findall(r"\b(sparrow_[a-z_]+)\s*\(", header))
+    assert declared == set(B.EXPORTS)
+    L = B.lib()
+    for name in declared:
+        assert hasattr(L, name), name
+
+
+def test_ancestor_masks_match_oracle_all_small_trees():
+    for T in range(1, 7):
+        for par in itertools.product(*[range(-1, i) for i in range(T)]):
+            assert B.sparrow_build_ancestor_masks(list(par)) == [int(x) for x in oracle.ancestor_masks(np.array(par, np.int32))]
+    for seed in range(20):
+        par = W.random_tree_parents(seed, 4, 64)
+        assert B.sparrow_build_ancestor_masks(par) == [int(x) for x in oracle.ancestor_masks(np.array(par, np.int32))]
+
+
+def test_ancestor_masks_reject_bad_trees():
+    for bad in ([0], [-1, 1], [-1, 2, 0], [-2]):
+        with pytest.raises(B.SparrowError) as e:
+            B.sparrow_build_ancestor_masks(bad)
+        assert e.value.status == 3
+
+
+def test_anchor_idx_matches_oracle():
+    rng = np.random.default_rng(3)
+    for _ in range(50):
+        L = int(rng.integers(0, 300))
+        cuts = sorted(rng.integers(0, L + 1, size=4).tolist())
+        spans = [[cuts[0], cuts[1]], [cuts[2], cuts[3]]]
+        Wn = int(rng.integers(-1, 100)); T = int(rng.integers(0, 9))
+        assert B.sparrow_build_anchor_idx(L, spans, Wn, T) == oracle.anchor_idx(L, spans, Wn, T).tolist()
+    got = B.sparrow_build_anchor_idx(26112, [[64, 25664]], 1024, 8)
+    assert got == oracle.anchor_idx(26112, [[64, 25664]], 1024, 8).tolist() and len(got) == 456
+
+
+def test_split_plan_properties():
+    cases = [([26128], 16), ([16448], 64), ([2056], 8), ([456], 8), ([1], 1),
+             ([n + 32 for n in W.ragged_lengths(W.config_seed(4), 5, 8)], 32)]
+    for n_keys, T in cases:
+        for n_sm in (148, 132, 16):
+            splits, n_items = B.sparrow_plan_splits(n_sm, 4, n_keys, T)
+            groups = -(-7 * T // 128)
+            assert n_items == sum(4 * groups * s for s in splits)
+            assert all(1 <= s <= n for s, n in zip(splits, n_keys))
+            units = 4 * groups * len(n_keys)
+            assert n_items <= max(n_sm, units)
+            # pieces tile the key range exactly
+            for s, n in zip(splits, n_keys):
+                edges = [n * i // s for i in range(s + 1)]
+                assert edges[0] == 0 and edges[-1] == n and all(a < b for a, b in zip(edges, edges[1:]))
+    assert B.sparrow_plan_splits(148, 4, [26128], 16) == ([37], 148)
+
+
+def test_plan_rejects_bad_arguments():
+    for args in ((148, 4, [0], 8), (148, 4, [100], 0), (148, 4, [100], 65), (0, 4, [100], 8)):
+        with pytest.raises(B.SparrowError):
+            B.sparrow_plan_splits(*args)
+
+
+def test_create_without_gpu_fails_loudly():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("has a GPU")
+    with pytest.raises(B.SparrowError):
+        B.Context(1, 100, 4 * 100 * 128, 100 * 128, 0.1, allocate_workspace=False)
+
+
+def test_status_strings():
+    assert B.sparrow_status_string(0) == "ok"
+    assert "anchor" in B.sparrow_status_string(4)

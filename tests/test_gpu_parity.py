@@ -1,0 +1,274 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle on the same seeded inputs.
+
+Tolerances (bf16 inputs, fp32 accumulation): max |d out| <= 1e-2, max |d lse| <= 1e-3; masks and
+indices bit-exact.  Small cases are compared element by element; the full-size configurations are
+compared on seeded samples of (sequence, token, head) rows the oracle computes one by one.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2602_15318_b200 import binding as B
+from paper_2602_15318_b200 import workloads as W
+
+from gpu_util import (check, compare, oracle_anchor, oracle_verify, run_anchor, run_verify,
+                      sample_rows)
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+# ---- verification mode: small shapes spanning several tiles and ragged tails ---------------
+
+@pytest.mark.parametrize("kv_len,T,tree", [
+    ([300], 5, "chain"),
+    ([1], 1, "chain"),
+    ([0], 7, "chain"),             # no prefix at all: only the draft block
+    ([0], 1, "chain"),             # a single key
+    ([63], 3, "forest"),
+    ([64], 8, "random"),
+    ([129], 19, "random"),         # 133 packed rows: two row groups
+    ([1000], 64, "random"),        # 448 packed rows
+    ([4099], 16, "chain"),
+    ([1, 130, 517], 9, "random"),  # ragged batch
+    ([777, 5, 2048, 64], 32, "random"),
+])
+def test_verify_small(kv_len, T, tree):
+    case = W.make_verify_case(1234 + T + len(kv_len), kv_len, T, tree, DEV)
+    out, lse, _ = run_verify(case)
+    ref_out, ref_lse = oracle_verify(case)
+    check(out, lse, ref_out, ref_lse)
+
+
+def test_verify_capacity_larger_than_used_and_garbage_tail():
+    """Rows past kv_len+T may hold anything, NaN and Inf patterns included."""
+    case = W.make_verify_case(77, [200, 333], 6, "random", DEV, capacity=700)
+    for b, n in enumerate(case.kv_len):
+        case.k[b, :, n + case.T:, :] = float("nan")
+        case.v[b, :, n + case.T:, :] = float("inf")
+        case.v[b, :, n + case.T + 3:, :] = float("nan")
+    out, lse, _ = run_verify(case)
+    ref_out, ref_lse = oracle_verify(case)
+    check(out, lse, ref_out, ref_lse)
+
+
+def test_verify_strided_cache_view():
+    """A cache whose head stride is larger than capacity*128 (a view into a bigger buffer)."""
+    big = W.make_verify_case(78, [150], 4, "chain", DEV, capacity=400)
+    kview, vview = big.k[:, :, :200, :], big.v[:, :, :200, :]
+    ctx = B.Context(1, 200, kview.stride(0), kview.stride(1), W.SCALE)
+    out = torch.empty_like(big.q)
+    lse = torch.empty((1, W.HQ, 4), dtype=torch.float32, device=DEV)
+    B.sparrow_verify_attn(ctx, big.q, kview, vview, big.kv_len, big.parents, 4, out, lse)
+    torch.cuda.synchronize()
+    ref_out, ref_lse = oracle_verify(big)
+    check(out, lse, ref_out, ref_lse)
+
+
+def test_verify_deterministic_and_context_reuse():
+    case = W.make_verify_case(79, [3000, 1500], 12, "random", DEV)
+    out1, lse1, ctx = run_verify(case)
+    out2, lse2, _ = run_verify(case, ctx)
+    assert torch.equal(out1.view(torch.int16), out2.view(torch.int16))
+    assert torch.equal(lse1, lse2)
+    other = W.make_verify_case(80, [100, 2900], 3, "chain", DEV, capacity=case.capacity)
+    out3, lse3, _ = run_verify(other, ctx)          # different T and lengths, same context
+    ref_out, ref_lse = oracle_verify(other)
+    check(out3, lse3, ref_out, ref_lse)
+
+
+def test_verify_on_side_stream():
+    case = W.make_verify_case(81, [2000], 8, "chain", DEV)
+    ctx = B.Context.for_cache(case.k, W.SCALE)
+    out = torch.empty_like(case.q)
+    lse = torch.empty((1, W.HQ, 8), dtype=torch.float32, device=DEV)
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        B.sparrow_verify_attn(ctx, case.q, case.k, case.v, case.kv_len, case.parents, 8, out, lse)
+    s.synchronize()
+    ref_out, ref_lse = oracle_verify(case)
+    check(out, lse, ref_out, ref_lse)
+
+
+# ---- masks and indices: bit-exact -----------------------------------------------------------
+
+def test_device_ancestor_masks_bit_exact():
+    ctx = B.Context(1, 128, 4 * 128 * 128, 128 * 128, W.SCALE)
+    trees = [W.chain_parents(64), [-1] * 64, [-1], [-1, 0, 0, 2, 1, 1, 5]]
+    trees += [W.random_tree_parents(s, 4, T) for s, T in [(1, 64), (2, 48), (3, 30), (4, 25), (5, 2)]]
+    for par in trees:
+        dev = torch.tensor(par, dtype=torch.int32, device=DEV)
+        masks = B.sparrow_debug_ancestor_masks_device(ctx, dev, len(par))
+        torch.cuda.synchronize()
+        got = masks.cpu().numpy().view(np.uint64)
+        assert np.array_equal(got, oracle.ancestor_masks(np.array(par, np.int32)))
+    assert ctx.last_device_status() == 0
+
+
+def test_device_reports_malformed_parents_without_faulting():
+    ctx = B.Context(1, 128, 4 * 128 * 128, 128 * 128, W.SCALE)
+    dev = torch.tensor([-1, 0, 5, 1, -3, 2], dtype=torch.int32, device=DEV)   # 5 >= 2, -3 < -1
+    masks = B.sparrow_debug_ancestor_masks_device(ctx, dev, 6)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == 3            # SPARROW_ERR_TREE, sticky until read
+    assert ctx.last_device_status() == 0
+    got = masks.cpu().numpy().view(np.uint64)
+    assert int(got[2]) == 0b100 and int(got[4]) == 0b10000        # bad parent treated as root
+
+
+def test_masking_is_exact_under_one_hot_values():
+    """With V = one-hot rows the output row is the softmax weight vector itself: entries of
+    invisible draft keys must be exactly zero, visible ones positive."""
+    T, kv_len = 16, 40
+    case = W.make_verify_case(90, [kv_len], T, "random", DEV, capacity=128)
+    case.v.zero_()
+    n = kv_len + T
+    case.v[0, :, torch.arange(n), torch.arange(n)] = 1.0
+    out, lse, _ = run_verify(case)
+    anc = oracle.ancestor_masks(case.parents[0].cpu().numpy())
+    vis = oracle.verify_visibility(kv_len, anc).astype(bool)           # [T, n]
+    w = out[0].float().cpu().numpy()                                   # [T, Hq, 128]
+    for t in range(T):
+        assert np.all(w[t][:, :n][:, ~vis[t]] == 0.0)
+        assert np.all(w[t][:, :n][:, vis[t]] >= 0.0)
+        assert np.all(w[t][:, n:] == 0.0)
+        np.testing.assert_allclose(w[t].sum(axis=1), 1.0, atol=2e-2)
+
+
+# ---- anchored mode ---------------------------------------------------------------------------
+
+@pytest.mark.parametrize("seq_len,spans,window,T,batch", [
+    (300, [[10, 250]], 0, 4, 1),
+    (500, [[0, 100], [200, 420]], 64, 8, 2),
+    (1000, [], 0, 3, 1),                  # nothing visual: plain causal over everything
+    (2000, [[5, 1990]], 100, 16, 1),
+    (90, [[0, 90]], 0, 5, 1),             # only the draft block remains
+])
+def test_anchor_small(seq_len, spans, window, T, batch):
+    case = W.make_anchor_case(4321 + T, seq_len, spans, window, T, batch, DEV)
+    assert case.anchor_idx[0].tolist() == B.sparrow_build_anchor_idx(seq_len, spans, window, T)
+    out, lse, _ = run_anchor(case)
+    ref_out, ref_lse = oracle_anchor(case)
+    check(out, lse, ref_out, ref_lse)
+
+
+def test_anchor_window_drops_old_anchors():
+    """An explicit anchor list where the per-query window bound cuts inside the list."""
+    T = 3
+    idx = list(range(0, 400, 3)) + [1000, 1001, 1002]
+    case = W.make_anchor_case(55, 1000, [], 0, T, 1, DEV)
+    case.anchor_idx = torch.tensor([idx], dtype=torch.int32, device=DEV)
+    case.n_anchor = len(idx)
+    case.window = 700
+    out, lse, _ = run_anchor(case)
+    ref_out, ref_lse = oracle_anchor(case)
+    check(out, lse, ref_out, ref_lse)
+
+
+def test_anchor_out_of_range_index_is_reported_not_read():
+    case = W.make_anchor_case(56, 200, [[20, 150]], 0, 4, 1, DEV)
+    bad = case.anchor_idx.clone()
+    bad[0, 3] = 10 ** 6
+    case.anchor_idx = bad
+    ctx = B.Context.for_cache(case.k, W.SCALE)
+    out = torch.empty_like(case.q)
+    lse = torch.empty((1, W.HQ, 4), dtype=torch.float32, device=DEV)
+    B.sparrow_anchor_attn(ctx, case.q, case.k, case.v, case.anchor_idx, case.n_anchor, 0, 4, out, lse)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == 4
+    assert torch.isfinite(out.float()).all()
+
+
+# ---- the five configurations at full size ---------------------------------------------------
+
+def test_config1_full():
+    case = W.make_config(0, DEV)
+    out, lse, _ = run_verify(case)
+    ref_out, ref_lse = oracle_verify(case)
+    check(out, lse, ref_out, ref_lse)
+
+
+def test_config2_sampled_rows():
+    case = W.make_config(1, DEV)
+    out, lse, _ = run_verify(case)
+    rows = sample_rows(2, 1, case.T, 48)
+    ref_out, ref_lse = oracle_verify(case, rows)
+    check(out, lse, ref_out, ref_lse, rows)
+    assert torch.isfinite(out.float()).all() and torch.isfinite(lse).all()
+
+
+def test_config3_sampled_rows():
+    case = W.make_config(2, DEV)
+    out, lse, _ = run_verify(case)
+    rows = sample_rows(3, 1, case.T, 64)
+    ref_out, ref_lse = oracle_verify(case, rows)
+    check(out, lse, ref_out, ref_lse, rows)
+    assert torch.isfinite(out.float()).all() and torch.isfinite(lse).all()
+
+
+def test_config4_full():
+    case = W.make_config(3, DEV)
+    assert case.n_anchor == 456
+    out, lse, _ = run_anchor(case)
+    ref_out, ref_lse = oracle_anchor(case)
+    check(out, lse, ref_out, ref_lse)
+
+
+@pytest.mark.parametrize("layer", [0, 13, 27])
+def test_config5_layer_sampled_rows(layer):
+    case = W.make_config(4, DEV, layer=layer)
+    out, lse, _ = run_verify(case)
+    rows = sample_rows(5 + layer, 8, case.T, 40)
+    ref_out, ref_lse = oracle_verify(case, rows)
+    check(out, lse, ref_out, ref_lse, rows)
+    assert torch.isfinite(out.float()).all() and torch.isfinite(lse).all()
+
+
+# ---- host-buffer entry point and argument errors --------------------------------------------
+
+def test_verify_step_host_matches_device_call():
+    case = W.make_verify_case(91, [900, 411], 10, "random", DEV, capacity=1024)
+    ref_out, ref_lse = oracle_verify(case)
+    ctx = B.Context.for_cache(case.k, W.SCALE)
+    T = case.T
+    q_h = case.q.cpu().pin_memory()
+    k_new = torch.stack([case.k[b, :, n:n + T, :] for b, n in enumerate(case.kv_len)]).cpu().pin_memory()
+    v_new = torch.stack([case.v[b, :, n:n + T, :] for b, n in enumerate(case.kv_len)]).cpu().pin_memory()
+    for b, n in enumerate(case.kv_len):            # the call must write the draft rows itself
+        case.k[b, :, n:n + T, :] = 0
+        case.v[b, :, n:n + T, :] = 0
+    out_h = torch.empty_like(q_h).pin_memory()
+    lse_h = torch.empty((2, W.HQ, T), dtype=torch.float32).pin_memory()
+    B.sparrow_verify_step_host(ctx, q_h, k_new, v_new, case.k, case.v, case.kv_len,
+                               case.parents.cpu(), T, out_h, lse_h)
+    check(out_h, lse_h, ref_out, ref_lse)
+
+
+def test_argument_errors_launch_nothing():
+    case = W.make_verify_case(92, [100], 4, "chain", DEV)
+    ctx = B.Context.for_cache(case.k, W.SCALE)
+    out = torch.empty_like(case.q)
+    lse = torch.empty((1, W.HQ, 4), dtype=torch.float32, device=DEV)
+    n0 = ctx.launch_count()
+    for kw, status in [(dict(T=0), 2), (dict(T=65), 2), (dict(kv_len=[-1]), 2), (dict(kv_len=[101]), 2),
+                       (dict(q=None), 1), (dict(parents=None), 1)]:
+        args = dict(q=case.q, kv_len=case.kv_len, parents=case.parents, T=4)
+        args.update(kw)
+        with pytest.raises(B.SparrowError) as e:
+            B.sparrow_verify_attn(ctx, args["q"], case.k, case.v, args["kv_len"], args["parents"],
+                                  args["T"], out, lse)
+        assert e.value.status == status
+    with pytest.raises(B.SparrowError) as e:
+        B.sparrow_anchor_attn(ctx, case.q, case.k, case.v, case.parents, 2, 0, 4, out, lse)
+    assert e.value.status == 4                      # n_anchor < T
+    bare = B.Context.for_cache(case.k, W.SCALE, allocate_workspace=False)
+    with pytest.raises(B.SparrowError) as e:
+        B.sparrow_verify_attn(bare, case.q, case.k, case.v, case.kv_len, case.parents, 4, out, lse)
+    assert e.value.status == 5
+    with pytest.raises(B.SparrowError):
+        B.Context(1, 100, 51200, 12800, W.SCALE, n_q_heads=32)       # not 7:1
+    with pytest.raises(B.SparrowError):
+        B.Context(1, 100, 51200, 12800, W.SCALE, head_dim=64, n_q_heads=28)
+    assert ctx.launch_count() == n0
