@@ -1,0 +1,384 @@
+#!/usr/bin/env python
+"""Benchmark of the speculative-step attention path.
+
+Headline (the metric quoted on the long-video configuration): verification attention, batch 1,
+28/4 heads, head_dim 128, KV length 26,112 (25,600 visual + 512 text), T = 16 chain, bf16.
+A step = one sparrow_verify_attn call (split-KV pass + LSE combine).  Steps rotate over R distinct
+K/V caches whose total size is several times the L2 capacity, so every step streams its cache
+from HBM.  Timing is by CUDA events on the launching stream, after warm-up, synchronised on both
+sides; the calls are enqueued from C (sparrow_verify_attn_batch) so Python is not in the loop.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--all-configs]
+
+Prints ONE JSON line on stdout.  With --gpus N > 1 (launched under torch.distributed.run) every
+rank runs an independent replica on its own GPU -- the path has no cross-GPU exchange -- and the
+reported time is the maximum over ranks.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "verify_attn_us_per_call_kv26112_T16_bf16"
+UNIT = "us"
+WORKLOAD = "C2: verify attention, batch 1, 28/4 heads, head_dim 128, kv_len 26112, T=16 chain"
+L2_BYTES_FALLBACK = 126 * 1024 * 1024
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json)", d
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)", {}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks / throttle reasons of one GPU while a timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"], "samples": 0}
+        # keep the samples taken under load (upper half of the observed clocks)
+        sm_sorted = sorted(sm)
+        return {"sm_mhz": sm_sorted[len(sm_sorted) // 2], "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def oracle_time_c2(min_seconds=8.0, max_reps=40):
+    """Times the CPU oracle, as it stands, on full C2 calls (all 448 (token, head) rows)."""
+    import oracle
+    from paper_2602_15318_b200 import workloads as W
+    case = W.make_config(1, "cpu")
+    qb, kb, vb = W.bf16_bits(case.q), W.bf16_bits(case.k), W.bf16_bits(case.v)
+    par = case.parents.numpy()
+    cores = oracle.host_threads()
+    oracle.verify_attn(qb, kb, vb, case.kv_len, par, W.SCALE, rows=[(0, 0, 0)])      # loads the library
+    reps, t0 = 0, time.perf_counter()
+    while True:
+        oracle.verify_attn(qb, kb, vb, case.kv_len, par, W.SCALE, n_threads=cores)
+        reps += 1
+        dt = time.perf_counter() - t0
+        if dt >= min_seconds or reps >= max_reps:
+            break
+    return dt / reps * 1e6, cores, reps
+
+
+def run_reference(args, rank):
+    """The reference arm of this build is the CPU oracle timed on the host cores (rank 0 only)."""
+    if rank != 0:
+        return
+    steps, warmup = max(1, args.steps), max(0, args.warmup)
+    import oracle
+    from paper_2602_15318_b200 import workloads as W
+    case = W.make_config(1, "cpu")
+    qb, kb, vb = W.bf16_bits(case.q), W.bf16_bits(case.k), W.bf16_bits(case.v)
+    par = case.parents.numpy()
+    cores = oracle.host_threads()
+    # a step = a bounded sample of one C2 call: 56 of its 448 (token, head) rows, scaled up
+    rows = [(0, t, h) for t in range(0, 16, 2) for h in range(0, 28, 4)]
+    scale_up = 448.0 / len(rows)
+    for _ in range(min(warmup, 3)):
+        oracle.verify_attn(qb, kb, vb, case.kv_len, par, W.SCALE, rows=rows, n_threads=cores)
+    steps = min(steps, 200)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle.verify_attn(qb, kb, vb, case.kv_len, par, W.SCALE, rows=rows, n_threads=cores)
+    dt = time.perf_counter() - t0
+    us = dt / steps * scale_up * 1e6
+    line = {"impl": "reference", "metric": METRIC, "value": us, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": steps, "warmup": min(warmup, 3), "ms_per_step": us / 1e3, "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD},
+            "cpu_baseline": {"value": us, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": f"{len(rows)} of 448 (token, head) rows per step, scaled by {scale_up:g}"},
+            "e2e": {"value": us, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def time_calls(ctx, batch, n_steps, B, torch):
+    """Enqueues n_steps calls (cycling through the prepared batch) between two CUDA events."""
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    R = batch.n
+    torch.cuda.synchronize()
+    start.record()
+    done = 0
+    while done < n_steps:
+        n = min(R, n_steps - done)
+        B.sparrow_verify_attn_batch(ctx, batch, n)
+        done += n
+    stop.record()
+    torch.cuda.synchronize()
+    return start.elapsed_time(stop) * 1e3 / n_steps          # us per call
+
+
+def build_rotation(W, B, torch, dev, cfg_index, n_caches):
+    """R distinct (q, K, V) sets of one configuration, one context sized for them."""
+    cases = [W.make_config(cfg_index, dev, layer=r) for r in range(n_caches)]
+    ctx = B.Context.for_cache(cases[0].k, W.SCALE)
+    outs = [torch.empty_like(c.q) for c in cases]
+    lses = [torch.empty((c.B, W.HQ, c.T), dtype=torch.float32, device=dev) for c in cases]
+    batch = B.VerifyBatch([(c.q, c.k, c.v, c.kv_len, c.parents, c.T, o, l)
+                           for c, o, l in zip(cases, outs, lses)])
+    return cases, ctx, outs, lses, batch
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100000)
+    ap.add_argument("--warmup", type=int, default=2000)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--all-configs", action="store_true",
+                    help="also time the other configurations; extra JSON lines go to stderr")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    from paper_2602_15318_b200 import binding as B
+    from paper_2602_15318_b200 import workloads as W
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the attention path has no CPU fallback")
+    B.lib()                                   # fails loudly if the CUDA library is not built
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    steps, warmup = max(1, args.steps), max(3, args.warmup)
+    l2 = torch.cuda.get_device_properties(local_rank).L2_cache_size or L2_BYTES_FALLBACK
+    probe = W.make_config(1, "cpu")
+    kv_bytes, io_bytes, flops = probe.kv_bytes(), probe.io_bytes(), probe.flops()
+    n_caches = max(4, -(-4 * l2 // kv_bytes))                 # R * bytes >= 4 x L2
+    cases, ctx, outs, lses, batch = build_rotation(W, B, torch, dev, 1, n_caches)
+    launches0 = ctx.launch_count()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # -- device-resident throughput: whole calls ------------------------------------------------
+    time_calls(ctx, batch, warmup, B, torch)
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    launches_before = ctx.launch_count()
+    us_call = time_calls(ctx, batch, steps, B, torch)
+    launches_timed = ctx.launch_count() - launches_before
+    barrier()
+    clocks = sampler.stop()
+    if dist is not None:
+        t = torch.tensor([us_call], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        us_call = float(t.item())
+
+    # -- the dominant kernel on its own (split-KV pass), same rotation ---------------------------
+    B.sparrow_debug_set_stages(ctx, True, False)
+    time_calls(ctx, batch, max(3, warmup // 4), B, torch)
+    us_split = time_calls(ctx, batch, max(1, steps // 4), B, torch)
+    B.sparrow_debug_set_stages(ctx, True, True)
+    # -- L2-warm figure (one cache, labelled as such) --------------------------------------------
+    warm = B.VerifyBatch([(cases[0].q, cases[0].k, cases[0].v, cases[0].kv_len, cases[0].parents,
+                           cases[0].T, outs[0], lses[0])])
+    time_calls(ctx, warm, 50, B, torch)
+    us_warm = time_calls(ctx, warm, max(1, steps // 10), B, torch)
+
+    # -- end to end through the host-buffer entry point -----------------------------------------
+    c0 = cases[0]
+    T = c0.T
+    q_h = c0.q.cpu().pin_memory()
+    k_new = torch.stack([c0.k[b, :, n:n + T, :] for b, n in enumerate(c0.kv_len)]).cpu().pin_memory()
+    v_new = torch.stack([c0.v[b, :, n:n + T, :] for b, n in enumerate(c0.kv_len)]).cpu().pin_memory()
+    par_h = c0.parents.cpu().pin_memory()
+    out_h = torch.empty_like(q_h).pin_memory()
+    lse_h = torch.empty((c0.B, W.HQ, T), dtype=torch.float32).pin_memory()
+    h2d = q_h.numel() * 2 + k_new.numel() * 2 + v_new.numel() * 2 + par_h.numel() * 4
+    d2h = out_h.numel() * 2 + lse_h.numel() * 4
+    e2e_steps = max(10, min(steps // 20, 5000))
+
+    def e2e_loop(n):
+        for i in range(n):
+            c = cases[i % len(cases)]
+            B.sparrow_verify_step_host(ctx, q_h, k_new, v_new, c.k, c.v, c.kv_len, par_h, T, out_h, lse_h)
+    e2e_loop(20)
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    t0 = time.perf_counter()
+    e2e_loop(e2e_steps)
+    ev1.record()
+    torch.cuda.synchronize()
+    us_e2e = max(ev0.elapsed_time(ev1) * 1e3, (time.perf_counter() - t0) * 1e6) / e2e_steps
+    if dist is not None:
+        t = torch.tensor([us_e2e], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        us_e2e = float(t.item())
+    status = ctx.last_device_status()
+    if status != 0:
+        raise SystemExit(f"device status {status} after the timed region")
+
+    peak, peak_kind, peaks = measured_peaks()
+    alg_bytes = kv_bytes + io_bytes
+    achieved = alg_bytes / (us_split * 1e-6) / 1e9
+    traffic = None
+    tp = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(tp):
+        try:
+            traffic = json.load(open(tp)).get("verify_split_c2_dram_bytes_per_launch")
+        except Exception:
+            traffic = None
+
+    line = {
+        "metric": METRIC, "value": us_call, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+        "ms_per_step": us_call / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "l2_policy": f"rotation over {n_caches} distinct K/V caches "
+                   f"({n_caches * kv_bytes / 1e6:.0f} MB > 4 x L2 {l2 / 1e6:.0f} MB)",
+                   "launch": "plain stream launches enqueued from C (sparrow_verify_attn_batch)",
+                   "parallelism": "replicas only" if world > 1 else "1 GPU"},
+        "hbm_gbs_per_call": alg_bytes / (us_call * 1e-6) / 1e9,
+        "pct_of_8tbs_nominal": 100.0 * alg_bytes / (us_call * 1e-6) / 8e12,
+        "tflops_per_call": flops / (us_call * 1e-6) / 1e12,
+        "us_per_call_l2_warm": us_warm,
+        "us_split_kernel_only": us_split,
+        "calls_per_s_all_gpus": world * 1e6 / us_call,
+        "roofline": {"bound": "hbm", "kernel": "split-KV pass (timed alone: calls with the combine stage off)",
+                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_source": "of " + peak_kind, "algorithmic_bytes_per_launch": alg_bytes,
+                     "traffic": traffic},
+        "clocks": clocks,
+        "e2e": {"value": us_e2e, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_steps,
+                "what": "sparrow_verify_step_host: pinned host q / new K,V rows / parents in, out + lse back, "
+                        "stream synchronised every step; the committed KV prefix stays resident"},
+        "gpu_launches": launches_timed,
+    }
+    if rank == 0 and not args.no_cpu_baseline and world == 1:
+        us_cpu, cores, reps = oracle_time_c2()
+        line["cpu_baseline"] = {"value": us_cpu, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "sample": f"{reps} full C2 calls (448 (token, head) rows x 26,128 keys each)"}
+    elif rank == 0:
+        line["cpu_baseline"] = None
+
+    if args.all_configs and rank == 0 and world == 1:
+        del cases, batch, outs, lses, warm
+        torch.cuda.empty_cache()
+        extra_configs(W, B, torch, dev, l2, peak)
+
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def extra_configs(W, B, torch, dev, l2, peak):
+    """Times C1, C3, C4 and the 28-layer C5 step; one JSON line each on stderr."""
+    def emit(d):
+        print(json.dumps(d), file=sys.stderr, flush=True)
+
+    for ci, name in ((0, "C1"), (2, "C3")):
+        probe = W.make_config(ci, "cpu")
+        n_caches = max(4, -(-4 * l2 // probe.kv_bytes()))
+        cases, ctx, outs, lses, batch = build_rotation(W, B, torch, dev, ci, n_caches)
+        time_calls(ctx, batch, 500, B, torch)
+        us = time_calls(ctx, batch, 20000, B, torch)
+        by = probe.kv_bytes() + probe.io_bytes()
+        emit({"config": name, "workload": probe.name, "us_per_call": us, "hbm_gbs": by / us / 1e3,
+              "pct_of_measured_hbm": 100 * by / us / 1e3 / peak, "tflops": probe.flops() / us / 1e6,
+              "rotation": n_caches})
+        del cases, ctx, outs, lses, batch
+        torch.cuda.empty_cache()
+    # C4: anchored mode, rotate over full-length buffers
+    ac = [W.make_config(3, dev, layer=r) for r in range(8)]
+    actx = B.Context.for_cache(ac[0].k, W.SCALE)
+    aout = torch.empty_like(ac[0].q)
+    alse = torch.empty((1, W.HQ, ac[0].T), dtype=torch.float32, device=dev)
+
+    def anchor_loop(n):
+        for i in range(n):
+            c = ac[i % len(ac)]
+            B.sparrow_anchor_attn(actx, c.q, c.k, c.v, c.anchor_idx, c.n_anchor, c.window, c.T, aout, alse)
+    anchor_loop(200)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize(); ev0.record(); anchor_loop(5000); ev1.record(); torch.cuda.synchronize()
+    emit({"config": "C4", "workload": ac[0].name, "us_per_call": ev0.elapsed_time(ev1) * 1e3 / 5000,
+          "gathered_bytes": ac[0].kv_bytes(), "note": "launched from Python; latency-bound"})
+    del ac, actx
+    torch.cuda.empty_cache()
+    # C5: 28 layers, each with its own cache (about 15 GB resident)
+    layers = [W.make_config(4, dev, layer=l) for l in range(28)]
+    ctx = B.Context.for_cache(layers[0].k, W.SCALE)
+    outs = [torch.empty_like(c.q) for c in layers]
+    lses = [torch.empty((c.B, W.HQ, c.T), dtype=torch.float32, device=dev) for c in layers]
+    batch = B.VerifyBatch([(c.q, c.k, c.v, c.kv_len, c.parents, c.T, o, l) for c, o, l in zip(layers, outs, lses)])
+    time_calls(ctx, batch, 28 * 5, B, torch)
+    us = time_calls(ctx, batch, 28 * 50, B, torch)
+    by = sum(c.kv_bytes() + c.io_bytes() for c in layers)
+    fl = sum(c.flops() for c in layers)
+    emit({"config": "C5", "workload": "batch 8 ragged, T=32 tree, 28 layers per step", "us_per_step": us * 28,
+          "us_per_layer": us, "hbm_gbs": by / (us * 28) / 1e3, "pct_of_measured_hbm": 100 * by / (us * 28) / 1e3 / peak,
+          "tflops": fl / (us * 28) / 1e6, "kv_len": layers[0].kv_len})
+
+
+if __name__ == "__main__":
+    main()

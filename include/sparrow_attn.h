@@ -104,6 +104,23 @@ sparrow_status sparrow_verify_attn(sparrow_ctx* ctx, const void* q, const void* 
                                    const int32_t* parents, int32_t T, void* out, float* lse,
                                    void* stream);
 
+/* Several verification calls enqueued back to back on one stream -- e.g. the layers of one
+ * decode step, each with its own KV cache (Section 4: the target verifies the draft tree in one
+ * forward pass, i.e. one such call per decoder layer).  Equivalent to calling
+ * sparrow_verify_attn() n_calls times; stops at the first error.  `calls` is HOST memory. */
+typedef struct {
+    const void*    q;
+    const void*    k_cache;
+    const void*    v_cache;
+    const int32_t* kv_len;    /* HOST */
+    const int32_t* parents;   /* DEV */
+    int32_t        T;
+    void*          out;
+    float*         lse;
+} sparrow_verify_call;
+sparrow_status sparrow_verify_attn_batch(sparrow_ctx* ctx, const sparrow_verify_call* calls,
+                                         int32_t n_calls, void* stream);
+
 /* (b) Text-anchored window attention (Eq. 2, Section 3.1).
  *   k, v        DEV bf16 full-length buffers (layout above); only rows named by anchor_idx are read
  *   anchor_idx  DEV int32 [batch][n_anchor], strictly increasing per sequence, every entry in
@@ -156,6 +173,10 @@ sparrow_status sparrow_debug_ancestor_masks_device(sparrow_ctx* ctx, const int32
 sparrow_status sparrow_plan_splits(int32_t n_sm, int32_t batch, int32_t n_kv_heads,
                                    const int32_t* n_keys, int32_t T, int32_t* splits_out,
                                    int32_t* n_items_out);
+
+/* Profiling aid: selects which of the two kernels of a call are launched (both by default), so
+ * the split-KV pass can be timed on its own.  With run_combine == 0 out / lse are not written. */
+sparrow_status sparrow_debug_set_stages(sparrow_ctx* ctx, int32_t run_split, int32_t run_combine);
 
 /* Synchronises `stream`, returns the sticky device status (SPARROW_OK, SPARROW_ERR_TREE,
  * SPARROW_ERR_ANCHOR or SPARROW_ERR_TIMEOUT) and clears it.  Not for the hot path. */

@@ -20,7 +20,8 @@ STATUS_NAMES = {0: "SPARROW_OK", 1: "SPARROW_ERR_NULL", 2: "SPARROW_ERR_SHAPE", 
                 7: "SPARROW_ERR_TIMEOUT", 8: "SPARROW_ERR_ARCH"}
 
 EXPORTS = ["sparrow_create", "sparrow_destroy", "sparrow_workspace_bytes", "sparrow_set_workspace",
-           "sparrow_verify_attn", "sparrow_anchor_attn", "sparrow_verify_step_host",
+           "sparrow_verify_attn", "sparrow_verify_attn_batch", "sparrow_anchor_attn",
+           "sparrow_verify_step_host", "sparrow_debug_set_stages",
            "sparrow_build_ancestor_masks", "sparrow_build_anchor_idx",
            "sparrow_debug_ancestor_masks_device", "sparrow_plan_splits",
            "sparrow_last_device_status", "sparrow_launch_count", "sparrow_status_string"]
@@ -57,6 +58,8 @@ def lib():
         L.sparrow_workspace_bytes.restype = ctypes.c_size_t
         L.sparrow_set_workspace.argtypes = [vp, vp, ctypes.c_size_t]
         L.sparrow_verify_attn.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp, vp, vp]
+        L.sparrow_verify_attn_batch.argtypes = [vp, vp, i32, vp]
+        L.sparrow_debug_set_stages.argtypes = [vp, i32, i32]
         L.sparrow_anchor_attn.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp]
         L.sparrow_verify_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp]
         L.sparrow_build_ancestor_masks.argtypes = [vp, i32, vp]
@@ -155,6 +158,39 @@ def sparrow_verify_attn(ctx: Context, q, k_cache, v_cache, kv_len: Sequence[int]
     kl = _i32_array(kv_len)
     _chk(lib().sparrow_verify_attn(ctx.handle, _ptr(q), _ptr(k_cache), _ptr(v_cache), kl, _ptr(parents),
                                    T, _ptr(out), _ptr(lse), _stream_handle(stream)), "sparrow_verify_attn")
+
+
+class VerifyCall(ctypes.Structure):
+    _fields_ = [("q", ctypes.c_void_p), ("k_cache", ctypes.c_void_p), ("v_cache", ctypes.c_void_p),
+                ("kv_len", ctypes.c_void_p), ("parents", ctypes.c_void_p), ("T", ctypes.c_int32),
+                ("out", ctypes.c_void_p), ("lse", ctypes.c_void_p)]
+
+
+class VerifyBatch:
+    """A prepared array of sparrow_verify_call records (keeps the host kv_len arrays alive)."""
+
+    def __init__(self, calls):
+        """calls: iterable of (q, k_cache, v_cache, kv_len, parents, T, out, lse)."""
+        calls = list(calls)
+        self._keep = []
+        self.array = (VerifyCall * len(calls))()
+        for i, (q, k, v, kv_len, parents, T, out, lse) in enumerate(calls):
+            kl = _i32_array(kv_len)
+            self._keep.append((kl, q, k, v, parents, out, lse))
+            self.array[i] = VerifyCall(_ptr(q), _ptr(k), _ptr(v), ctypes.cast(kl, ctypes.c_void_p), _ptr(parents),
+                                       T, _ptr(out), _ptr(lse))
+        self.n = len(calls)
+
+
+def sparrow_verify_attn_batch(ctx: Context, batch: VerifyBatch, n_calls: Optional[int] = None, stream=None):
+    n = batch.n if n_calls is None else n_calls
+    _chk(lib().sparrow_verify_attn_batch(ctx.handle, batch.array, n, _stream_handle(stream)),
+         "sparrow_verify_attn_batch")
+
+
+def sparrow_debug_set_stages(ctx: Context, run_split: bool, run_combine: bool):
+    _chk(lib().sparrow_debug_set_stages(ctx.handle, int(run_split), int(run_combine)),
+         "sparrow_debug_set_stages")
 
 
 def sparrow_anchor_attn(ctx: Context, q, k, v, anchor_idx, n_anchor: int, window: int, T: int, out, lse,

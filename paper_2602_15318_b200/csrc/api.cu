@@ -26,6 +26,8 @@ struct sparrow_ctx {
     size_t ws_bytes;
     std::atomic<long long> launches;
     bool use_pdl;
+    bool run_split;
+    bool run_combine;
 };
 
 namespace {
@@ -246,6 +248,7 @@ sparrow_status sparrow_create(sparrow_ctx** out, const sparrow_layout* L, int de
     c->launches.store(0);
     const char* e = std::getenv("SPARROW_NO_PDL");
     c->use_pdl = !(e && e[0] == '1');
+    c->run_split = c->run_combine = true;
     *out = c;
     return SPARROW_OK;
 }
@@ -313,8 +316,28 @@ sparrow_status sparrow_verify_attn(sparrow_ctx* c, const void* q, const void* k,
     DeviceGuard guard(c->device);
     if (!guard.ok) return SPARROW_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if ((s = launch_split_gather(c, plan, q, k, v, parents, nullptr, 0, 0, st)) != SPARROW_OK) return s;
-    return launch_combine(c, plan, out, lse, st);
+    if (c->run_split && (s = launch_split_gather(c, plan, q, k, v, parents, nullptr, 0, 0, st)) != SPARROW_OK) return s;
+    return c->run_combine ? launch_combine(c, plan, out, lse, st) : SPARROW_OK;
+}
+
+sparrow_status sparrow_verify_attn_batch(sparrow_ctx* c, const sparrow_verify_call* calls, int32_t n_calls, void* stream)
+{
+    if (!c || !calls) return SPARROW_ERR_NULL;
+    if (n_calls < 0) return SPARROW_ERR_SHAPE;
+    for (int i = 0; i < n_calls; ++i) {
+        const sparrow_verify_call& k = calls[i];
+        const sparrow_status s = sparrow_verify_attn(c, k.q, k.k_cache, k.v_cache, k.kv_len, k.parents, k.T, k.out, k.lse, stream);
+        if (s != SPARROW_OK) return s;
+    }
+    return SPARROW_OK;
+}
+
+sparrow_status sparrow_debug_set_stages(sparrow_ctx* c, int32_t run_split, int32_t run_combine)
+{
+    if (!c) return SPARROW_ERR_NULL;
+    c->run_split = run_split != 0;
+    c->run_combine = run_combine != 0;
+    return SPARROW_OK;
 }
 
 sparrow_status sparrow_anchor_attn(sparrow_ctx* c, const void* q, const void* k, const void* v,
@@ -334,8 +357,8 @@ sparrow_status sparrow_anchor_attn(sparrow_ctx* c, const void* q, const void* k,
     DeviceGuard guard(c->device);
     if (!guard.ok) return SPARROW_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if ((s = launch_split_gather(c, plan, q, k, v, nullptr, anchor_idx, n_anchor, window, st)) != SPARROW_OK) return s;
-    return launch_combine(c, plan, out, lse, st);
+    if (c->run_split && (s = launch_split_gather(c, plan, q, k, v, nullptr, anchor_idx, n_anchor, window, st)) != SPARROW_OK) return s;
+    return c->run_combine ? launch_combine(c, plan, out, lse, st) : SPARROW_OK;
 }
 
 sparrow_status sparrow_verify_step_host(sparrow_ctx* c, const void* q_host, const void* k_new_host,
