@@ -3,6 +3,7 @@
 // calls, no host synchronisation on the hot calls.
 #include "sparrow_attn.h"
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 
 #include <atomic>
@@ -15,10 +16,26 @@
 #include "combine.cuh"
 #include "common.cuh"
 #include "split_gather.cuh"
+#include "verify_tc.cuh"
 
 using namespace sparrow;
 
+typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                      const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                      CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct TensorMapEntry {
+    const void* base;
+    CUtensorMap map;
+};
+constexpr int kMapCacheSize = 128;
+
 struct sparrow_ctx {
+    TensorMapEntry maps[kMapCacheSize];      // K/V tensor maps, keyed by base pointer
+    int n_maps;
+    int next_evict;
+    TensorMapEncodeFn encode;
+    bool verify_on_gather;                   // bring-up aid: route verification through the gather kernel
     sparrow_layout layout;
     int device;
     int n_sm;
@@ -53,7 +70,7 @@ Staging staging_layout(const sparrow_layout& L)
     return s;
 }
 
-int rows_per_group_for(int /*M*/) { return gather::kRows; }
+int rows_per_group_tc(int M) { return M <= 128 ? 128 : 256; }
 
 int max_items(int n_sm, int batch, int n_kv_heads, int n_groups)
 {
@@ -62,14 +79,15 @@ int max_items(int n_sm, int batch, int n_kv_heads, int n_groups)
 
 // Chooses the number of key-range pieces per sequence so that the total number of work items is
 // close to (and not above) the SM count while every item streams about the same number of keys.
-sparrow_status make_plan(int n_sm, int batch, int n_kv_heads, const int32_t* n_keys, int T, SplitPlan* p)
+sparrow_status make_plan(int n_sm, int batch, int n_kv_heads, const int32_t* n_keys, int T, int rows_per_group,
+                         SplitPlan* p)
 {
     if (batch < 1 || batch > kMaxBatch || T < 1 || T > kMaxT || n_kv_heads < 1 || n_sm < 1) return SPARROW_ERR_SHAPE;
     std::memset(p, 0, sizeof(*p));
     p->batch = batch;
     p->T = T;
     p->M = kGroup * T;
-    p->rows_per_group = rows_per_group_for(p->M);
+    p->rows_per_group = rows_per_group;
     p->n_groups = (p->M + p->rows_per_group - 1) / p->rows_per_group;
     p->n_kv_heads = n_kv_heads;
     p->part_rows = p->rows_per_group;
@@ -171,6 +189,65 @@ sparrow_status launch_split_gather(sparrow_ctx* c, const SplitPlan& plan, const 
     return SPARROW_OK;
 }
 
+// Tensor map over one K or V buffer: dims (128 dims, capacity rows, KV heads, batch), boxes of
+// 64 dims x 128 rows, 128-byte swizzle; rows past the capacity read as zero.
+const CUtensorMap* tensor_map_for(sparrow_ctx* c, const void* base)
+{
+    for (int i = 0; i < c->n_maps; ++i)
+        if (c->maps[i].base == base) return &c->maps[i].map;
+    if (!c->encode) return nullptr;
+    const sparrow_layout& L = c->layout;
+    int slot;
+    if (c->n_maps < kMapCacheSize) slot = c->n_maps++;
+    else { slot = c->next_evict; c->next_evict = (c->next_evict + 1) % kMapCacheSize; }
+    const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)L.kv_capacity, (cuuint64_t)L.n_kv_heads, (cuuint64_t)L.batch};
+    const cuuint64_t batch_stride = L.batch > 1 ? (cuuint64_t)L.kv_stride_batch : (cuuint64_t)L.kv_stride_head * L.n_kv_heads;
+    const cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)L.kv_stride_head * 2, batch_stride * 2};
+    const cuuint32_t box[4] = {64, 128, 1, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    const CUresult r = c->encode(&c->maps[slot].map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims,
+                                 strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { c->maps[slot].base = nullptr; if (slot == c->n_maps - 1) --c->n_maps; return nullptr; }
+    c->maps[slot].base = base;
+    return &c->maps[slot].map;
+}
+
+sparrow_status launch_verify_tc(sparrow_ctx* c, const SplitPlan& plan, const void* q, const void* k, const void* v,
+                                const int32_t* parents, cudaStream_t st)
+{
+    const CUtensorMap* mk = tensor_map_for(c, k);
+    const CUtensorMap* mv = tensor_map_for(c, v);
+    if (!mk || !mv) return SPARROW_ERR_CUDA;
+    TcArgs a;
+    a.q = static_cast<const __nv_bfloat16*>(q);
+    a.parents = parents;
+    a.n_q_heads = c->layout.n_q_heads;
+    a.n_blocks = plan.rows_per_group / 128;
+    a.n_stages = a.n_blocks == 1 ? 3 : 2;
+    a.use_pdl = c->use_pdl ? 1 : 0;
+    a.scale_log2e = c->layout.softmax_scale * 1.4426950408889634f;
+    a.o_part = o_part_ptr(c, plan);
+    a.lse_part = lse_part_ptr(c);
+    a.status = reinterpret_cast<unsigned*>(c->ws);
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(plan.n_items);
+    cfg.blockDim = dim3(tc::threads_for(a.n_blocks));
+    cfg.dynamicSmemBytes = tc::smem_bytes(a.n_blocks, a.n_stages);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = c->use_pdl ? 1 : 0;
+    const cudaError_t e = a.n_blocks == 1 ? cudaLaunchKernelEx(&cfg, tc::verify_tc_kernel<1>, *mk, *mv, plan, a)
+                                          : cudaLaunchKernelEx(&cfg, tc::verify_tc_kernel<2>, *mk, *mv, plan, a);
+    if (e != cudaSuccess) return SPARROW_ERR_CUDA;
+    c->launches.fetch_add(1);
+    return SPARROW_OK;
+}
+
 __global__ void ancestor_masks_kernel(const int32_t* parents, int T, unsigned long long* masks, unsigned* status)
 {
     const int i = threadIdx.x;
@@ -238,8 +315,23 @@ sparrow_status sparrow_create(sparrow_ctx** out, const sparrow_layout* L, int de
     if (cudaFuncSetAttribute(gather::split_gather_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              gather::kSmemBytes) != cudaSuccess)
         return SPARROW_ERR_CUDA;
+    if (cudaFuncSetAttribute(tc::verify_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             tc::smem_bytes(1, 3)) != cudaSuccess ||
+        cudaFuncSetAttribute(tc::verify_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             tc::smem_bytes(2, 2)) != cudaSuccess)
+        return SPARROW_ERR_CUDA;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || !fn)
+        return SPARROW_ERR_CUDA;
     sparrow_ctx* c = new (std::nothrow) sparrow_ctx();
     if (!c) return SPARROW_ERR_CUDA;
+    c->n_maps = 0;
+    c->next_evict = 0;
+    c->encode = reinterpret_cast<TensorMapEncodeFn>(fn);
+    const char* eg = std::getenv("SPARROW_VERIFY_GATHER");
+    c->verify_on_gather = eg && eg[0] == '1';
     c->layout = *L;
     c->device = device;
     c->n_sm = prop.multiProcessorCount;
@@ -264,11 +356,14 @@ size_t sparrow_workspace_bytes(const sparrow_ctx* c, int32_t max_T)
 {
     if (!c || max_T < 1 || max_T > kMaxT) return 0;
     const int M = kGroup * max_T;
-    const int rpg = rows_per_group_for(M);
-    const int groups = (M + rpg - 1) / rpg;
-    const size_t items = (size_t)max_items(c->n_sm, c->layout.batch, c->layout.n_kv_heads, groups);
-    return kStatusBytes + staging_layout(c->layout).total + align_up(items * rpg * sizeof(float), 256) +
-           items * rpg * kD * sizeof(float) + 256;
+    size_t worst = 0;
+    for (int rpg : {gather::kRows, rows_per_group_tc(M)}) {
+        const int groups = (M + rpg - 1) / rpg;
+        const size_t rows = (size_t)max_items(c->n_sm, c->layout.batch, c->layout.n_kv_heads, groups) * rpg;
+        const size_t need = (align_up(rows, 64) + rows * kD) * sizeof(float);
+        if (need > worst) worst = need;
+    }
+    return kStatusBytes + staging_layout(c->layout).total + worst + 256;
 }
 
 sparrow_status sparrow_set_workspace(sparrow_ctx* c, void* p, size_t bytes)
@@ -289,7 +384,8 @@ sparrow_status sparrow_plan_splits(int32_t n_sm, int32_t batch, int32_t n_kv_hea
 {
     if (!n_keys || !splits_out || !n_items_out) return SPARROW_ERR_NULL;
     SplitPlan p;
-    const sparrow_status s = make_plan(n_sm, batch, n_kv_heads, n_keys, T, &p);
+    if (T < 1 || T > kMaxT) return SPARROW_ERR_SHAPE;
+    const sparrow_status s = make_plan(n_sm, batch, n_kv_heads, n_keys, T, rows_per_group_tc(kGroup * T), &p);
     if (s != SPARROW_OK) return s;
     for (int b = 0; b < batch; ++b) splits_out[b] = p.n_splits[b];
     *n_items_out = p.n_items;
@@ -309,14 +405,19 @@ sparrow_status sparrow_verify_attn(sparrow_ctx* c, const void* q, const void* k,
         n_keys[b] = kv_len[b] + T;
     }
     SplitPlan plan;
-    sparrow_status s = make_plan(c->n_sm, c->layout.batch, c->layout.n_kv_heads, n_keys, T, &plan);
+    const int rpg = c->verify_on_gather ? gather::kRows : rows_per_group_tc(kGroup * T);
+    sparrow_status s = make_plan(c->n_sm, c->layout.batch, c->layout.n_kv_heads, n_keys, T, rpg, &plan);
     if (s != SPARROW_OK) return s;
     for (int b = 0; b < c->layout.batch; ++b) plan.kv_len[b] = kv_len[b];
     if ((s = check_ws(c, plan)) != SPARROW_OK) return s;
     DeviceGuard guard(c->device);
     if (!guard.ok) return SPARROW_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (c->run_split && (s = launch_split_gather(c, plan, q, k, v, parents, nullptr, 0, 0, st)) != SPARROW_OK) return s;
+    if (c->run_split) {
+        s = c->verify_on_gather ? launch_split_gather(c, plan, q, k, v, parents, nullptr, 0, 0, st)
+                                : launch_verify_tc(c, plan, q, k, v, parents, st);
+        if (s != SPARROW_OK) return s;
+    }
     return c->run_combine ? launch_combine(c, plan, out, lse, st) : SPARROW_OK;
 }
 
@@ -351,7 +452,7 @@ sparrow_status sparrow_anchor_attn(sparrow_ctx* c, const void* q, const void* k,
     int32_t n_keys[kMaxBatch];
     for (int b = 0; b < c->layout.batch; ++b) n_keys[b] = n_anchor;
     SplitPlan plan;
-    sparrow_status s = make_plan(c->n_sm, c->layout.batch, c->layout.n_kv_heads, n_keys, T, &plan);
+    sparrow_status s = make_plan(c->n_sm, c->layout.batch, c->layout.n_kv_heads, n_keys, T, gather::kRows, &plan);
     if (s != SPARROW_OK) return s;
     if ((s = check_ws(c, plan)) != SPARROW_OK) return s;
     DeviceGuard guard(c->device);

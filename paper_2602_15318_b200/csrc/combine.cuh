@@ -27,7 +27,10 @@ combine_kernel(const __grid_constant__ SplitPlan plan, const __grid_constant__ C
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rows_total = plan.batch * plan.n_kv_heads * plan.M;
     const int row_id = blockIdx.x * kWarps + warp;
-    if (args.use_pdl) asm volatile("griddepcontrol.wait;\n" ::: "memory");
+    if (args.use_pdl) {
+        asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
+        asm volatile("griddepcontrol.wait;\n" ::: "memory");
+    }
     if (row_id >= rows_total) return;
     const int R = row_id % plan.M;                    // packed row: t*7 + g
     const int unit_bh = row_id / plan.M;
