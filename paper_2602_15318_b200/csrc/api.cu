@@ -4,6 +4,7 @@
 #include "sparrow_attn.h"
 
 #include <cuda.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
 #include <atomic>
@@ -49,7 +50,7 @@ struct sparrow_ctx {
 
 namespace {
 
-constexpr size_t kStatusBytes = 256;
+constexpr size_t kStatusBytes = 1024;      // word 0: sticky status; the rest is spare (tuning builds use it)
 constexpr int kMinPieceKeys = 128;
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -128,14 +129,14 @@ sparrow_status check_ws(const sparrow_ctx* c, const SplitPlan& p)
     if (!c->ws) return SPARROW_ERR_WORKSPACE;
     const Staging st = staging_layout(c->layout);
     const size_t rows = (size_t)p.n_items * p.part_rows;
-    const size_t need = kStatusBytes + st.total + (align_up(rows, 64) + rows * kD) * sizeof(float);
+    const size_t need = kStatusBytes + st.total + align_up(rows, 64) * sizeof(float) + rows * kD * sizeof(__half);
     return need <= c->ws_bytes ? SPARROW_OK : SPARROW_ERR_WORKSPACE;
 }
 
 float* lse_part_ptr(const sparrow_ctx* c) { return reinterpret_cast<float*>(c->ws + kStatusBytes + staging_layout(c->layout).total); }
-float* o_part_ptr(const sparrow_ctx* c, const SplitPlan& p)
+__half* o_part_ptr(const sparrow_ctx* c, const SplitPlan& p)
 {
-    return lse_part_ptr(c) + align_up((size_t)p.n_items * p.part_rows, 64);
+    return reinterpret_cast<__half*>(lse_part_ptr(c) + align_up((size_t)p.n_items * p.part_rows, 64));
 }
 
 sparrow_status launch_combine(sparrow_ctx* c, const SplitPlan& plan, void* out, float* lse, cudaStream_t st)
@@ -150,7 +151,7 @@ sparrow_status launch_combine(sparrow_ctx* c, const SplitPlan& plan, void* out, 
     const int rows = plan.batch * plan.n_kv_heads * plan.M;
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof cfg);
-    cfg.gridDim = dim3((rows + combine::kWarps - 1) / combine::kWarps);
+    cfg.gridDim = dim3(rows);
     cfg.blockDim = dim3(combine::kWarps * 32);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -165,7 +166,7 @@ sparrow_status launch_combine(sparrow_ctx* c, const SplitPlan& plan, void* out, 
 
 sparrow_status launch_split_gather(sparrow_ctx* c, const SplitPlan& plan, const void* q, const void* k, const void* v,
                                    const int32_t* parents, const int32_t* anchor_idx, int n_anchor, int window,
-                                   cudaStream_t st)
+                                   void* out, float* lse, cudaStream_t st)
 {
     SplitArgs a;
     a.q = static_cast<const __nv_bfloat16*>(q);
@@ -182,6 +183,8 @@ sparrow_status launch_split_gather(sparrow_ctx* c, const SplitPlan& plan, const 
     a.scale_log2e = c->layout.softmax_scale * 1.4426950408889634f;
     a.o_part = o_part_ptr(c, plan);
     a.lse_part = lse_part_ptr(c);
+    a.out = static_cast<__nv_bfloat16*>(out);
+    a.lse = lse;
     a.status = reinterpret_cast<unsigned*>(c->ws);
     gather::split_gather_kernel<<<plan.n_items, gather::kThreads, gather::kSmemBytes, st>>>(plan, a);
     if (cudaGetLastError() != cudaSuccess) return SPARROW_ERR_CUDA;
@@ -214,7 +217,7 @@ const CUtensorMap* tensor_map_for(sparrow_ctx* c, const void* base)
 }
 
 sparrow_status launch_verify_tc(sparrow_ctx* c, const SplitPlan& plan, const void* q, const void* k, const void* v,
-                                const int32_t* parents, cudaStream_t st)
+                                const int32_t* parents, void* out, float* lse, cudaStream_t st)
 {
     const CUtensorMap* mk = tensor_map_for(c, k);
     const CUtensorMap* mv = tensor_map_for(c, v);
@@ -229,7 +232,10 @@ sparrow_status launch_verify_tc(sparrow_ctx* c, const SplitPlan& plan, const voi
     a.scale_log2e = c->layout.softmax_scale * 1.4426950408889634f;
     a.o_part = o_part_ptr(c, plan);
     a.lse_part = lse_part_ptr(c);
+    a.out = static_cast<__nv_bfloat16*>(out);
+    a.lse = lse;
     a.status = reinterpret_cast<unsigned*>(c->ws);
+    a.tl_all = reinterpret_cast<unsigned long long*>(c->ws + ((c->ws_bytes - 65536) & ~(size_t)255));
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof cfg);
     cfg.gridDim = dim3(plan.n_items);
@@ -360,7 +366,7 @@ size_t sparrow_workspace_bytes(const sparrow_ctx* c, int32_t max_T)
     for (int rpg : {gather::kRows, rows_per_group_tc(M)}) {
         const int groups = (M + rpg - 1) / rpg;
         const size_t rows = (size_t)max_items(c->n_sm, c->layout.batch, c->layout.n_kv_heads, groups) * rpg;
-        const size_t need = (align_up(rows, 64) + rows * kD) * sizeof(float);
+        const size_t need = align_up(rows, 64) * sizeof(float) + rows * kD * sizeof(__half);
         if (need > worst) worst = need;
     }
     return kStatusBytes + staging_layout(c->layout).total + worst + 256;
@@ -414,8 +420,8 @@ sparrow_status sparrow_verify_attn(sparrow_ctx* c, const void* q, const void* k,
     if (!guard.ok) return SPARROW_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (c->run_split) {
-        s = c->verify_on_gather ? launch_split_gather(c, plan, q, k, v, parents, nullptr, 0, 0, st)
-                                : launch_verify_tc(c, plan, q, k, v, parents, st);
+        s = c->verify_on_gather ? launch_split_gather(c, plan, q, k, v, parents, nullptr, 0, 0, out, lse, st)
+                                : launch_verify_tc(c, plan, q, k, v, parents, out, lse, st);
         if (s != SPARROW_OK) return s;
     }
     return c->run_combine ? launch_combine(c, plan, out, lse, st) : SPARROW_OK;
@@ -458,7 +464,7 @@ sparrow_status sparrow_anchor_attn(sparrow_ctx* c, const void* q, const void* k,
     DeviceGuard guard(c->device);
     if (!guard.ok) return SPARROW_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (c->run_split && (s = launch_split_gather(c, plan, q, k, v, nullptr, anchor_idx, n_anchor, window, st)) != SPARROW_OK) return s;
+    if (c->run_split && (s = launch_split_gather(c, plan, q, k, v, nullptr, anchor_idx, n_anchor, window, out, lse, st)) != SPARROW_OK) return s;
     return c->run_combine ? launch_combine(c, plan, out, lse, st) : SPARROW_OK;
 }
 

@@ -7,8 +7,11 @@
 // with 16-byte cp.async (row index = key index, or anchor_idx[key] when gathering) into a
 // two-stage XOR-swizzled shared-memory ring; S = QK^T and O += PV run on mma.sync m16n8k16 bf16
 // with fp32 accumulation; the online softmax is fp32 with quad shuffles.  Per item the kernel
-// writes a normalised fp32 partial output and a natural-log LSE for the combine step.
+// writes a normalised fp16 partial output and a natural-log LSE for the combine step (or, when
+// the sequence has a single piece, the final bf16 output and LSE).
 #pragma once
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 
 namespace sparrow {
@@ -26,8 +29,10 @@ struct SplitArgs {
     int64_t kv_stride_batch;
     int64_t kv_stride_head;
     float scale_log2e;           // softmax_scale * log2(e)
-    float* o_part;               // [n_items][part_rows][128]
+    __half* o_part;              // [n_items][part_rows][128] normalised partial outputs (fp16)
     float* lse_part;             // [n_items][part_rows]
+    __nv_bfloat16* out;          // final output, written directly for sequences with one piece
+    float* lse;
     unsigned* status;
 };
 
@@ -102,16 +107,26 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
             anc_s[tid] = ancestor_word(args.parents + (size_t)it.b * T, T, tid, args.status);
         }
     }
-    for (int i = tid; i < kRows * 16; i += kThreads) {
-        const int r = i >> 4, c = i & 15;
-        const int R = it.group * plan.rows_per_group + r;
-        uint4 val = make_uint4(0, 0, 0, 0);
-        if (R < M && r < plan.rows_per_group) {
-            const int t = R / kGroup, g = R % kGroup;
-            const __nv_bfloat16* src = args.q + (((size_t)it.b * T + t) * args.n_q_heads + it.kvh * kGroup + g) * kD + c * 8;
-            val = *reinterpret_cast<const uint4*>(src);
+    {
+        constexpr int kChunksPerThread = kRows * 16 / kThreads;      // 8: all loads first, then the stores
+        uint4 val[kChunksPerThread];
+        #pragma unroll
+        for (int u = 0; u < kChunksPerThread; ++u) {
+            const int i = tid + u * kThreads;
+            const int r = i >> 4, c = i & 15;
+            const int R = it.group * plan.rows_per_group + r;
+            val[u] = make_uint4(0, 0, 0, 0);
+            if (R < M && r < plan.rows_per_group) {
+                const int t = R / kGroup, g = R % kGroup;
+                val[u] = __ldg(reinterpret_cast<const uint4*>(
+                    args.q + (((size_t)it.b * T + t) * args.n_q_heads + it.kvh * kGroup + g) * kD + c * 8));
+            }
         }
-        *reinterpret_cast<uint4*>(kv_smem + swz(r, c)) = val;
+        #pragma unroll
+        for (int u = 0; u < kChunksPerThread; ++u) {
+            const int i = tid + u * kThreads;
+            *reinterpret_cast<uint4*>(kv_smem + swz(i >> 4, i & 15)) = val[u];
+        }
     }
     __syncthreads();
     uint32_t qf[8][4];
@@ -281,15 +296,22 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
         if (!row_ok[rr]) continue;
         const int lr = warp * 16 + g4 + rr * 8;
         const float inv = l > 0.f ? 1.f / l : 0.f;
-        const size_t prow = (size_t)blockIdx.x * plan.part_rows + lr;
-        float* dst = args.o_part + prow * kD;
-        #pragma unroll
-        for (int nt = 0; nt < 16; ++nt) {
-            float2 val = make_float2(o[nt][2 * rr] * inv, o[nt][2 * rr + 1] * inv);
-            *reinterpret_cast<float2*>(dst + nt * 8 + 2 * c4) = val;
+        const float lse_val = l > 0.f ? (m_run[rr] * c2 + log2f(l)) * 0.6931471805599453f : -INFINITY;
+        if (plan.n_splits[it.b] == 1) {                 // the only piece: write the final result
+            const int t = rowR[rr] / kGroup, h = it.kvh * kGroup + rowR[rr] % kGroup;
+            __nv_bfloat16* dst = args.out + (((size_t)it.b * T + t) * args.n_q_heads + h) * kD;
+            #pragma unroll
+            for (int nt = 0; nt < 16; ++nt)
+                *reinterpret_cast<uint32_t*>(dst + nt * 8 + 2 * c4) = pack_bf16(o[nt][2 * rr] * inv, o[nt][2 * rr + 1] * inv);
+            if (c4 == 0) args.lse[((size_t)it.b * args.n_q_heads + h) * T + t] = lse_val;
+        } else {
+            const size_t prow = (size_t)blockIdx.x * plan.part_rows + lr;
+            __half* dst = args.o_part + prow * kD;
+            #pragma unroll
+            for (int nt = 0; nt < 16; ++nt)
+                *reinterpret_cast<__half2*>(dst + nt * 8 + 2 * c4) = __floats2half2_rn(o[nt][2 * rr] * inv, o[nt][2 * rr + 1] * inv);
+            if (c4 == 0) args.lse_part[prow] = lse_val;
         }
-        if (c4 == 0)
-            args.lse_part[prow] = l > 0.f ? (m_run[rr] * c2 + log2f(l)) * 0.6931471805599453f : -INFINITY;
     }
 }
 

@@ -22,6 +22,7 @@
 // drains and exits.  TMEM is always released.
 #pragma once
 #include <cuda.h>
+#include <cuda_fp16.h>
 
 #include "common.cuh"
 
@@ -35,9 +36,12 @@ struct TcArgs {
     int32_t n_blocks;            // 128-row blocks per work item (1 or 2)
     int32_t use_pdl;
     float scale_log2e;           // softmax_scale * log2(e)
-    float* o_part;               // [n_items][part_rows][128]
+    __half* o_part;              // [n_items][part_rows][128] normalised partial outputs (fp16)
     float* lse_part;             // [n_items][part_rows]
+    __nv_bfloat16* out;          // final output, written here directly for sequences with one piece
+    float* lse;
     unsigned* status;
+    unsigned long long* tl_all;  // tuning builds only: [n_items][8] wall-clock stamps
 };
 
 namespace tc {
@@ -204,12 +208,27 @@ struct Bars {
     __device__ __forceinline__ uint32_t o_done(int i) const { return base + 96u + 8u * (uint32_t)i; }
 };
 
+// Optional timeline for tuning builds (-DSPARROW_TIMELINE): CTA 0 stores SM clock deltas into the
+// spare words of the status block.  Compiled out of the product build.
+#ifdef SPARROW_TIMELINE
+#define SPARROW_TL(word) do { if (blockIdx.x == 0 && (word) < 240) args.status[16 + (word)] = (unsigned)(clock64() - tl_t0); } while (0)
+// every CTA: wall-clock (globaltimer, ns) stamps into a per-CTA record of 8 words
+#define SPARROW_TLG(word) do { unsigned long long gt_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt_)); args.tl_all[blockIdx.x * 8 + (word)] = gt_; } while (0)
+#else
+#define SPARROW_TL(word) do { } while (0)
+#define SPARROW_TLG(word) do { } while (0)
+#endif
+
 template <int NB>
 __global__ void __launch_bounds__(threads_for(NB), 1)
 verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
                  const __grid_constant__ SplitPlan plan, const __grid_constant__ TcArgs args)
 {
+#ifdef SPARROW_TIMELINE
+    const long long tl_t0 = clock64();
+#endif
     extern __shared__ unsigned char smem_raw[];
+    if (threadIdx.x == 0) { SPARROW_TLG(0); }
     const uint32_t raw = smem_u32(smem_raw);
     unsigned char* sm = smem_raw + ((1024u - (raw & 1023u)) & 1023u);
     const int NS = args.n_stages;
@@ -252,6 +271,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    if (tid == 0) SPARROW_TL(0);
     if (args.use_pdl) {
         asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
         asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -268,29 +288,56 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
         tma_load_4d(dst + 3 * kSubTileBytes, &tmap_v, 64, row, it.kvh, it.b, B.kv_full(st));
     };
 
-    // The first ring-full of tiles goes out before anything else touches memory.
-    if (warp == kProducerWarp && lane == 0)
-        for (int j = 0; j < n_tiles && j < NS; ++j) issue_tile(j);
-
-    // ---- prologue: ancestor words and the packed Q block(s) -> shared memory (swizzled) ---------
+    // ---- prologue --------------------------------------------------------------------------------
+    // The small reads (parents, the packed Q block) are issued first and the K/V stream second:
+    // requests are served roughly in order, and Q queued behind a ring-full of K/V tiles would
+    // hold up the first S = Q K^T for several microseconds.
+    constexpr int kChunksPerThread = 16;             // 16-byte chunks of Q per softmax thread
+    uint4 qv[kChunksPerThread];
+    int32_t par0 = -1, par1 = -1;
     if (warp < 4 * NB) {
-        if (tid < T) anc_s[tid] = ancestor_word(args.parents + (size_t)it.b * T, T, tid, args.status);
-        for (int i = tid; i < NB * 128 * 16; i += NB * 128) {
+        if (warp == 0) {
+            const int32_t* par_g = args.parents + (size_t)it.b * T;
+            if (lane < T) par0 = __ldg(par_g + lane);
+            if (lane + 32 < T) par1 = __ldg(par_g + lane + 32);
+        }
+        #pragma unroll
+        for (int u = 0; u < kChunksPerThread; ++u) {
+            const int i = tid + u * NB * 128;
             const int r = i >> 4, c = i & 15;                       // row in the item, 16-byte chunk
             const int R = it.group * plan.rows_per_group + r;
-            uint4 val = make_uint4(0, 0, 0, 0);
+            qv[u] = make_uint4(0, 0, 0, 0);
             if (R < M && r < plan.rows_per_group) {
                 const int t = R / kGroup, g = R % kGroup;
-                val = *reinterpret_cast<const uint4*>(
-                    args.q + (((size_t)it.b * T + t) * args.n_q_heads + it.kvh * kGroup + g) * kD + c * 8);
+                qv[u] = __ldg(reinterpret_cast<const uint4*>(
+                    args.q + (((size_t)it.b * T + t) * args.n_q_heads + it.kvh * kGroup + g) * kD + c * 8));
             }
+        }
+    }
+    __syncthreads();                                 // every Q / parents request is in flight
+    if (warp == kProducerWarp && lane == 0)
+        for (int j = 0; j < n_tiles && j < NS; ++j) issue_tile(j);
+    if (warp < 4 * NB) {
+        if (warp == 0) {
+            int32_t* par_s = reinterpret_cast<int32_t*>(misc + 768);               // [64]
+            if (lane < T) par_s[lane] = par0;
+            if (lane + 32 < T) par_s[lane + 32] = par1;
+            __syncwarp();
+            for (int i = lane; i < T; i += 32) anc_s[i] = ancestor_word(par_s, T, i, args.status);
+        }
+        #pragma unroll
+        for (int u = 0; u < kChunksPerThread; ++u) {
+            const int i = tid + u * NB * 128;
+            const int r = i >> 4, c = i & 15;
             const int blk = r >> 7, rr = r & 127;
             unsigned char* dst = q_sm + blk * kQBlockBytes + (c >> 3) * kSubTileBytes + rr * 128 + (((c & 7) ^ (rr & 7)) << 4);
-            *reinterpret_cast<uint4*>(dst) = val;
+            *reinterpret_cast<uint4*>(dst) = qv[u];
         }
         fence_proxy_async();
     }
+    if (tid == 0) SPARROW_TL(1);
     __syncthreads();
+    if (tid == 0) SPARROW_TL(2);
 
     if (warp == kProducerWarp) {
         // ================= TMA producer =================
@@ -314,6 +361,9 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
                 if (blk == 0) {                                       // first use of this tile
                     if (!mbar_wait(B.kv_full(st), (j / NS) & 1)) { ok = false; return; }
                     tc_fence_after();
+                    SPARROW_TL(100 + 4 * n);
+                    if (j == 0) { SPARROW_TLG(1); }
+                    if (j == n_tiles - 1) { SPARROW_TLG(2); }
                 }
                 const uint32_t qa = smem_u32(q_sm + blk * kQBlockBytes);
                 const uint32_t ka = smem_u32(kv_sm + st * kStageBytes);
@@ -323,6 +373,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
                     mma_ss(tmem + slot * 128, smem_desc(qa + off, 16, 1024), smem_desc(ka + off, 16, 1024), idesc_qk, ks > 0);
                 }
                 tc_commit(B.s_full(slot));
+                SPARROW_TL(101 + 4 * n);
             };
             if (n_jobs > 0) issue_qk(0);
             for (int n = 0; n < n_jobs && ok; ++n) {
@@ -330,6 +381,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
                 const int j = n / NB, blk = n % NB, slot = n & 1, st = j % NS;
                 if (!mbar_wait(B.p_full(slot), (n >> 1) & 1)) { ok = false; break; }
                 tc_fence_after();
+                SPARROW_TL(102 + 4 * n);
                 const uint32_t va = smem_u32(kv_sm + st * kStageBytes + 2 * kSubTileBytes);
                 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk)
@@ -337,7 +389,9 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
                            smem_desc(va + kk * 2048, kSubTileBytes, 1024), idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);
                 tc_commit(B.o_done(blk));
                 if (blk == NB - 1) tc_commit(B.kv_empty(st));
+                SPARROW_TL(103 + 4 * n);
             }
+            SPARROW_TLG(3);
             if (!ok) { atomicOr(args.status, kStatTimeout); *abort_flag = 1; }
         }
     } else if (warp < 4 * NB) {
@@ -359,20 +413,35 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
             const int j = n / NB, slot = n & 1, st = j % NS;
             if (!mbar_wait_warp(B.s_full(slot), (n >> 1) & 1)) { ok = false; break; }
             tc_fence_after();
+            if (tid == 0) SPARROW_TL(8 + 6 * n);
             float s[128];
             const uint32_t s_addr = lane_addr + slot * 128;
             tmem_ld32(s_addr, s); tmem_ld32(s_addr + 32, s + 32);
             tmem_ld32(s_addr + 64, s + 64); tmem_ld32(s_addr + 96, s + 96);
             tmem_wait_ld();
+            if (tid == 0) SPARROW_TL(9 + 6 * n);
 
             const int j0 = it.key_begin + j * kTile;
             if (j0 + kTile > it.key_end || j0 + kTile > kv_len) {          // tile touches the draft block / range end
+                // 128-bit visibility word of this row for the tile's columns: prefix columns, then the
+                // ancestor word shifted to the draft block's column, cut at the end of the key range.
+                const int d0 = kv_len - j0;                                 // column of draft token 0 (any sign)
+                const int nval = it.key_end - j0;                           // valid columns (>= 1)
+                unsigned long long lo, hi;
+                if (d0 >= 128) { lo = ~0ull; hi = ~0ull; }
+                else if (d0 >= 64) { lo = ~0ull; hi = ((1ull << (d0 - 64)) - 1ull) | (anc << (d0 - 64)); }
+                else if (d0 > 0) { lo = ((1ull << d0) - 1ull) | (anc << d0); hi = anc >> (64 - d0); }
+                else if (d0 > -64) { lo = anc >> (-d0); hi = 0ull; }
+                else { lo = 0ull; hi = 0ull; }
+                if (nval < 64) { lo &= (1ull << nval) - 1ull; hi = 0ull; }
+                else if (nval < 128) { hi &= (1ull << (nval - 64)) - 1ull; }
+                const uint32_t w0 = (uint32_t)lo, w1 = (uint32_t)(lo >> 32), w2 = (uint32_t)hi, w3 = (uint32_t)(hi >> 32);
                 #pragma unroll
-                for (int c = 0; c < 128; ++c) {
-                    const int key = j0 + c;
-                    bool vis = key < it.key_end;
-                    if (vis && key >= kv_len) vis = (anc >> (key - kv_len)) & 1ull;
-                    if (!vis) s[c] = -INFINITY;
+                for (int c = 0; c < 32; ++c) {
+                    if (!((w0 >> c) & 1u)) s[c] = -INFINITY;
+                    if (!((w1 >> c) & 1u)) s[32 + c] = -INFINITY;
+                    if (!((w2 >> c) & 1u)) s[64 + c] = -INFINITY;
+                    if (!((w3 >> c) & 1u)) s[96 + c] = -INFINITY;
                 }
                 // V rows past the end of the sequence may hold anything: zero them so 0 * x stays 0
                 if (wg == 0 && j0 + kTile > n_keys_seq && row_local >= n_keys_seq - j0) {
@@ -386,10 +455,15 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
                     fence_proxy_async();
                 }
             }
-            float mx = s[0];
+            float mx4[4] = {s[0], s[1], s[2], s[3]};                   // four independent chains
             #pragma unroll
-            for (int c = 1; c < 128; ++c) mx = fmaxf(mx, s[c]);
+            for (int c = 4; c < 128; c += 4) {
+                mx4[0] = fmaxf(mx4[0], s[c]); mx4[1] = fmaxf(mx4[1], s[c + 1]);
+                mx4[2] = fmaxf(mx4[2], s[c + 2]); mx4[3] = fmaxf(mx4[3], s[c + 3]);
+            }
+            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
 
+            if (tid == 0) SPARROW_TL(10 + 6 * n);
             const bool need = mx > m_ref + thr || (m_ref == -INFINITY && mx > -INFINITY);
             if (__any_sync(0xffffffffu, need)) {
                 float alpha = 1.f;
@@ -415,8 +489,9 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
                     tmem_wait_st();
                 }
             }
+            if (tid == 0) SPARROW_TL(11 + 6 * n);
             const float mc = (m_ref == -INFINITY) ? 0.f : m_ref * c2;
-            float sum = 0.f;
+            float sum4[4] = {0.f, 0.f, 0.f, 0.f};
             #pragma unroll
             for (int ch = 0; ch < 4; ++ch) {                          // 32 scores -> 16 packed bf16 pairs
                 uint32_t p[16];
@@ -424,15 +499,17 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
                 for (int c = 0; c < 16; ++c) {
                     const float p0 = ex2(fmaf(s[ch * 32 + 2 * c], c2, -mc));
                     const float p1 = ex2(fmaf(s[ch * 32 + 2 * c + 1], c2, -mc));
-                    sum += p0 + p1;
+                    sum4[c & 3] += p0 + p1;
                     p[c] = pack_bf16x2(p0, p1);
                 }
                 tmem_st16(s_addr + ch * 16, p);
             }
-            l_run += sum;
+            l_run += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+            if (tid == 0) SPARROW_TL(12 + 6 * n);
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(B.p_full(slot));
+            if (tid == 0) SPARROW_TL(13 + 6 * n);
         }
 
         // ---- epilogue: normalised partial output + natural-log LSE -------------------------------
@@ -440,23 +517,45 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
             const int blk = NB == 2 ? wg : 0;
             if (mbar_wait_warp(B.o_done(blk), (n_tiles - 1) & 1)) {
                 tc_fence_after();
+                if (tid == 0) { SPARROW_TL(3); SPARROW_TLG(4); }
                 const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-                const size_t prow = (size_t)blockIdx.x * plan.part_rows + r_item;
+                const float lse_val = l_run > 0.f ? (m_ref * c2 + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
                 const uint32_t o_addr = lane_addr + 256 + blk * 128;
+                const bool direct = plan.n_splits[it.b] == 1;           // the only piece: write the final result
+                const size_t prow = (size_t)blockIdx.x * plan.part_rows + r_item;
+                const int t_row = row_ok ? R / kGroup : 0, h_row = it.kvh * kGroup + (row_ok ? R % kGroup : 0);
                 #pragma unroll
                 for (int ch = 0; ch < 4; ++ch) {
                     float o[32];
                     tmem_ld32(o_addr + ch * 32, o);
                     tmem_wait_ld();
                     if (row_ok) {
-                        float4* dst = reinterpret_cast<float4*>(args.o_part + prow * kD + ch * 32);
-                        #pragma unroll
-                        for (int c = 0; c < 8; ++c)
-                            dst[c] = make_float4(o[4 * c] * inv, o[4 * c + 1] * inv, o[4 * c + 2] * inv, o[4 * c + 3] * inv);
+                        uint4 pk[4];
+                        uint32_t* w = reinterpret_cast<uint32_t*>(pk);
+                        if (direct) {
+                            #pragma unroll
+                            for (int c = 0; c < 16; ++c) w[c] = pack_bf16x2(o[2 * c] * inv, o[2 * c + 1] * inv);
+                            uint4* dst = reinterpret_cast<uint4*>(
+                                args.out + (((size_t)it.b * T + t_row) * args.n_q_heads + h_row) * kD + ch * 32);
+                            #pragma unroll
+                            for (int c = 0; c < 4; ++c) dst[c] = pk[c];
+                        } else {
+                            #pragma unroll
+                            for (int c = 0; c < 16; ++c) {
+                                const __half2 h2 = __floats2half2_rn(o[2 * c] * inv, o[2 * c + 1] * inv);
+                                w[c] = *reinterpret_cast<const uint32_t*>(&h2);
+                            }
+                            uint4* dst = reinterpret_cast<uint4*>(args.o_part + prow * kD + ch * 32);
+                            #pragma unroll
+                            for (int c = 0; c < 4; ++c) dst[c] = pk[c];
+                        }
                     }
                 }
-                if (row_ok)
-                    args.lse_part[prow] = l_run > 0.f ? (m_ref * c2 + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
+                if (row_ok) {
+                    if (direct) args.lse[((size_t)it.b * args.n_q_heads + h_row) * T + t_row] = lse_val;
+                    else args.lse_part[prow] = lse_val;
+                }
+                if (tid == 0) SPARROW_TL(4);
             } else {
                 ok = false;
             }
@@ -474,6 +573,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
         for (int i = 0; i < 2000; ++i) __nanosleep(1000);
         __syncthreads();
     }
+    if (tid == 0) { SPARROW_TL(5); SPARROW_TLG(5); }
     if (warp == kMmaWarp) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
