@@ -198,14 +198,18 @@ __host__ __device__ constexpr uint32_t idesc_bf16(bool b_mn_major)
     return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 }
 
-// Shared-memory addresses of the mbarriers (16 consecutive 8-byte slots).
+// Shared-memory addresses of the mbarriers (8-byte slots).  K and V tiles have their own full /
+// empty pairs: a K tile is released as soon as its S = Q K^T has been computed, a V tile only
+// after its O += P V, so the K stream runs ahead of the V stream.
 struct Bars {
     uint32_t base;
-    __device__ __forceinline__ uint32_t kv_full(int i) const { return base + 8u * (uint32_t)i; }
-    __device__ __forceinline__ uint32_t kv_empty(int i) const { return base + 32u + 8u * (uint32_t)i; }
-    __device__ __forceinline__ uint32_t s_full(int i) const { return base + 64u + 8u * (uint32_t)i; }
-    __device__ __forceinline__ uint32_t p_full(int i) const { return base + 80u + 8u * (uint32_t)i; }
-    __device__ __forceinline__ uint32_t o_done(int i) const { return base + 96u + 8u * (uint32_t)i; }
+    __device__ __forceinline__ uint32_t k_full(int i) const { return base + 8u * (uint32_t)i; }
+    __device__ __forceinline__ uint32_t k_empty(int i) const { return base + 32u + 8u * (uint32_t)i; }
+    __device__ __forceinline__ uint32_t v_full(int i) const { return base + 64u + 8u * (uint32_t)i; }
+    __device__ __forceinline__ uint32_t v_empty(int i) const { return base + 96u + 8u * (uint32_t)i; }
+    __device__ __forceinline__ uint32_t s_full(int i) const { return base + 128u + 8u * (uint32_t)i; }
+    __device__ __forceinline__ uint32_t p_full(int i) const { return base + 144u + 8u * (uint32_t)i; }
+    __device__ __forceinline__ uint32_t o_done(int i) const { return base + 160u + 8u * (uint32_t)i; }
 };
 
 // Optional timeline for tuning builds (-DSPARROW_TIMELINE): CTA 0 stores SM clock deltas into the
@@ -236,9 +240,9 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
     unsigned char* q_sm = sm;
     unsigned char* kv_sm = sm + NB * kQBlockBytes;
     unsigned char* misc = kv_sm + NS * kStageBytes;
-    uint64_t* bar_mem = reinterpret_cast<uint64_t*>(misc);                  // 16 barriers
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 128);
-    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(misc + 132);
+    uint64_t* bar_mem = reinterpret_cast<uint64_t*>(misc);                  // 22 barriers in 176 bytes
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 192);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(misc + 196);
     unsigned long long* anc_s = reinterpret_cast<unsigned long long*>(misc + 256);   // [64]
 
     Bars B;
@@ -254,7 +258,9 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
 
     // ---- setup: barriers, TMEM ------------------------------------------------------------------
     if (tid == 0) {
-        for (int i = 0; i < 4; ++i) { mbar_init(B.kv_full(i), 1); mbar_init(B.kv_empty(i), 1); }
+        for (int i = 0; i < 4; ++i) {
+            mbar_init(B.k_full(i), 1); mbar_init(B.k_empty(i), 1); mbar_init(B.v_full(i), 1); mbar_init(B.v_empty(i), 1);
+        }
         for (int i = 0; i < 2; ++i) { mbar_init(B.s_full(i), 1); mbar_init(B.p_full(i), 128); mbar_init(B.o_done(i), 1); }
         *abort_flag = 0;
         fence_barrier_init();
@@ -277,15 +283,21 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
         asm volatile("griddepcontrol.wait;" ::: "memory");
     }
 
-    auto issue_tile = [&](int j) {                  // producer thread only
+    auto issue_k = [&](int j) {                     // producer thread only
         const int st = j % NS;
         const uint32_t dst = smem_u32(kv_sm + st * kStageBytes);
         const int row = it.key_begin + j * kTile;
-        mbar_expect_tx(B.kv_full(st), kStageBytes);
-        tma_load_4d(dst, &tmap_k, 0, row, it.kvh, it.b, B.kv_full(st));
-        tma_load_4d(dst + kSubTileBytes, &tmap_k, 64, row, it.kvh, it.b, B.kv_full(st));
-        tma_load_4d(dst + 2 * kSubTileBytes, &tmap_v, 0, row, it.kvh, it.b, B.kv_full(st));
-        tma_load_4d(dst + 3 * kSubTileBytes, &tmap_v, 64, row, it.kvh, it.b, B.kv_full(st));
+        mbar_expect_tx(B.k_full(st), 2 * kSubTileBytes);
+        tma_load_4d(dst, &tmap_k, 0, row, it.kvh, it.b, B.k_full(st));
+        tma_load_4d(dst + kSubTileBytes, &tmap_k, 64, row, it.kvh, it.b, B.k_full(st));
+    };
+    auto issue_v = [&](int j) {
+        const int st = j % NS;
+        const uint32_t dst = smem_u32(kv_sm + st * kStageBytes + 2 * kSubTileBytes);
+        const int row = it.key_begin + j * kTile;
+        mbar_expect_tx(B.v_full(st), 2 * kSubTileBytes);
+        tma_load_4d(dst, &tmap_v, 0, row, it.kvh, it.b, B.v_full(st));
+        tma_load_4d(dst + kSubTileBytes, &tmap_v, 64, row, it.kvh, it.b, B.v_full(st));
     };
 
     // ---- prologue --------------------------------------------------------------------------------
@@ -316,7 +328,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
     }
     __syncthreads();                                 // every Q / parents request is in flight
     if (warp == kProducerWarp && lane == 0)
-        for (int j = 0; j < n_tiles && j < NS; ++j) issue_tile(j);
+        for (int j = 0; j < n_tiles && j < NS; ++j) { issue_k(j); issue_v(j); }
     if (warp < 4 * NB) {
         if (warp == 0) {
             int32_t* par_s = reinterpret_cast<int32_t*>(misc + 768);               // [64]
@@ -343,10 +355,15 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
         // ================= TMA producer =================
         if (NB == 2) asm volatile("setmaxnreg.dec.sync.aligned.u32 40;" ::: "memory");
         if (lane == 0) {
-            for (int j = NS; j < n_tiles; ++j) {
-                const int st = j % NS, k = j / NS;
-                if (!mbar_wait(B.kv_empty(st), (k - 1) & 1)) { atomicOr(args.status, kStatTimeout); *abort_flag = 1; break; }
-                issue_tile(j);
+            // refill whichever ring has a free slot; K slots free up about one tile before V slots
+            int jk = NS < n_tiles ? NS : n_tiles, jv = jk;
+            uint32_t idle = 0;
+            while (jk < n_tiles || jv < n_tiles) {
+                bool progress = false;
+                if (jk < n_tiles && mbar_try_wait(B.k_empty(jk % NS), (jk / NS - 1) & 1)) { issue_k(jk); ++jk; progress = true; }
+                if (jv < n_tiles && mbar_try_wait(B.v_empty(jv % NS), (jv / NS - 1) & 1)) { issue_v(jv); ++jv; progress = true; }
+                if (progress) idle = 0;
+                else if (++idle > kSpinLimit) { atomicOr(args.status, kStatTimeout); *abort_flag = 1; break; }
             }
         }
     } else if (warp == kMmaWarp) {
@@ -358,8 +375,8 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
             bool ok = true;
             auto issue_qk = [&](int n) {
                 const int j = n / NB, blk = n % NB, slot = n & 1, st = j % NS;
-                if (blk == 0) {                                       // first use of this tile
-                    if (!mbar_wait(B.kv_full(st), (j / NS) & 1)) { ok = false; return; }
+                if (blk == 0) {                                       // first use of this K tile
+                    if (!mbar_wait(B.k_full(st), (j / NS) & 1)) { ok = false; return; }
                     tc_fence_after();
                     SPARROW_TL(100 + 4 * n);
                     if (j == 0) { SPARROW_TLG(1); }
@@ -373,12 +390,14 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
                     mma_ss(tmem + slot * 128, smem_desc(qa + off, 16, 1024), smem_desc(ka + off, 16, 1024), idesc_qk, ks > 0);
                 }
                 tc_commit(B.s_full(slot));
+                if (blk == NB - 1) tc_commit(B.k_empty(st));
                 SPARROW_TL(101 + 4 * n);
             };
             if (n_jobs > 0) issue_qk(0);
             for (int n = 0; n < n_jobs && ok; ++n) {
                 if (n + 1 < n_jobs) { issue_qk(n + 1); if (!ok) break; }
                 const int j = n / NB, blk = n % NB, slot = n & 1, st = j % NS;
+                if (blk == 0 && !mbar_wait(B.v_full(st), (j / NS) & 1)) { ok = false; break; }
                 if (!mbar_wait(B.p_full(slot), (n >> 1) & 1)) { ok = false; break; }
                 tc_fence_after();
                 SPARROW_TL(102 + 4 * n);
@@ -388,7 +407,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
                     mma_ts(tmem + 256 + blk * 128, tmem + slot * 128 + kk * 8,
                            smem_desc(va + kk * 2048, kSubTileBytes, 1024), idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);
                 tc_commit(B.o_done(blk));
-                if (blk == NB - 1) tc_commit(B.kv_empty(st));
+                if (blk == NB - 1) tc_commit(B.v_empty(st));
                 SPARROW_TL(103 + 4 * n);
             }
             SPARROW_TLG(3);
@@ -445,7 +464,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
                 }
                 // V rows past the end of the sequence may hold anything: zero them so 0 * x stays 0
                 if (wg == 0 && j0 + kTile > n_keys_seq && row_local >= n_keys_seq - j0) {
-                    mbar_wait(B.kv_full(st), (j / NS) & 1);
+                    mbar_wait(B.v_full(st), (j / NS) & 1);
                     unsigned char* vrow = kv_sm + st * kStageBytes + 2 * kSubTileBytes + row_local * 128;
                     #pragma unroll
                     for (int c = 0; c < 8; ++c) {
@@ -522,38 +541,57 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
                 const float lse_val = l_run > 0.f ? (m_ref * c2 + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
                 const uint32_t o_addr = lane_addr + 256 + blk * 128;
                 const bool direct = plan.n_splits[it.b] == 1;           // the only piece: write the final result
-                const size_t prow = (size_t)blockIdx.x * plan.part_rows + r_item;
+                const size_t prow0 = (size_t)blockIdx.x * plan.part_rows + blk * 128;    // first partial row of this block
                 const int t_row = row_ok ? R / kGroup : 0, h_row = it.kvh * kGroup + (row_ok ? R % kGroup : 0);
+                // Staging area: this row block's Q tile (every MMA that read it has completed).  Row r
+                // holds 16 chunks of 16 bytes (128 halves), chunk c stored at position c ^ (r & 15).
+                unsigned char* stage = q_sm + blk * kQBlockBytes;
                 #pragma unroll
                 for (int ch = 0; ch < 4; ++ch) {
                     float o[32];
                     tmem_ld32(o_addr + ch * 32, o);
                     tmem_wait_ld();
-                    if (row_ok) {
-                        uint4 pk[4];
-                        uint32_t* w = reinterpret_cast<uint32_t*>(pk);
-                        if (direct) {
+                    uint4 pk[4];
+                    uint32_t* w = reinterpret_cast<uint32_t*>(pk);
+                    if (direct) {
+                        if (row_ok) {
                             #pragma unroll
                             for (int c = 0; c < 16; ++c) w[c] = pack_bf16x2(o[2 * c] * inv, o[2 * c + 1] * inv);
                             uint4* dst = reinterpret_cast<uint4*>(
                                 args.out + (((size_t)it.b * T + t_row) * args.n_q_heads + h_row) * kD + ch * 32);
                             #pragma unroll
                             for (int c = 0; c < 4; ++c) dst[c] = pk[c];
-                        } else {
-                            #pragma unroll
-                            for (int c = 0; c < 16; ++c) {
-                                const __half2 h2 = __floats2half2_rn(o[2 * c] * inv, o[2 * c + 1] * inv);
-                                w[c] = *reinterpret_cast<const uint32_t*>(&h2);
-                            }
-                            uint4* dst = reinterpret_cast<uint4*>(args.o_part + prow * kD + ch * 32);
-                            #pragma unroll
-                            for (int c = 0; c < 4; ++c) dst[c] = pk[c];
                         }
+                    } else {
+                        #pragma unroll
+                        for (int c = 0; c < 16; ++c) {
+                            const __half2 h2 = __floats2half2_rn(o[2 * c] * inv, o[2 * c + 1] * inv);
+                            w[c] = *reinterpret_cast<const uint32_t*>(&h2);
+                        }
+                        #pragma unroll
+                        for (int c = 0; c < 4; ++c)
+                            *reinterpret_cast<uint4*>(stage + row_local * 256 + (((ch * 4 + c) ^ (row_local & 15)) << 4)) = pk[c];
                     }
                 }
+                if (tid == 0) SPARROW_TL(6);
                 if (row_ok) {
                     if (direct) args.lse[((size_t)it.b * args.n_q_heads + h_row) * T + t_row] = lse_val;
-                    else args.lse_part[prow] = lse_val;
+                    else args.lse_part[prow0 + row_local] = lse_val;
+                }
+                if (tid == 0) SPARROW_TL(7);
+                if (!direct) {
+                    // each warp wrote its own 32 rows; read them back two rows per instruction so a warp
+                    // store covers 512 contiguous bytes of the partial buffer
+                    __syncwarp();
+                    const int rows_here = min(128, min(plan.rows_per_group - blk * 128, M - (it.group * plan.rows_per_group + blk * 128)));
+                    #pragma unroll 4
+                    for (int i = 0; i < 16; ++i) {
+                        const int r = (warp & 3) * 32 + 2 * i + (lane >> 4), c = lane & 15;
+                        if (r < rows_here) {
+                            const uint4 val = *reinterpret_cast<const uint4*>(stage + r * 256 + ((c ^ (r & 15)) << 4));
+                            *reinterpret_cast<uint4*>(args.o_part + (prow0 + r) * kD + c * 8) = val;
+                        }
+                    }
                 }
                 if (tid == 0) SPARROW_TL(4);
             } else {
