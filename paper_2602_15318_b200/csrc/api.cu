@@ -91,7 +91,7 @@ sparrow_status make_plan(int n_sm, int batch, int n_kv_heads, const int32_t* n_k
     p->rows_per_group = rows_per_group;
     p->n_groups = (p->M + p->rows_per_group - 1) / p->rows_per_group;
     p->n_kv_heads = n_kv_heads;
-    p->part_rows = p->rows_per_group;
+    p->part_rows = p->rows_per_group + 1;    // odd pitch: partial rows of successive pieces must not share L2 sets
     const int units = n_kv_heads * p->n_groups;
     int max_keys = 1;
     for (int b = 0; b < batch; ++b) {
@@ -151,7 +151,7 @@ sparrow_status launch_combine(sparrow_ctx* c, const SplitPlan& plan, void* out, 
     const int rows = plan.batch * plan.n_kv_heads * plan.M;
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof cfg);
-    cfg.gridDim = dim3(rows);
+    cfg.gridDim = dim3((rows + combine::kWarps - 1) / combine::kWarps);
     cfg.blockDim = dim3(combine::kWarps * 32);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -365,7 +365,7 @@ size_t sparrow_workspace_bytes(const sparrow_ctx* c, int32_t max_T)
     size_t worst = 0;
     for (int rpg : {gather::kRows, rows_per_group_tc(M)}) {
         const int groups = (M + rpg - 1) / rpg;
-        const size_t rows = (size_t)max_items(c->n_sm, c->layout.batch, c->layout.n_kv_heads, groups) * rpg;
+        const size_t rows = (size_t)max_items(c->n_sm, c->layout.batch, c->layout.n_kv_heads, groups) * (rpg + 1);
         const size_t need = align_up(rows, 64) * sizeof(float) + rows * kD * sizeof(__half);
         if (need > worst) worst = need;
     }

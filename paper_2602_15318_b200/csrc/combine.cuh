@@ -1,11 +1,16 @@
 // Split-combine step: merges the per-piece partial outputs of the split-KV pass by log-sum-exp,
 //     lse = log sum_s exp(lse_s),   out = sum_s exp(lse_s - lse) * o_s,
-// (partials are fp16, normalised, so their magnitude is bounded by max |v|) and writes bf16 out [B][T][Hq][128] and fp32 lse [B][Hq][T].  Pieces that saw no visible key
-// carry lse_s = -inf and weigh zero; a row with no visible key anywhere gets out = 0, lse = -inf.
+// (partials are fp16, normalised, so their magnitude is bounded by max |v|) and writes bf16 out
+// [B][T][Hq][128] and fp32 lse [B][Hq][T].  Pieces that saw no visible key carry lse_s = -inf and
+// weigh zero; a row with no visible key anywhere gets out = 0, lse = -inf.
 //
-// One CTA of 4 warps per packed query row.  The piece LSEs go to shared memory with one read per
-// thread; warp w then accumulates pieces w, w+4, ... (each lane owns 4 of the 128 output dims, all
-// its loads issued before the first use), and the four warp sums are added through shared memory.
+// One warp per packed query row, registers and shuffles only: the kernel uses no shared memory, so
+// its CTAs can become resident next to the split-KV CTAs (which fill the SM's shared memory) and
+// sit in griddepcontrol.wait until the partials are complete.  Lane l keeps the LSEs of pieces
+// l, l+32, ...  The four quarter-warps take pieces q, q+4, q+8, ...; inside a quarter each of the 8
+// lanes owns 16 of the 128 output dims (two 16-byte loads per piece), and the quarters' sums meet
+// through two shuffle steps.  The code is kept small on purpose: every warp runs it exactly once,
+// so instruction fetch, not arithmetic, is what a long unrolled body would pay for.
 #pragma once
 #include <cuda_fp16.h>
 
@@ -24,16 +29,32 @@ struct CombineArgs {
 
 namespace combine {
 
-constexpr int kWarps = 4;
-constexpr int kMaxPieces = 1024;       // upper bound on pieces per row held in shared memory
+constexpr int kWarps = 4;             // rows per CTA
+constexpr int kPerLane = 8;           // pieces per lane held in registers (256 pieces per row)
+constexpr int kIter = 5;              // pieces per quarter-warp fetched in one go (20 per warp pass)
+
+__device__ __forceinline__ void fma8(float (&acc)[16], int base, float w, const uint4& v)
+{
+    const __half2* h = reinterpret_cast<const __half2*>(&v);
+    #pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float2 f = __half22float2(h[i]);
+        acc[base + 2 * i] = fmaf(w, f.x, acc[base + 2 * i]);
+        acc[base + 2 * i + 1] = fmaf(w, f.y, acc[base + 2 * i + 1]);
+    }
+}
 
 __global__ void __launch_bounds__(kWarps * 32)
 combine_kernel(const __grid_constant__ SplitPlan plan, const __grid_constant__ CombineArgs args)
 {
-    __shared__ float lse_s[kMaxPieces];
-    __shared__ float4 acc_s[kWarps][32];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int row_id = blockIdx.x;
+    const int rows_total = plan.batch * plan.n_kv_heads * plan.M;
+    const int row_id = blockIdx.x * kWarps + warp;
+    if (args.use_pdl) {
+        asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
+        asm volatile("griddepcontrol.wait;\n" ::: "memory");
+    }
+    if (row_id >= rows_total) return;
     const int R = row_id % plan.M;                    // packed row: t*7 + g
     const int unit_bh = row_id / plan.M;
     const int kvh = unit_bh % plan.n_kv_heads;
@@ -41,68 +62,92 @@ combine_kernel(const __grid_constant__ SplitPlan plan, const __grid_constant__ C
     const int group = R / plan.rows_per_group;
     const int lr = R % plan.rows_per_group;
     const int ns = plan.n_splits[b];
-    const int item0 = plan.item_begin[b] + (kvh * plan.n_groups + group) * ns;
-    if (args.use_pdl) {
-        asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
-        asm volatile("griddepcontrol.wait;\n" ::: "memory");
-    }
     if (ns == 1) return;                              // the split pass wrote this row's result itself
-    for (int s = threadIdx.x; s < ns; s += kWarps * 32)
-        lse_s[s] = args.lse_part[(size_t)(item0 + s) * plan.part_rows + lr];
-    __syncthreads();
+    const int item0 = plan.item_begin[b] + (kvh * plan.n_groups + group) * ns;
+    const float* lse_row = args.lse_part + (size_t)item0 * plan.part_rows + lr;      // piece s at s * part_rows
+    const int quarter = lane >> 3, sub = lane & 7;
+    const __half* o_row = args.o_part + ((size_t)item0 * plan.part_rows + lr) * kD + sub * 16;
+    const size_t o_pitch = (size_t)plan.part_rows * kD;
+
+    // first pass of partial loads goes out together with the LSE loads (they are independent)
+    uint4 o0[kIter], o1[kIter];
+    #pragma unroll
+    for (int i = 0; i < kIter; ++i) {
+        const int s = 4 * i + quarter;
+        if (s < ns) {
+            const uint4* src = reinterpret_cast<const uint4*>(o_row + (size_t)s * o_pitch);
+            o0[i] = __ldcg(src); o1[i] = __ldcg(src + 1);
+        }
+    }
+    float lv[kPerLane];
+    #pragma unroll
+    for (int i = 0; i < kPerLane; ++i) {
+        const int s = lane + 32 * i;
+        lv[i] = s < ns ? __ldcg(lse_row + (size_t)s * plan.part_rows) : -INFINITY;
+    }
     float mx = -INFINITY;
-    for (int s = lane; s < ns; s += 32) mx = fmaxf(mx, lse_s[s]);
+    #pragma unroll
+    for (int i = 0; i < kPerLane; ++i) mx = fmaxf(mx, lv[i]);
+    for (int s = lane + 32 * kPerLane; s < ns; s += 32) mx = fmaxf(mx, __ldcg(lse_row + (size_t)s * plan.part_rows));
     #pragma unroll
     for (int d = 16; d > 0; d >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, d));
+    const bool any = mx != -INFINITY;
     float sum = 0.f;
-    if (mx != -INFINITY)
-        for (int s = lane; s < ns; s += 32) sum += expf(lse_s[s] - mx);
+    #pragma unroll
+    for (int i = 0; i < kPerLane; ++i) sum += any ? __expf(lv[i] - mx) : 0.f;        // 0 for absent pieces
+    for (int s = lane + 32 * kPerLane; s < ns; s += 32) sum += any ? __expf(__ldcg(lse_row + (size_t)s * plan.part_rows) - mx) : 0.f;
     #pragma unroll
     for (int d = 16; d > 0; d >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, d);
-    const float total = (mx == -INFINITY) ? -INFINITY : mx + logf(sum);
+    const float total = any ? mx + logf(sum) : -INFINITY;
+    #pragma unroll
+    for (int i = 0; i < kPerLane; ++i) lv[i] = any ? __expf(lv[i] - total) : 0.f;     // now the weights
 
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (mx != -INFINITY) {
-        constexpr int kBatch = 8;
-        for (int s0 = warp; s0 < ns; s0 += kWarps * kBatch) {
-            uint2 o[kBatch];                                   // 4 halves per lane and piece
+    float acc[16];
+    #pragma unroll
+    for (int i = 0; i < 16; ++i) acc[i] = 0.f;
+    #pragma unroll 1
+    for (int s0 = 0; s0 < ns; s0 += 4 * kIter) {                 // warp-uniform trip count
+        if (s0 > 0) {
             #pragma unroll
-            for (int u = 0; u < kBatch; ++u) {
-                const int s = s0 + u * kWarps;
-                if (s < ns)
-                    o[u] = __ldcg(reinterpret_cast<const uint2*>(
-                        args.o_part + ((size_t)(item0 + s) * plan.part_rows + lr) * kD + lane * 4));
-            }
-            #pragma unroll
-            for (int u = 0; u < kBatch; ++u) {
-                const int s = s0 + u * kWarps;
+            for (int i = 0; i < kIter; ++i) {
+                const int s = s0 + 4 * i + quarter;
                 if (s < ns) {
-                    const float w = expf(lse_s[s] - total);
-                    const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&o[u].x));
-                    const float2 c = __half22float2(*reinterpret_cast<const __half2*>(&o[u].y));
-                    acc.x = fmaf(w, a.x, acc.x); acc.y = fmaf(w, a.y, acc.y);
-                    acc.z = fmaf(w, c.x, acc.z); acc.w = fmaf(w, c.y, acc.w);
+                    const uint4* src = reinterpret_cast<const uint4*>(o_row + (size_t)s * o_pitch);
+                    o0[i] = __ldcg(src); o1[i] = __ldcg(src + 1);
                 }
             }
         }
-    }
-    acc_s[warp][lane] = acc;
-    __syncthreads();
-    if (warp == 0) {
         #pragma unroll
-        for (int w = 1; w < kWarps; ++w) {
-            const float4 o = acc_s[w][lane];
-            acc.x += o.x; acc.y += o.y; acc.z += o.z; acc.w += o.w;
+        for (int i = 0; i < kIter; ++i) {
+            const int s = s0 + 4 * i + quarter;
+            // weight of piece s lives in lane s & 31, register s >> 5 (the same register for all quarters)
+            const int reg = (s0 + 4 * i) >> 5;
+            float mine = 0.f;
+            #pragma unroll
+            for (int k = 0; k < kPerLane; ++k) if (reg == k) mine = lv[k];
+            float w = __shfl_sync(0xffffffffu, mine, s & 31);
+            if (reg >= kPerLane && s < ns) w = any ? __expf(__ldcg(lse_row + (size_t)s * plan.part_rows) - total) : 0.f;
+            if (s < ns) { fma8(acc, 0, w, o0[i]); fma8(acc, 8, w, o1[i]); }
         }
+    }
+    #pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        acc[i] += __shfl_xor_sync(0xffffffffu, acc[i], 8);
+        acc[i] += __shfl_xor_sync(0xffffffffu, acc[i], 16);
+    }
+    if (quarter == 0) {
         const int t = R / kGroup, g = R % kGroup;
         const int h = kvh * kGroup + g;
-        __nv_bfloat16* dst = args.out + (((size_t)b * plan.T + t) * args.n_q_heads + h) * kD + lane * 4;
-        __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y);
-        __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z, acc.w);
-        uint2 packed;
-        packed.x = *reinterpret_cast<uint32_t*>(&lo);
-        packed.y = *reinterpret_cast<uint32_t*>(&hi);
-        *reinterpret_cast<uint2*>(dst) = packed;
+        __nv_bfloat16* dst = args.out + (((size_t)b * plan.T + t) * args.n_q_heads + h) * kD + sub * 16;
+        uint4 pk[2];
+        uint32_t* w32 = reinterpret_cast<uint32_t*>(pk);
+        #pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            __nv_bfloat162 v = __floats2bfloat162_rn(acc[2 * i], acc[2 * i + 1]);
+            w32[i] = *reinterpret_cast<uint32_t*>(&v);
+        }
+        reinterpret_cast<uint4*>(dst)[0] = pk[0];
+        reinterpret_cast<uint4*>(dst)[1] = pk[1];
         if (lane == 0) args.lse[((size_t)b * args.n_q_heads + h) * plan.T + t] = total;
     }
 }

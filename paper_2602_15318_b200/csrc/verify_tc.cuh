@@ -313,16 +313,19 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
             if (lane < T) par0 = __ldg(par_g + lane);
             if (lane + 32 < T) par1 = __ldg(par_g + lane + 32);
         }
-        #pragma unroll
-        for (int u = 0; u < kChunksPerThread; ++u) {
-            const int i = tid + u * NB * 128;
-            const int r = i >> 4, c = i & 15;                       // row in the item, 16-byte chunk
-            const int R = it.group * plan.rows_per_group + r;
-            qv[u] = make_uint4(0, 0, 0, 0);
-            if (R < M && r < plan.rows_per_group) {
-                const int t = R / kGroup, g = R % kGroup;
-                qv[u] = __ldg(reinterpret_cast<const uint4*>(
-                    args.q + (((size_t)it.b * T + t) * args.n_q_heads + it.kvh * kGroup + g) * kD + c * 8));
+        {
+            // thread tid owns 16-byte chunk (tid & 15) of rows (tid >> 4) + u * 8 * NB, u = 0..15
+            const int c = tid & 15;
+            const __nv_bfloat16* qbase = args.q + ((size_t)it.b * T * args.n_q_heads + it.kvh * kGroup) * kD + c * 8;
+            #pragma unroll
+            for (int u = 0; u < kChunksPerThread; ++u) {
+                const int r = (tid >> 4) + u * 8 * NB;
+                const int R = it.group * plan.rows_per_group + r;
+                qv[u] = make_uint4(0, 0, 0, 0);
+                if (R < M && r < plan.rows_per_group) {
+                    const int t = R / kGroup, g = R - t * kGroup;
+                    qv[u] = __ldg(reinterpret_cast<const uint4*>(qbase + ((size_t)t * args.n_q_heads + g) * kD));
+                }
             }
         }
     }
@@ -358,6 +361,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
             // refill whichever ring has a free slot; K slots free up about one tile before V slots
             int jk = NS < n_tiles ? NS : n_tiles, jv = jk;
             uint32_t idle = 0;
+            #pragma unroll 1
             while (jk < n_tiles || jv < n_tiles) {
                 bool progress = false;
                 if (jk < n_tiles && mbar_try_wait(B.k_empty(jk % NS), (jk / NS - 1) & 1)) { issue_k(jk); ++jk; progress = true; }
@@ -373,39 +377,44 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
             constexpr uint32_t idesc_qk = idesc_bf16(false);
             constexpr uint32_t idesc_pv = idesc_bf16(true);
             bool ok = true;
-            auto issue_qk = [&](int n) {
-                const int j = n / NB, blk = n % NB, slot = n & 1, st = j % NS;
-                if (blk == 0) {                                       // first use of this K tile
-                    if (!mbar_wait(B.k_full(st), (j / NS) & 1)) { ok = false; return; }
-                    tc_fence_after();
-                    SPARROW_TL(100 + 4 * n);
-                    if (j == 0) { SPARROW_TLG(1); }
-                    if (j == n_tiles - 1) { SPARROW_TLG(2); }
+            // descriptors differ from tile to tile only in their 14-bit address field
+            const uint64_t q_desc0 = smem_desc(smem_u32(q_sm), 16, 1024);
+            const uint64_t k_desc0 = smem_desc(smem_u32(kv_sm), 16, 1024);
+            const uint64_t v_desc0 = smem_desc(smem_u32(kv_sm) + 2 * kSubTileBytes, kSubTileBytes, 1024);
+            #pragma unroll 1
+            for (int n = -1; n < n_jobs && ok; ++n) {
+                if (n + 1 < n_jobs) {                                     // S = Q K^T of the next job
+                    const int m = n + 1;
+                    const int j = m / NB, blk = m % NB, slot = m & 1, st = j % NS;
+                    if (blk == 0) {                                       // first use of this K tile
+                        if (!mbar_wait(B.k_full(st), (j / NS) & 1)) { ok = false; break; }
+                        tc_fence_after();
+                        SPARROW_TL(100 + 4 * m);
+                        if (j == 0) { SPARROW_TLG(1); }
+                        if (j == n_tiles - 1) { SPARROW_TLG(2); }
+                    }
+                    const uint64_t qd = q_desc0 + (uint64_t)((blk * kQBlockBytes) >> 4);
+                    const uint64_t kd = k_desc0 + (uint64_t)((st * kStageBytes) >> 4);
+                    #pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint32_t off = ((ks >> 2) * kSubTileBytes + (ks & 3) * 32) >> 4;
+                        mma_ss(tmem + slot * 128, qd + off, kd + off, idesc_qk, ks > 0);
+                    }
+                    tc_commit(B.s_full(slot));
+                    if (blk == NB - 1) tc_commit(B.k_empty(st));
+                    SPARROW_TL(101 + 4 * m);
                 }
-                const uint32_t qa = smem_u32(q_sm + blk * kQBlockBytes);
-                const uint32_t ka = smem_u32(kv_sm + st * kStageBytes);
-                #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint32_t off = (ks >> 2) * kSubTileBytes + (ks & 3) * 32;
-                    mma_ss(tmem + slot * 128, smem_desc(qa + off, 16, 1024), smem_desc(ka + off, 16, 1024), idesc_qk, ks > 0);
-                }
-                tc_commit(B.s_full(slot));
-                if (blk == NB - 1) tc_commit(B.k_empty(st));
-                SPARROW_TL(101 + 4 * n);
-            };
-            if (n_jobs > 0) issue_qk(0);
-            for (int n = 0; n < n_jobs && ok; ++n) {
-                if (n + 1 < n_jobs) { issue_qk(n + 1); if (!ok) break; }
+                if (n < 0) continue;
                 const int j = n / NB, blk = n % NB, slot = n & 1, st = j % NS;
                 if (blk == 0 && !mbar_wait(B.v_full(st), (j / NS) & 1)) { ok = false; break; }
                 if (!mbar_wait(B.p_full(slot), (n >> 1) & 1)) { ok = false; break; }
                 tc_fence_after();
                 SPARROW_TL(102 + 4 * n);
-                const uint32_t va = smem_u32(kv_sm + st * kStageBytes + 2 * kSubTileBytes);
+                const uint64_t vd = v_desc0 + (uint64_t)((st * kStageBytes) >> 4);
                 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk)
-                    mma_ts(tmem + 256 + blk * 128, tmem + slot * 128 + kk * 8,
-                           smem_desc(va + kk * 2048, kSubTileBytes, 1024), idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);
+                    mma_ts(tmem + 256 + blk * 128, tmem + slot * 128 + kk * 8, vd + (uint64_t)((kk * 2048) >> 4),
+                           idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);
                 tc_commit(B.o_done(blk));
                 if (blk == NB - 1) tc_commit(B.v_empty(st));
                 SPARROW_TL(103 + 4 * n);
@@ -428,6 +437,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
         float m_ref = -INFINITY, l_run = 0.f;
         bool ok = true;
 
+        #pragma unroll 1
         for (int n = (NB == 2 ? wg : 0); n < n_jobs; n += NB) {
             const int j = n / NB, slot = n & 1, st = j % NS;
             if (!mbar_wait_warp(B.s_full(slot), (n >> 1) & 1)) { ok = false; break; }
@@ -496,7 +506,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
                     if (!mbar_wait_warp(B.o_done(NB == 2 ? wg : 0), (i_blk - 1) & 1)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t o_addr = lane_addr + 256 + (NB == 2 ? wg : 0) * 128;
-                    #pragma unroll
+                    #pragma unroll 1
                     for (int ch = 0; ch < 4; ++ch) {
                         float o[32];
                         tmem_ld32(o_addr + ch * 32, o);
@@ -546,7 +556,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
                 // Staging area: this row block's Q tile (every MMA that read it has completed).  Row r
                 // holds 16 chunks of 16 bytes (128 halves), chunk c stored at position c ^ (r & 15).
                 unsigned char* stage = q_sm + blk * kQBlockBytes;
-                #pragma unroll
+                #pragma unroll 1
                 for (int ch = 0; ch < 4; ++ch) {
                     float o[32];
                     tmem_ld32(o_addr + ch * 32, o);
@@ -608,6 +618,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
     __syncthreads();
     if (*abort_flag) {
         // give copies that are still in flight time to land before the CTA's memory is released
+        #pragma unroll 1
         for (int i = 0; i < 2000; ++i) __nanosleep(1000);
         __syncthreads();
     }
