@@ -62,7 +62,8 @@ def test_split_plan_properties():
     for n_keys, T in cases:
         for n_sm in (148, 132, 16):
             splits, n_items = B.sparrow_plan_splits(n_sm, 4, n_keys, T)
-            groups = -(-7 * T // 128)
+            M = 7 * T
+            groups = -(-M // (128 if M <= 128 else 256))    # row groups of one or two 128-row blocks
             assert n_items == sum(4 * groups * s for s in splits)
             assert all(1 <= s <= n for s, n in zip(splits, n_keys))
             units = 4 * groups * len(n_keys)
