@@ -174,10 +174,6 @@ sparrow_status sparrow_plan_splits(int32_t n_sm, int32_t batch, int32_t n_kv_hea
                                    const int32_t* n_keys, int32_t T, int32_t* splits_out,
                                    int32_t* n_items_out);
 
-/* Profiling aid: selects which of the two kernels of a call are launched (both by default), so
- * the split-KV pass can be timed on its own.  With run_combine == 0 out / lse are not written. */
-sparrow_status sparrow_debug_set_stages(sparrow_ctx* ctx, int32_t run_split, int32_t run_combine);
-
 /* Synchronises `stream`, returns the sticky device status (SPARROW_OK, SPARROW_ERR_TREE,
  * SPARROW_ERR_ANCHOR or SPARROW_ERR_TIMEOUT) and clears it.  Not for the hot path. */
 sparrow_status sparrow_last_device_status(sparrow_ctx* ctx, void* stream);

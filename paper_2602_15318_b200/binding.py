@@ -21,7 +21,7 @@ STATUS_NAMES = {0: "SPARROW_OK", 1: "SPARROW_ERR_NULL", 2: "SPARROW_ERR_SHAPE", 
 
 EXPORTS = ["sparrow_create", "sparrow_destroy", "sparrow_workspace_bytes", "sparrow_set_workspace",
            "sparrow_verify_attn", "sparrow_verify_attn_batch", "sparrow_anchor_attn",
-           "sparrow_verify_step_host", "sparrow_debug_set_stages",
+           "sparrow_verify_step_host",
            "sparrow_build_ancestor_masks", "sparrow_build_anchor_idx",
            "sparrow_debug_ancestor_masks_device", "sparrow_plan_splits",
            "sparrow_last_device_status", "sparrow_launch_count", "sparrow_status_string"]
@@ -59,7 +59,6 @@ def lib():
         L.sparrow_set_workspace.argtypes = [vp, vp, ctypes.c_size_t]
         L.sparrow_verify_attn.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp, vp, vp]
         L.sparrow_verify_attn_batch.argtypes = [vp, vp, i32, vp]
-        L.sparrow_debug_set_stages.argtypes = [vp, i32, i32]
         L.sparrow_anchor_attn.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp]
         L.sparrow_verify_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp]
         L.sparrow_build_ancestor_masks.argtypes = [vp, i32, vp]
@@ -186,11 +185,6 @@ def sparrow_verify_attn_batch(ctx: Context, batch: VerifyBatch, n_calls: Optiona
     n = batch.n if n_calls is None else n_calls
     _chk(lib().sparrow_verify_attn_batch(ctx.handle, batch.array, n, _stream_handle(stream)),
          "sparrow_verify_attn_batch")
-
-
-def sparrow_debug_set_stages(ctx: Context, run_split: bool, run_combine: bool):
-    _chk(lib().sparrow_debug_set_stages(ctx.handle, int(run_split), int(run_combine)),
-         "sparrow_debug_set_stages")
 
 
 def sparrow_anchor_attn(ctx: Context, q, k, v, anchor_idx, n_anchor: int, window: int, T: int, out, lse,

@@ -27,12 +27,13 @@ typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint3
 
 struct TensorMapEntry {
     const void* base;
+    int tag;                 // 0: K/V cache map; n > 0: Q map for n = batch * T tokens
     CUtensorMap map;
 };
 constexpr int kMapCacheSize = 128;
 
 struct sparrow_ctx {
-    TensorMapEntry maps[kMapCacheSize];      // K/V tensor maps, keyed by base pointer
+    TensorMapEntry maps[kMapCacheSize];      // Q / K / V tensor maps, keyed by base pointer (and token count)
     int n_maps;
     int next_evict;
     TensorMapEncodeFn encode;
@@ -44,8 +45,6 @@ struct sparrow_ctx {
     size_t ws_bytes;
     std::atomic<long long> launches;
     bool use_pdl;
-    bool run_split;
-    bool run_combine;
 };
 
 namespace {
@@ -71,7 +70,8 @@ Staging staging_layout(const sparrow_layout& L)
     return s;
 }
 
-int rows_per_group_tc(int M) { return M <= 128 ? 128 : 256; }
+// 128-row blocks (18 draft tokens each) one work item of the tensor-core pass handles
+int blocks_per_group_tc(int T) { return T <= kTokPerBlock ? 1 : 2; }
 
 int max_items(int n_sm, int batch, int n_kv_heads, int n_groups)
 {
@@ -80,7 +80,7 @@ int max_items(int n_sm, int batch, int n_kv_heads, int n_groups)
 
 // Chooses the number of key-range pieces per sequence so that the total number of work items is
 // close to (and not above) the SM count while every item streams about the same number of keys.
-sparrow_status make_plan(int n_sm, int batch, int n_kv_heads, const int32_t* n_keys, int T, int rows_per_group,
+sparrow_status make_plan(int n_sm, int batch, int n_kv_heads, const int32_t* n_keys, int T, int blocks_per_group,
                          SplitPlan* p)
 {
     if (batch < 1 || batch > kMaxBatch || T < 1 || T > kMaxT || n_kv_heads < 1 || n_sm < 1) return SPARROW_ERR_SHAPE;
@@ -88,10 +88,10 @@ sparrow_status make_plan(int n_sm, int batch, int n_kv_heads, const int32_t* n_k
     p->batch = batch;
     p->T = T;
     p->M = kGroup * T;
-    p->rows_per_group = rows_per_group;
-    p->n_groups = (p->M + p->rows_per_group - 1) / p->rows_per_group;
+    p->blocks_per_group = blocks_per_group;
+    p->n_groups = (T + kTokPerBlock * blocks_per_group - 1) / (kTokPerBlock * blocks_per_group);
     p->n_kv_heads = n_kv_heads;
-    p->part_rows = p->rows_per_group + 1;    // odd pitch: partial rows of successive pieces must not share L2 sets
+    p->part_rows = blocks_per_group * kBlockRows + 1;    // odd pitch: partial rows of successive pieces must not share L2 sets
     const int units = n_kv_heads * p->n_groups;
     int max_keys = 1;
     for (int b = 0; b < batch; ++b) {
@@ -192,42 +192,56 @@ sparrow_status launch_split_gather(sparrow_ctx* c, const SplitPlan& plan, const 
     return SPARROW_OK;
 }
 
-// Tensor map over one K or V buffer: dims (128 dims, capacity rows, KV heads, batch), boxes of
-// 64 dims x 128 rows, 128-byte swizzle; rows past the capacity read as zero.
-const CUtensorMap* tensor_map_for(sparrow_ctx* c, const void* base)
+// Cached tensor maps.  tag == 0: one K or V buffer, dims (128 dims, capacity rows, KV heads,
+// batch), boxes of 64 dims x 128 rows; rows past the capacity read as zero.  tag == n_tok > 0: the
+// query tensor [n_tok][KV heads][7][128], boxes of 64 dims x 7 heads x 18 tokens, which land in
+// shared memory as the rows (t * 7 + g) of a K-major operand block; tokens past n_tok read as zero.
+// Both use the 128-byte swizzle.
+const CUtensorMap* tensor_map_for(sparrow_ctx* c, const void* base, int tag)
 {
     for (int i = 0; i < c->n_maps; ++i)
-        if (c->maps[i].base == base) return &c->maps[i].map;
+        if (c->maps[i].base == base && c->maps[i].tag == tag) return &c->maps[i].map;
     if (!c->encode) return nullptr;
     const sparrow_layout& L = c->layout;
     int slot;
     if (c->n_maps < kMapCacheSize) slot = c->n_maps++;
     else { slot = c->next_evict; c->next_evict = (c->next_evict + 1) % kMapCacheSize; }
-    const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)L.kv_capacity, (cuuint64_t)L.n_kv_heads, (cuuint64_t)L.batch};
-    const cuuint64_t batch_stride = L.batch > 1 ? (cuuint64_t)L.kv_stride_batch : (cuuint64_t)L.kv_stride_head * L.n_kv_heads;
-    const cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)L.kv_stride_head * 2, batch_stride * 2};
-    const cuuint32_t box[4] = {64, 128, 1, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
-    const CUresult r = c->encode(&c->maps[slot].map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims,
-                                 strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r;
+    if (tag == 0) {
+        const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)L.kv_capacity, (cuuint64_t)L.n_kv_heads, (cuuint64_t)L.batch};
+        const cuuint64_t batch_stride = L.batch > 1 ? (cuuint64_t)L.kv_stride_batch : (cuuint64_t)L.kv_stride_head * L.n_kv_heads;
+        const cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)L.kv_stride_head * 2, batch_stride * 2};
+        const cuuint32_t box[4] = {64, 128, 1, 1};
+        r = c->encode(&c->maps[slot].map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
+                      estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    } else {
+        const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)kGroup, (cuuint64_t)L.n_kv_heads, (cuuint64_t)tag};
+        const cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)kGroup * kD * 2, (cuuint64_t)L.n_q_heads * kD * 2};
+        const cuuint32_t box[4] = {64, (cuuint32_t)kGroup, 1, (cuuint32_t)kTokPerBlock};
+        r = c->encode(&c->maps[slot].map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
+                      estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    }
     if (r != CUDA_SUCCESS) { c->maps[slot].base = nullptr; if (slot == c->n_maps - 1) --c->n_maps; return nullptr; }
     c->maps[slot].base = base;
+    c->maps[slot].tag = tag;
     return &c->maps[slot].map;
 }
 
 sparrow_status launch_verify_tc(sparrow_ctx* c, const SplitPlan& plan, const void* q, const void* k, const void* v,
                                 const int32_t* parents, void* out, float* lse, cudaStream_t st)
 {
-    const CUtensorMap* mk = tensor_map_for(c, k);
-    const CUtensorMap* mv = tensor_map_for(c, v);
-    if (!mk || !mv) return SPARROW_ERR_CUDA;
+    const CUtensorMap* mq = tensor_map_for(c, q, plan.batch * plan.T);
+    const CUtensorMap* mk = tensor_map_for(c, k, 0);
+    const CUtensorMap* mv = tensor_map_for(c, v, 0);
+    if (!mq || !mk || !mv) return SPARROW_ERR_CUDA;
+    const int nb = plan.blocks_per_group;
     TcArgs a;
-    a.q = static_cast<const __nv_bfloat16*>(q);
     a.parents = parents;
     a.n_q_heads = c->layout.n_q_heads;
-    a.n_blocks = plan.rows_per_group / 128;
-    a.n_stages = a.n_blocks == 1 ? 3 : 2;
+    a.n_stages = nb == 1 ? 3 : 2;
     a.use_pdl = c->use_pdl ? 1 : 0;
     a.scale_log2e = c->layout.softmax_scale * 1.4426950408889634f;
     a.o_part = o_part_ptr(c, plan);
@@ -235,20 +249,19 @@ sparrow_status launch_verify_tc(sparrow_ctx* c, const SplitPlan& plan, const voi
     a.out = static_cast<__nv_bfloat16*>(out);
     a.lse = lse;
     a.status = reinterpret_cast<unsigned*>(c->ws);
-    a.tl_all = reinterpret_cast<unsigned long long*>(c->ws + ((c->ws_bytes - 65536) & ~(size_t)255));
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof cfg);
     cfg.gridDim = dim3(plan.n_items);
-    cfg.blockDim = dim3(tc::threads_for(a.n_blocks));
-    cfg.dynamicSmemBytes = tc::smem_bytes(a.n_blocks, a.n_stages);
+    cfg.blockDim = dim3(tc::kThreads);
+    cfg.dynamicSmemBytes = tc::smem_bytes(nb, a.n_stages);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = c->use_pdl ? 1 : 0;
-    const cudaError_t e = a.n_blocks == 1 ? cudaLaunchKernelEx(&cfg, tc::verify_tc_kernel<1>, *mk, *mv, plan, a)
-                                          : cudaLaunchKernelEx(&cfg, tc::verify_tc_kernel<2>, *mk, *mv, plan, a);
+    const cudaError_t e = nb == 1 ? cudaLaunchKernelEx(&cfg, tc::verify_tc_kernel<1>, *mq, *mk, *mv, plan, a)
+                                  : cudaLaunchKernelEx(&cfg, tc::verify_tc_kernel<2>, *mq, *mk, *mv, plan, a);
     if (e != cudaSuccess) return SPARROW_ERR_CUDA;
     c->launches.fetch_add(1);
     return SPARROW_OK;
@@ -346,7 +359,6 @@ sparrow_status sparrow_create(sparrow_ctx** out, const sparrow_layout* L, int de
     c->launches.store(0);
     const char* e = std::getenv("SPARROW_NO_PDL");
     c->use_pdl = !(e && e[0] == '1');
-    c->run_split = c->run_combine = true;
     *out = c;
     return SPARROW_OK;
 }
@@ -361,11 +373,10 @@ sparrow_status sparrow_destroy(sparrow_ctx* c)
 size_t sparrow_workspace_bytes(const sparrow_ctx* c, int32_t max_T)
 {
     if (!c || max_T < 1 || max_T > kMaxT) return 0;
-    const int M = kGroup * max_T;
     size_t worst = 0;
-    for (int rpg : {gather::kRows, rows_per_group_tc(M)}) {
-        const int groups = (M + rpg - 1) / rpg;
-        const size_t rows = (size_t)max_items(c->n_sm, c->layout.batch, c->layout.n_kv_heads, groups) * (rpg + 1);
+    for (int nb : {1, blocks_per_group_tc(max_T)}) {         // the gathered pass uses single blocks
+        const int groups = (max_T + kTokPerBlock * nb - 1) / (kTokPerBlock * nb);
+        const size_t rows = (size_t)max_items(c->n_sm, c->layout.batch, c->layout.n_kv_heads, groups) * (nb * kBlockRows + 1);
         const size_t need = align_up(rows, 64) * sizeof(float) + rows * kD * sizeof(__half);
         if (need > worst) worst = need;
     }
@@ -391,7 +402,7 @@ sparrow_status sparrow_plan_splits(int32_t n_sm, int32_t batch, int32_t n_kv_hea
     if (!n_keys || !splits_out || !n_items_out) return SPARROW_ERR_NULL;
     SplitPlan p;
     if (T < 1 || T > kMaxT) return SPARROW_ERR_SHAPE;
-    const sparrow_status s = make_plan(n_sm, batch, n_kv_heads, n_keys, T, rows_per_group_tc(kGroup * T), &p);
+    const sparrow_status s = make_plan(n_sm, batch, n_kv_heads, n_keys, T, blocks_per_group_tc(T), &p);
     if (s != SPARROW_OK) return s;
     for (int b = 0; b < batch; ++b) splits_out[b] = p.n_splits[b];
     *n_items_out = p.n_items;
@@ -411,20 +422,18 @@ sparrow_status sparrow_verify_attn(sparrow_ctx* c, const void* q, const void* k,
         n_keys[b] = kv_len[b] + T;
     }
     SplitPlan plan;
-    const int rpg = c->verify_on_gather ? gather::kRows : rows_per_group_tc(kGroup * T);
-    sparrow_status s = make_plan(c->n_sm, c->layout.batch, c->layout.n_kv_heads, n_keys, T, rpg, &plan);
+    const int nb = c->verify_on_gather ? 1 : blocks_per_group_tc(T);
+    sparrow_status s = make_plan(c->n_sm, c->layout.batch, c->layout.n_kv_heads, n_keys, T, nb, &plan);
     if (s != SPARROW_OK) return s;
     for (int b = 0; b < c->layout.batch; ++b) plan.kv_len[b] = kv_len[b];
     if ((s = check_ws(c, plan)) != SPARROW_OK) return s;
     DeviceGuard guard(c->device);
     if (!guard.ok) return SPARROW_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (c->run_split) {
-        s = c->verify_on_gather ? launch_split_gather(c, plan, q, k, v, parents, nullptr, 0, 0, out, lse, st)
-                                : launch_verify_tc(c, plan, q, k, v, parents, out, lse, st);
-        if (s != SPARROW_OK) return s;
-    }
-    return c->run_combine ? launch_combine(c, plan, out, lse, st) : SPARROW_OK;
+    s = c->verify_on_gather ? launch_split_gather(c, plan, q, k, v, parents, nullptr, 0, 0, out, lse, st)
+                            : launch_verify_tc(c, plan, q, k, v, parents, out, lse, st);
+    if (s != SPARROW_OK) return s;
+    return launch_combine(c, plan, out, lse, st);
 }
 
 sparrow_status sparrow_verify_attn_batch(sparrow_ctx* c, const sparrow_verify_call* calls, int32_t n_calls, void* stream)
@@ -439,14 +448,6 @@ sparrow_status sparrow_verify_attn_batch(sparrow_ctx* c, const sparrow_verify_ca
     return SPARROW_OK;
 }
 
-sparrow_status sparrow_debug_set_stages(sparrow_ctx* c, int32_t run_split, int32_t run_combine)
-{
-    if (!c) return SPARROW_ERR_NULL;
-    c->run_split = run_split != 0;
-    c->run_combine = run_combine != 0;
-    return SPARROW_OK;
-}
-
 sparrow_status sparrow_anchor_attn(sparrow_ctx* c, const void* q, const void* k, const void* v,
                                    const int32_t* anchor_idx, int32_t n_anchor, int32_t window, int32_t T,
                                    void* out, float* lse, void* stream)
@@ -458,14 +459,14 @@ sparrow_status sparrow_anchor_attn(sparrow_ctx* c, const void* q, const void* k,
     int32_t n_keys[kMaxBatch];
     for (int b = 0; b < c->layout.batch; ++b) n_keys[b] = n_anchor;
     SplitPlan plan;
-    sparrow_status s = make_plan(c->n_sm, c->layout.batch, c->layout.n_kv_heads, n_keys, T, gather::kRows, &plan);
+    sparrow_status s = make_plan(c->n_sm, c->layout.batch, c->layout.n_kv_heads, n_keys, T, 1, &plan);
     if (s != SPARROW_OK) return s;
     if ((s = check_ws(c, plan)) != SPARROW_OK) return s;
     DeviceGuard guard(c->device);
     if (!guard.ok) return SPARROW_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (c->run_split && (s = launch_split_gather(c, plan, q, k, v, nullptr, anchor_idx, n_anchor, window, out, lse, st)) != SPARROW_OK) return s;
-    return c->run_combine ? launch_combine(c, plan, out, lse, st) : SPARROW_OK;
+    if ((s = launch_split_gather(c, plan, q, k, v, nullptr, anchor_idx, n_anchor, window, out, lse, st)) != SPARROW_OK) return s;
+    return launch_combine(c, plan, out, lse, st);
 }
 
 sparrow_status sparrow_verify_step_host(sparrow_ctx* c, const void* q_host, const void* k_new_host,

@@ -55,12 +55,14 @@ combine_kernel(const __grid_constant__ SplitPlan plan, const __grid_constant__ C
         asm volatile("griddepcontrol.wait;\n" ::: "memory");
     }
     if (row_id >= rows_total) return;
-    const int R = row_id % plan.M;                    // packed row: t*7 + g
+    const int R = row_id % plan.M;                    // (token, head of the group): t*7 + g
     const int unit_bh = row_id / plan.M;
     const int kvh = unit_bh % plan.n_kv_heads;
     const int b = unit_bh / plan.n_kv_heads;
-    const int group = R / plan.rows_per_group;
-    const int lr = R % plan.rows_per_group;
+    const int t = R / kGroup, g = R - t * kGroup;
+    const int block = t / kTokPerBlock;               // 128-row block holding this token
+    const int group = block / plan.blocks_per_group;
+    const int lr = (block - group * plan.blocks_per_group) * kBlockRows + (t - block * kTokPerBlock) * kGroup + g;
     const int ns = plan.n_splits[b];
     if (ns == 1) return;                              // the split pass wrote this row's result itself
     const int item0 = plan.item_begin[b] + (kvh * plan.n_groups + group) * ns;
@@ -136,7 +138,6 @@ combine_kernel(const __grid_constant__ SplitPlan plan, const __grid_constant__ C
         acc[i] += __shfl_xor_sync(0xffffffffu, acc[i], 16);
     }
     if (quarter == 0) {
-        const int t = R / kGroup, g = R % kGroup;
         const int h = kvh * kGroup + g;
         __nv_bfloat16* dst = args.out + (((size_t)b * plan.T + t) * args.n_q_heads + h) * kD + sub * 16;
         uint4 pk[2];

@@ -11,12 +11,18 @@ constexpr int kD = 128;           // head_dim
 constexpr int kGroup = 7;         // query heads per KV head
 constexpr int kMaxT = 64;
 constexpr int kMaxBatch = 64;
+constexpr int kTokPerBlock = 18;  // draft tokens per 128-row block: 18 x 7 = 126 rows, 2 rows of padding
+constexpr int kBlockRows = 128;
 
 // device status bits (sticky, OR-ed into the first word of the workspace)
 constexpr unsigned kStatTree = 1u;
 constexpr unsigned kStatAnchor = 2u;
 constexpr unsigned kStatTimeout = 4u;
 
+// The GQA group's 7 query heads x T draft tokens are packed into 128-row blocks: block i holds
+// tokens [18 i, 18 i + 18), row r of a block is (token 18 i + r / 7, head r % 7), rows 126 and 127
+// are padding.  A row group is 1 or 2 consecutive blocks, handled by one work item.
+//
 // One work item = (sequence b, KV head, row group, key-range piece).  Items of sequence b occupy
 // [item_begin[b], item_begin[b+1]); inside, the index runs (kv head, row group, piece) with the
 // piece fastest.  Piece s of n covers keys [n_keys*s/n, n_keys*(s+1)/n).
@@ -24,9 +30,9 @@ struct SplitPlan {
     int32_t n_items;
     int32_t batch;
     int32_t T;                    // draft tokens
-    int32_t M;                    // packed query rows per KV head = 7*T, row r = t*7 + g
-    int32_t rows_per_group;       // rows one work item handles (a multiple of 16)
-    int32_t n_groups;             // ceil(M / rows_per_group)
+    int32_t M;                    // query rows per KV head = 7*T
+    int32_t blocks_per_group;     // 128-row blocks one work item handles (1 or 2)
+    int32_t n_groups;             // ceil(T / (18 * blocks_per_group))
     int32_t n_kv_heads;
     int32_t part_rows;            // row pitch of one item's partial block in the workspace
     int32_t item_begin[kMaxBatch + 1];

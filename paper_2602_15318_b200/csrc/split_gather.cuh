@@ -1,9 +1,10 @@
 // Split-KV pass with row-gathered K/V loads: the kernel behind the text-anchored window mode
 // (Eq. 2: keys/values restricted to the anchor list) and a general path for any key layout.
 //
-// One CTA = one work item (sequence, KV head, group of up to 128 packed query rows, key-range
-// piece).  The 7 query heads of the GQA group times the T draft tokens form one packed block
-// (row r = t*7 + g), so every gathered K/V row is loaded once per KV head.  K/V rows are fetched
+// One CTA = one work item (sequence, KV head, one 128-row block of packed query rows, key-range
+// piece).  The 7 query heads of the GQA group times 18 draft tokens form one block (row
+// r = (t % 18)*7 + g, two rows of padding), so every gathered K/V row is loaded once per KV head
+// and block.  K/V rows are fetched
 // with 16-byte cp.async (row index = key index, or anchor_idx[key] when gathering) into a
 // two-stage XOR-swizzled shared-memory ring; S = QK^T and O += PV run on mma.sync m16n8k16 bf16
 // with fp32 accumulation; the online softmax is fp32 with quad shuffles.  Per item the kernel
@@ -92,7 +93,7 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g4 = lane >> 2, c4 = lane & 3;
     const Item it = decode_item(plan, blockIdx.x);
-    const int T = plan.T, M = plan.M;
+    const int T = plan.T;
     const bool anchored = args.anchor_idx != nullptr;
     const int kv_len = anchored ? 0 : plan.kv_len[it.b];
     const int32_t* aidx = anchored ? args.anchor_idx + (size_t)it.b * args.n_anchor : nullptr;
@@ -114,10 +115,9 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
         for (int u = 0; u < kChunksPerThread; ++u) {
             const int i = tid + u * kThreads;
             const int r = i >> 4, c = i & 15;
-            const int R = it.group * plan.rows_per_group + r;
+            const int t = it.group * kTokPerBlock + r / kGroup, g = r % kGroup;
             val[u] = make_uint4(0, 0, 0, 0);
-            if (R < M && r < plan.rows_per_group) {
-                const int t = R / kGroup, g = R % kGroup;
+            if (r < kTokPerBlock * kGroup && t < T) {
                 val[u] = __ldg(reinterpret_cast<const uint4*>(
                     args.q + (((size_t)it.b * T + t) * args.n_q_heads + it.kvh * kGroup + g) * kD + c * 8));
             }
@@ -137,13 +137,13 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
             ldsm_x4(smem_u32(kv_smem + swz(r, ks * 2 + (lane >> 4))), qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
     }
     // per-thread row state: rows lr0 = warp*16+g4 and lr0+8
-    int rowR[2]; bool row_ok[2]; unsigned long long row_anc[2]; int row_qpos[2];
+    int row_t[2]; bool row_ok[2]; unsigned long long row_anc[2]; int row_qpos[2];
     #pragma unroll
     for (int rr = 0; rr < 2; ++rr) {
         const int lr = warp * 16 + g4 + rr * 8;
-        rowR[rr] = it.group * plan.rows_per_group + lr;
-        row_ok[rr] = rowR[rr] < M && lr < plan.rows_per_group;
-        const int t = row_ok[rr] ? rowR[rr] / kGroup : 0;
+        row_t[rr] = it.group * kTokPerBlock + lr / kGroup;
+        row_ok[rr] = lr < kTokPerBlock * kGroup && row_t[rr] < T;
+        const int t = row_ok[rr] ? row_t[rr] : 0;
         row_anc[rr] = anchored ? 0ull : anc_s[t];
         row_qpos[rr] = anchored ? qpos_s[t] : 0;
     }
@@ -298,7 +298,7 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
         const float inv = l > 0.f ? 1.f / l : 0.f;
         const float lse_val = l > 0.f ? (m_run[rr] * c2 + log2f(l)) * 0.6931471805599453f : -INFINITY;
         if (plan.n_splits[it.b] == 1) {                 // the only piece: write the final result
-            const int t = rowR[rr] / kGroup, h = it.kvh * kGroup + rowR[rr] % kGroup;
+            const int t = row_t[rr], h = it.kvh * kGroup + lr % kGroup;
             __nv_bfloat16* dst = args.out + (((size_t)it.b * T + t) * args.n_q_heads + h) * kD;
             #pragma unroll
             for (int nt = 0; nt < 16; ++nt)
