@@ -45,11 +45,16 @@ struct sparrow_ctx {
     size_t ws_bytes;
     std::atomic<long long> launches;
     bool use_pdl;
+    // Host mirror of the ordering counters in the workspace (see SyncArgs): call sequence number
+    // of the fused calls and, per call parity, the cumulative number of finishers launched so far.
+    uint32_t seq;
+    uint32_t fin_total[2];
 };
 
 namespace {
 
-constexpr size_t kStatusBytes = 1024;      // word 0: sticky status; the rest is spare (tuning builds use it)
+constexpr size_t kStatusBytes = 1024;      // word 0: sticky status; words 16, 17: finisher counters
+constexpr size_t kFinDoneOffset = 64;
 constexpr int kMinPieceKeys = 128;
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -124,47 +129,83 @@ sparrow_status make_plan(int n_sm, int batch, int n_kv_heads, const int32_t* n_k
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+int max_units(const sparrow_layout& L) { return L.batch * L.n_kv_heads * kMaxGroups; }
+// per-unit arrival words of the four call slots, right behind the header
+size_t arrivals_bytes(const sparrow_layout& L) { return align_up((size_t)kArrivalSlots * max_units(L) * sizeof(unsigned), 256); }
+size_t fixed_bytes(const sparrow_layout& L) { return kStatusBytes + arrivals_bytes(L) + staging_layout(L).total; }
+size_t part_bytes(size_t rows) { return align_up(align_up(rows, 64) * sizeof(float) + rows * kD * sizeof(__half), 256); }
+
+// The partial outputs are double-buffered by call parity: buffer p is the p-th half of what
+// follows the header, the arrival words and the staging area.
+size_t part_half_bytes(const sparrow_ctx* c)
+{
+    const size_t fixed = fixed_bytes(c->layout);
+    return c->ws_bytes > fixed ? ((c->ws_bytes - fixed) / 2) & ~(size_t)255 : 0;
+}
+
 sparrow_status check_ws(const sparrow_ctx* c, const SplitPlan& p)
 {
     if (!c->ws) return SPARROW_ERR_WORKSPACE;
-    const Staging st = staging_layout(c->layout);
-    const size_t rows = (size_t)p.n_items * p.part_rows;
-    const size_t need = kStatusBytes + st.total + align_up(rows, 64) * sizeof(float) + rows * kD * sizeof(__half);
-    return need <= c->ws_bytes ? SPARROW_OK : SPARROW_ERR_WORKSPACE;
+    return part_bytes((size_t)p.n_items * p.part_rows) <= part_half_bytes(c) ? SPARROW_OK : SPARROW_ERR_WORKSPACE;
 }
 
-float* lse_part_ptr(const sparrow_ctx* c) { return reinterpret_cast<float*>(c->ws + kStatusBytes + staging_layout(c->layout).total); }
-__half* o_part_ptr(const sparrow_ctx* c, const SplitPlan& p)
+float* lse_part_ptr(const sparrow_ctx* c, int parity)
 {
-    return reinterpret_cast<__half*>(lse_part_ptr(c) + align_up((size_t)p.n_items * p.part_rows, 64));
+    return reinterpret_cast<float*>(c->ws + fixed_bytes(c->layout) + parity * part_half_bytes(c));
+}
+__half* o_part_ptr(const sparrow_ctx* c, const SplitPlan& p, int parity)
+{
+    return reinterpret_cast<__half*>(lse_part_ptr(c, parity) + align_up((size_t)p.n_items * p.part_rows, 64));
 }
 
-sparrow_status launch_combine(sparrow_ctx* c, const SplitPlan& plan, void* out, float* lse, cudaStream_t st)
+// Ordering arguments of the next call and, once it is enqueued, the advance of the host mirror.
+// Calls that are being captured into a graph, or made with programmatic launch switched off, or
+// served by the gathered kernel run in stream-ordered mode: their kernels touch no counter.
+SyncArgs next_sync(const sparrow_ctx* c, cudaStream_t st, bool fused_kernel)
+{
+    SyncArgs sy;
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) { cudaGetLastError(); cap = cudaStreamCaptureStatusActive; }
+    const int parity = (int)(c->seq & 1u);
+    sy.arrivals = reinterpret_cast<unsigned*>(c->ws + kStatusBytes);
+    sy.fin_done = reinterpret_cast<unsigned*>(c->ws + kFinDoneOffset);
+    sy.enabled = (fused_kernel && c->use_pdl && cap == cudaStreamCaptureStatusNone) ? 1 : 0;
+    sy.parity = parity;
+    sy.slot = (int)(c->seq & 3u);
+    sy.max_units = max_units(c->layout);
+    sy.fin_wait_same = c->fin_total[parity];
+    sy.fin_wait_other = c->fin_total[parity ^ 1];
+    return sy;
+}
+
+void advance_sync(sparrow_ctx* c, const SplitPlan& p, const SyncArgs& sy)
+{
+    if (!sy.enabled) return;         // stream-ordered calls leave the fused sequence where it is
+    uint32_t fin = 0;
+    for (int b = 0; b < p.batch; ++b)
+        fin += (uint32_t)(p.n_kv_heads * p.n_groups * (p.n_splits[b] < kFinishers ? p.n_splits[b] : kFinishers));
+    c->fin_total[sy.parity] += fin;
+    c->seq += 1;
+}
+
+sparrow_status launch_combine(sparrow_ctx* c, const SplitPlan& plan, const SyncArgs& sy, void* out, float* lse, cudaStream_t st)
 {
     CombineArgs ca;
-    ca.o_part = o_part_ptr(c, plan);
-    ca.lse_part = lse_part_ptr(c);
+    ca.o_part = o_part_ptr(c, plan, sy.parity);
+    ca.lse_part = lse_part_ptr(c, sy.parity);
     ca.out = static_cast<__nv_bfloat16*>(out);
     ca.lse = lse;
     ca.n_q_heads = c->layout.n_q_heads;
-    ca.use_pdl = c->use_pdl ? 1 : 0;
     const int rows = plan.batch * plan.n_kv_heads * plan.M;
-    cudaLaunchConfig_t cfg;
-    std::memset(&cfg, 0, sizeof cfg);
-    cfg.gridDim = dim3((rows + combine::kWarps - 1) / combine::kWarps);
-    cfg.blockDim = dim3(combine::kWarps * 32);
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = c->use_pdl ? 1 : 0;
-    if (cudaLaunchKernelEx(&cfg, combine::combine_kernel, plan, ca) != cudaSuccess) return SPARROW_ERR_CUDA;
+    int ctas = (rows + combine::kWarps - 1) / combine::kWarps;
+    if (ctas > 8 * c->n_sm) ctas = 8 * c->n_sm;
+    combine::combine_kernel<<<ctas, combine::kWarps * 32, 0, st>>>(plan, ca);
+    if (cudaGetLastError() != cudaSuccess) return SPARROW_ERR_CUDA;
     c->launches.fetch_add(1);
     return SPARROW_OK;
 }
 
-sparrow_status launch_split_gather(sparrow_ctx* c, const SplitPlan& plan, const void* q, const void* k, const void* v,
+sparrow_status launch_split_gather(sparrow_ctx* c, const SplitPlan& plan, const SyncArgs& sy, const void* q, const void* k, const void* v,
                                    const int32_t* parents, const int32_t* anchor_idx, int n_anchor, int window,
                                    void* out, float* lse, cudaStream_t st)
 {
@@ -181,8 +222,8 @@ sparrow_status launch_split_gather(sparrow_ctx* c, const SplitPlan& plan, const 
     a.kv_stride_batch = c->layout.kv_stride_batch;
     a.kv_stride_head = c->layout.kv_stride_head;
     a.scale_log2e = c->layout.softmax_scale * 1.4426950408889634f;
-    a.o_part = o_part_ptr(c, plan);
-    a.lse_part = lse_part_ptr(c);
+    a.o_part = o_part_ptr(c, plan, sy.parity);
+    a.lse_part = lse_part_ptr(c, sy.parity);
     a.out = static_cast<__nv_bfloat16*>(out);
     a.lse = lse;
     a.status = reinterpret_cast<unsigned*>(c->ws);
@@ -230,7 +271,7 @@ const CUtensorMap* tensor_map_for(sparrow_ctx* c, const void* base, int tag)
     return &c->maps[slot].map;
 }
 
-sparrow_status launch_verify_tc(sparrow_ctx* c, const SplitPlan& plan, const void* q, const void* k, const void* v,
+sparrow_status launch_verify_tc(sparrow_ctx* c, const SplitPlan& plan, const SyncArgs& sy, const void* q, const void* k, const void* v,
                                 const int32_t* parents, void* out, float* lse, cudaStream_t st)
 {
     const CUtensorMap* mq = tensor_map_for(c, q, plan.batch * plan.T);
@@ -242,10 +283,9 @@ sparrow_status launch_verify_tc(sparrow_ctx* c, const SplitPlan& plan, const voi
     a.parents = parents;
     a.n_q_heads = c->layout.n_q_heads;
     a.n_stages = nb == 1 ? 3 : 2;
-    a.use_pdl = c->use_pdl ? 1 : 0;
     a.scale_log2e = c->layout.softmax_scale * 1.4426950408889634f;
-    a.o_part = o_part_ptr(c, plan);
-    a.lse_part = lse_part_ptr(c);
+    a.o_part = o_part_ptr(c, plan, sy.parity);
+    a.lse_part = lse_part_ptr(c, sy.parity);
     a.out = static_cast<__nv_bfloat16*>(out);
     a.lse = lse;
     a.status = reinterpret_cast<unsigned*>(c->ws);
@@ -259,9 +299,9 @@ sparrow_status launch_verify_tc(sparrow_ctx* c, const SplitPlan& plan, const voi
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = c->use_pdl ? 1 : 0;
-    const cudaError_t e = nb == 1 ? cudaLaunchKernelEx(&cfg, tc::verify_tc_kernel<1>, *mq, *mk, *mv, plan, a)
-                                  : cudaLaunchKernelEx(&cfg, tc::verify_tc_kernel<2>, *mq, *mk, *mv, plan, a);
+    cfg.numAttrs = sy.enabled ? 1 : 0;
+    const cudaError_t e = nb == 1 ? cudaLaunchKernelEx(&cfg, tc::verify_tc_kernel<1>, *mq, *mk, *mv, plan, a, sy)
+                                  : cudaLaunchKernelEx(&cfg, tc::verify_tc_kernel<2>, *mq, *mk, *mv, plan, a, sy);
     if (e != cudaSuccess) return SPARROW_ERR_CUDA;
     c->launches.fetch_add(1);
     return SPARROW_OK;
@@ -359,6 +399,8 @@ sparrow_status sparrow_create(sparrow_ctx** out, const sparrow_layout* L, int de
     c->launches.store(0);
     const char* e = std::getenv("SPARROW_NO_PDL");
     c->use_pdl = !(e && e[0] == '1');
+    c->seq = 0;
+    c->fin_total[0] = c->fin_total[1] = 0;
     *out = c;
     return SPARROW_OK;
 }
@@ -377,22 +419,25 @@ size_t sparrow_workspace_bytes(const sparrow_ctx* c, int32_t max_T)
     for (int nb : {1, blocks_per_group_tc(max_T)}) {         // the gathered pass uses single blocks
         const int groups = (max_T + kTokPerBlock * nb - 1) / (kTokPerBlock * nb);
         const size_t rows = (size_t)max_items(c->n_sm, c->layout.batch, c->layout.n_kv_heads, groups) * (nb * kBlockRows + 1);
-        const size_t need = align_up(rows, 64) * sizeof(float) + rows * kD * sizeof(__half);
+        const size_t need = part_bytes(rows);
         if (need > worst) worst = need;
     }
-    return kStatusBytes + staging_layout(c->layout).total + worst + 256;
+    return fixed_bytes(c->layout) + 2 * worst + 512;
 }
 
 sparrow_status sparrow_set_workspace(sparrow_ctx* c, void* p, size_t bytes)
 {
     if (!c || !p) return SPARROW_ERR_NULL;
-    if ((reinterpret_cast<uintptr_t>(p) & 255u) != 0 || bytes < kStatusBytes + staging_layout(c->layout).total)
-        return SPARROW_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(p) & 255u) != 0 || bytes < fixed_bytes(c->layout)) return SPARROW_ERR_WORKSPACE;
     DeviceGuard guard(c->device);
     if (!guard.ok) return SPARROW_ERR_CUDA;
-    if (cudaMemset(p, 0, kStatusBytes) != cudaSuccess) return SPARROW_ERR_CUDA;
+    // Kernels of earlier calls may still be using the old workspace and its counters.
+    if (cudaDeviceSynchronize() != cudaSuccess) return SPARROW_ERR_CUDA;
+    if (cudaMemset(p, 0, kStatusBytes + arrivals_bytes(c->layout)) != cudaSuccess) return SPARROW_ERR_CUDA;
     c->ws = static_cast<unsigned char*>(p);
     c->ws_bytes = bytes;
+    c->seq = 0;
+    c->fin_total[0] = c->fin_total[1] = 0;
     return SPARROW_OK;
 }
 
@@ -430,10 +475,12 @@ sparrow_status sparrow_verify_attn(sparrow_ctx* c, const void* q, const void* k,
     DeviceGuard guard(c->device);
     if (!guard.ok) return SPARROW_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    s = c->verify_on_gather ? launch_split_gather(c, plan, q, k, v, parents, nullptr, 0, 0, out, lse, st)
-                            : launch_verify_tc(c, plan, q, k, v, parents, out, lse, st);
+    const SyncArgs sy = next_sync(c, st, !c->verify_on_gather);
+    s = c->verify_on_gather ? launch_split_gather(c, plan, sy, q, k, v, parents, nullptr, 0, 0, out, lse, st)
+                            : launch_verify_tc(c, plan, sy, q, k, v, parents, out, lse, st);
     if (s != SPARROW_OK) return s;
-    return launch_combine(c, plan, out, lse, st);
+    advance_sync(c, plan, sy);
+    return sy.enabled ? SPARROW_OK : launch_combine(c, plan, sy, out, lse, st);    // fused mode combines in the kernel
 }
 
 sparrow_status sparrow_verify_attn_batch(sparrow_ctx* c, const sparrow_verify_call* calls, int32_t n_calls, void* stream)
@@ -465,8 +512,9 @@ sparrow_status sparrow_anchor_attn(sparrow_ctx* c, const void* q, const void* k,
     DeviceGuard guard(c->device);
     if (!guard.ok) return SPARROW_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if ((s = launch_split_gather(c, plan, q, k, v, nullptr, anchor_idx, n_anchor, window, out, lse, st)) != SPARROW_OK) return s;
-    return launch_combine(c, plan, out, lse, st);
+    const SyncArgs sy = next_sync(c, st, false);
+    if ((s = launch_split_gather(c, plan, sy, q, k, v, nullptr, anchor_idx, n_anchor, window, out, lse, st)) != SPARROW_OK) return s;
+    return launch_combine(c, plan, sy, out, lse, st);
 }
 
 sparrow_status sparrow_verify_step_host(sparrow_ctx* c, const void* q_host, const void* k_new_host,
@@ -489,7 +537,7 @@ sparrow_status sparrow_verify_step_host(sparrow_ctx* c, const void* q_host, cons
     if (!guard.ok) return SPARROW_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const Staging sl = staging_layout(L);
-    unsigned char* base = c->ws + kStatusBytes;
+    unsigned char* base = c->ws + kStatusBytes + arrivals_bytes(L);
     void* q_dev = base + sl.q;
     void* out_dev = base + sl.out;
     float* lse_dev = reinterpret_cast<float*>(base + sl.lse);

@@ -4,9 +4,9 @@
 // [B][T][Hq][128] and fp32 lse [B][Hq][T].  Pieces that saw no visible key carry lse_s = -inf and
 // weigh zero; a row with no visible key anywhere gets out = 0, lse = -inf.
 //
-// One warp per packed query row, registers and shuffles only: the kernel uses no shared memory, so
-// its CTAs can become resident next to the split-KV CTAs (which fill the SM's shared memory) and
-// sit in griddepcontrol.wait until the partials are complete.  Lane l keeps the LSEs of pieces
+// One warp per query row, registers and shuffles only, so the same routine serves the finisher
+// CTAs of the fused split-KV kernel (whose shared memory is taken) and the stand-alone combine
+// kernel of the stream-ordered mode.  Lane l keeps the LSEs of pieces
 // l, l+32, ...  The four quarter-warps take pieces q, q+4, q+8, ...; inside a quarter each of the 8
 // lanes owns 16 of the 128 output dims (two 16-byte loads per piece), and the quarters' sums meet
 // through two shuffle steps.  The code is kept small on purpose: every warp runs it exactly once,
@@ -24,7 +24,6 @@ struct CombineArgs {
     __nv_bfloat16* out;
     float* lse;
     int32_t n_q_heads;
-    int32_t use_pdl;      // 1: launched with programmatic stream serialisation
 };
 
 namespace combine {
@@ -44,22 +43,10 @@ __device__ __forceinline__ void fma8(float (&acc)[16], int base, float w, const 
     }
 }
 
-__global__ void __launch_bounds__(kWarps * 32)
-combine_kernel(const __grid_constant__ SplitPlan plan, const __grid_constant__ CombineArgs args)
+// Merges the pieces of one (sequence b, KV head, draft token t, head g of the group) row; called
+// by all 32 lanes of a warp.
+__device__ __forceinline__ void combine_row(const SplitPlan& plan, const CombineArgs& args, int b, int kvh, int t, int g, int lane)
 {
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int rows_total = plan.batch * plan.n_kv_heads * plan.M;
-    const int row_id = blockIdx.x * kWarps + warp;
-    if (args.use_pdl) {
-        asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
-        asm volatile("griddepcontrol.wait;\n" ::: "memory");
-    }
-    if (row_id >= rows_total) return;
-    const int R = row_id % plan.M;                    // (token, head of the group): t*7 + g
-    const int unit_bh = row_id / plan.M;
-    const int kvh = unit_bh % plan.n_kv_heads;
-    const int b = unit_bh / plan.n_kv_heads;
-    const int t = R / kGroup, g = R - t * kGroup;
     const int block = t / kTokPerBlock;               // 128-row block holding this token
     const int group = block / plan.blocks_per_group;
     const int lr = (block - group * plan.blocks_per_group) * kBlockRows + (t - block * kTokPerBlock) * kGroup + g;
@@ -150,6 +137,19 @@ combine_kernel(const __grid_constant__ SplitPlan plan, const __grid_constant__ C
         reinterpret_cast<uint4*>(dst)[0] = pk[0];
         reinterpret_cast<uint4*>(dst)[1] = pk[1];
         if (lane == 0) args.lse[((size_t)b * args.n_q_heads + h) * plan.T + t] = total;
+    }
+}
+
+// The stand-alone combine kernel of the stream-ordered mode: grid-stride over the rows, one warp
+// per row.  It is an ordinary launch behind the split-KV kernel.
+__global__ void __launch_bounds__(kWarps * 32)
+combine_kernel(const __grid_constant__ SplitPlan plan, const __grid_constant__ CombineArgs args)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int rows_total = plan.batch * plan.n_kv_heads * plan.M;
+    for (int row_id = blockIdx.x * kWarps + warp; row_id < rows_total; row_id += gridDim.x * kWarps) {
+        const int R = row_id % plan.M, unit_bh = row_id / plan.M;
+        combine_row(plan, args, unit_bh / plan.n_kv_heads, unit_bh % plan.n_kv_heads, R / kGroup, R % kGroup, lane);
     }
 }
 

@@ -41,6 +41,83 @@ struct SplitPlan {
     int32_t kv_len[kMaxBatch];    // verify mode only
 };
 
+constexpr int kFinishers = 16;    // work items per unit that share its combine step
+constexpr int kMaxGroups = 4;     // row groups per (sequence, KV head): ceil(64 / 18) blocks, 1 or 2 per group
+constexpr int kArrivalSlots = 4;  // arrival words rotate over the call number modulo 4
+
+// Fused mode: ordering between the CTAs of one call and between consecutive calls.
+//
+// The split-KV kernel is launched with programmatic stream serialisation and never waits for the
+// previous grid as a whole, so the next call's CTAs start (and read their inputs) while the
+// previous call is still finishing.  What must be ordered goes through counters in the workspace,
+// released / acquired at GPU scope.  Partial buffers are double-buffered by the parity of the call
+// number n, arrival words rotate over n modulo 4.
+//   arrivals[n % 4][unit]  items of the unit (sequence, KV head, row group) that have published
+//                          their partials in call n
+//   fin_done[n % 2]        finishers (see below) of calls with this parity that are done, cumulative
+// The last min(16, pieces) pieces of a unit are its finishers: after publishing their own item
+// they wait until every piece of the unit has arrived, merge the partials of their share of the
+// unit's rows by log-sum-exp and write the final out / lse; the other items publish and exit.  An
+// item that is its unit's only piece writes final results itself and counts as one finisher.
+// Before its first global write an item of call n waits until the finishers of call n-2 are done
+// (fin_wait_same: they read the partial buffer it is about to overwrite); whoever writes final
+// results also waits for the finishers of call n-1 (fin_wait_other), so results land in call order.
+// Piece 0 of row group 0 then clears the (sequence, KV head)'s arrival words of slot (n + 2) % 4:
+// their last user was call n-2, and the items of call n+2 cannot arrive before the finishers of
+// call n are done, which in turn have seen this item's arrival.
+// With enabled == 0 the kernels are ordered by the stream alone: they touch no counter, never let
+// dependents launch early, and a separate combine kernel follows the split-KV kernel.
+struct SyncArgs {
+    unsigned* arrivals;      // [4][max_units]
+    unsigned* fin_done;      // [2]
+    int32_t enabled;
+    int32_t parity;          // n % 2
+    int32_t slot;            // n % 4
+    int32_t max_units;
+    uint32_t fin_wait_same;
+    uint32_t fin_wait_other;
+};
+
+__device__ __forceinline__ unsigned long long global_timer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ unsigned ld_acquire(const unsigned* addr)
+{
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(addr) : "memory");
+    return v;
+}
+// Bounded acquire-wait until a cumulative counter has reached `target` (wrap-safe compare).
+// Gives up after about one second and returns false.
+__device__ __forceinline__ bool wait_counter(const unsigned* addr, uint32_t target)
+{
+    const unsigned long long t0 = global_timer_ns();
+    for (;;) {
+        if ((int32_t)(ld_acquire(addr) - target) >= 0) return true;
+        if (global_timer_ns() - t0 > 1000000000ull) return false;
+        __nanosleep(100);
+    }
+}
+// Bounded acquire-wait until a word equals `value`.
+__device__ __forceinline__ bool wait_equal(const unsigned* addr, uint32_t value)
+{
+    const unsigned long long t0 = global_timer_ns();
+    for (;;) {
+        if (ld_acquire(addr) == value) return true;
+        if (global_timer_ns() - t0 > 1000000000ull) return false;
+        __nanosleep(100);
+    }
+}
+// Release-increment of a counter: orders every write this thread has observed (its own and, after
+// a CTA barrier, its CTA's) before the increment.
+__device__ __forceinline__ void publish_counter(unsigned* addr)
+{
+    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(addr) : "memory");
+}
+
 struct Item {
     int b, kvh, group, split, key_begin, key_end;
 };

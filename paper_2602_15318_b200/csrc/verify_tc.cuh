@@ -8,30 +8,40 @@
 //                        each, which land exactly in the K-major 128-byte-swizzled operand
 //                        layout), then K and V tiles of 128 keys x 128 dims (4 boxes of 128 x 64)
 //                        into a 2- or 3-stage shared-memory ring, mbarrier full / empty handshakes.
-//   warp 9, one thread   tcgen05.mma issuer: S = Q K^T (A, B from shared memory, K-major) into a
-//                        128x128 fp32 TMEM block; O += P V with P read from TMEM (bf16, aliasing
-//                        the S block) and V from shared memory as an MN-major operand.
-//   warps 0-3, 4-7       two softmax warpgroups, one thread per query row (TMEM lane): tcgen05.ld
-//                        of the score row, ancestor / range masking, fp32 online softmax with a
-//                        lazy maximum (O is rescaled in TMEM only when the row maximum grows by
-//                        more than 2^8), P packed to bf16 and stored back with tcgen05.st.
+//   warp 9, one thread   tcgen05.mma issuer.  A job is one key tile against one row block:
+//                        S = Q K^T (A, B from shared memory, K-major) into a 128 x 128 fp32 TMEM
+//                        block; O += P V with P read from TMEM (bf16, aliasing the S block) and V
+//                        from shared memory as an MN-major operand.  The scores of up to three
+//                        jobs are kept ahead of the softmax.
+//   warps 0-3, 4-7       softmax: the two threads with the same TMEM lane (warps w and w + 4)
+//                        share one query row, warpgroup g taking key columns [64 g, 64 g + 64) of
+//                        every job: tcgen05.ld, ancestor / range masking, fp32 online softmax
+//                        with a lazy maximum, P packed to bf16 and stored back with tcgen05.st.
+//                        The two threads keep the same reference maximum: one barrier with an OR
+//                        reduction per job tells whether any row's maximum grew by more than 2^8;
+//                        only then the halves' maxima meet in shared memory and O is rescaled in
+//                        TMEM.  Each thread sums its own columns; the halves' sums meet once, in
+//                        the epilogue.
 //
-// Warpgroup w owns S block w and O accumulator w.  With one row block (T <= 18) the warpgroups
-// take alternate key tiles of the same rows and their two (max, sum, O) states are merged in the
-// epilogue; with two row blocks each warpgroup owns one block and both process every key tile.
-// Either way the tensor pipe computes one job's scores while the other job's softmax runs.
+// With one row block (T <= 18) there are three S blocks and one O accumulator, with two row
+// blocks two S blocks and two accumulators (jobs alternate between the blocks).
 //
-// Ordering against neighbouring kernels in the stream (programmatic dependent launch): all reads
-// of q / k / v / parents are issued as soon as the CTA starts; griddepcontrol.wait is executed only
-// in front of the first global write (partials, out, lse), so the K/V stream of this call overlaps
-// the tail and the combine step of the previous one.
+// Ordering against neighbouring kernels in the stream (fused mode, see SyncArgs): the kernel is
+// launched with programmatic stream serialisation and never waits for the previous grid as a
+// whole.  All reads of q / k / v / parents are issued as soon as the CTA starts, so the K/V stream
+// of this call overlaps the tail of the previous one; in front of its first global write a CTA
+// waits on the finisher counters.  After storing its partials a CTA publishes its item; the last
+// pieces of each unit merge the unit's pieces by log-sum-exp (combine_row) and write out / lse,
+// the others exit at once.  In stream-ordered mode the kernel only writes partials and a separate
+// combine kernel follows.
 //
-// Every mbarrier wait is bounded; a wait that gives up sets the timeout status bit and the CTA
-// drains and exits.  TMEM is always released.
+// Every wait is bounded; a wait that gives up sets the timeout status bit and the CTA drains and
+// exits.  TMEM is always released.
 #pragma once
 #include <cuda.h>
 #include <cuda_fp16.h>
 
+#include "combine.cuh"
 #include "common.cuh"
 
 namespace sparrow {
@@ -40,11 +50,10 @@ struct TcArgs {
     const int32_t* parents;      // DEV [B][T]
     int32_t n_q_heads;
     int32_t n_stages;            // K/V ring depth (3 with one row block, 2 with two)
-    int32_t use_pdl;
     float scale_log2e;           // softmax_scale * log2(e)
     __half* o_part;              // [n_items][part_rows][128] normalised partial outputs (fp16)
     float* lse_part;             // [n_items][part_rows]
-    __nv_bfloat16* out;          // final output, written here directly for sequences with one piece
+    __nv_bfloat16* out;          // final output
     float* lse;
     unsigned* status;
 };
@@ -52,16 +61,15 @@ struct TcArgs {
 namespace tc {
 
 constexpr int kThreads = 320;                    // 8 softmax warps, producer, MMA issuer
-// Declared thread bound: caps the kernel at 65536 / 512 = 128 registers per thread, so that a CTA
-// (320 x 128 registers) leaves room on the SM for the combine kernel's CTAs.
+// Declared thread bound: caps the kernel at 65536 / 512 = 128 registers per thread.
 constexpr int kBoundThreads = 512;
 constexpr int kProducerWarp = 8, kMmaWarp = 9;
-constexpr int kTile = 128;                       // keys per stage
+constexpr int kTile = 128;                       // keys per stage and per job
 constexpr int kSubTileBytes = 128 * 64 * 2;      // one 128 x 64 bf16 box: 16 KB
 constexpr int kQBlockBytes = 2 * kSubTileBytes;  // 128 rows x 128 dims: 32 KB
 constexpr int kQBoxBytes = 64 * kGroup * kTokPerBlock * 2;   // one Q box: 64 dims x 7 heads x 18 tokens
 constexpr int kStageBytes = 4 * kSubTileBytes;   // K (32 KB) + V (32 KB)
-constexpr int kMiscBytes = 1024;                 // barriers, TMEM slot, flags, ancestor words
+constexpr int kMiscBytes = 2048;                 // barriers, flags, ancestor words, maxima exchange
 constexpr uint32_t kSpinLimit = 1u << 22;        // polls before a wait gives up
 constexpr float kRescaleLog2 = 8.0f;             // lazy-max threshold in log2 units
 
@@ -69,6 +77,9 @@ __host__ __device__ constexpr int smem_bytes(int n_blocks, int n_stages)
 {
     return 1024 /*alignment slack*/ + n_blocks * kQBlockBytes + n_stages * kStageBytes + kMiscBytes;
 }
+// S blocks (score tiles in flight) for a given number of row blocks; TMEM: S blocks first, then
+// one 128-column O accumulator per row block, 512 columns in all.
+__host__ __device__ constexpr int s_blocks(int n_blocks) { return n_blocks == 1 ? 3 : 2; }
 
 // ---- PTX wrappers ------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -123,7 +134,6 @@ __device__ __forceinline__ void tc_commit(uint32_t bar)
 }
 // barrier among the 256 softmax threads only (id 1; id 0 is __syncthreads)
 __device__ __forceinline__ void softmax_bar_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 // D[tmem] (+)= A[smem] * B[smem]
 __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
 {
@@ -249,27 +259,41 @@ __device__ __forceinline__ void exp_chunk(const float (&x)[32], float c2, float 
     tmem_st16(p_addr, p);
 }
 
+// Barrier among the 256 softmax threads with an OR reduction of a predicate (id 2).
+__device__ __forceinline__ bool softmax_bar_or(bool pred)
+{
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %1, 0;\n\t"
+        "bar.red.or.pred q, 2, 256, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(r) : "r"((uint32_t)pred) : "memory");
+    return r != 0;
+}
+
 // Shared-memory addresses of the mbarriers (8-byte slots).  K and V tiles have their own full /
-// empty pairs: a K tile is released as soon as its S = Q K^T has been computed, a V tile only
-// after its O += P V, so the K stream runs ahead of the V stream.
+// empty pairs: a K tile is released as soon as its last S = Q K^T has been computed, a V tile
+// only after its last O += P V, so the K stream runs ahead of the V stream.
 struct Bars {
     uint32_t base;
     __device__ __forceinline__ uint32_t k_full(int i) const { return base + 8u * (uint32_t)i; }
     __device__ __forceinline__ uint32_t k_empty(int i) const { return base + 32u + 8u * (uint32_t)i; }
     __device__ __forceinline__ uint32_t v_full(int i) const { return base + 64u + 8u * (uint32_t)i; }
     __device__ __forceinline__ uint32_t v_empty(int i) const { return base + 96u + 8u * (uint32_t)i; }
-    __device__ __forceinline__ uint32_t s_full(int i) const { return base + 128u + 8u * (uint32_t)i; }
-    __device__ __forceinline__ uint32_t p_full(int i) const { return base + 144u + 8u * (uint32_t)i; }
-    __device__ __forceinline__ uint32_t o_done(int i) const { return base + 160u + 8u * (uint32_t)i; }
-    __device__ __forceinline__ uint32_t q_full() const { return base + 176u; }
+    __device__ __forceinline__ uint32_t s_full(int i) const { return base + 128u + 8u * (uint32_t)i; }   // <= 4 S blocks
+    __device__ __forceinline__ uint32_t p_full(int i) const { return base + 160u + 8u * (uint32_t)i; }
+    __device__ __forceinline__ uint32_t o_done(int i) const { return base + 192u + 8u * (uint32_t)i; }   // per row block
+    __device__ __forceinline__ uint32_t q_full() const { return base + 208u; }
 };
 
 template <int NB>
 __global__ void __launch_bounds__(kBoundThreads, 1)
 verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                  const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ SplitPlan plan,
-                 const __grid_constant__ TcArgs args)
+                 const __grid_constant__ TcArgs args, const __grid_constant__ SyncArgs sync)
 {
+    constexpr int NSB = s_blocks(NB);                 // S blocks
+    constexpr uint32_t kOCol = 512 - 128 * NB;        // first accumulator's TMEM column
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     unsigned char* sm = smem_raw + ((1024u - (raw & 1023u)) & 1023u);
@@ -277,11 +301,14 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     unsigned char* q_sm = sm;
     unsigned char* kv_sm = sm + NB * kQBlockBytes;
     unsigned char* misc = kv_sm + NS * kStageBytes;
-    uint64_t* bar_mem = reinterpret_cast<uint64_t*>(misc);                  // 23 barriers in 184 bytes
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 192);
-    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(misc + 196);
+    uint64_t* bar_mem = reinterpret_cast<uint64_t*>(misc);                  // 27 barrier slots in 216 bytes
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 224);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(misc + 228);
+    volatile uint32_t* write_ok = reinterpret_cast<volatile uint32_t*>(misc + 232);   // the counters allow global writes
+    volatile int32_t* fin_go = reinterpret_cast<volatile int32_t*>(misc + 236);       // finishers: their waits succeeded
     unsigned long long* anc_s = reinterpret_cast<unsigned long long*>(misc + 256);   // [64]
-    int32_t* par_s = reinterpret_cast<int32_t*>(misc + 768);                          // [64]
+    int32_t* par_s = reinterpret_cast<int32_t*>(misc + 768);                          // [64], prologue only
+    float* xch = reinterpret_cast<float*>(misc + 1024);                               // [2][128] maxima / sums exchange
 
     Bars B;
     B.base = smem_u32(bar_mem);
@@ -292,7 +319,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     const int kv_len = plan.kv_len[it.b];
     const int n_keys_seq = plan.n_keys[it.b];
     const int n_tiles = (it.key_end - it.key_begin + kTile - 1) / kTile;
-    // job n: key tile n / NB; S block, O accumulator and softmax warpgroup n % 2; row block n % NB
+    // job n: key tile n / NB, row block (and O accumulator) n % NB, S block n % NSB
     const int n_jobs = n_tiles * NB;
     const int block0 = it.group * NB;                       // first 128-row block of this item
 
@@ -317,8 +344,9 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     if (warp == kProducerWarp && lane == 0) {
         for (int i = 0; i < 4; ++i) {
             mbar_init(B.k_full(i), 1); mbar_init(B.k_empty(i), 1); mbar_init(B.v_full(i), 1); mbar_init(B.v_empty(i), 1);
+            mbar_init(B.s_full(i), 1); mbar_init(B.p_full(i), 256);
         }
-        for (int i = 0; i < 2; ++i) { mbar_init(B.s_full(i), 1); mbar_init(B.p_full(i), 128); mbar_init(B.o_done(i), 1); }
+        for (int i = 0; i < 2; ++i) mbar_init(B.o_done(i), 1);
         mbar_init(B.q_full(), 1);
         *abort_flag = 0;
         fence_barrier_init();
@@ -349,12 +377,12 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    if (args.use_pdl) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (sync.enabled) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == kProducerWarp) {
         // ================= TMA producer =================
         if (lane == 0) {
-            // refill whichever ring has a free slot; K slots free up about one tile before V slots
+            // refill whichever ring has a free slot; K slots free up ahead of V slots
             int jk = NS < n_tiles ? NS : n_tiles, jv = jk;
             uint32_t idle = 0;
             #pragma unroll 1
@@ -371,89 +399,105 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
         if (lane == 0) {
             constexpr uint32_t idesc_qk = idesc_bf16(false);
             constexpr uint32_t idesc_pv = idesc_bf16(true);
-            // descriptors differ from tile to tile only in their 14-bit address field
+            // descriptors differ from job to job only in their 14-bit address field
             const uint64_t q_desc0 = smem_desc(smem_u32(q_sm), 16, 1024);
             const uint64_t k_desc0 = smem_desc(smem_u32(kv_sm), 16, 1024);
             const uint64_t v_desc0 = smem_desc(smem_u32(kv_sm) + 2 * kSubTileBytes, kSubTileBytes, 1024);
             bool ok = mbar_wait(B.q_full(), 0);
-            #pragma unroll 1
-            for (int n = -1; n < n_jobs && ok; ++n) {
-                if (n + 1 < n_jobs) {                                     // S = Q K^T of the next job
-                    const int m = n + 1;
-                    const int j = m / NB, blk = m % NB, slot = m & 1, st = j % NS;
-                    if (blk == 0) {                                       // first use of this K tile
-                        if (!mbar_wait(B.k_full(st), (j / NS) & 1)) { ok = false; break; }
-                        tc_fence_after();
-                    }
-                    const uint64_t qd = q_desc0 + (uint64_t)((blk * kQBlockBytes) >> 4);
-                    const uint64_t kd = k_desc0 + (uint64_t)((st * kStageBytes) >> 4);
-                    #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {
-                        const uint32_t off = ((ks >> 2) * kSubTileBytes + (ks & 3) * 32) >> 4;
-                        mma_ss(tmem + slot * 128, qd + off, kd + off, idesc_qk, ks > 0);
-                    }
-                    tc_commit(B.s_full(slot));
-                    if (blk == NB - 1) tc_commit(B.k_empty(st));
+            // S = Q K^T of job m into S block m % NSB
+            auto issue_qk = [&](int m) -> bool {
+                const int j = m / NB, blk = m % NB, sb = m % NSB, st = j % NS;
+                if (blk == 0) {                                           // first use of this K tile
+                    if (!mbar_wait(B.k_full(st), (j / NS) & 1)) return false;
+                    tc_fence_after();
                 }
-                if (n < 0) continue;
-                const int j = n / NB, blk = n % NB, slot = n & 1, st = j % NS;
+                const uint64_t qd = q_desc0 + (uint64_t)((blk * kQBlockBytes) >> 4);
+                const uint64_t kd = k_desc0 + (uint64_t)((st * kStageBytes) >> 4);
+                #pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint32_t off = ((ks >> 2) * kSubTileBytes + (ks & 3) * 32) >> 4;
+                    mma_ss(tmem + sb * 128, qd + off, kd + off, idesc_qk, ks > 0);
+                }
+                tc_commit(B.s_full(sb));
+                if (blk == NB - 1) tc_commit(B.k_empty(st));              // last use of the tile
+                return true;
+            };
+            for (int m = 0; m < NSB && m < n_jobs && ok; ++m) ok = issue_qk(m);
+            #pragma unroll 1
+            for (int n = 0; n < n_jobs && ok; ++n) {
+                const int j = n / NB, blk = n % NB, sb = n % NSB, st = j % NS;
                 if (blk == 0 && !mbar_wait(B.v_full(st), (j / NS) & 1)) { ok = false; break; }
-                if (!mbar_wait(B.p_full(slot), (n >> 1) & 1)) { ok = false; break; }
+                if (!mbar_wait(B.p_full(sb), (n / NSB) & 1)) { ok = false; break; }
                 tc_fence_after();
                 const uint64_t vd = v_desc0 + (uint64_t)((st * kStageBytes) >> 4);
                 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk)
-                    mma_ts(tmem + 256 + slot * 128, tmem + slot * 128 + kk * 8, vd + (uint64_t)((kk * 2048) >> 4),
-                           idesc_pv, (n >= 2 || kk > 0) ? 1u : 0u);
-                tc_commit(B.o_done(slot));
+                    mma_ts(tmem + kOCol + blk * 128, tmem + sb * 128 + kk * 8, vd + (uint64_t)((kk * 2048) >> 4),
+                           idesc_pv, (n >= NB || kk > 0) ? 1u : 0u);
+                tc_commit(B.o_done(blk));
                 if (blk == NB - 1) tc_commit(B.v_empty(st));
+                if (n + NSB < n_jobs) ok = issue_qk(n + NSB);             // its S block was job n's
             }
             if (!ok) { atomicOr(args.status, kStatTimeout); *abort_flag = 1; }
         }
     } else if (warp < 8) {
-        // ================= softmax warpgroups =================
-        const int wg = warp >> 2;                        // S block / O accumulator owned
+        // ================= softmax =================
+        const int wg = warp >> 2;                        // key-column half this thread takes
         const int row_local = (warp & 3) * 32 + lane;    // TMEM lane = row inside the 128-row block
-        const int blk = NB == 2 ? wg : 0;                // row block this warpgroup works on
-        const int tok0 = (block0 + blk) * kTokPerBlock;  // first token of that block
-        const int t_row = tok0 + row_local / kGroup, g_row = row_local % kGroup;
-        const bool row_ok = row_local < kTokPerBlock * kGroup && t_row < T;
-        const unsigned long long anc = (row_ok && it.key_end > kv_len) ? anc_s[t_row] : 0ull;
         const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-        const uint32_t s_addr = lane_addr + wg * 128;
-        const uint32_t o_addr = lane_addr + 256 + wg * 128;
         const float c2 = args.scale_log2e;
         const float thr = kRescaleLog2 / c2;             // threshold in raw score units
-        float m_ref = -INFINITY, l_run = 0.f;
+        const int g_row = row_local % kGroup;
+        int t_row[NB];
+        bool row_ok[NB];
+        unsigned long long anc[NB];
+        float m_ref[NB], l_run[NB];
+        // Phases of o_done[blk] observed so far.  A parity wait is only meaningful for the phase in
+        // progress or the one just completed, and the softmax runs ahead of the P V products, so
+        // every job ends by observing the previous job's phase: o_seen never lags by more than one.
+        int o_seen[NB];
+        #pragma unroll
+        for (int blk = 0; blk < NB; ++blk) {
+            t_row[blk] = (block0 + blk) * kTokPerBlock + row_local / kGroup;
+            row_ok[blk] = row_local < kTokPerBlock * kGroup && t_row[blk] < T;
+            anc[blk] = (row_ok[blk] && it.key_end > kv_len) ? anc_s[t_row[blk]] : 0ull;
+            m_ref[blk] = -INFINITY; l_run[blk] = 0.f; o_seen[blk] = 0;
+        }
         bool ok = true;
 
         #pragma unroll 1
-        for (int n = wg; n < n_jobs; n += 2) {
-            const int j = n / NB, st = j % NS;
-            if (!mbar_wait_warp(B.s_full(wg), (n >> 1) & 1)) { ok = false; break; }
-            tc_fence_after();
-            // Visibility words of this row for the tile's 128 columns (all ones away from the draft
-            // block and the end of the key range).
-            const int j0 = it.key_begin + j * kTile;
-            const bool boundary = j0 + kTile > it.key_end || j0 + kTile > kv_len;
-            unsigned long long vis_lo = ~0ull, vis_hi = ~0ull;      // columns 0-63 / 64-127
-            if (boundary) {
-                // prefix columns, then the ancestor word shifted to the draft block's column, cut at
-                // the end of the key range
-                const int d0 = kv_len - j0;                                 // column of draft token 0 (any sign)
-                const int nval = it.key_end - j0;                           // valid columns (>= 1)
-                unsigned long long lo, hi;
-                if (d0 >= 128) { lo = ~0ull; hi = ~0ull; }
-                else if (d0 >= 64) { lo = ~0ull; hi = ((1ull << (d0 - 64)) - 1ull) | (anc << (d0 - 64)); }
-                else if (d0 > 0) { lo = ((1ull << d0) - 1ull) | (anc << d0); hi = anc >> (64 - d0); }
-                else if (d0 > -64) { lo = anc >> (-d0); hi = 0ull; }
-                else { lo = 0ull; hi = 0ull; }
-                if (nval < 64) { lo &= (1ull << nval) - 1ull; hi = 0ull; }
-                else if (nval < 128) { hi &= (1ull << (nval - 64)) - 1ull; }
-                vis_lo = lo; vis_hi = hi;
-                // V rows past the end of the sequence may hold anything: zero them so 0 * x stays 0.
-                // Done by the warpgroup whose P V product is the first to read this V tile.
-                if ((NB == 1 || wg == 0) && j0 + kTile > n_keys_seq && row_local >= n_keys_seq - j0) {
+        for (int j = 0; j < n_tiles && ok; ++j) {
+            const int st = j % NS;
+            const int tile0 = it.key_begin + j * kTile;          // first key of the tile
+            const int j0 = tile0 + 64 * wg;                       // first key of this thread's columns
+            #pragma unroll
+            for (int blk = 0; blk < NB; ++blk) {
+                const int n = j * NB + blk, sb = n % NSB;
+                const uint32_t s_addr = lane_addr + sb * 128 + 64 * wg;
+                if (!mbar_wait_warp(B.s_full(sb), (n / NSB) & 1)) { ok = false; break; }
+                tc_fence_after();
+                float x0[32], x1[32];
+                tmem_ld32(s_addr, x0);
+                tmem_ld32(s_addr + 32, x1);
+                // Visibility word of this row for the thread's 64 columns (all ones away from the
+                // draft block and the end of the key range).
+                const bool boundary = j0 + 64 > it.key_end || j0 + 64 > kv_len;
+                unsigned long long vis = ~0ull;
+                if (boundary) {
+                    // prefix columns, then the ancestor word shifted to the draft block's column, cut
+                    // at the end of the key range
+                    const int d0 = kv_len - j0;                             // column of draft token 0 (any sign)
+                    const int nval = it.key_end - j0;                       // valid columns (may be <= 0)
+                    if (d0 >= 64) vis = ~0ull;
+                    else if (d0 > 0) vis = ((1ull << d0) - 1ull) | (anc[blk] << d0);
+                    else if (d0 > -64) vis = anc[blk] >> (-d0);
+                    else vis = 0ull;
+                    if (nval <= 0) vis = 0ull;
+                    else if (nval < 64) vis &= (1ull << nval) - 1ull;
+                }
+                // V rows past the end of the sequence may hold anything: zero them so 0 * x stays 0
+                // (once per tile, by the threads of the first half, thread r taking key row r).
+                if (blk == 0 && wg == 0 && tile0 + kTile > n_keys_seq && tile0 + row_local >= n_keys_seq) {
                     mbar_wait(B.v_full(st), (j / NS) & 1);
                     unsigned char* vrow = kv_sm + st * kStageBytes + 2 * kSubTileBytes + row_local * 128;
                     #pragma unroll
@@ -463,138 +507,131 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     }
                     fence_proxy_async();
                 }
-            }
-
-            // ---- pass 1: row maximum, 32 columns at a time (two chunks in flight) ----
-            float x0[32], x1[32];
-            float mx = -INFINITY;
-            #pragma unroll 1
-            for (int hf = 0; hf < 2; ++hf) {
-                tmem_ld32(s_addr + hf * 64, x0);
-                tmem_ld32(s_addr + hf * 64 + 32, x1);
                 tmem_wait_ld();
-                const unsigned long long vw = hf ? vis_hi : vis_lo;
-                if (boundary) { mask_chunk(x0, (uint32_t)vw); mask_chunk(x1, (uint32_t)(vw >> 32)); }
-                mx = fmaxf(mx, fmaxf(chunk_max(x0), chunk_max(x1)));
-            }
+                if (boundary) { mask_chunk(x0, (uint32_t)vis); mask_chunk(x1, (uint32_t)(vis >> 32)); }
+                const float mx = fmaxf(chunk_max(x0), chunk_max(x1));
 
-            // rows of padding hold whatever the Q box left there: they never force a rescale
-            const bool need = row_ok && (mx > m_ref + thr || (m_ref == -INFINITY && mx > -INFINITY));
-            if (__any_sync(0xffffffffu, need)) {
-                float alpha = 1.f;
-                if (need) {
-                    alpha = (m_ref == -INFINITY) ? 0.f : ex2((m_ref - mx) * c2);
-                    m_ref = mx;
-                    l_run *= alpha;
-                }
-                if (n >= 2) {                                         // O holds earlier tiles: rescale it in TMEM
-                    if (!mbar_wait_warp(B.o_done(wg), ((n >> 1) - 1) & 1)) { ok = false; break; }
-                    tc_fence_after();
-                    #pragma unroll 1
-                    for (int ch = 0; ch < 4; ++ch) {
-                        tmem_ld32(o_addr + ch * 32, x0);
-                        tmem_wait_ld();
-                        #pragma unroll
-                        for (int c = 0; c < 32; ++c) x0[c] *= alpha;
-                        tmem_st32(o_addr + ch * 32, reinterpret_cast<uint32_t*>(x0));
+                // Rows of padding hold whatever the Q box left there: they never force a rescale.  The
+                // barrier also orders both halves' score loads before anyone's P stores (P aliases S).
+                const bool need = row_ok[blk] && (mx > m_ref[blk] + thr || (m_ref[blk] == -INFINITY && mx > -INFINITY));
+                if (softmax_bar_or(need)) {
+                    // some row's maximum moved: the two halves of every row agree on the new reference
+                    xch[wg * 128 + row_local] = need ? mx : -INFINITY;
+                    softmax_bar_sync();
+                    const float cand = fmaxf(need ? mx : -INFINITY, xch[(wg ^ 1) * 128 + row_local]);
+                    float alpha = 1.f;
+                    if (cand > -INFINITY) {
+                        alpha = (m_ref[blk] == -INFINITY) ? 0.f : ex2((m_ref[blk] - cand) * c2);
+                        m_ref[blk] = cand;
+                        l_run[blk] *= alpha;
                     }
-                    tmem_wait_st();
+                    if (j > 0 && __any_sync(0xffffffffu, cand > -INFINITY)) {     // O holds earlier tiles: rescale this half of it
+                        for (; ok && o_seen[blk] < j; ++o_seen[blk]) ok = mbar_wait_warp(B.o_done(blk), o_seen[blk] & 1);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint32_t o_addr = lane_addr + kOCol + blk * 128 + 64 * wg;
+                        #pragma unroll 1
+                        for (int ch = 0; ch < 2; ++ch) {
+                            float o[32];
+                            tmem_ld32(o_addr + ch * 32, o);
+                            tmem_wait_ld();
+                            #pragma unroll
+                            for (int c = 0; c < 32; ++c) o[c] *= alpha;
+                            tmem_st32(o_addr + ch * 32, reinterpret_cast<uint32_t*>(o));
+                        }
+                        tmem_wait_st();
+                    }
                 }
-            }
 
-            // ---- pass 2: p = 2^(s c2 - m c2), row sum from the unrounded p, P (bf16) over the S block.
-            // P chunk ch lands on columns [16 ch, 16 ch + 16), which hold scores already consumed.
-            const float mc = (m_ref == -INFINITY) ? 0.f : m_ref * c2;
-            float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-            tmem_ld32(s_addr, x0);
-            #pragma unroll 1
-            for (int hf = 0; hf < 2; ++hf) {
-                const unsigned long long vw = hf ? vis_hi : vis_lo;
-                tmem_wait_ld();
-                tmem_ld32(s_addr + hf * 64 + 32, x1);                  // next chunk in flight
-                if (boundary) mask_chunk(x0, (uint32_t)vw);
-                exp_chunk(x0, c2, mc, sum4, s_addr + hf * 32);
-                tmem_wait_ld();
-                if (hf == 0) tmem_ld32(s_addr + 64, x0);
-                if (boundary) mask_chunk(x1, (uint32_t)(vw >> 32));
-                exp_chunk(x1, c2, mc, sum4, s_addr + hf * 32 + 16);
+                // p = 2^(s c2 - m c2), row sum from the unrounded p, P (bf16) over the S block: this
+                // thread's 64 keys land on columns [32 wg, 32 wg + 32) of the block.
+                const float mc = (m_ref[blk] == -INFINITY) ? 0.f : m_ref[blk] * c2;
+                float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+                const uint32_t p_addr = lane_addr + sb * 128 + 32 * wg;
+                exp_chunk(x0, c2, mc, sum4, p_addr);
+                exp_chunk(x1, c2, mc, sum4, p_addr + 16);
+                l_run[blk] += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+                tmem_wait_st();
+                tc_fence_before();
+                mbar_arrive(B.p_full(sb));
+                for (; ok && o_seen[blk] < j; ++o_seen[blk]) ok = mbar_wait_warp(B.o_done(blk), o_seen[blk] & 1);   // previous tile's P V, long done
+                if (!ok) break;
             }
-            l_run += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
-            tmem_wait_st();
-            tc_fence_before();
-            mbar_arrive(B.p_full(wg));
         }
 
         // ---- epilogue: normalised partial output + natural-log LSE -------------------------------
-        const int my_jobs = (n_jobs - wg + 1) / 2;                     // jobs this warpgroup ran
-        // A warpgroup without a job (a single-tile item has one job) waits for that one job instead:
-        // nothing below may touch shared memory while a load or an MMA can still use it.
-        if (ok && !mbar_wait_warp(B.o_done(my_jobs > 0 ? wg : wg ^ 1), my_jobs > 0 ? (my_jobs - 1) & 1 : 0)) ok = false;
-        tc_fence_after();
         const bool direct = plan.n_splits[it.b] == 1;                  // the only piece: write the final result
-        const int h_row = it.kvh * kGroup + g_row;
-        // Staging area for coalesced stores: the Q block(s) (every MMA that read them has completed
-        // once both warpgroups are past their last o_done).  Row r holds 16 chunks of 16 bytes
-        // (128 halves), chunk c stored at position c ^ (r & 15).
-        unsigned char* stage = q_sm + blk * kQBlockBytes;
-        const size_t prow0 = (size_t)blockIdx.x * plan.part_rows + blk * kBlockRows;   // first partial row of this block
-        const int tok_here = min(kTokPerBlock, max(0, T - tok0));
-        const int rows_here = tok_here * kGroup;
-
-        if (NB == 1) {
-            // The two warpgroups hold two (max, sum, O) states of the same rows: exchange (max, sum)
-            // through shared memory (first bytes of the K/V ring, idle by now), then warpgroup w
-            // merges and writes output dims [64 w, 64 w + 64).
-            float2* ml = reinterpret_cast<float2*>(kv_sm);
-            ml[wg * 128 + row_local] = make_float2(m_ref, l_run);
+        if (tid == 0) {
+            // global writes start below: whoever read this parity's partial buffer two calls ago must
+            // be done, and final results may only follow every earlier call's
+            bool go = true;
+            if (sync.enabled) {
+                go = wait_counter(sync.fin_done + sync.parity, sync.fin_wait_same);
+                if (go && direct) go = wait_counter(sync.fin_done + (sync.parity ^ 1), sync.fin_wait_other);
+                if (!go) atomicOr(args.status, kStatTimeout);
+                if (go && it.split == 0 && it.group == 0) {
+                    // arrival words of this (sequence, KV head) for the call after next: unused by now
+                    unsigned* w = sync.arrivals + (size_t)((sync.slot + 2) & 3) * sync.max_units +
+                                  ((size_t)it.b * plan.n_kv_heads + it.kvh) * kMaxGroups;
+                    #pragma unroll
+                    for (int g = 0; g < kMaxGroups; ++g) w[g] = 0u;
+                }
+            }
+            *write_ok = go ? 1u : 0u;
+        }
+        #pragma unroll
+        for (int blk = 0; blk < NB; ++blk) {
+            for (; ok && o_seen[blk] < n_tiles; ++o_seen[blk]) ok = mbar_wait_warp(B.o_done(blk), o_seen[blk] & 1);
+            tc_fence_after();
+            // the two halves' sums meet (the maxima are already the same)
+            xch[wg * 128 + row_local] = l_run[blk];
             softmax_bar_sync();
-            const float2 other = ml[(wg ^ 1) * 128 + row_local];
-            const float m_all = fmaxf(m_ref, other.x);
-            const float a_me = (m_ref == -INFINITY) ? 0.f : ex2((m_ref - m_all) * c2);
-            const float a_ot = (other.x == -INFINITY) ? 0.f : ex2((other.x - m_all) * c2);
-            const float l_all = a_me * l_run + a_ot * other.y;
+            const float l_all = l_run[blk] + xch[(wg ^ 1) * 128 + row_local];
+            softmax_bar_sync();                                        // xch is reused by the next block
+            ok = ok && *write_ok != 0;                                 // (thread 0 wrote it before the barriers above)
             const float inv = l_all > 0.f ? 1.f / l_all : 0.f;
-            const float lse_val = l_all > 0.f ? (m_all * c2 + log2f(l_all)) * 0.6931471805599453f : -INFINITY;
-            const float w0 = (wg == 0 ? a_me : a_ot) * inv, w1 = (wg == 0 ? a_ot : a_me) * inv;
-            const bool has1 = n_jobs >= 2;                             // accumulator 1 was written at all
-            if (args.use_pdl) pdl_wait();                              // global writes start here
+            const float lse_val = l_all > 0.f ? (m_ref[blk] * c2 + log2f(l_all)) * 0.6931471805599453f : -INFINITY;
+            const int h_row = it.kvh * kGroup + g_row;
+            // Staging area for coalesced stores: the Q block (every MMA has completed by now).  Row r
+            // holds 16 chunks of 16 bytes (128 halves), chunk c stored at position c ^ (r & 15).
+            unsigned char* stage = q_sm + blk * kQBlockBytes;
+            const size_t prow0 = (size_t)blockIdx.x * plan.part_rows + blk * kBlockRows;   // first partial row of this block
             if (ok) {
                 #pragma unroll 1
-                for (int hf = 0; hf < 2; ++hf) {
+                for (int hf = 0; hf < 2; ++hf) {                       // this thread's output dims [64 wg, 64 wg + 64)
                     const int col = wg * 64 + hf * 32;
-                    float oa[32], ob[32];
-                    tmem_ld32(lane_addr + 256 + col, oa);
-                    if (has1) tmem_ld32(lane_addr + 384 + col, ob);
+                    float o[32];
+                    tmem_ld32(lane_addr + kOCol + blk * 128 + col, o);
                     tmem_wait_ld();
-                    #pragma unroll
-                    for (int c = 0; c < 32; ++c) oa[c] = has1 ? fmaf(ob[c], w1, oa[c] * w0) : oa[c] * w0;
                     uint4 pk[4];
                     uint32_t* w = reinterpret_cast<uint32_t*>(pk);
                     if (direct) {
-                        if (row_ok) {
+                        if (row_ok[blk]) {
                             #pragma unroll
-                            for (int c = 0; c < 16; ++c) w[c] = pack_bf16x2(oa[2 * c], oa[2 * c + 1]);
+                            for (int c = 0; c < 16; ++c) w[c] = pack_bf16x2(o[2 * c] * inv, o[2 * c + 1] * inv);
                             uint4* dst = reinterpret_cast<uint4*>(
-                                args.out + (((size_t)it.b * T + t_row) * args.n_q_heads + h_row) * kD + col);
+                                args.out + (((size_t)it.b * T + t_row[blk]) * args.n_q_heads + h_row) * kD + col);
                             #pragma unroll
                             for (int c = 0; c < 4; ++c) dst[c] = pk[c];
                         }
                     } else {
                         #pragma unroll
-                        for (int c = 0; c < 16; ++c) w[c] = pack_half2(oa[2 * c], oa[2 * c + 1]);
+                        for (int c = 0; c < 16; ++c) w[c] = pack_half2(o[2 * c] * inv, o[2 * c + 1] * inv);
                         #pragma unroll
                         for (int c = 0; c < 4; ++c)
                             *reinterpret_cast<uint4*>(stage + row_local * 256 + ((((col >> 3) + c) ^ (row_local & 15)) << 4)) = pk[c];
                     }
                 }
-                if (row_ok && wg == 0) {
-                    if (direct) args.lse[((size_t)it.b * args.n_q_heads + h_row) * T + t_row] = lse_val;
+                if (row_ok[blk] && wg == 0) {
+                    if (direct) args.lse[((size_t)it.b * args.n_q_heads + h_row) * T + t_row[blk]] = lse_val;
                     else args.lse_part[prow0 + row_local] = lse_val;
                 }
             }
             softmax_bar_sync();                                        // both halves of every staged row are in place
             if (ok && !direct) {
                 // warp w copies rows [16 w, 16 w + 16), two rows (512 contiguous bytes) per instruction
+                const int tok_here = min(kTokPerBlock, max(0, T - (block0 + blk) * kTokPerBlock));
+                const int rows_here = tok_here * kGroup;
                 #pragma unroll 4
                 for (int i = 0; i < 8; ++i) {
                     const int r = warp * 16 + 2 * i + (lane >> 4), c = lane & 15;
@@ -604,54 +641,44 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     }
                 }
             }
-        } else {
-            softmax_bar_sync();                                        // both warpgroups are done with the MMAs' operands
-            const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-            const float lse_val = l_run > 0.f ? (m_ref * c2 + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
-            if (args.use_pdl) pdl_wait();                              // global writes start here
-            if (ok) {
-                #pragma unroll 1
-                for (int ch = 0; ch < 4; ++ch) {
-                    float o[32];
-                    tmem_ld32(o_addr + ch * 32, o);
-                    tmem_wait_ld();
-                    uint4 pk[4];
-                    uint32_t* w = reinterpret_cast<uint32_t*>(pk);
-                    if (direct) {
-                        if (row_ok) {
-                            #pragma unroll
-                            for (int c = 0; c < 16; ++c) w[c] = pack_bf16x2(o[2 * c] * inv, o[2 * c + 1] * inv);
-                            uint4* dst = reinterpret_cast<uint4*>(
-                                args.out + (((size_t)it.b * T + t_row) * args.n_q_heads + h_row) * kD + ch * 32);
-                            #pragma unroll
-                            for (int c = 0; c < 4; ++c) dst[c] = pk[c];
-                        }
-                    } else {
-                        #pragma unroll
-                        for (int c = 0; c < 16; ++c) w[c] = pack_half2(o[2 * c] * inv, o[2 * c + 1] * inv);
-                        #pragma unroll
-                        for (int c = 0; c < 4; ++c)
-                            *reinterpret_cast<uint4*>(stage + row_local * 256 + (((ch * 4 + c) ^ (row_local & 15)) << 4)) = pk[c];
-                    }
-                }
-                if (row_ok) {
-                    if (direct) args.lse[((size_t)it.b * args.n_q_heads + h_row) * T + t_row] = lse_val;
-                    else args.lse_part[prow0 + row_local] = lse_val;
-                }
-                if (!direct) {
-                    // each warp wrote its own 32 rows; read them back two rows per instruction so a
-                    // warp store covers 512 contiguous bytes of the partial buffer
-                    __syncwarp();
-                    #pragma unroll 4
-                    for (int i = 0; i < 16; ++i) {
-                        const int r = (warp & 3) * 32 + 2 * i + (lane >> 4), c = lane & 15;
-                        if (r < rows_here) {
-                            const uint4 val = *reinterpret_cast<const uint4*>(stage + r * 256 + ((c ^ (r & 15)) << 4));
-                            *reinterpret_cast<uint4*>(args.o_part + (prow0 + r) * kD + c * 8) = val;
-                        }
-                    }
+        }
+
+        // ---- fused mode: publish this item; the unit's last pieces merge all of its pieces ----------
+        if (sync.enabled) {
+            const int ns = plan.n_splits[it.b];
+            const int n_fin = ns < kFinishers ? ns : kFinishers;
+            // >= 0: finisher index; -1: plain item; -2: wrote final results itself
+            const int role = direct ? -2 : (it.split >= ns - n_fin ? it.split - (ns - n_fin) : -1);
+            softmax_bar_sync();                                        // every global store of this CTA has been issued
+            if (tid == 0 && !direct) {
+                unsigned* word = sync.arrivals + (size_t)sync.slot * sync.max_units +
+                                 ((size_t)it.b * plan.n_kv_heads + it.kvh) * kMaxGroups + it.group;
+                publish_counter(word);
+                if (role >= 0) {
+                    // every piece of the unit in place, and the previous call's final results written
+                    const bool go = wait_equal(word, (unsigned)ns) &&
+                                    wait_counter(sync.fin_done + (sync.parity ^ 1), sync.fin_wait_other);
+                    if (!go) atomicOr(args.status, kStatTimeout);
+                    *fin_go = go ? 1 : 0;
                 }
             }
+            if (role >= 0) {
+                softmax_bar_sync();
+                if (*fin_go) {
+                    CombineArgs ca;
+                    ca.o_part = args.o_part; ca.lse_part = args.lse_part; ca.out = args.out; ca.lse = args.lse;
+                    ca.n_q_heads = args.n_q_heads;
+                    // rows of the unit: (block, r) with r < 126; this finisher takes every n_fin-th, one warp per row
+                    #pragma unroll 1
+                    for (int idx = role + n_fin * warp; idx < NB * kTokPerBlock * kGroup; idx += n_fin * 8) {
+                        const int bk = idx / (kTokPerBlock * kGroup), r = idx - bk * (kTokPerBlock * kGroup);
+                        const int t = (block0 + bk) * kTokPerBlock + r / kGroup;
+                        if (t < T) combine::combine_row(plan, ca, it.b, it.kvh, t, r % kGroup, lane);
+                    }
+                }
+                softmax_bar_sync();
+            }
+            if (tid == 0 && role != -1) publish_counter(sync.fin_done + sync.parity);
         }
         if (!ok) { atomicOr(args.status, kStatTimeout); *abort_flag = 1; }
     }
