@@ -124,6 +124,12 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
         "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar) : "memory");
 }
+// 1-D bulk copy global -> shared (16-byte aligned, size a multiple of 16), completion on an mbarrier
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -198,6 +204,13 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
 }
+// Two non-negative finite floats -> packed bf16, rounded to nearest (ties up) with integer
+// instructions: the conversion instruction shares the quarter-rate pipe with ex2, which is the
+// softmax's bottleneck.
+__device__ __forceinline__ uint32_t pack_bf16x2_pos(float lo, float hi)
+{
+    return __byte_perm(__float_as_uint(lo) + 0x8000u, __float_as_uint(hi) + 0x8000u, 0x7632);
+}
 __device__ __forceinline__ uint32_t pack_half2(float lo, float hi)
 {
     const __half2 h2 = __floats2half2_rn(lo, hi);
@@ -254,7 +267,7 @@ __device__ __forceinline__ void exp_chunk(const float (&x)[32], float c2, float 
         const float p0 = ex2(fmaf(x[2 * c], c2, -mc));
         const float p1 = ex2(fmaf(x[2 * c + 1], c2, -mc));
         sum4[c & 3] += p0 + p1;
-        p[c] = pack_bf16x2(p0, p1);
+        p[c] = pack_bf16x2_pos(p0, p1);
     }
     tmem_st16(p_addr, p);
 }
@@ -284,6 +297,7 @@ struct Bars {
     __device__ __forceinline__ uint32_t p_full(int i) const { return base + 160u + 8u * (uint32_t)i; }
     __device__ __forceinline__ uint32_t o_done(int i) const { return base + 192u + 8u * (uint32_t)i; }   // per row block
     __device__ __forceinline__ uint32_t q_full() const { return base + 208u; }
+    __device__ __forceinline__ uint32_t fin() const { return base + 216u; }       // finishers' bulk copies
 };
 
 template <int NB>
@@ -301,7 +315,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     unsigned char* q_sm = sm;
     unsigned char* kv_sm = sm + NB * kQBlockBytes;
     unsigned char* misc = kv_sm + NS * kStageBytes;
-    uint64_t* bar_mem = reinterpret_cast<uint64_t*>(misc);                  // 27 barrier slots in 216 bytes
+    uint64_t* bar_mem = reinterpret_cast<uint64_t*>(misc);                  // 28 barrier slots in 224 bytes
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 224);
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(misc + 228);
     volatile uint32_t* write_ok = reinterpret_cast<volatile uint32_t*>(misc + 232);   // the counters allow global writes
@@ -348,6 +362,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
         }
         for (int i = 0; i < 2; ++i) mbar_init(B.o_done(i), 1);
         mbar_init(B.q_full(), 1);
+        mbar_init(B.fin(), 1);
         *abort_flag = 0;
         fence_barrier_init();
         // Q first (the first S = Q K^T needs it and it is small), then K and V tiles in the order
@@ -665,16 +680,80 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
             if (role >= 0) {
                 softmax_bar_sync();
                 if (*fin_go) {
-                    CombineArgs ca;
-                    ca.o_part = args.o_part; ca.lse_part = args.lse_part; ca.out = args.out; ca.lse = args.lse;
-                    ca.n_q_heads = args.n_q_heads;
-                    // rows of the unit: (block, r) with r < 126; this finisher takes every n_fin-th, one warp per row
+                    // This finisher's rows: entries role, role + n_fin, ... of the unit's row list
+                    // (block, r) with r < 126.  Their pieces are copied into the (idle) K/V ring in
+                    // bulk -- one memory round trip for all of them -- and merged from there, one
+                    // warp per row, lane l owning output dims [4 l, 4 l + 4).
+                    const int list_len = NB * kTokPerBlock * kGroup;
+                    const int my_rows = (list_len - role + n_fin - 1) / n_fin;
+                    int batch_rows = (NS * kStageBytes) / (ns * 256);          // rows whose pieces fit the ring at once
+                    if (batch_rows > 64) batch_rows = 64;
+                    const size_t item0 = (size_t)plan.item_begin[it.b] + (size_t)(it.kvh * plan.n_groups + it.group) * ns;
+                    bool fin_ok = true;
                     #pragma unroll 1
-                    for (int idx = role + n_fin * warp; idx < NB * kTokPerBlock * kGroup; idx += n_fin * 8) {
-                        const int bk = idx / (kTokPerBlock * kGroup), r = idx - bk * (kTokPerBlock * kGroup);
-                        const int t = (block0 + bk) * kTokPerBlock + r / kGroup;
-                        if (t < T) combine::combine_row(plan, ca, it.b, it.kvh, t, r % kGroup, lane);
+                    for (int r0 = 0, phase = 0; r0 < my_rows; r0 += batch_rows, phase ^= 1) {     // same trip count in every warp
+                        const int n_here = min(batch_rows, my_rows - r0);
+                        if (tid == 0) mbar_expect_tx(B.fin(), (uint32_t)(n_here * ns * 256));
+                        softmax_bar_sync();                                    // previous batch consumed, byte count posted
+                        for (int c = tid; c < n_here * ns; c += 256) {
+                            const int i = c / ns, sp = c - i * ns;
+                            const int idx = role + n_fin * (r0 + i);
+                            const int bk = idx / (kTokPerBlock * kGroup), r = idx - bk * (kTokPerBlock * kGroup);
+                            bulk_load(smem_u32(kv_sm + (size_t)c * 256),
+                                      args.o_part + ((item0 + sp) * plan.part_rows + bk * kBlockRows + r) * kD, 256, B.fin());
+                        }
+                        fin_ok = fin_ok && mbar_wait_warp(B.fin(), phase);
+                        #pragma unroll 1
+                        for (int i = warp; i < n_here && fin_ok; i += 8) {
+                            const int idx = role + n_fin * (r0 + i);
+                            const int bk = idx / (kTokPerBlock * kGroup), r = idx - bk * (kTokPerBlock * kGroup);
+                            const int t = (block0 + bk) * kTokPerBlock + r / kGroup, g = r % kGroup;
+                            if (t >= T) continue;
+                            const float* lse_row = args.lse_part + item0 * plan.part_rows + bk * kBlockRows + r;
+                            float lv[8];
+                            float mxl = -INFINITY;
+                            #pragma unroll
+                            for (int k = 0; k < 8; ++k) {
+                                const int sp = lane + 32 * k;
+                                lv[k] = sp < ns ? __ldcg(lse_row + (size_t)sp * plan.part_rows) : -INFINITY;
+                                mxl = fmaxf(mxl, lv[k]);
+                            }
+                            #pragma unroll
+                            for (int d = 16; d > 0; d >>= 1) mxl = fmaxf(mxl, __shfl_xor_sync(0xffffffffu, mxl, d));
+                            const bool any = mxl != -INFINITY;
+                            float suml = 0.f;
+                            #pragma unroll
+                            for (int k = 0; k < 8; ++k) suml += any ? __expf(lv[k] - mxl) : 0.f;
+                            #pragma unroll
+                            for (int d = 16; d > 0; d >>= 1) suml += __shfl_xor_sync(0xffffffffu, suml, d);
+                            const float total = any ? mxl + logf(suml) : -INFINITY;
+                            #pragma unroll
+                            for (int k = 0; k < 8; ++k) lv[k] = any ? __expf(lv[k] - total) : 0.f;   // now the weights
+                            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                            const unsigned char* src = kv_sm + (size_t)i * ns * 256 + lane * 8;
+                            #pragma unroll
+                            for (int k = 0; k < 8; ++k) {
+                                if (32 * k < ns) {                             // warp-uniform
+                                    const int cnt = min(32, ns - 32 * k);
+                                    #pragma unroll 4
+                                    for (int jj = 0; jj < cnt; ++jj) {
+                                        const float w = __shfl_sync(0xffffffffu, lv[k], jj);
+                                        const uint2 raw = *reinterpret_cast<const uint2*>(src + (size_t)(32 * k + jj) * 256);
+                                        const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
+                                        const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
+                                        acc[0] = fmaf(w, f0.x, acc[0]); acc[1] = fmaf(w, f0.y, acc[1]);
+                                        acc[2] = fmaf(w, f1.x, acc[2]); acc[3] = fmaf(w, f1.y, acc[3]);
+                                    }
+                                }
+                            }
+                            const int h = it.kvh * kGroup + g;
+                            uint2 pk;
+                            pk.x = pack_bf16x2(acc[0], acc[1]); pk.y = pack_bf16x2(acc[2], acc[3]);
+                            *reinterpret_cast<uint2*>(args.out + (((size_t)it.b * T + t) * args.n_q_heads + h) * kD + lane * 4) = pk;
+                            if (lane == 0) args.lse[((size_t)it.b * args.n_q_heads + h) * T + t] = total;
+                        }
                     }
+                    if (!fin_ok) atomicOr(args.status, kStatTimeout);
                 }
                 softmax_bar_sync();
             }
