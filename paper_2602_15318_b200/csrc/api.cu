@@ -55,6 +55,7 @@ namespace {
 
 constexpr size_t kStatusBytes = 1024;      // word 0: sticky status; words 16, 17: finisher counters
 constexpr size_t kFinDoneOffset = 64;
+constexpr size_t kArrivalsOffset = 128;     // words 32..35: arrival words of the four call slots
 constexpr int kMinPieceKeys = 128;
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -129,14 +130,11 @@ sparrow_status make_plan(int n_sm, int batch, int n_kv_heads, const int32_t* n_k
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-int max_units(const sparrow_layout& L) { return L.batch * L.n_kv_heads * kMaxGroups; }
-// per-unit arrival words of the four call slots, right behind the header
-size_t arrivals_bytes(const sparrow_layout& L) { return align_up((size_t)kArrivalSlots * max_units(L) * sizeof(unsigned), 256); }
-size_t fixed_bytes(const sparrow_layout& L) { return kStatusBytes + arrivals_bytes(L) + staging_layout(L).total; }
-size_t part_bytes(size_t rows) { return align_up(align_up(rows, 64) * sizeof(float) + rows * kD * sizeof(__half), 256); }
+size_t fixed_bytes(const sparrow_layout& L) { return kStatusBytes + staging_layout(L).total; }
+size_t part_bytes(size_t rows) { return align_up(rows * kPartRowHalves * sizeof(__half), 256); }
 
 // The partial outputs are double-buffered by call parity: buffer p is the p-th half of what
-// follows the header, the arrival words and the staging area.
+// follows the header and the staging area.
 size_t part_half_bytes(const sparrow_ctx* c)
 {
     const size_t fixed = fixed_bytes(c->layout);
@@ -149,30 +147,30 @@ sparrow_status check_ws(const sparrow_ctx* c, const SplitPlan& p)
     return part_bytes((size_t)p.n_items * p.part_rows) <= part_half_bytes(c) ? SPARROW_OK : SPARROW_ERR_WORKSPACE;
 }
 
-float* lse_part_ptr(const sparrow_ctx* c, int parity)
+__half* o_part_ptr(const sparrow_ctx* c, int parity)
 {
-    return reinterpret_cast<float*>(c->ws + fixed_bytes(c->layout) + parity * part_half_bytes(c));
-}
-__half* o_part_ptr(const sparrow_ctx* c, const SplitPlan& p, int parity)
-{
-    return reinterpret_cast<__half*>(lse_part_ptr(c, parity) + align_up((size_t)p.n_items * p.part_rows, 64));
+    return reinterpret_cast<__half*>(c->ws + fixed_bytes(c->layout) + parity * part_half_bytes(c));
 }
 
 // Ordering arguments of the next call and, once it is enqueued, the advance of the host mirror.
 // Calls that are being captured into a graph, or made with programmatic launch switched off, or
 // served by the gathered kernel run in stream-ordered mode: their kernels touch no counter.
-SyncArgs next_sync(const sparrow_ctx* c, cudaStream_t st, bool fused_kernel)
+SyncArgs next_sync(const sparrow_ctx* c, const SplitPlan& p, cudaStream_t st, bool fused_kernel)
 {
     SyncArgs sy;
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
     if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) { cudaGetLastError(); cap = cudaStreamCaptureStatusActive; }
     const int parity = (int)(c->seq & 1u);
-    sy.arrivals = reinterpret_cast<unsigned*>(c->ws + kStatusBytes);
+    sy.arrivals = reinterpret_cast<unsigned*>(c->ws + kArrivalsOffset);
     sy.fin_done = reinterpret_cast<unsigned*>(c->ws + kFinDoneOffset);
     sy.enabled = (fused_kernel && c->use_pdl && cap == cudaStreamCaptureStatusNone) ? 1 : 0;
     sy.parity = parity;
     sy.slot = (int)(c->seq & 3u);
-    sy.max_units = max_units(c->layout);
+    int n_arrive = 0;
+    for (int b = 0; b < p.batch; ++b)
+        if (p.n_splits[b] > 1) n_arrive += p.n_kv_heads * p.n_groups * p.n_splits[b];
+    sy.n_arrive = n_arrive;
+    sy.n_fin = n_arrive == 0 ? 0 : (p.n_items < kFinisherCtas ? p.n_items : kFinisherCtas);
     sy.fin_wait_same = c->fin_total[parity];
     sy.fin_wait_other = c->fin_total[parity ^ 1];
     return sy;
@@ -181,18 +179,14 @@ SyncArgs next_sync(const sparrow_ctx* c, cudaStream_t st, bool fused_kernel)
 void advance_sync(sparrow_ctx* c, const SplitPlan& p, const SyncArgs& sy)
 {
     if (!sy.enabled) return;         // stream-ordered calls leave the fused sequence where it is
-    uint32_t fin = 0;
-    for (int b = 0; b < p.batch; ++b)
-        fin += (uint32_t)(p.n_kv_heads * p.n_groups * (p.n_splits[b] < kFinishers ? p.n_splits[b] : kFinishers));
-    c->fin_total[sy.parity] += fin;
+    c->fin_total[sy.parity] += (uint32_t)(p.n_items - sy.n_arrive + sy.n_fin);    // single-piece items + finishers
     c->seq += 1;
 }
 
 sparrow_status launch_combine(sparrow_ctx* c, const SplitPlan& plan, const SyncArgs& sy, void* out, float* lse, cudaStream_t st)
 {
     CombineArgs ca;
-    ca.o_part = o_part_ptr(c, plan, sy.parity);
-    ca.lse_part = lse_part_ptr(c, sy.parity);
+    ca.o_part = o_part_ptr(c, sy.parity);
     ca.out = static_cast<__nv_bfloat16*>(out);
     ca.lse = lse;
     ca.n_q_heads = c->layout.n_q_heads;
@@ -222,8 +216,7 @@ sparrow_status launch_split_gather(sparrow_ctx* c, const SplitPlan& plan, const 
     a.kv_stride_batch = c->layout.kv_stride_batch;
     a.kv_stride_head = c->layout.kv_stride_head;
     a.scale_log2e = c->layout.softmax_scale * 1.4426950408889634f;
-    a.o_part = o_part_ptr(c, plan, sy.parity);
-    a.lse_part = lse_part_ptr(c, sy.parity);
+    a.o_part = o_part_ptr(c, sy.parity);
     a.out = static_cast<__nv_bfloat16*>(out);
     a.lse = lse;
     a.status = reinterpret_cast<unsigned*>(c->ws);
@@ -284,8 +277,7 @@ sparrow_status launch_verify_tc(sparrow_ctx* c, const SplitPlan& plan, const Syn
     a.n_q_heads = c->layout.n_q_heads;
     a.n_stages = nb == 1 ? 3 : 2;
     a.scale_log2e = c->layout.softmax_scale * 1.4426950408889634f;
-    a.o_part = o_part_ptr(c, plan, sy.parity);
-    a.lse_part = lse_part_ptr(c, sy.parity);
+    a.o_part = o_part_ptr(c, sy.parity);
     a.out = static_cast<__nv_bfloat16*>(out);
     a.lse = lse;
     a.status = reinterpret_cast<unsigned*>(c->ws);
@@ -433,7 +425,7 @@ sparrow_status sparrow_set_workspace(sparrow_ctx* c, void* p, size_t bytes)
     if (!guard.ok) return SPARROW_ERR_CUDA;
     // Kernels of earlier calls may still be using the old workspace and its counters.
     if (cudaDeviceSynchronize() != cudaSuccess) return SPARROW_ERR_CUDA;
-    if (cudaMemset(p, 0, kStatusBytes + arrivals_bytes(c->layout)) != cudaSuccess) return SPARROW_ERR_CUDA;
+    if (cudaMemset(p, 0, kStatusBytes) != cudaSuccess) return SPARROW_ERR_CUDA;
     c->ws = static_cast<unsigned char*>(p);
     c->ws_bytes = bytes;
     c->seq = 0;
@@ -475,7 +467,7 @@ sparrow_status sparrow_verify_attn(sparrow_ctx* c, const void* q, const void* k,
     DeviceGuard guard(c->device);
     if (!guard.ok) return SPARROW_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const SyncArgs sy = next_sync(c, st, !c->verify_on_gather);
+    const SyncArgs sy = next_sync(c, plan, st, !c->verify_on_gather);
     s = c->verify_on_gather ? launch_split_gather(c, plan, sy, q, k, v, parents, nullptr, 0, 0, out, lse, st)
                             : launch_verify_tc(c, plan, sy, q, k, v, parents, out, lse, st);
     if (s != SPARROW_OK) return s;
@@ -512,7 +504,7 @@ sparrow_status sparrow_anchor_attn(sparrow_ctx* c, const void* q, const void* k,
     DeviceGuard guard(c->device);
     if (!guard.ok) return SPARROW_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const SyncArgs sy = next_sync(c, st, false);
+    const SyncArgs sy = next_sync(c, plan, st, false);
     if ((s = launch_split_gather(c, plan, sy, q, k, v, nullptr, anchor_idx, n_anchor, window, out, lse, st)) != SPARROW_OK) return s;
     return launch_combine(c, plan, sy, out, lse, st);
 }
@@ -537,7 +529,7 @@ sparrow_status sparrow_verify_step_host(sparrow_ctx* c, const void* q_host, cons
     if (!guard.ok) return SPARROW_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const Staging sl = staging_layout(L);
-    unsigned char* base = c->ws + kStatusBytes + arrivals_bytes(L);
+    unsigned char* base = c->ws + kStatusBytes;
     void* q_dev = base + sl.q;
     void* out_dev = base + sl.out;
     float* lse_dev = reinterpret_cast<float*>(base + sl.lse);

@@ -19,8 +19,7 @@
 namespace sparrow {
 
 struct CombineArgs {
-    const __half* o_part;       // [n_items][part_rows][128] normalised partial outputs (fp16)
-    const float* lse_part;
+    const __half* o_part;       // [n_items][part_rows] partial rows: 128 fp16 outputs + fp32 LSE (kPartRowHalves)
     __nv_bfloat16* out;
     float* lse;
     int32_t n_q_heads;
@@ -53,10 +52,11 @@ __device__ __forceinline__ void combine_row(const SplitPlan& plan, const Combine
     const int ns = plan.n_splits[b];
     if (ns == 1) return;                              // the split pass wrote this row's result itself
     const int item0 = plan.item_begin[b] + (kvh * plan.n_groups + group) * ns;
-    const float* lse_row = args.lse_part + (size_t)item0 * plan.part_rows + lr;      // piece s at s * part_rows
+    const size_t lse_pitch = (size_t)plan.part_rows * (kPartRowHalves / 2);          // floats between pieces
+    const float* lse_row = reinterpret_cast<const float*>(args.o_part + ((size_t)item0 * plan.part_rows + lr) * kPartRowHalves + kD);
     const int quarter = lane >> 3, sub = lane & 7;
-    const __half* o_row = args.o_part + ((size_t)item0 * plan.part_rows + lr) * kD + sub * 16;
-    const size_t o_pitch = (size_t)plan.part_rows * kD;
+    const __half* o_row = args.o_part + ((size_t)item0 * plan.part_rows + lr) * kPartRowHalves + sub * 16;
+    const size_t o_pitch = (size_t)plan.part_rows * kPartRowHalves;
 
     // first pass of partial loads goes out together with the LSE loads (they are independent)
     uint4 o0[kIter], o1[kIter];
@@ -72,19 +72,19 @@ __device__ __forceinline__ void combine_row(const SplitPlan& plan, const Combine
     #pragma unroll
     for (int i = 0; i < kPerLane; ++i) {
         const int s = lane + 32 * i;
-        lv[i] = s < ns ? __ldcg(lse_row + (size_t)s * plan.part_rows) : -INFINITY;
+        lv[i] = s < ns ? __ldcg(lse_row + (size_t)s * lse_pitch) : -INFINITY;
     }
     float mx = -INFINITY;
     #pragma unroll
     for (int i = 0; i < kPerLane; ++i) mx = fmaxf(mx, lv[i]);
-    for (int s = lane + 32 * kPerLane; s < ns; s += 32) mx = fmaxf(mx, __ldcg(lse_row + (size_t)s * plan.part_rows));
+    for (int s = lane + 32 * kPerLane; s < ns; s += 32) mx = fmaxf(mx, __ldcg(lse_row + (size_t)s * lse_pitch));
     #pragma unroll
     for (int d = 16; d > 0; d >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, d));
     const bool any = mx != -INFINITY;
     float sum = 0.f;
     #pragma unroll
     for (int i = 0; i < kPerLane; ++i) sum += any ? __expf(lv[i] - mx) : 0.f;        // 0 for absent pieces
-    for (int s = lane + 32 * kPerLane; s < ns; s += 32) sum += any ? __expf(__ldcg(lse_row + (size_t)s * plan.part_rows) - mx) : 0.f;
+    for (int s = lane + 32 * kPerLane; s < ns; s += 32) sum += any ? __expf(__ldcg(lse_row + (size_t)s * lse_pitch) - mx) : 0.f;
     #pragma unroll
     for (int d = 16; d > 0; d >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, d);
     const float total = any ? mx + logf(sum) : -INFINITY;
@@ -115,7 +115,7 @@ __device__ __forceinline__ void combine_row(const SplitPlan& plan, const Combine
             #pragma unroll
             for (int k = 0; k < kPerLane; ++k) if (reg == k) mine = lv[k];
             float w = __shfl_sync(0xffffffffu, mine, s & 31);
-            if (reg >= kPerLane && s < ns) w = any ? __expf(__ldcg(lse_row + (size_t)s * plan.part_rows) - total) : 0.f;
+            if (reg >= kPerLane && s < ns) w = any ? __expf(__ldcg(lse_row + (size_t)s * lse_pitch) - total) : 0.f;
             if (s < ns) { fma8(acc, 0, w, o0[i]); fma8(acc, 8, w, o1[i]); }
         }
     }

@@ -41,9 +41,12 @@ struct SplitPlan {
     int32_t kv_len[kMaxBatch];    // verify mode only
 };
 
-constexpr int kFinishers = 16;    // work items per unit that share its combine step
-constexpr int kMaxGroups = 4;     // row groups per (sequence, KV head): ceil(64 / 18) blocks, 1 or 2 per group
-constexpr int kArrivalSlots = 4;  // arrival words rotate over the call number modulo 4
+constexpr int kFinisherCtas = 32;  // CTAs of a call that share its combine step
+constexpr int kMaxGroups = 4;      // row groups per (sequence, KV head): ceil(64 / 18) blocks, 1 or 2 per group
+constexpr int kArrivalSlots = 4;   // arrival words rotate over the call number modulo 4
+// A partial row in the workspace: 128 fp16 outputs, then the row's fp32 LSE, padded to 16 bytes,
+// so that one bulk copy brings a run of rows with everything needed to merge them.
+constexpr int kPartRowHalves = 136;
 
 // Fused mode: ordering between the CTAs of one call and between consecutive calls.
 //
@@ -52,28 +55,31 @@ constexpr int kArrivalSlots = 4;  // arrival words rotate over the call number m
 // previous call is still finishing.  What must be ordered goes through counters in the workspace,
 // released / acquired at GPU scope.  Partial buffers are double-buffered by the parity of the call
 // number n, arrival words rotate over n modulo 4.
-//   arrivals[n % 4][unit]  items of the unit (sequence, KV head, row group) that have published
-//                          their partials in call n
-//   fin_done[n % 2]        finishers (see below) of calls with this parity that are done, cumulative
-// The last min(16, pieces) pieces of a unit are its finishers: after publishing their own item
-// they wait until every piece of the unit has arrived, merge the partials of their share of the
-// unit's rows by log-sum-exp and write the final out / lse; the other items publish and exit.  An
-// item that is its unit's only piece writes final results itself and counts as one finisher.
-// Before its first global write an item of call n waits until the finishers of call n-2 are done
-// (fin_wait_same: they read the partial buffer it is about to overwrite); whoever writes final
-// results also waits for the finishers of call n-1 (fin_wait_other), so results land in call order.
-// Piece 0 of row group 0 then clears the (sequence, KV head)'s arrival words of slot (n + 2) % 4:
-// their last user was call n-2, and the items of call n+2 cannot arrive before the finishers of
-// call n are done, which in turn have seen this item's arrival.
+//   arrivals[n % 4]   items of call n that have published their partials
+//   fin_done[n % 2]   final-result writers of calls with this parity that are done, cumulative
+// An item whose unit (sequence, KV head, row group) has several key-range pieces stores a partial
+// and arrives; an item that is its unit's only piece writes final results itself.  The last
+// n_fin CTAs of the grid are the call's finishers -- they are the last to start, so by the time
+// they are through with their own items little is left to wait for: they wait until every
+// partial of the call has arrived, then each merges a contiguous share of the call's rows by
+// log-sum-exp and writes the final out / lse.  Every final-result writer (finisher or single
+// piece) bumps fin_done once.
+// Before its first global write an item of call n waits until the writers of call n-2 are done
+// (fin_wait_same: the finishers among them read the partial buffer it is about to overwrite);
+// whoever writes final results also waits for the writers of call n-1 (fin_wait_other), so
+// results land in call order.  CTA 0 then clears the arrival word of slot (n + 2) % 4: its last
+// user was call n-2, and the items of call n+2 cannot arrive before the finishers of call n are
+// done, which in turn have seen CTA 0's arrival (or, if it had none, follow it in the stream).
 // With enabled == 0 the kernels are ordered by the stream alone: they touch no counter, never let
 // dependents launch early, and a separate combine kernel follows the split-KV kernel.
 struct SyncArgs {
-    unsigned* arrivals;      // [4][max_units]
+    unsigned* arrivals;      // [4]
     unsigned* fin_done;      // [2]
     int32_t enabled;
     int32_t parity;          // n % 2
     int32_t slot;            // n % 4
-    int32_t max_units;
+    int32_t n_arrive;        // items of this call that store partials
+    int32_t n_fin;           // finisher CTAs of this call (0 when no unit has several pieces)
     uint32_t fin_wait_same;
     uint32_t fin_wait_other;
 };

@@ -30,8 +30,7 @@ struct SplitArgs {
     int64_t kv_stride_batch;
     int64_t kv_stride_head;
     float scale_log2e;           // softmax_scale * log2(e)
-    __half* o_part;              // [n_items][part_rows][128] normalised partial outputs (fp16)
-    float* lse_part;             // [n_items][part_rows]
+    __half* o_part;              // [n_items][part_rows] partial rows: 128 fp16 outputs + fp32 LSE (kPartRowHalves)
     __nv_bfloat16* out;          // final output, written directly for sequences with one piece
     float* lse;
     unsigned* status;
@@ -306,11 +305,11 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
             if (c4 == 0) args.lse[((size_t)it.b * args.n_q_heads + h) * T + t] = lse_val;
         } else {
             const size_t prow = (size_t)blockIdx.x * plan.part_rows + lr;
-            __half* dst = args.o_part + prow * kD;
+            __half* dst = args.o_part + prow * kPartRowHalves;
             #pragma unroll
             for (int nt = 0; nt < 16; ++nt)
                 *reinterpret_cast<__half2*>(dst + nt * 8 + 2 * c4) = __floats2half2_rn(o[nt][2 * rr] * inv, o[nt][2 * rr + 1] * inv);
-            if (c4 == 0) args.lse_part[prow] = lse_val;
+            if (c4 == 0) *reinterpret_cast<float*>(dst + kD) = lse_val;
         }
     }
 }

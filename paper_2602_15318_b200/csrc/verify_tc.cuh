@@ -51,8 +51,7 @@ struct TcArgs {
     int32_t n_q_heads;
     int32_t n_stages;            // K/V ring depth (3 with one row block, 2 with two)
     float scale_log2e;           // softmax_scale * log2(e)
-    __half* o_part;              // [n_items][part_rows][128] normalised partial outputs (fp16)
-    float* lse_part;             // [n_items][part_rows]
+    __half* o_part;              // [n_items][part_rows] partial rows: 128 fp16 outputs + fp32 LSE (kPartRowHalves)
     __nv_bfloat16* out;          // final output
     float* lse;
     unsigned* status;
@@ -584,13 +583,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                 go = wait_counter(sync.fin_done + sync.parity, sync.fin_wait_same);
                 if (go && direct) go = wait_counter(sync.fin_done + (sync.parity ^ 1), sync.fin_wait_other);
                 if (!go) atomicOr(args.status, kStatTimeout);
-                if (go && it.split == 0 && it.group == 0) {
-                    // arrival words of this (sequence, KV head) for the call after next: unused by now
-                    unsigned* w = sync.arrivals + (size_t)((sync.slot + 2) & 3) * sync.max_units +
-                                  ((size_t)it.b * plan.n_kv_heads + it.kvh) * kMaxGroups;
-                    #pragma unroll
-                    for (int g = 0; g < kMaxGroups; ++g) w[g] = 0u;
-                }
+                if (go && blockIdx.x == 0) sync.arrivals[(sync.slot + 2) & 3] = 0u;   // the call after next: unused by now
             }
             *write_ok = go ? 1u : 0u;
         }
@@ -639,7 +632,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                 }
                 if (row_ok[blk] && wg == 0) {
                     if (direct) args.lse[((size_t)it.b * args.n_q_heads + h_row) * T + t_row[blk]] = lse_val;
-                    else args.lse_part[prow0 + row_local] = lse_val;
+                    else *reinterpret_cast<float*>(args.o_part + (prow0 + row_local) * kPartRowHalves + kD) = lse_val;
                 }
             }
             softmax_bar_sync();                                        // both halves of every staged row are in place
@@ -652,112 +645,136 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     const int r = warp * 16 + 2 * i + (lane >> 4), c = lane & 15;
                     if (r < rows_here) {
                         const uint4 val = *reinterpret_cast<const uint4*>(stage + r * 256 + ((c ^ (r & 15)) << 4));
-                        *reinterpret_cast<uint4*>(args.o_part + (prow0 + r) * kD + c * 8) = val;
+                        *reinterpret_cast<uint4*>(args.o_part + (prow0 + r) * kPartRowHalves + c * 8) = val;
                     }
                 }
             }
         }
 
-        // ---- fused mode: publish this item; the unit's last pieces merge all of its pieces ----------
+        // ---- fused mode: publish this item; the grid's last CTAs merge the call's partials -----------
         if (sync.enabled) {
-            const int ns = plan.n_splits[it.b];
-            const int n_fin = ns < kFinishers ? ns : kFinishers;
-            // >= 0: finisher index; -1: plain item; -2: wrote final results itself
-            const int role = direct ? -2 : (it.split >= ns - n_fin ? it.split - (ns - n_fin) : -1);
+            const int fin_idx = (int)blockIdx.x - (plan.n_items - sync.n_fin);     // >= 0: this CTA is a finisher
             softmax_bar_sync();                                        // every global store of this CTA has been issued
-            if (tid == 0 && !direct) {
-                unsigned* word = sync.arrivals + (size_t)sync.slot * sync.max_units +
-                                 ((size_t)it.b * plan.n_kv_heads + it.kvh) * kMaxGroups + it.group;
-                publish_counter(word);
-                if (role >= 0) {
-                    // every piece of the unit in place, and the previous call's final results written
-                    const bool go = wait_equal(word, (unsigned)ns) &&
+            if (tid == 0) {
+                if (!direct) publish_counter(sync.arrivals + sync.slot);
+                if (fin_idx >= 0) {
+                    // every partial of the call in place, and the previous call's final results written
+                    const bool go = wait_equal(sync.arrivals + sync.slot, (unsigned)sync.n_arrive) &&
                                     wait_counter(sync.fin_done + (sync.parity ^ 1), sync.fin_wait_other);
                     if (!go) atomicOr(args.status, kStatTimeout);
                     *fin_go = go ? 1 : 0;
                 }
             }
-            if (role >= 0) {
+            if (fin_idx >= 0) {
                 softmax_bar_sync();
                 if (*fin_go) {
-                    // This finisher's rows: entries role, role + n_fin, ... of the unit's row list
-                    // (block, r) with r < 126.  Their pieces are copied into the (idle) K/V ring in
-                    // bulk -- one memory round trip for all of them -- and merged from there, one
-                    // warp per row, lane l owning output dims [4 l, 4 l + 4).
-                    const int list_len = NB * kTokPerBlock * kGroup;
-                    const int my_rows = (list_len - role + n_fin - 1) / n_fin;
-                    int batch_rows = (NS * kStageBytes) / (ns * 256);          // rows whose pieces fit the ring at once
-                    if (batch_rows > 64) batch_rows = 64;
-                    const size_t item0 = (size_t)plan.item_begin[it.b] + (size_t)(it.kvh * plan.n_groups + it.group) * ns;
+                    // The call's row list: for every unit with several pieces, its (block, r) rows,
+                    // r < 126.  This finisher takes a contiguous chunk of the list.  Per unit, the
+                    // pieces' rows are copied into the (idle) K/V ring in bulk -- per piece one copy per
+                    // block touched, one memory round trip for a whole batch -- and merged from
+                    // there, one warp per row, lane l owning output dims [4 l, 4 l + 4).
+                    constexpr int kRowsPerBlock = kTokPerBlock * kGroup;       // 126
+                    constexpr int kRowBytes = kPartRowHalves * 2;              // 272
+                    const int list_len = NB * kRowsPerBlock;                   // rows per unit
+                    int n_units = 0;
+                    for (int b = 0; b < plan.batch; ++b)
+                        if (plan.n_splits[b] > 1) n_units += plan.n_kv_heads * plan.n_groups;
+                    const int total = n_units * list_len;
+                    const int chunk = (total + sync.n_fin - 1) / sync.n_fin;
+                    const int my_begin = fin_idx * chunk, my_end = min(total, my_begin + chunk);
                     bool fin_ok = true;
+                    int phase = 0, ubase = 0;
                     #pragma unroll 1
-                    for (int r0 = 0, phase = 0; r0 < my_rows; r0 += batch_rows, phase ^= 1) {     // same trip count in every warp
-                        const int n_here = min(batch_rows, my_rows - r0);
-                        if (tid == 0) mbar_expect_tx(B.fin(), (uint32_t)(n_here * ns * 256));
-                        softmax_bar_sync();                                    // previous batch consumed, byte count posted
-                        for (int c = tid; c < n_here * ns; c += 256) {
-                            const int i = c / ns, sp = c - i * ns;
-                            const int idx = role + n_fin * (r0 + i);
-                            const int bk = idx / (kTokPerBlock * kGroup), r = idx - bk * (kTokPerBlock * kGroup);
-                            bulk_load(smem_u32(kv_sm + (size_t)c * 256),
-                                      args.o_part + ((item0 + sp) * plan.part_rows + bk * kBlockRows + r) * kD, 256, B.fin());
-                        }
-                        fin_ok = fin_ok && mbar_wait_warp(B.fin(), phase);
+                    for (int b = 0; b < plan.batch; ++b) {
+                        const int ns = plan.n_splits[b];
+                        if (ns == 1) continue;
+                        int batch_rows = (NS * kStageBytes) / (ns * kRowBytes);    // rows whose pieces fit the ring at once
+                        if (batch_rows > kRowsPerBlock) batch_rows = kRowsPerBlock;
                         #pragma unroll 1
-                        for (int i = warp; i < n_here && fin_ok; i += 8) {
-                            const int idx = role + n_fin * (r0 + i);
-                            const int bk = idx / (kTokPerBlock * kGroup), r = idx - bk * (kTokPerBlock * kGroup);
-                            const int t = (block0 + bk) * kTokPerBlock + r / kGroup, g = r % kGroup;
-                            if (t >= T) continue;
-                            const float* lse_row = args.lse_part + item0 * plan.part_rows + bk * kBlockRows + r;
-                            float lv[8];
-                            float mxl = -INFINITY;
-                            #pragma unroll
-                            for (int k = 0; k < 8; ++k) {
-                                const int sp = lane + 32 * k;
-                                lv[k] = sp < ns ? __ldcg(lse_row + (size_t)sp * plan.part_rows) : -INFINITY;
-                                mxl = fmaxf(mxl, lv[k]);
-                            }
-                            #pragma unroll
-                            for (int d = 16; d > 0; d >>= 1) mxl = fmaxf(mxl, __shfl_xor_sync(0xffffffffu, mxl, d));
-                            const bool any = mxl != -INFINITY;
-                            float suml = 0.f;
-                            #pragma unroll
-                            for (int k = 0; k < 8; ++k) suml += any ? __expf(lv[k] - mxl) : 0.f;
-                            #pragma unroll
-                            for (int d = 16; d > 0; d >>= 1) suml += __shfl_xor_sync(0xffffffffu, suml, d);
-                            const float total = any ? mxl + logf(suml) : -INFINITY;
-                            #pragma unroll
-                            for (int k = 0; k < 8; ++k) lv[k] = any ? __expf(lv[k] - total) : 0.f;   // now the weights
-                            float acc[4] = {0.f, 0.f, 0.f, 0.f};
-                            const unsigned char* src = kv_sm + (size_t)i * ns * 256 + lane * 8;
-                            #pragma unroll
-                            for (int k = 0; k < 8; ++k) {
-                                if (32 * k < ns) {                             // warp-uniform
-                                    const int cnt = min(32, ns - 32 * k);
-                                    #pragma unroll 4
-                                    for (int jj = 0; jj < cnt; ++jj) {
-                                        const float w = __shfl_sync(0xffffffffu, lv[k], jj);
-                                        const uint2 raw = *reinterpret_cast<const uint2*>(src + (size_t)(32 * k + jj) * 256);
-                                        const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
-                                        const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
-                                        acc[0] = fmaf(w, f0.x, acc[0]); acc[1] = fmaf(w, f0.y, acc[1]);
-                                        acc[2] = fmaf(w, f1.x, acc[2]); acc[3] = fmaf(w, f1.y, acc[3]);
+                        for (int u = 0; u < plan.n_kv_heads * plan.n_groups; ++u, ubase += list_len) {
+                            const int row_begin = max(my_begin, ubase) - ubase, row_end = min(my_end, ubase + list_len) - ubase;
+                            if (row_begin >= row_end) continue;                    // (the same in every thread of the CTA)
+                            const int kvh = u / plan.n_groups, grp = u - kvh * plan.n_groups;
+                            const size_t item0 = (size_t)plan.item_begin[b] + (size_t)u * ns;
+                            #pragma unroll 1
+                            for (int r0 = row_begin; r0 < row_end; r0 += batch_rows, phase ^= 1) {
+                                const int n_here = min(batch_rows, row_end - r0);
+                                // the batch may straddle the two blocks: rows [r0, split) and [split, r0 + n_here)
+                                const int split = (r0 < kRowsPerBlock && r0 + n_here > kRowsPerBlock) ? kRowsPerBlock : r0 + n_here;
+                                if (tid == 0) mbar_expect_tx(B.fin(), (uint32_t)(n_here * ns * kRowBytes));
+                                softmax_bar_sync();                                // previous batch consumed, byte count posted
+                                for (int sp = tid; sp < ns; sp += 256) {           // shared memory: [piece][row of the batch][272 bytes]
+                                    const __half* piece = args.o_part + (item0 + sp) * plan.part_rows * kPartRowHalves;
+                                    const uint32_t dst = smem_u32(kv_sm + (size_t)sp * n_here * kRowBytes);
+                                    const int bk0 = r0 / kRowsPerBlock;
+                                    bulk_load(dst, piece + (size_t)(bk0 * kBlockRows + r0 - bk0 * kRowsPerBlock) * kPartRowHalves,
+                                              (uint32_t)(split - r0) * kRowBytes, B.fin());
+                                    if (split < r0 + n_here)
+                                        bulk_load(dst + (uint32_t)(split - r0) * kRowBytes, piece + (size_t)kBlockRows * kPartRowHalves,
+                                                  (uint32_t)(r0 + n_here - split) * kRowBytes, B.fin());
+                                }
+                                fin_ok = fin_ok && mbar_wait_warp(B.fin(), phase);
+                                #pragma unroll 1
+                                for (int i = warp; i < n_here && fin_ok; i += 8) {
+                                    const int idx = r0 + i;
+                                    const int bk = idx / kRowsPerBlock, r = idx - bk * kRowsPerBlock;
+                                    const int t = (grp * NB + bk) * kTokPerBlock + r / kGroup, g = r % kGroup;
+                                    if (t >= T) continue;
+                                    const unsigned char* row0 = kv_sm + (size_t)i * kRowBytes;   // piece stride: n_here rows
+                                    const size_t pstride = (size_t)n_here * kRowBytes;
+                                    float lv[8];
+                                    float mxl = -INFINITY;
+                                    #pragma unroll
+                                    for (int k = 0; k < 8; ++k) {
+                                        const int sp = lane + 32 * k;
+                                        lv[k] = sp < ns ? *reinterpret_cast<const float*>(row0 + sp * pstride + 2 * kD) : -INFINITY;
+                                        mxl = fmaxf(mxl, lv[k]);
                                     }
+                                    #pragma unroll
+                                    for (int d = 16; d > 0; d >>= 1) mxl = fmaxf(mxl, __shfl_xor_sync(0xffffffffu, mxl, d));
+                                    const bool any = mxl != -INFINITY;
+                                    float suml = 0.f;
+                                    #pragma unroll
+                                    for (int k = 0; k < 8; ++k) suml += any ? __expf(lv[k] - mxl) : 0.f;
+                                    #pragma unroll
+                                    for (int d = 16; d > 0; d >>= 1) suml += __shfl_xor_sync(0xffffffffu, suml, d);
+                                    const float total_lse = any ? mxl + logf(suml) : -INFINITY;
+                                    #pragma unroll
+                                    for (int k = 0; k < 8; ++k) lv[k] = any ? __expf(lv[k] - total_lse) : 0.f;   // now the weights
+                                    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                                    const unsigned char* src = row0 + lane * 8;
+                                    #pragma unroll
+                                    for (int k = 0; k < 8; ++k) {
+                                        if (32 * k < ns) {                         // warp-uniform
+                                            const int cnt = min(32, ns - 32 * k);
+                                            #pragma unroll 4
+                                            for (int jj = 0; jj < cnt; ++jj) {
+                                                const float w = __shfl_sync(0xffffffffu, lv[k], jj);
+                                                const uint2 raw = *reinterpret_cast<const uint2*>(src + (size_t)(32 * k + jj) * pstride);
+                                                const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
+                                                const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
+                                                acc[0] = fmaf(w, f0.x, acc[0]); acc[1] = fmaf(w, f0.y, acc[1]);
+                                                acc[2] = fmaf(w, f1.x, acc[2]); acc[3] = fmaf(w, f1.y, acc[3]);
+                                            }
+                                        }
+                                    }
+                                    const int h = kvh * kGroup + g;
+                                    uint2 pk;
+                                    pk.x = pack_bf16x2(acc[0], acc[1]); pk.y = pack_bf16x2(acc[2], acc[3]);
+                                    *reinterpret_cast<uint2*>(args.out + (((size_t)b * T + t) * args.n_q_heads + h) * kD + lane * 4) = pk;
+                                    if (lane == 0) args.lse[((size_t)b * args.n_q_heads + h) * T + t] = total_lse;
                                 }
                             }
-                            const int h = it.kvh * kGroup + g;
-                            uint2 pk;
-                            pk.x = pack_bf16x2(acc[0], acc[1]); pk.y = pack_bf16x2(acc[2], acc[3]);
-                            *reinterpret_cast<uint2*>(args.out + (((size_t)it.b * T + t) * args.n_q_heads + h) * kD + lane * 4) = pk;
-                            if (lane == 0) args.lse[((size_t)it.b * args.n_q_heads + h) * T + t] = total;
                         }
                     }
                     if (!fin_ok) atomicOr(args.status, kStatTimeout);
                 }
                 softmax_bar_sync();
             }
-            if (tid == 0 && role != -1) publish_counter(sync.fin_done + sync.parity);
+            if (tid == 0) {
+                if (direct) publish_counter(sync.fin_done + sync.parity);
+                if (fin_idx >= 0) publish_counter(sync.fin_done + sync.parity);
+            }
         }
         if (!ok) { atomicOr(args.status, kStatTimeout); *abort_flag = 1; }
     }
