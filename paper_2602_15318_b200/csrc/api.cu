@@ -118,12 +118,11 @@ sparrow_status make_plan(int n_sm, int batch, int n_kv_heads, const int32_t* n_k
     }
     int total = 0;
     for (int b = 0; b < batch; ++b) {
-        p->n_keys[b] = n_keys[b];
-        p->n_splits[b] = (int)((n_keys[b] + lo - 1) / lo);
-        p->item_begin[b] = total;
-        total += units * p->n_splits[b];
+        p->seq[b].n_keys = n_keys[b];
+        p->seq[b].n_splits = (int)((n_keys[b] + lo - 1) / lo);
+        p->seq[b].item_begin = total;
+        total += units * p->seq[b].n_splits;
     }
-    p->item_begin[batch] = total;
     p->n_items = total;
     return SPARROW_OK;
 }
@@ -168,7 +167,7 @@ SyncArgs next_sync(const sparrow_ctx* c, const SplitPlan& p, cudaStream_t st, bo
     sy.slot = (int)(c->seq & 3u);
     int n_arrive = 0;
     for (int b = 0; b < p.batch; ++b)
-        if (p.n_splits[b] > 1) n_arrive += p.n_kv_heads * p.n_groups * p.n_splits[b];
+        if (p.seq[b].n_splits > 1) n_arrive += p.n_kv_heads * p.n_groups * p.seq[b].n_splits;
     sy.n_arrive = n_arrive;
     sy.n_fin = n_arrive == 0 ? 0 : (p.n_items < kFinisherCtas ? p.n_items : kFinisherCtas);
     sy.fin_wait_same = c->fin_total[parity];
@@ -275,7 +274,6 @@ sparrow_status launch_verify_tc(sparrow_ctx* c, const SplitPlan& plan, const Syn
     TcArgs a;
     a.parents = parents;
     a.n_q_heads = c->layout.n_q_heads;
-    a.n_stages = nb == 1 ? 3 : 2;
     a.scale_log2e = c->layout.softmax_scale * 1.4426950408889634f;
     a.o_part = o_part_ptr(c, sy.parity);
     a.out = static_cast<__nv_bfloat16*>(out);
@@ -285,15 +283,15 @@ sparrow_status launch_verify_tc(sparrow_ctx* c, const SplitPlan& plan, const Syn
     std::memset(&cfg, 0, sizeof cfg);
     cfg.gridDim = dim3(plan.n_items);
     cfg.blockDim = dim3(tc::kThreads);
-    cfg.dynamicSmemBytes = tc::smem_bytes(nb, a.n_stages);
+    cfg.dynamicSmemBytes = tc::smem_bytes(nb, nb == 1 ? 3 : 2);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = sy.enabled ? 1 : 0;
-    const cudaError_t e = nb == 1 ? cudaLaunchKernelEx(&cfg, tc::verify_tc_kernel<1>, *mq, *mk, *mv, plan, a, sy)
-                                  : cudaLaunchKernelEx(&cfg, tc::verify_tc_kernel<2>, *mq, *mk, *mv, plan, a, sy);
+    const cudaError_t e = nb == 1 ? cudaLaunchKernelEx(&cfg, tc::verify_tc_kernel<1>, a, sy, plan, *mq, *mk, *mv)
+                                  : cudaLaunchKernelEx(&cfg, tc::verify_tc_kernel<2>, a, sy, plan, *mq, *mk, *mv);
     if (e != cudaSuccess) return SPARROW_ERR_CUDA;
     c->launches.fetch_add(1);
     return SPARROW_OK;
@@ -441,7 +439,7 @@ sparrow_status sparrow_plan_splits(int32_t n_sm, int32_t batch, int32_t n_kv_hea
     if (T < 1 || T > kMaxT) return SPARROW_ERR_SHAPE;
     const sparrow_status s = make_plan(n_sm, batch, n_kv_heads, n_keys, T, blocks_per_group_tc(T), &p);
     if (s != SPARROW_OK) return s;
-    for (int b = 0; b < batch; ++b) splits_out[b] = p.n_splits[b];
+    for (int b = 0; b < batch; ++b) splits_out[b] = p.seq[b].n_splits;
     *n_items_out = p.n_items;
     return SPARROW_OK;
 }
@@ -462,7 +460,7 @@ sparrow_status sparrow_verify_attn(sparrow_ctx* c, const void* q, const void* k,
     const int nb = c->verify_on_gather ? 1 : blocks_per_group_tc(T);
     sparrow_status s = make_plan(c->n_sm, c->layout.batch, c->layout.n_kv_heads, n_keys, T, nb, &plan);
     if (s != SPARROW_OK) return s;
-    for (int b = 0; b < c->layout.batch; ++b) plan.kv_len[b] = kv_len[b];
+    for (int b = 0; b < c->layout.batch; ++b) plan.seq[b].kv_len = kv_len[b];
     if ((s = check_ws(c, plan)) != SPARROW_OK) return s;
     DeviceGuard guard(c->device);
     if (!guard.ok) return SPARROW_ERR_CUDA;

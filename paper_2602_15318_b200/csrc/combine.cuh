@@ -49,9 +49,9 @@ __device__ __forceinline__ void combine_row(const SplitPlan& plan, const Combine
     const int block = t / kTokPerBlock;               // 128-row block holding this token
     const int group = block / plan.blocks_per_group;
     const int lr = (block - group * plan.blocks_per_group) * kBlockRows + (t - block * kTokPerBlock) * kGroup + g;
-    const int ns = plan.n_splits[b];
+    const int ns = plan.seq[b].n_splits;
     if (ns == 1) return;                              // the split pass wrote this row's result itself
-    const int item0 = plan.item_begin[b] + (kvh * plan.n_groups + group) * ns;
+    const int item0 = plan.seq[b].item_begin + (kvh * plan.n_groups + group) * ns;
     const size_t lse_pitch = (size_t)plan.part_rows * (kPartRowHalves / 2);          // floats between pieces
     const float* lse_row = reinterpret_cast<const float*>(args.o_part + ((size_t)item0 * plan.part_rows + lr) * kPartRowHalves + kD);
     const int quarter = lane >> 3, sub = lane & 7;

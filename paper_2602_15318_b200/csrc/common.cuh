@@ -24,8 +24,16 @@ constexpr unsigned kStatTimeout = 4u;
 // are padding.  A row group is 1 or 2 consecutive blocks, handled by one work item.
 //
 // One work item = (sequence b, KV head, row group, key-range piece).  Items of sequence b occupy
-// [item_begin[b], item_begin[b+1]); inside, the index runs (kv head, row group, piece) with the
+// [seq[b].item_begin, seq[b+1].item_begin); inside, the index runs (kv head, row group, piece) with the
 // piece fastest.  Piece s of n covers keys [n_keys*s/n, n_keys*(s+1)/n).
+struct SeqPlan {                  // per sequence
+    int32_t item_begin;           // first work item of the sequence
+    int32_t n_splits;             // key-range pieces per unit
+    int32_t n_keys;               // kv_len + T (verify) or n_anchor (anchored)
+    int32_t kv_len;               // verify mode only
+};
+// Scalars first and the per-sequence entries as an array of structs: what a CTA reads of the plan
+// then sits in one or two lines of the constant bank the kernel parameters live in.
 struct SplitPlan {
     int32_t n_items;
     int32_t batch;
@@ -35,10 +43,7 @@ struct SplitPlan {
     int32_t n_groups;             // ceil(T / (18 * blocks_per_group))
     int32_t n_kv_heads;
     int32_t part_rows;            // row pitch of one item's partial block in the workspace
-    int32_t item_begin[kMaxBatch + 1];
-    int32_t n_splits[kMaxBatch];
-    int32_t n_keys[kMaxBatch];    // keys per sequence: kv_len + T (verify) or n_anchor (anchored)
-    int32_t kv_len[kMaxBatch];    // verify mode only
+    SeqPlan seq[kMaxBatch];
 };
 
 constexpr int kFinisherCtas = 32;  // CTAs of a call that share its combine step
@@ -131,16 +136,16 @@ struct Item {
 __device__ __forceinline__ Item decode_item(const SplitPlan& p, int item)
 {
     int b = 0;
-    while (b + 1 < p.batch && item >= p.item_begin[b + 1]) ++b;
-    const int local = item - p.item_begin[b];
-    const int ns = p.n_splits[b];
+    while (b + 1 < p.batch && item >= p.seq[b + 1].item_begin) ++b;
+    const int local = item - p.seq[b].item_begin;
+    const int ns = p.seq[b].n_splits;
     Item it;
     it.b = b;
     it.split = local % ns;
     const int unit = local / ns;
     it.group = unit % p.n_groups;
     it.kvh = unit / p.n_groups;
-    const long long nk = p.n_keys[b];
+    const long long nk = p.seq[b].n_keys;
     it.key_begin = (int)(nk * it.split / ns);
     it.key_end = (int)(nk * (it.split + 1) / ns);
     return it;

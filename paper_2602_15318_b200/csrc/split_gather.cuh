@@ -94,7 +94,7 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
     const Item it = decode_item(plan, blockIdx.x);
     const int T = plan.T;
     const bool anchored = args.anchor_idx != nullptr;
-    const int kv_len = anchored ? 0 : plan.kv_len[it.b];
+    const int kv_len = anchored ? 0 : plan.seq[it.b].kv_len;
     const int32_t* aidx = anchored ? args.anchor_idx + (size_t)it.b * args.n_anchor : nullptr;
 
     // ---- prologue: masks / query positions, packed Q block -> registers --------------------
@@ -296,7 +296,7 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
         const int lr = warp * 16 + g4 + rr * 8;
         const float inv = l > 0.f ? 1.f / l : 0.f;
         const float lse_val = l > 0.f ? (m_run[rr] * c2 + log2f(l)) * 0.6931471805599453f : -INFINITY;
-        if (plan.n_splits[it.b] == 1) {                 // the only piece: write the final result
+        if (plan.seq[it.b].n_splits == 1) {                 // the only piece: write the final result
             const int t = row_t[rr], h = it.kvh * kGroup + lr % kGroup;
             __nv_bfloat16* dst = args.out + (((size_t)it.b * T + t) * args.n_q_heads + h) * kD;
             #pragma unroll

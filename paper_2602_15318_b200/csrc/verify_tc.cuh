@@ -49,7 +49,6 @@ namespace sparrow {
 struct TcArgs {
     const int32_t* parents;      // DEV [B][T]
     int32_t n_q_heads;
-    int32_t n_stages;            // K/V ring depth (3 with one row block, 2 with two)
     float scale_log2e;           // softmax_scale * log2(e)
     __half* o_part;              // [n_items][part_rows] partial rows: 128 fp16 outputs + fp32 LSE (kPartRowHalves)
     __nv_bfloat16* out;          // final output
@@ -301,16 +300,16 @@ struct Bars {
 
 template <int NB>
 __global__ void __launch_bounds__(kBoundThreads, 1)
-verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
-                 const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ SplitPlan plan,
-                 const __grid_constant__ TcArgs args, const __grid_constant__ SyncArgs sync)
+verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ SyncArgs sync,
+                 const __grid_constant__ SplitPlan plan, const __grid_constant__ CUtensorMap tmap_q,
+                 const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v)
 {
     constexpr int NSB = s_blocks(NB);                 // S blocks
     constexpr uint32_t kOCol = 512 - 128 * NB;        // first accumulator's TMEM column
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     unsigned char* sm = smem_raw + ((1024u - (raw & 1023u)) & 1023u);
-    const int NS = args.n_stages;
+    constexpr int NS = NB == 1 ? 3 : 2;               // K/V ring depth
     unsigned char* q_sm = sm;
     unsigned char* kv_sm = sm + NB * kQBlockBytes;
     unsigned char* misc = kv_sm + NS * kStageBytes;
@@ -329,8 +328,8 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const Item it = decode_item(plan, blockIdx.x);
     const int T = plan.T;
-    const int kv_len = plan.kv_len[it.b];
-    const int n_keys_seq = plan.n_keys[it.b];
+    const int kv_len = plan.seq[it.b].kv_len;
+    const int n_keys_seq = plan.seq[it.b].n_keys;
     const int n_tiles = (it.key_end - it.key_begin + kTile - 1) / kTile;
     // job n: key tile n / NB, row block (and O accumulator) n % NB, S block n % NSB
     const int n_jobs = n_tiles * NB;
@@ -355,6 +354,9 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
 
     // ---- setup: barriers and the first ring-full of loads, TMEM, ancestor words ------------------
     if (warp == kProducerWarp && lane == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_q) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_k) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_v) : "memory");
         for (int i = 0; i < 4; ++i) {
             mbar_init(B.k_full(i), 1); mbar_init(B.k_empty(i), 1); mbar_init(B.v_full(i), 1); mbar_init(B.v_empty(i), 1);
             mbar_init(B.s_full(i), 1); mbar_init(B.p_full(i), 256);
@@ -574,7 +576,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
         }
 
         // ---- epilogue: normalised partial output + natural-log LSE -------------------------------
-        const bool direct = plan.n_splits[it.b] == 1;                  // the only piece: write the final result
+        const bool direct = plan.seq[it.b].n_splits == 1;                  // the only piece: write the final result
         if (tid == 0) {
             // global writes start below: whoever read this parity's partial buffer two calls ago must
             // be done, and final results may only follow every earlier call's
@@ -675,10 +677,13 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     // there, one warp per row, lane l owning output dims [4 l, 4 l + 4).
                     constexpr int kRowsPerBlock = kTokPerBlock * kGroup;       // 126
                     constexpr int kRowBytes = kPartRowHalves * 2;              // 272
+                    constexpr int kMaxPieces = 256;                            // pieces per unit (<= SMs)
+                    constexpr int kWtsBytes = 8 * kMaxPieces * 4;              // per-warp piece weights, at the end of the ring
+                    float* wts = reinterpret_cast<float*>(kv_sm + NS * kStageBytes - kWtsBytes);
                     const int list_len = NB * kRowsPerBlock;                   // rows per unit
                     int n_units = 0;
                     for (int b = 0; b < plan.batch; ++b)
-                        if (plan.n_splits[b] > 1) n_units += plan.n_kv_heads * plan.n_groups;
+                        if (plan.seq[b].n_splits > 1) n_units += plan.n_kv_heads * plan.n_groups;
                     const int total = n_units * list_len;
                     const int chunk = (total + sync.n_fin - 1) / sync.n_fin;
                     const int my_begin = fin_idx * chunk, my_end = min(total, my_begin + chunk);
@@ -686,16 +691,16 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     int phase = 0, ubase = 0;
                     #pragma unroll 1
                     for (int b = 0; b < plan.batch; ++b) {
-                        const int ns = plan.n_splits[b];
+                        const int ns = plan.seq[b].n_splits;
                         if (ns == 1) continue;
-                        int batch_rows = (NS * kStageBytes) / (ns * kRowBytes);    // rows whose pieces fit the ring at once
+                        int batch_rows = (NS * kStageBytes - kWtsBytes) / (ns * kRowBytes);    // rows whose pieces fit the ring at once
                         if (batch_rows > kRowsPerBlock) batch_rows = kRowsPerBlock;
                         #pragma unroll 1
                         for (int u = 0; u < plan.n_kv_heads * plan.n_groups; ++u, ubase += list_len) {
                             const int row_begin = max(my_begin, ubase) - ubase, row_end = min(my_end, ubase + list_len) - ubase;
                             if (row_begin >= row_end) continue;                    // (the same in every thread of the CTA)
                             const int kvh = u / plan.n_groups, grp = u - kvh * plan.n_groups;
-                            const size_t item0 = (size_t)plan.item_begin[b] + (size_t)u * ns;
+                            const size_t item0 = (size_t)plan.seq[b].item_begin + (size_t)u * ns;
                             #pragma unroll 1
                             for (int r0 = row_begin; r0 < row_end; r0 += batch_rows, phase ^= 1) {
                                 const int n_here = min(batch_rows, row_end - r0);
@@ -720,44 +725,42 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                                     const int bk = idx / kRowsPerBlock, r = idx - bk * kRowsPerBlock;
                                     const int t = (grp * NB + bk) * kTokPerBlock + r / kGroup, g = r % kGroup;
                                     if (t >= T) continue;
+                                    // (small rolled loops on purpose: this code runs once per finisher and
+                                    // would otherwise be paid for in instruction fetch)
                                     const unsigned char* row0 = kv_sm + (size_t)i * kRowBytes;   // piece stride: n_here rows
                                     const size_t pstride = (size_t)n_here * kRowBytes;
-                                    float lv[8];
+                                    float* wsm = wts + warp * kMaxPieces;                        // this warp's piece weights
                                     float mxl = -INFINITY;
-                                    #pragma unroll
-                                    for (int k = 0; k < 8; ++k) {
-                                        const int sp = lane + 32 * k;
-                                        lv[k] = sp < ns ? *reinterpret_cast<const float*>(row0 + sp * pstride + 2 * kD) : -INFINITY;
-                                        mxl = fmaxf(mxl, lv[k]);
-                                    }
+                                    for (int sp = lane; sp < ns; sp += 32)
+                                        mxl = fmaxf(mxl, *reinterpret_cast<const float*>(row0 + sp * pstride + 2 * kD));
                                     #pragma unroll
                                     for (int d = 16; d > 0; d >>= 1) mxl = fmaxf(mxl, __shfl_xor_sync(0xffffffffu, mxl, d));
                                     const bool any = mxl != -INFINITY;
                                     float suml = 0.f;
-                                    #pragma unroll
-                                    for (int k = 0; k < 8; ++k) suml += any ? __expf(lv[k] - mxl) : 0.f;
+                                    for (int sp = lane; sp < ns; sp += 32) {
+                                        const float w = any ? __expf(*reinterpret_cast<const float*>(row0 + sp * pstride + 2 * kD) - mxl) : 0.f;
+                                        wsm[sp] = w;
+                                        suml += w;
+                                    }
                                     #pragma unroll
                                     for (int d = 16; d > 0; d >>= 1) suml += __shfl_xor_sync(0xffffffffu, suml, d);
+                                    __syncwarp();
                                     const float total_lse = any ? mxl + logf(suml) : -INFINITY;
-                                    #pragma unroll
-                                    for (int k = 0; k < 8; ++k) lv[k] = any ? __expf(lv[k] - total_lse) : 0.f;   // now the weights
+                                    const float inv = any ? 1.f / suml : 0.f;
                                     float acc[4] = {0.f, 0.f, 0.f, 0.f};
                                     const unsigned char* src = row0 + lane * 8;
-                                    #pragma unroll
-                                    for (int k = 0; k < 8; ++k) {
-                                        if (32 * k < ns) {                         // warp-uniform
-                                            const int cnt = min(32, ns - 32 * k);
-                                            #pragma unroll 4
-                                            for (int jj = 0; jj < cnt; ++jj) {
-                                                const float w = __shfl_sync(0xffffffffu, lv[k], jj);
-                                                const uint2 raw = *reinterpret_cast<const uint2*>(src + (size_t)(32 * k + jj) * pstride);
-                                                const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
-                                                const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
-                                                acc[0] = fmaf(w, f0.x, acc[0]); acc[1] = fmaf(w, f0.y, acc[1]);
-                                                acc[2] = fmaf(w, f1.x, acc[2]); acc[3] = fmaf(w, f1.y, acc[3]);
-                                            }
-                                        }
+                                    #pragma unroll 4
+                                    for (int sp = 0; sp < ns; ++sp) {
+                                        const float w = wsm[sp];
+                                        const uint2 raw = *reinterpret_cast<const uint2*>(src + sp * pstride);
+                                        const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
+                                        const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
+                                        acc[0] = fmaf(w, f0.x, acc[0]); acc[1] = fmaf(w, f0.y, acc[1]);
+                                        acc[2] = fmaf(w, f1.x, acc[2]); acc[3] = fmaf(w, f1.y, acc[3]);
                                     }
+                                    __syncwarp();                                                // wsm is rewritten for the next row
+                                    #pragma unroll
+                                    for (int c = 0; c < 4; ++c) acc[c] *= inv;
                                     const int h = kvh * kGroup + g;
                                     uint2 pk;
                                     pk.x = pack_bf16x2(acc[0], acc[1]); pk.y = pack_bf16x2(acc[2], acc[3]);
