@@ -111,10 +111,14 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
-// Same, with a warp-uniform result (every lane polls; used around warp-collective tcgen05 ops).
+// Same for a whole warp, with a warp-uniform result.  One lane polls (32 lanes hammering the same
+// barrier word serialise and cost hundreds of cycles per wait); the shuffle carries the verdict to
+// the others and orders their later accesses behind the observation.
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity)
 {
-    return __all_sync(0xffffffffu, mbar_wait(bar, parity) ? 1 : 0) != 0;
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity) ? 1 : 0;
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, uint32_t bar)
 {
