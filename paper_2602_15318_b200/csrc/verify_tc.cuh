@@ -682,7 +682,8 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                     constexpr int kRowsPerBlock = kTokPerBlock * kGroup;       // 126
                     constexpr int kRowBytes = kPartRowHalves * 2;              // 272
                     constexpr int kMaxPieces = 256;                            // pieces per unit (<= SMs)
-                    constexpr int kWtsBytes = 8 * kMaxPieces * 4;              // per-warp piece weights, at the end of the ring
+                    constexpr int kBatchRowsMax = 32;                          // rows merged at once
+                    constexpr int kWtsBytes = kBatchRowsMax * kMaxPieces * 4;  // their piece weights, at the end of the ring
                     float* wts = reinterpret_cast<float*>(kv_sm + NS * kStageBytes - kWtsBytes);
                     const int list_len = NB * kRowsPerBlock;                   // rows per unit
                     int n_units = 0;
@@ -698,7 +699,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                         const int ns = plan.seq[b].n_splits;
                         if (ns == 1) continue;
                         int batch_rows = (NS * kStageBytes - kWtsBytes) / (ns * kRowBytes);    // rows whose pieces fit the ring at once
-                        if (batch_rows > kRowsPerBlock) batch_rows = kRowsPerBlock;
+                        if (batch_rows > kBatchRowsMax) batch_rows = kBatchRowsMax;
                         #pragma unroll 1
                         for (int u = 0; u < plan.n_kv_heads * plan.n_groups; ++u, ubase += list_len) {
                             const int row_begin = max(my_begin, ubase) - ubase, row_end = min(my_end, ubase + list_len) - ubase;
@@ -723,53 +724,59 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                                                   (uint32_t)(r0 + n_here - split) * kRowBytes, B.fin());
                                 }
                                 fin_ok = fin_ok && mbar_wait_warp(B.fin(), phase);
+                                // (a) weights: one warp per row -- LSE = log sum exp(lse_s); w[row][s] = exp(lse_s - LSE)
                                 #pragma unroll 1
                                 for (int i = warp; i < n_here && fin_ok; i += 8) {
                                     const int idx = r0 + i;
                                     const int bk = idx / kRowsPerBlock, r = idx - bk * kRowsPerBlock;
-                                    const int t = (grp * NB + bk) * kTokPerBlock + r / kGroup, g = r % kGroup;
-                                    if (t >= T) continue;
-                                    // (small rolled loops on purpose: this code runs once per finisher and
-                                    // would otherwise be paid for in instruction fetch)
-                                    const unsigned char* row0 = kv_sm + (size_t)i * kRowBytes;   // piece stride: n_here rows
-                                    const size_t pstride = (size_t)n_here * kRowBytes;
-                                    float* wsm = wts + warp * kMaxPieces;                        // this warp's piece weights
+                                    const int t = (grp * NB + bk) * kTokPerBlock + r / kGroup;
+                                    const uint32_t pstride = (uint32_t)n_here * kRowBytes;             // bytes between pieces
+                                    const unsigned char* lse0 = kv_sm + (uint32_t)i * kRowBytes + 2 * kD + lane * pstride;
                                     float mxl = -INFINITY;
-                                    for (int sp = lane; sp < ns; sp += 32)
-                                        mxl = fmaxf(mxl, *reinterpret_cast<const float*>(row0 + sp * pstride + 2 * kD));
+                                    for (uint32_t sp = lane, off = 0; sp < (uint32_t)ns; sp += 32, off += 32 * pstride)
+                                        mxl = fmaxf(mxl, *reinterpret_cast<const float*>(lse0 + off));
                                     #pragma unroll
                                     for (int d = 16; d > 0; d >>= 1) mxl = fmaxf(mxl, __shfl_xor_sync(0xffffffffu, mxl, d));
                                     const bool any = mxl != -INFINITY;
                                     float suml = 0.f;
-                                    for (int sp = lane; sp < ns; sp += 32) {
-                                        const float w = any ? __expf(*reinterpret_cast<const float*>(row0 + sp * pstride + 2 * kD) - mxl) : 0.f;
-                                        wsm[sp] = w;
-                                        suml += w;
-                                    }
+                                    for (uint32_t sp = lane, off = 0; sp < (uint32_t)ns; sp += 32, off += 32 * pstride)
+                                        suml += any ? __expf(*reinterpret_cast<const float*>(lse0 + off) - mxl) : 0.f;
                                     #pragma unroll
                                     for (int d = 16; d > 0; d >>= 1) suml += __shfl_xor_sync(0xffffffffu, suml, d);
-                                    __syncwarp();
                                     const float total_lse = any ? mxl + logf(suml) : -INFINITY;
-                                    const float inv = any ? 1.f / suml : 0.f;
-                                    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-                                    const unsigned char* src = row0 + lane * 8;
+                                    for (uint32_t sp = lane, off = 0; sp < (uint32_t)ns; sp += 32, off += 32 * pstride)
+                                        wts[i * kMaxPieces + sp] = any ? __expf(*reinterpret_cast<const float*>(lse0 + off) - total_lse) : 0.f;
+                                    if (lane == 0 && t < T)
+                                        args.lse[((size_t)b * args.n_q_heads + kvh * kGroup + r % kGroup) * T + t] = total_lse;
+                                }
+                                softmax_bar_sync();
+                                // (b) outputs: one thread per (row, 8 output dims), all rows of the batch at once
+                                #pragma unroll 1
+                                for (int e = tid; e < n_here * 16 && fin_ok; e += 256) {
+                                    const int i = e >> 4, c = e & 15;
+                                    const int idx = r0 + i;
+                                    const int bk = idx / kRowsPerBlock, r = idx - bk * kRowsPerBlock;
+                                    const int t = (grp * NB + bk) * kTokPerBlock + r / kGroup;
+                                    if (t >= T) continue;
+                                    const uint32_t pstride = (uint32_t)n_here * kRowBytes;
+                                    const unsigned char* src = kv_sm + (uint32_t)i * kRowBytes + c * 16;
+                                    const float* w = wts + i * kMaxPieces;
+                                    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
                                     #pragma unroll 4
-                                    for (int sp = 0; sp < ns; ++sp) {
-                                        const float w = wsm[sp];
-                                        const uint2 raw = *reinterpret_cast<const uint2*>(src + sp * pstride);
-                                        const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
-                                        const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
-                                        acc[0] = fmaf(w, f0.x, acc[0]); acc[1] = fmaf(w, f0.y, acc[1]);
-                                        acc[2] = fmaf(w, f1.x, acc[2]); acc[3] = fmaf(w, f1.y, acc[3]);
+                                    for (int sp = 0; sp < ns; ++sp, src += pstride) {
+                                        const uint4 raw = *reinterpret_cast<const uint4*>(src);
+                                        const float ws = w[sp];
+                                        const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
+                                        #pragma unroll
+                                        for (int q = 0; q < 4; ++q) {
+                                            const float2 f = __half22float2(h2[q]);
+                                            acc[2 * q] = fmaf(ws, f.x, acc[2 * q]); acc[2 * q + 1] = fmaf(ws, f.y, acc[2 * q + 1]);
+                                        }
                                     }
-                                    __syncwarp();                                                // wsm is rewritten for the next row
-                                    #pragma unroll
-                                    for (int c = 0; c < 4; ++c) acc[c] *= inv;
-                                    const int h = kvh * kGroup + g;
-                                    uint2 pk;
+                                    uint4 pk;
                                     pk.x = pack_bf16x2(acc[0], acc[1]); pk.y = pack_bf16x2(acc[2], acc[3]);
-                                    *reinterpret_cast<uint2*>(args.out + (((size_t)b * T + t) * args.n_q_heads + h) * kD + lane * 4) = pk;
-                                    if (lane == 0) args.lse[((size_t)b * args.n_q_heads + h) * T + t] = total_lse;
+                                    pk.z = pack_bf16x2(acc[4], acc[5]); pk.w = pack_bf16x2(acc[6], acc[7]);
+                                    *reinterpret_cast<uint4*>(args.out + (((size_t)b * T + t) * args.n_q_heads + kvh * kGroup + r % kGroup) * kD + c * 8) = pk;
                                 }
                             }
                         }
