@@ -97,8 +97,15 @@ sparrow_status sparrow_set_workspace(sparrow_ctx* ctx, void* dev_ptr, size_t byt
  *   out      DEV bf16 [batch][T][n_q_heads][128]
  *   lse      DEV fp32 [batch][n_q_heads][T], natural log of the softmax normaliser
  *   stream   cudaStream_t (NULL = default stream)
- * Split-KV pass over ~one work item per SM followed by a log-sum-exp combine, both enqueued on
- * `stream`.  Results are deterministic for fixed arguments. */
+ * One kernel per call: a split-KV pass over ~one work item per SM whose last CTAs merge the
+ * pieces by log-sum-exp.  Consecutive calls on one stream overlap: the kernel is launched with
+ * programmatic stream serialisation and starts reading q / k_cache / v_cache / parents while the
+ * previous kernel in the stream is finishing, as soon as that kernel lets its dependents launch
+ * (the library's own kernels do; an ordinary kernel never does before it completes).  Writes of
+ * consecutive calls are ordered through counters in the workspace.  While a stream is being
+ * captured into a graph, or with SPARROW_NO_PDL=1 in the environment when the context is created,
+ * a call is two ordinary launches (split-KV pass, combine) ordered by the stream alone.
+ * Results are deterministic for fixed arguments. */
 sparrow_status sparrow_verify_attn(sparrow_ctx* ctx, const void* q, const void* k_cache,
                                    const void* v_cache, const int32_t* kv_len,
                                    const int32_t* parents, int32_t T, void* out, float* lse,
@@ -173,6 +180,13 @@ sparrow_status sparrow_debug_ancestor_masks_device(sparrow_ctx* ctx, const int32
 sparrow_status sparrow_plan_splits(int32_t n_sm, int32_t batch, int32_t n_kv_heads,
                                    const int32_t* n_keys, int32_t T, int32_t* splits_out,
                                    int32_t* n_items_out);
+
+/* Exercises the bounded device-side wait the kernels use between consecutive calls: enqueues a
+ * one-thread kernel that waits until the finisher counter of even calls reaches its current
+ * expected value plus `ahead`.  With ahead == 0 it returns once all earlier calls are done; with
+ * ahead > 0 nothing will ever satisfy it, the wait gives up after about one second, the kernel
+ * sets the timeout status bit and ends -- the context stays usable. */
+sparrow_status sparrow_debug_wait_counter(sparrow_ctx* ctx, uint32_t ahead, void* stream);
 
 /* Synchronises `stream`, returns the sticky device status (SPARROW_OK, SPARROW_ERR_TREE,
  * SPARROW_ERR_ANCHOR or SPARROW_ERR_TIMEOUT) and clears it.  Not for the hot path. */

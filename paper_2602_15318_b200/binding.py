@@ -23,7 +23,7 @@ EXPORTS = ["sparrow_create", "sparrow_destroy", "sparrow_workspace_bytes", "spar
            "sparrow_verify_attn", "sparrow_verify_attn_batch", "sparrow_anchor_attn",
            "sparrow_verify_step_host",
            "sparrow_build_ancestor_masks", "sparrow_build_anchor_idx",
-           "sparrow_debug_ancestor_masks_device", "sparrow_plan_splits",
+           "sparrow_debug_ancestor_masks_device", "sparrow_debug_wait_counter", "sparrow_plan_splits",
            "sparrow_last_device_status", "sparrow_launch_count", "sparrow_status_string"]
 
 
@@ -64,6 +64,7 @@ def lib():
         L.sparrow_build_ancestor_masks.argtypes = [vp, i32, vp]
         L.sparrow_build_anchor_idx.argtypes = [i32, vp, i32, i32, i32, vp, vp]
         L.sparrow_debug_ancestor_masks_device.argtypes = [vp, vp, i32, vp, vp]
+        L.sparrow_debug_wait_counter.argtypes = [vp, ctypes.c_uint32, vp]
         L.sparrow_plan_splits.argtypes = [i32, i32, i32, vp, i32, vp, vp]
         L.sparrow_last_device_status.argtypes = [vp, vp]
         L.sparrow_launch_count.argtypes = [vp]
@@ -228,6 +229,10 @@ def sparrow_debug_ancestor_masks_device(ctx: Context, parents_dev: torch.Tensor,
                                                    _stream_handle(stream)),
          "sparrow_debug_ancestor_masks_device")
     return masks
+
+
+def sparrow_debug_wait_counter(ctx: Context, ahead: int, stream=None):
+    _chk(lib().sparrow_debug_wait_counter(ctx.handle, ahead, _stream_handle(stream)), "sparrow_debug_wait_counter")
 
 
 def sparrow_plan_splits(n_sm: int, n_kv_heads: int, n_keys: Sequence[int], T: int):

@@ -303,6 +303,12 @@ __global__ void ancestor_masks_kernel(const int32_t* parents, int T, unsigned lo
     if (i < T) masks[i] = ancestor_word(parents, T, i, status);
 }
 
+// One thread waits (bounded) on a finisher counter; see sparrow_debug_wait_counter().
+__global__ void wait_counter_kernel(const unsigned* counter, unsigned target, unsigned* status)
+{
+    if (!wait_counter(counter, target)) atomicOr(status, kStatTimeout);
+}
+
 struct DeviceGuard {
     int prev = -1;
     bool ok = true;
@@ -601,6 +607,20 @@ sparrow_status sparrow_debug_ancestor_masks_device(sparrow_ctx* c, const int32_t
     if (!guard.ok) return SPARROW_ERR_CUDA;
     ancestor_masks_kernel<<<1, kMaxT, 0, static_cast<cudaStream_t>(stream)>>>(
         parents_dev, T, reinterpret_cast<unsigned long long*>(masks_dev), reinterpret_cast<unsigned*>(c->ws));
+    if (cudaGetLastError() != cudaSuccess) return SPARROW_ERR_CUDA;
+    c->launches.fetch_add(1);
+    return SPARROW_OK;
+}
+
+sparrow_status sparrow_debug_wait_counter(sparrow_ctx* c, uint32_t ahead, void* stream)
+{
+    if (!c) return SPARROW_ERR_NULL;
+    if (!c->ws) return SPARROW_ERR_WORKSPACE;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return SPARROW_ERR_CUDA;
+    const unsigned* counter = reinterpret_cast<const unsigned*>(c->ws + kFinDoneOffset);
+    wait_counter_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(counter, c->fin_total[0] + ahead,
+                                                                         reinterpret_cast<unsigned*>(c->ws));
     if (cudaGetLastError() != cudaSuccess) return SPARROW_ERR_CUDA;
     c->launches.fetch_add(1);
     return SPARROW_OK;

@@ -1,0 +1,131 @@
+"""GPU tests of how calls are ordered: back-to-back fused calls (programmatic dependent launch with
+counter-ordered writes), the stream-ordered two-kernel mode, calls captured into a CUDA graph, and
+the bounded device-side wait.  Results are always compared with the CPU oracle."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2602_15318_b200 import binding as B
+from paper_2602_15318_b200 import workloads as W
+
+from gpu_util import check, oracle_verify, run_verify
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _new(case):
+    out = torch.full_like(case.q, float("nan"))
+    lse = torch.full((case.B, W.HQ, case.T), float("nan"), dtype=torch.float32, device=DEV)
+    return out, lse
+
+
+def test_back_to_back_calls_keep_their_results_apart():
+    """Many calls enqueued without any synchronisation, alternating between inputs with different
+    shapes of work (several pieces / single piece, one and two row blocks) on one context: every
+    call's outputs must be its own."""
+    cap = 3000 + 64
+    cases = [W.make_verify_case(500 + i, kv, T, tree, DEV, capacity=cap)
+             for i, (kv, T, tree) in enumerate([([3000], 16, "chain"), ([90], 5, "random"), ([2500], 24, "random"),
+                                                ([1700], 8, "chain"), ([40], 19, "chain")])]
+    refs = [oracle_verify(c) for c in cases]
+    ctx = B.Context.for_cache(cases[0].k, W.SCALE)
+    results = []
+    for rep in range(6):
+        for c in cases:
+            out, lse = _new(c)
+            B.sparrow_verify_attn(ctx, c.q, c.k, c.v, c.kv_len, c.parents, c.T, out, lse)
+            results.append((out, lse))
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == 0
+    for i, (out, lse) in enumerate(results):
+        check(out, lse, *refs[i % len(cases)])
+
+
+def test_same_output_buffer_reused_by_consecutive_calls():
+    """Calls that write the same out / lse buffers land in call order: after the stream drains the
+    buffers hold the last call's result."""
+    a = W.make_verify_case(601, [2800], 12, "random", DEV)
+    b = W.make_verify_case(602, [2800], 12, "chain", DEV)
+    ctx = B.Context.for_cache(a.k, W.SCALE)
+    out, lse = _new(a)
+    for _ in range(5):
+        B.sparrow_verify_attn(ctx, a.q, a.k, a.v, a.kv_len, a.parents, a.T, out, lse)
+        B.sparrow_verify_attn(ctx, b.q, b.k, b.v, b.kv_len, b.parents, b.T, out, lse)
+    torch.cuda.synchronize()
+    check(out, lse, *oracle_verify(b))
+    B.sparrow_verify_attn(ctx, a.q, a.k, a.v, a.kv_len, a.parents, a.T, out, lse)
+    torch.cuda.synchronize()
+    check(out, lse, *oracle_verify(a))
+
+
+def test_anchor_and_verify_calls_interleave():
+    v = W.make_verify_case(603, [2000], 8, "chain", DEV, capacity=2100)
+    a = W.make_anchor_case(604, 2000, [[50, 1800]], 0, 8, 1, DEV, capacity=2100)
+    ctx = B.Context.for_cache(v.k, W.SCALE)
+    outs = []
+    for _ in range(3):
+        ov, lv = _new(v)
+        B.sparrow_verify_attn(ctx, v.q, v.k, v.v, v.kv_len, v.parents, v.T, ov, lv)
+        oa, la = _new(a)
+        B.sparrow_anchor_attn(ctx, a.q, a.k, a.v, a.anchor_idx, a.n_anchor, a.window, a.T, oa, la)
+        outs.append((ov, lv, oa, la))
+    torch.cuda.synchronize()
+    import oracle
+    ra = oracle.anchor_attn(W.bf16_bits(a.q), W.bf16_bits(a.k), W.bf16_bits(a.v), a.anchor_idx.cpu().numpy(), a.window, W.SCALE)
+    rv = oracle_verify(v)
+    for ov, lv, oa, la in outs:
+        check(ov, lv, *rv)
+        check(oa, la, *ra)
+
+
+def test_stream_ordered_mode(monkeypatch):
+    """SPARROW_NO_PDL=1 at context creation: two ordinary launches per call, no counters."""
+    monkeypatch.setenv("SPARROW_NO_PDL", "1")
+    for kv, T, tree in [([3000, 1500], 12, "random"), ([129], 19, "random"), ([64], 8, "chain")]:
+        case = W.make_verify_case(610 + T, kv, T, tree, DEV)
+        ctx = B.Context.for_cache(case.k, W.SCALE)
+        n0 = ctx.launch_count()
+        out, lse, _ = run_verify(case, ctx)
+        assert ctx.launch_count() - n0 == 2
+        check(out, lse, *oracle_verify(case))
+
+
+def test_call_captured_into_a_graph_replays():
+    case = W.make_verify_case(620, [2500, 900], 10, "random", DEV)
+    ctx = B.Context.for_cache(case.k, W.SCALE)
+    out, lse = _new(case)
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        B.sparrow_verify_attn(ctx, case.q, case.k, case.v, case.kv_len, case.parents, case.T, out, lse)   # warm-up
+    s.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=s):
+        B.sparrow_verify_attn(ctx, case.q, case.k, case.v, case.kv_len, case.parents, case.T, out, lse, stream=s)
+    ref = oracle_verify(case)
+    for _ in range(3):
+        out.fill_(float("nan")); lse.fill_(float("nan"))
+        g.replay()
+        torch.cuda.synchronize()
+        check(out, lse, *ref)
+    # ordinary calls after the replays still work on the same context
+    out2, lse2, _ = run_verify(case, ctx)
+    check(out2, lse2, *ref)
+
+
+def test_bounded_wait_gives_up_and_context_survives():
+    case = W.make_verify_case(630, [1500], 8, "chain", DEV)
+    ctx = B.Context.for_cache(case.k, W.SCALE)
+    out, lse, _ = run_verify(case, ctx)
+    B.sparrow_debug_wait_counter(ctx, 0)                  # everything it waits for has happened
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == 0
+    B.sparrow_debug_wait_counter(ctx, 5)                  # nothing will ever bump the counter that far
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == 7                  # SPARROW_ERR_TIMEOUT, then cleared
+    assert ctx.last_device_status() == 0
+    out2, lse2, _ = run_verify(case, ctx)
+    check(out2, lse2, *oracle_verify(case))
