@@ -157,6 +157,41 @@ sparrow_status sparrow_verify_step_host(sparrow_ctx* ctx, const void* q_host,
                                         const int32_t* parents_host, int32_t T, void* out_host,
                                         float* lse_host, void* stream);
 
+/* Verification attention without a context and without a caller-provided workspace.
+ * (The paper has no counterpart to this call; it exists for integration reasons only.)
+ *
+ * Who it is for: callers that are not allowed to allocate.  Some hosts own every byte of device
+ * memory themselves (a serving engine with a fixed pool, a plugin loaded into another framework)
+ * and forbid cudaMalloc in extension code; others run a latency-critical loop in which
+ * cudaMalloc's device-wide synchronisation, or its failure under fragmentation, is not
+ * acceptable.  sparrow_create / sparrow_set_workspace push that problem to the caller; this call
+ * removes it: the scratch memory (split-KV partials, status word) is a fixed array of
+ * SPARROW_STATIC_SCRATCH_BYTES that is part of the library's device image.  Every GPU that loads
+ * the library therefore holds that much memory until the process exits, whether or not the call
+ * is ever used.
+ *
+ * Arguments are those of sparrow_verify_attn(), with the layout passed by value of pointer in
+ * place of a context; the call works on the CURRENT device.  It calls no cudaMalloc / cudaFree
+ * and no allocating library routine, and keeps its bookkeeping in static host storage.
+ *   - First call on a device: one-time set-up (device query, kernel attributes, address of the
+ *     scratch array, clearing its header with a synchronising cudaMemset).  Make that first call
+ *     outside any stream capture.
+ *   - SPARROW_ERR_WORKSPACE when the layout / T need more scratch than the array holds (on a
+ *     148-SM part: blocks of more than 36 draft tokens, or large batches); nothing is launched then.
+ *   - The call always runs in the stream-ordered mode: two ordinary kernel launches on `stream`.
+ *   - All calls on a device share the one array, which keeps the previous call's contents.  What
+ *     must start clean (the status word) is cleared on `stream` at the start of every call;
+ *     partials are always written before they are read.  Calls that overlap on the GPU (two
+ *     streams without an event between them) race on the array and give undefined results; so do
+ *     concurrent calls from several host threads.
+ *   - Device-detected input problems (a parent index outside [-1, i)) are handled as everywhere
+ *     else (the node is treated as a root) but cannot be queried: there is no context to ask. */
+#define SPARROW_STATIC_SCRATCH_BYTES (16u * 1024u * 1024u)
+sparrow_status sparrow_verify_attn_static(const sparrow_layout* layout, const void* q, const void* k_cache,
+                                          const void* v_cache, const int32_t* kv_len,
+                                          const int32_t* parents, int32_t T, void* out, float* lse,
+                                          void* stream);
+
 /* Host helpers, exported so mask / index construction can be checked bit for bit.
  * Ancestor words of a draft tree (Section 4: dynamic draft trees): masks[i] has bit a set iff
  * a == i or a is an ancestor of i.  SPARROW_ERR_TREE unless -1 <= parents[i] < i. */

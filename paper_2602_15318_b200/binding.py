@@ -21,7 +21,7 @@ STATUS_NAMES = {0: "SPARROW_OK", 1: "SPARROW_ERR_NULL", 2: "SPARROW_ERR_SHAPE", 
 
 EXPORTS = ["sparrow_create", "sparrow_destroy", "sparrow_workspace_bytes", "sparrow_set_workspace",
            "sparrow_verify_attn", "sparrow_verify_attn_batch", "sparrow_anchor_attn",
-           "sparrow_verify_step_host",
+           "sparrow_verify_step_host", "sparrow_verify_attn_static",
            "sparrow_build_ancestor_masks", "sparrow_build_anchor_idx",
            "sparrow_debug_ancestor_masks_device", "sparrow_debug_wait_counter", "sparrow_plan_splits",
            "sparrow_last_device_status", "sparrow_launch_count", "sparrow_status_string"]
@@ -59,6 +59,7 @@ def lib():
         L.sparrow_set_workspace.argtypes = [vp, vp, ctypes.c_size_t]
         L.sparrow_verify_attn.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp, vp, vp]
         L.sparrow_verify_attn_batch.argtypes = [vp, vp, i32, vp]
+        L.sparrow_verify_attn_static.argtypes = [ctypes.POINTER(Layout), vp, vp, vp, vp, vp, i32, vp, vp, vp]
         L.sparrow_anchor_attn.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp]
         L.sparrow_verify_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp]
         L.sparrow_build_ancestor_masks.argtypes = [vp, i32, vp]
@@ -158,6 +159,18 @@ def sparrow_verify_attn(ctx: Context, q, k_cache, v_cache, kv_len: Sequence[int]
     kl = _i32_array(kv_len)
     _chk(lib().sparrow_verify_attn(ctx.handle, _ptr(q), _ptr(k_cache), _ptr(v_cache), kl, _ptr(parents),
                                    T, _ptr(out), _ptr(lse), _stream_handle(stream)), "sparrow_verify_attn")
+
+
+def sparrow_verify_attn_static(layout: Layout, q, k_cache, v_cache, kv_len: Sequence[int], parents, T: int,
+                               out, lse, stream=None):
+    """Verification attention for callers that may not allocate device memory (a host application
+    that owns the whole memory pool, or a loop that cannot afford cudaMalloc): no context, no
+    workspace -- the scratch is a fixed array inside the library.  Works on the current device;
+    calls sharing the device must not overlap on the GPU."""
+    kl = _i32_array(kv_len)
+    _chk(lib().sparrow_verify_attn_static(ctypes.byref(layout), _ptr(q), _ptr(k_cache), _ptr(v_cache), kl,
+                                          _ptr(parents), T, _ptr(out), _ptr(lse), _stream_handle(stream)),
+         "sparrow_verify_attn_static")
 
 
 class VerifyCall(ctypes.Structure):

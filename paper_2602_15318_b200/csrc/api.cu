@@ -479,6 +479,104 @@ sparrow_status sparrow_verify_attn(sparrow_ctx* c, const void* q, const void* k,
     return sy.enabled ? SPARROW_OK : launch_combine(c, plan, sy, out, lse, st);    // fused mode combines in the kernel
 }
 
+}  // extern "C"  (closed for the file-scope objects of the no-allocation entry point)
+
+// Scratch of sparrow_verify_attn_static(): part of the device image, one copy per GPU that loads
+// the library.  In host code this name is only a handle for cudaGetSymbolAddress().
+static __device__ __align__(256) unsigned char g_static_scratch[SPARROW_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxStaticDevices = 16;
+struct StaticSlot {
+    bool ready;
+    sparrow_ctx ctx;
+};
+StaticSlot g_static_slots[kMaxStaticDevices];      // static storage: no heap behind the entry point
+
+bool same_layout(const sparrow_layout& a, const sparrow_layout& b)
+{
+    return a.batch == b.batch && a.n_q_heads == b.n_q_heads && a.n_kv_heads == b.n_kv_heads && a.head_dim == b.head_dim &&
+           a.kv_capacity == b.kv_capacity && a.softmax_scale == b.softmax_scale &&
+           a.kv_stride_batch == b.kv_stride_batch && a.kv_stride_head == b.kv_stride_head;
+}
+}  // namespace
+
+extern "C" {
+
+sparrow_status sparrow_verify_attn_static(const sparrow_layout* L, const void* q, const void* k, const void* v,
+                                          const int32_t* kv_len, const int32_t* parents, int32_t T, void* out,
+                                          float* lse, void* stream)
+{
+    if (!L) return SPARROW_ERR_NULL;
+    if (L->batch < 1 || L->batch > kMaxBatch || L->head_dim != kD || L->n_kv_heads < 1 ||
+        L->n_q_heads != kGroup * L->n_kv_heads || L->kv_capacity < 1 ||
+        !(L->softmax_scale > 0.f) || !std::isfinite(L->softmax_scale) ||
+        L->kv_stride_head < (int64_t)L->kv_capacity * kD || (L->kv_stride_head % 8) != 0 ||
+        (L->kv_stride_batch % 8) != 0 ||
+        (L->batch > 1 && L->kv_stride_batch < L->kv_stride_head * (int64_t)L->n_kv_heads))
+        return SPARROW_ERR_SHAPE;
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess) { cudaGetLastError(); return SPARROW_ERR_CUDA; }
+    if (device < 0 || device >= kMaxStaticDevices) return SPARROW_ERR_SHAPE;
+    StaticSlot& slot = g_static_slots[device];
+    sparrow_ctx* c = &slot.ctx;
+    if (!slot.ready) {
+        // one-time set-up for this device (it is the current one)
+        cudaDeviceProp prop;
+        if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return SPARROW_ERR_CUDA;
+        if (prop.major != 10) return SPARROW_ERR_ARCH;
+        if (cudaFuncSetAttribute(gather::split_gather_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 gather::kSmemBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(tc::verify_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 tc::smem_bytes(1, 3)) != cudaSuccess ||
+            cudaFuncSetAttribute(tc::verify_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 tc::smem_bytes(2, 2)) != cudaSuccess)
+            return SPARROW_ERR_CUDA;
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess || !fn)
+            return SPARROW_ERR_CUDA;
+        void* scratch = nullptr;               // the array's device address on THIS device
+        if (cudaGetSymbolAddress(&scratch, g_static_scratch) != cudaSuccess || !scratch) return SPARROW_ERR_CUDA;
+        if (cudaMemset(scratch, 0, kStatusBytes) != cudaSuccess) return SPARROW_ERR_CUDA;
+        c->n_maps = 0;
+        c->next_evict = 0;
+        c->encode = reinterpret_cast<TensorMapEncodeFn>(fn);
+        c->verify_on_gather = false;
+        c->layout = *L;
+        c->device = device;
+        c->n_sm = prop.multiProcessorCount;
+        c->ws = static_cast<unsigned char*>(scratch);
+        c->ws_bytes = SPARROW_STATIC_SCRATCH_BYTES;
+        c->launches.store(0);
+        c->use_pdl = false;                    // stream-ordered mode: no counters live in the shared array
+        c->seq = 0;
+        c->fin_total[0] = c->fin_total[1] = 0;
+        slot.ready = true;
+    }
+    if (!same_layout(c->layout, *L)) {         // tensor maps depend on the layout
+        c->layout = *L;
+        c->n_maps = 0;
+        c->next_evict = 0;
+    }
+    if (T >= 1 && T <= kMaxT && kv_len) {      // refuse what does not fit the array before touching the GPU
+        int32_t n_keys[kMaxBatch];
+        bool lens_ok = true;
+        for (int b = 0; b < L->batch; ++b) {
+            lens_ok = lens_ok && kv_len[b] >= 0 && (int64_t)kv_len[b] + T <= L->kv_capacity;
+            n_keys[b] = kv_len[b] + T;
+        }
+        SplitPlan plan;
+        if (lens_ok && make_plan(c->n_sm, L->batch, L->n_kv_heads, n_keys, T, blocks_per_group_tc(T), &plan) == SPARROW_OK &&
+            check_ws(c, plan) != SPARROW_OK)
+            return SPARROW_ERR_WORKSPACE;
+    }
+    // the status word is the one thing that must start clean
+    if (cudaMemsetAsync(c->ws, 0, sizeof(unsigned), static_cast<cudaStream_t>(stream)) != cudaSuccess) return SPARROW_ERR_CUDA;
+    return sparrow_verify_attn(c, q, k, v, kv_len, parents, T, out, lse, stream);
+}
+
 sparrow_status sparrow_verify_attn_batch(sparrow_ctx* c, const sparrow_verify_call* calls, int32_t n_calls, void* stream)
 {
     if (!c || !calls) return SPARROW_ERR_NULL;
