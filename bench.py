@@ -192,6 +192,23 @@ def time_calls(ctx, batch, n_steps, B, torch):
     return start.elapsed_time(stop) * 1e3 / n_steps          # us per call
 
 
+def time_isolated_calls(ctx, cases, outs, lses, n_calls, B, torch):
+    """Latency of one call on an idle GPU: every call is bracketed by its own pair of events and
+    the stream is drained before the next one, so nothing overlaps.  Returns the median in us."""
+    singles = [B.VerifyBatch([(c.q, c.k, c.v, c.kv_len, c.parents, c.T, o, l)]) for c, o, l in zip(cases, outs, lses)]
+    times = []
+    for i in range(n_calls):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        B.sparrow_verify_attn_batch(ctx, singles[i % len(singles)])
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1) * 1e3)
+    times.sort()
+    return times[len(times) // 2]
+
+
 def build_rotation(W, B, torch, dev, cfg_index, n_caches):
     """R distinct (q, K, V) sets of one configuration, one context sized for them."""
     cases = [W.make_config(cfg_index, dev, layer=r) for r in range(n_caches)]
@@ -262,6 +279,9 @@ def main():
     clocks = sampler.stop()
     us_call = max_over_ranks(us_call, dist, dev)
 
+    # -- latency of an isolated call (cold cache: the rotation continues) ------------------------
+    us_isolated = time_isolated_calls(ctx, cases, outs, lses, 300, B, torch)
+
     # -- L2-warm figure (one cache, labelled as such) --------------------------------------------
     warm = B.VerifyBatch([(cases[0].q, cases[0].k, cases[0].v, cases[0].kv_len, cases[0].parents,
                            cases[0].T, outs[0], lses[0])])
@@ -315,6 +335,7 @@ def main():
         "hbm_gbs_per_call": alg_bytes / (us_call * 1e-6) / 1e9,
         "pct_of_8tbs_nominal": 100.0 * alg_bytes / (us_call * 1e-6) / 8e12,
         "tflops_per_call": flops / (us_call * 1e-6) / 1e12,
+        "us_per_call_isolated": us_isolated,
         "us_per_call_l2_warm": us_warm,
         "calls_per_s_all_gpus": world * 1e6 / us_call,
         "roofline": {"bound": "hbm", "kernel": "verify_tc_kernel<1> (the only kernel of a step: split-KV pass with the combine "

@@ -41,6 +41,7 @@ struct sparrow_ctx {
     sparrow_layout layout;
     int device;
     int n_sm;
+    int target_items;                        // work items the split plan aims for (<= n_sm)
     unsigned char* ws;
     size_t ws_bytes;
     std::atomic<long long> launches;
@@ -390,6 +391,11 @@ sparrow_status sparrow_create(sparrow_ctx** out, const sparrow_layout* L, int de
     c->layout = *L;
     c->device = device;
     c->n_sm = prop.multiProcessorCount;
+    c->target_items = c->n_sm;
+    if (const char* ti = std::getenv("SPARROW_TARGET_ITEMS")) {
+        const int v = std::atoi(ti);
+        if (v >= 1 && v <= c->n_sm) c->target_items = v;
+    }
     c->ws = nullptr;
     c->ws_bytes = 0;
     c->launches.store(0);
@@ -464,7 +470,7 @@ sparrow_status sparrow_verify_attn(sparrow_ctx* c, const void* q, const void* k,
     }
     SplitPlan plan;
     const int nb = c->verify_on_gather ? 1 : blocks_per_group_tc(T);
-    sparrow_status s = make_plan(c->n_sm, c->layout.batch, c->layout.n_kv_heads, n_keys, T, nb, &plan);
+    sparrow_status s = make_plan(c->target_items, c->layout.batch, c->layout.n_kv_heads, n_keys, T, nb, &plan);
     if (s != SPARROW_OK) return s;
     for (int b = 0; b < c->layout.batch; ++b) plan.seq[b].kv_len = kv_len[b];
     if ((s = check_ws(c, plan)) != SPARROW_OK) return s;
@@ -547,6 +553,7 @@ sparrow_status sparrow_verify_attn_static(const sparrow_layout* L, const void* q
         c->layout = *L;
         c->device = device;
         c->n_sm = prop.multiProcessorCount;
+        c->target_items = c->n_sm;
         c->ws = static_cast<unsigned char*>(scratch);
         c->ws_bytes = SPARROW_STATIC_SCRATCH_BYTES;
         c->launches.store(0);
@@ -568,7 +575,7 @@ sparrow_status sparrow_verify_attn_static(const sparrow_layout* L, const void* q
             n_keys[b] = kv_len[b] + T;
         }
         SplitPlan plan;
-        if (lens_ok && make_plan(c->n_sm, L->batch, L->n_kv_heads, n_keys, T, blocks_per_group_tc(T), &plan) == SPARROW_OK &&
+        if (lens_ok && make_plan(c->target_items, L->batch, L->n_kv_heads, n_keys, T, blocks_per_group_tc(T), &plan) == SPARROW_OK &&
             check_ws(c, plan) != SPARROW_OK)
             return SPARROW_ERR_WORKSPACE;
     }
@@ -600,7 +607,7 @@ sparrow_status sparrow_anchor_attn(sparrow_ctx* c, const void* q, const void* k,
     int32_t n_keys[kMaxBatch];
     for (int b = 0; b < c->layout.batch; ++b) n_keys[b] = n_anchor;
     SplitPlan plan;
-    sparrow_status s = make_plan(c->n_sm, c->layout.batch, c->layout.n_kv_heads, n_keys, T, 1, &plan);
+    sparrow_status s = make_plan(c->target_items, c->layout.batch, c->layout.n_kv_heads, n_keys, T, 1, &plan);
     if (s != SPARROW_OK) return s;
     if ((s = check_ws(c, plan)) != SPARROW_OK) return s;
     DeviceGuard guard(c->device);
