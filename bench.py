@@ -272,11 +272,20 @@ def main():
     sampler = ClockSampler(local_rank)
     barrier()
     sampler.start()
+    t_sample = time.perf_counter()
     launches_before = ctx.launch_count()
     us_call = time_calls(ctx, batch, steps, B, torch)
     launches_timed = ctx.launch_count() - launches_before
     barrier()
+    # nvidia-smi needs a second or so to deliver samples: a short timed region is followed by an
+    # untimed continuation of the same launches, so that the clocks are still read under this load
+    continued = 0
+    while time.perf_counter() - t_sample < 1.5:
+        time_calls(ctx, batch, 2000, B, torch)
+        continued += 2000
     clocks = sampler.stop()
+    if continued:
+        clocks["note"] = f"timed region shorter than the sampling period: {continued} more untimed calls of the same workload kept the load up while sampling"
     us_call = max_over_ranks(us_call, dist, dev)
 
     # -- latency of an isolated call (cold cache: the rotation continues) ------------------------
@@ -317,7 +326,7 @@ def main():
     us_e2e = max_over_ranks(us_e2e, dist, dev)
     status = ctx.last_device_status()
     if status != 0:
-        raise SystemExit(f"device status {status} after the timed region")
+        raise SystemExit(f"device status {status} (word {ctx.status_word():#x}) after the timed region")
 
     peak, peak_kind, peaks = measured_peaks()
     alg_bytes = kv_bytes + io_bytes

@@ -227,6 +227,14 @@ sparrow_status sparrow_debug_wait_counter(sparrow_ctx* ctx, uint32_t ahead, void
  * SPARROW_ERR_ANCHOR or SPARROW_ERR_TIMEOUT) and clears it.  Not for the hot path. */
 sparrow_status sparrow_last_device_status(sparrow_ctx* ctx, void* stream);
 
+/* The raw status word that the most recent sparrow_last_device_status() call on this context read
+ * (0 before the first call).  Bits 0..2: malformed tree, bad anchor, timeout.  A wait that gave up
+ * also sets bit 8 + site: 0 TMA producer, 1 MMA issuer, 2 softmax warps, 3 / 4 the waits in front
+ * of a CTA's first global write (same / other call parity), 5 finisher waiting for the call's
+ * pieces, 6 finisher waiting for the previous call, 7 finisher's bulk copies, 8 the debug wait.
+ * For diagnosis only. */
+uint32_t sparrow_debug_status_word(const sparrow_ctx* ctx);
+
 /* Number of kernels the library has launched through this context (for launch accounting). */
 int64_t sparrow_launch_count(const sparrow_ctx* ctx);
 

@@ -24,7 +24,8 @@ EXPORTS = ["sparrow_create", "sparrow_destroy", "sparrow_workspace_bytes", "spar
            "sparrow_verify_step_host", "sparrow_verify_attn_static",
            "sparrow_build_ancestor_masks", "sparrow_build_anchor_idx",
            "sparrow_debug_ancestor_masks_device", "sparrow_debug_wait_counter", "sparrow_plan_splits",
-           "sparrow_last_device_status", "sparrow_launch_count", "sparrow_status_string"]
+           "sparrow_last_device_status", "sparrow_debug_status_word", "sparrow_launch_count",
+           "sparrow_status_string"]
 
 
 class SparrowError(RuntimeError):
@@ -68,12 +69,15 @@ def lib():
         L.sparrow_debug_wait_counter.argtypes = [vp, ctypes.c_uint32, vp]
         L.sparrow_plan_splits.argtypes = [i32, i32, i32, vp, i32, vp, vp]
         L.sparrow_last_device_status.argtypes = [vp, vp]
+        L.sparrow_debug_status_word.argtypes = [vp]
+        L.sparrow_debug_status_word.restype = ctypes.c_uint32
         L.sparrow_launch_count.argtypes = [vp]
         L.sparrow_launch_count.restype = i64
         L.sparrow_status_string.argtypes = [ctypes.c_int]
         L.sparrow_status_string.restype = ctypes.c_char_p
         for name in EXPORTS:
-            if name not in ("sparrow_workspace_bytes", "sparrow_launch_count", "sparrow_status_string"):
+            if name not in ("sparrow_workspace_bytes", "sparrow_launch_count", "sparrow_status_string",
+                            "sparrow_debug_status_word"):
                 getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -139,6 +143,10 @@ class Context:
 
     def last_device_status(self, stream=None) -> int:
         return int(lib().sparrow_last_device_status(self.handle, _stream_handle(stream)))
+
+    def status_word(self) -> int:
+        """Raw status word read by the last last_device_status() call (wait-site bits above bit 8)."""
+        return int(lib().sparrow_debug_status_word(self.handle))
 
     def close(self):
         if self.handle:

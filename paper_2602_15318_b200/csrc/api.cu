@@ -50,6 +50,7 @@ struct sparrow_ctx {
     // of the fused calls and, per call parity, the cumulative number of finishers launched so far.
     uint32_t seq;
     uint32_t fin_total[2];
+    uint32_t last_status_word;   // raw word read by the last sparrow_last_device_status()
 };
 
 namespace {
@@ -307,7 +308,7 @@ __global__ void ancestor_masks_kernel(const int32_t* parents, int T, unsigned lo
 // One thread waits (bounded) on a finisher counter; see sparrow_debug_wait_counter().
 __global__ void wait_counter_kernel(const unsigned* counter, unsigned target, unsigned* status)
 {
-    if (!wait_counter(counter, target)) atomicOr(status, kStatTimeout);
+    if (!wait_counter(counter, target)) atomicOr(status, timeout_bits(kSiteDebug));
 }
 
 struct DeviceGuard {
@@ -403,6 +404,7 @@ sparrow_status sparrow_create(sparrow_ctx** out, const sparrow_layout* L, int de
     c->use_pdl = !(e && e[0] == '1');
     c->seq = 0;
     c->fin_total[0] = c->fin_total[1] = 0;
+    c->last_status_word = 0;
     *out = c;
     return SPARROW_OK;
 }
@@ -560,6 +562,7 @@ sparrow_status sparrow_verify_attn_static(const sparrow_layout* L, const void* q
         c->use_pdl = false;                    // stream-ordered mode: no counters live in the shared array
         c->seq = 0;
         c->fin_total[0] = c->fin_total[1] = 0;
+        c->last_status_word = 0;
         slot.ready = true;
     }
     if (!same_layout(c->layout, *L)) {         // tensor maps depend on the layout
@@ -742,11 +745,14 @@ sparrow_status sparrow_last_device_status(sparrow_ctx* c, void* stream)
     if (cudaMemcpyAsync(&word, c->ws, sizeof word, cudaMemcpyDeviceToHost, st) != cudaSuccess) return SPARROW_ERR_CUDA;
     if (cudaMemsetAsync(c->ws, 0, sizeof word, st) != cudaSuccess) return SPARROW_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return SPARROW_ERR_CUDA;
+    c->last_status_word = word;
     if (word & kStatTimeout) return SPARROW_ERR_TIMEOUT;
     if (word & kStatTree) return SPARROW_ERR_TREE;
     if (word & kStatAnchor) return SPARROW_ERR_ANCHOR;
     return SPARROW_OK;
 }
+
+uint32_t sparrow_debug_status_word(const sparrow_ctx* c) { return c ? c->last_status_word : 0u; }
 
 int64_t sparrow_launch_count(const sparrow_ctx* c) { return c ? (int64_t)c->launches.load() : 0; }
 

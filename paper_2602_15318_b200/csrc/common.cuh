@@ -18,6 +18,10 @@ constexpr int kBlockRows = 128;
 constexpr unsigned kStatTree = 1u;
 constexpr unsigned kStatAnchor = 2u;
 constexpr unsigned kStatTimeout = 4u;
+// A wait that gives up also sets bit (8 + site) of the status word, so that the raw word tells which wait it was.
+__host__ __device__ constexpr unsigned timeout_bits(int site) { return kStatTimeout | (1u << (8 + site)); }
+enum WaitSite { kSiteProducer = 0, kSiteMma = 1, kSiteSoftmax = 2, kSiteWriteSame = 3, kSiteWriteOther = 4,
+                kSiteArrivals = 5, kSiteFinOther = 6, kSiteFinCopies = 7, kSiteDebug = 8 };
 
 // The GQA group's 7 query heads x T draft tokens are packed into 128-row blocks: block i holds
 // tokens [18 i, 18 i + 18), row r of a block is (token 18 i + r / 7, head r % 7), rows 126 and 127
@@ -89,38 +93,35 @@ struct SyncArgs {
     uint32_t fin_wait_other;
 };
 
-__device__ __forceinline__ unsigned long long global_timer_ns()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
 __device__ __forceinline__ unsigned ld_acquire(const unsigned* addr)
 {
     unsigned v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(addr) : "memory");
     return v;
 }
+// Polls of a counter wait before it gives up: with the pause between polls this is of the order of
+// a second.  The bound counts polls rather than reading a timer, so it cannot misfire on a timer
+// glitch and does not depend on the timer's resolution.
+constexpr uint32_t kCounterPolls = 1u << 22;
 // Bounded acquire-wait until a cumulative counter has reached `target` (wrap-safe compare).
-// Gives up after about one second and returns false.
 __device__ __forceinline__ bool wait_counter(const unsigned* addr, uint32_t target)
 {
-    const unsigned long long t0 = global_timer_ns();
-    for (;;) {
+    #pragma unroll 1
+    for (uint32_t i = 0; i < kCounterPolls; ++i) {
         if ((int32_t)(ld_acquire(addr) - target) >= 0) return true;
-        if (global_timer_ns() - t0 > 1000000000ull) return false;
-        __nanosleep(100);
+        __nanosleep(i < 64 ? 40 : 200);
     }
+    return false;
 }
 // Bounded acquire-wait until a word equals `value`.
 __device__ __forceinline__ bool wait_equal(const unsigned* addr, uint32_t value)
 {
-    const unsigned long long t0 = global_timer_ns();
-    for (;;) {
+    #pragma unroll 1
+    for (uint32_t i = 0; i < kCounterPolls; ++i) {
         if (ld_acquire(addr) == value) return true;
-        if (global_timer_ns() - t0 > 1000000000ull) return false;
-        __nanosleep(100);
+        __nanosleep(i < 64 ? 40 : 200);
     }
+    return false;
 }
 // Release-increment of a counter: orders every write this thread has observed (its own and, after
 // a CTA barrier, its CTA's) before the increment.

@@ -411,7 +411,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                 if (jk < n_tiles && mbar_try_wait(B.k_empty(jk % NS), (jk / NS - 1) & 1)) { issue_k(jk); ++jk; progress = true; }
                 if (jv < n_tiles && mbar_try_wait(B.v_empty(jv % NS), (jv / NS - 1) & 1)) { issue_v(jv); ++jv; progress = true; }
                 if (progress) idle = 0;
-                else if (++idle > kSpinLimit) { atomicOr(args.status, kStatTimeout); *abort_flag = 1; break; }
+                else if (++idle > kSpinLimit) { atomicOr(args.status, timeout_bits(kSiteProducer)); *abort_flag = 1; break; }
             }
         }
     } else if (warp == kMmaWarp) {
@@ -458,7 +458,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                 if (blk == NB - 1) tc_commit(B.v_empty(st));
                 if (n + NSB < n_jobs) ok = issue_qk(n + NSB);             // its S block was job n's
             }
-            if (!ok) { atomicOr(args.status, kStatTimeout); *abort_flag = 1; }
+            if (!ok) { atomicOr(args.status, timeout_bits(kSiteMma)); *abort_flag = 1; }
         }
     } else if (warp < 8) {
         // ================= softmax =================
@@ -474,7 +474,8 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
         float m_ref[NB], l_run[NB];
         // Phases of o_done[blk] observed so far.  A parity wait is only meaningful for the phase in
         // progress or the one just completed, and the softmax runs ahead of the P V products, so
-        // every job ends by observing the previous job's phase: o_seen never lags by more than one.
+        // every job observes the previous job's phase before it releases its own P (which the next
+        // phase needs): o_seen never lags the barrier by more than one phase.
         int o_seen[NB];
         #pragma unroll
         for (int blk = 0; blk < NB; ++blk) {
@@ -571,11 +572,14 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                 exp_chunk(x0, c2, mc, sum4, p_addr);
                 exp_chunk(x1, c2, mc, sum4, p_addr + 16);
                 l_run[blk] += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+                // Observe the previous tile's P V (long done) BEFORE handing over this tile's P: the
+                // next phase of o_done cannot complete without this warp's arrival below, so the
+                // barrier never gets two phases ahead of a warp that has yet to look at it.
+                for (; ok && o_seen[blk] < j; ++o_seen[blk]) ok = mbar_wait_warp(B.o_done(blk), o_seen[blk] & 1);
+                if (!ok) break;
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(B.p_full(sb));
-                for (; ok && o_seen[blk] < j; ++o_seen[blk]) ok = mbar_wait_warp(B.o_done(blk), o_seen[blk] & 1);   // previous tile's P V, long done
-                if (!ok) break;
             }
         }
 
@@ -587,8 +591,11 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
             bool go = true;
             if (sync.enabled) {
                 go = wait_counter(sync.fin_done + sync.parity, sync.fin_wait_same);
-                if (go && direct) go = wait_counter(sync.fin_done + (sync.parity ^ 1), sync.fin_wait_other);
-                if (!go) atomicOr(args.status, kStatTimeout);
+                if (!go) atomicOr(args.status, timeout_bits(kSiteWriteSame));
+                if (go && direct) {
+                    go = wait_counter(sync.fin_done + (sync.parity ^ 1), sync.fin_wait_other);
+                    if (!go) atomicOr(args.status, timeout_bits(kSiteWriteOther));
+                }
                 if (go && blockIdx.x == 0) sync.arrivals[(sync.slot + 2) & 3] = 0u;   // the call after next: unused by now
             }
             *write_ok = go ? 1u : 0u;
@@ -665,9 +672,12 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                 if (!direct) publish_counter(sync.arrivals + sync.slot);
                 if (fin_idx >= 0) {
                     // every partial of the call in place, and the previous call's final results written
-                    const bool go = wait_equal(sync.arrivals + sync.slot, (unsigned)sync.n_arrive) &&
-                                    wait_counter(sync.fin_done + (sync.parity ^ 1), sync.fin_wait_other);
-                    if (!go) atomicOr(args.status, kStatTimeout);
+                    bool go = wait_equal(sync.arrivals + sync.slot, (unsigned)sync.n_arrive);
+                    if (!go) atomicOr(args.status, timeout_bits(kSiteArrivals));
+                    if (go) {
+                        go = wait_counter(sync.fin_done + (sync.parity ^ 1), sync.fin_wait_other);
+                        if (!go) atomicOr(args.status, timeout_bits(kSiteFinOther));
+                    }
                     *fin_go = go ? 1 : 0;
                 }
             }
@@ -681,10 +691,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                     // there, one warp per row, lane l owning output dims [4 l, 4 l + 4).
                     constexpr int kRowsPerBlock = kTokPerBlock * kGroup;       // 126
                     constexpr int kRowBytes = kPartRowHalves * 2;              // 272
-                    constexpr int kMaxPieces = 256;                            // pieces per unit (<= SMs)
-                    constexpr int kBatchRowsMax = 32;                          // rows merged at once
-                    constexpr int kWtsBytes = kBatchRowsMax * kMaxPieces * 4;  // their piece weights, at the end of the ring
-                    float* wts = reinterpret_cast<float*>(kv_sm + NS * kStageBytes - kWtsBytes);
+                    constexpr int kBatchRowsMax = 64;                          // rows merged at once
                     const int list_len = NB * kRowsPerBlock;                   // rows per unit
                     int n_units = 0;
                     for (int b = 0; b < plan.batch; ++b)
@@ -698,7 +705,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                     for (int b = 0; b < plan.batch; ++b) {
                         const int ns = plan.seq[b].n_splits;
                         if (ns == 1) continue;
-                        int batch_rows = (NS * kStageBytes - kWtsBytes) / (ns * kRowBytes);    // rows whose pieces fit the ring at once
+                        int batch_rows = (NS * kStageBytes) / (ns * kRowBytes);    // rows whose pieces fit the ring at once
                         if (batch_rows > kBatchRowsMax) batch_rows = kBatchRowsMax;
                         #pragma unroll 1
                         for (int u = 0; u < plan.n_kv_heads * plan.n_groups; ++u, ubase += list_len) {
@@ -724,33 +731,10 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                                                   (uint32_t)(r0 + n_here - split) * kRowBytes, B.fin());
                                 }
                                 fin_ok = fin_ok && mbar_wait_warp(B.fin(), phase);
-                                // (a) weights: one warp per row -- LSE = log sum exp(lse_s); w[row][s] = exp(lse_s - LSE)
-                                #pragma unroll 1
-                                for (int i = warp; i < n_here && fin_ok; i += 8) {
-                                    const int idx = r0 + i;
-                                    const int bk = idx / kRowsPerBlock, r = idx - bk * kRowsPerBlock;
-                                    const int t = (grp * NB + bk) * kTokPerBlock + r / kGroup;
-                                    const uint32_t pstride = (uint32_t)n_here * kRowBytes;             // bytes between pieces
-                                    const unsigned char* lse0 = kv_sm + (uint32_t)i * kRowBytes + 2 * kD + lane * pstride;
-                                    float mxl = -INFINITY;
-                                    for (uint32_t sp = lane, off = 0; sp < (uint32_t)ns; sp += 32, off += 32 * pstride)
-                                        mxl = fmaxf(mxl, *reinterpret_cast<const float*>(lse0 + off));
-                                    #pragma unroll
-                                    for (int d = 16; d > 0; d >>= 1) mxl = fmaxf(mxl, __shfl_xor_sync(0xffffffffu, mxl, d));
-                                    const bool any = mxl != -INFINITY;
-                                    float suml = 0.f;
-                                    for (uint32_t sp = lane, off = 0; sp < (uint32_t)ns; sp += 32, off += 32 * pstride)
-                                        suml += any ? __expf(*reinterpret_cast<const float*>(lse0 + off) - mxl) : 0.f;
-                                    #pragma unroll
-                                    for (int d = 16; d > 0; d >>= 1) suml += __shfl_xor_sync(0xffffffffu, suml, d);
-                                    const float total_lse = any ? mxl + logf(suml) : -INFINITY;
-                                    for (uint32_t sp = lane, off = 0; sp < (uint32_t)ns; sp += 32, off += 32 * pstride)
-                                        wts[i * kMaxPieces + sp] = any ? __expf(*reinterpret_cast<const float*>(lse0 + off) - total_lse) : 0.f;
-                                    if (lane == 0 && t < T)
-                                        args.lse[((size_t)b * args.n_q_heads + kvh * kGroup + r % kGroup) * T + t] = total_lse;
-                                }
-                                softmax_bar_sync();
-                                // (b) outputs: one thread per (row, 8 output dims), all rows of the batch at once
+                                // One thread per (row, 8 output dims), all rows of the batch at once.  Every
+                                // thread of a row scans the row's piece LSEs itself (broadcast reads): a first
+                                // pass for the maximum, a second that accumulates exp(lse_s - max) and the
+                                // weighted outputs; normalising by the sum at the end gives the merged row.
                                 #pragma unroll 1
                                 for (int e = tid; e < n_here * 16 && fin_ok; e += 256) {
                                     const int i = e >> 4, c = e & 15;
@@ -758,30 +742,40 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                                     const int bk = idx / kRowsPerBlock, r = idx - bk * kRowsPerBlock;
                                     const int t = (grp * NB + bk) * kTokPerBlock + r / kGroup;
                                     if (t >= T) continue;
-                                    const uint32_t pstride = (uint32_t)n_here * kRowBytes;
-                                    const unsigned char* src = kv_sm + (uint32_t)i * kRowBytes + c * 16;
-                                    const float* w = wts + i * kMaxPieces;
-                                    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                                    const uint32_t pstride = (uint32_t)n_here * kRowBytes;     // bytes between pieces
+                                    const unsigned char* row0 = kv_sm + (uint32_t)i * kRowBytes;
+                                    float mxl = -INFINITY;
                                     #pragma unroll 4
-                                    for (int sp = 0; sp < ns; ++sp, src += pstride) {
-                                        const uint4 raw = *reinterpret_cast<const uint4*>(src);
-                                        const float ws = w[sp];
+                                    for (uint32_t sp = 0, off = 2 * kD; sp < (uint32_t)ns; ++sp, off += pstride)
+                                        mxl = fmaxf(mxl, *reinterpret_cast<const float*>(row0 + off));
+                                    const bool any = mxl != -INFINITY;
+                                    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                                    float suml = 0.f;
+                                    const unsigned char* src = row0 + c * 16;
+                                    #pragma unroll 2
+                                    for (uint32_t sp = 0, off = 0; sp < (uint32_t)ns; ++sp, off += pstride) {
+                                        const float ws = any ? __expf(*reinterpret_cast<const float*>(row0 + off + 2 * kD) - mxl) : 0.f;
+                                        const uint4 raw = *reinterpret_cast<const uint4*>(src + off);
                                         const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
+                                        suml += ws;
                                         #pragma unroll
                                         for (int q = 0; q < 4; ++q) {
                                             const float2 f = __half22float2(h2[q]);
                                             acc[2 * q] = fmaf(ws, f.x, acc[2 * q]); acc[2 * q + 1] = fmaf(ws, f.y, acc[2 * q + 1]);
                                         }
                                     }
+                                    const float inv = any ? 1.f / suml : 0.f;
+                                    const int h = kvh * kGroup + r % kGroup;
                                     uint4 pk;
-                                    pk.x = pack_bf16x2(acc[0], acc[1]); pk.y = pack_bf16x2(acc[2], acc[3]);
-                                    pk.z = pack_bf16x2(acc[4], acc[5]); pk.w = pack_bf16x2(acc[6], acc[7]);
-                                    *reinterpret_cast<uint4*>(args.out + (((size_t)b * T + t) * args.n_q_heads + kvh * kGroup + r % kGroup) * kD + c * 8) = pk;
+                                    pk.x = pack_bf16x2(acc[0] * inv, acc[1] * inv); pk.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
+                                    pk.z = pack_bf16x2(acc[4] * inv, acc[5] * inv); pk.w = pack_bf16x2(acc[6] * inv, acc[7] * inv);
+                                    *reinterpret_cast<uint4*>(args.out + (((size_t)b * T + t) * args.n_q_heads + h) * kD + c * 8) = pk;
+                                    if (c == 0) args.lse[((size_t)b * args.n_q_heads + h) * T + t] = any ? mxl + logf(suml) : -INFINITY;
                                 }
                             }
                         }
                     }
-                    if (!fin_ok) atomicOr(args.status, kStatTimeout);
+                    if (!fin_ok) atomicOr(args.status, timeout_bits(kSiteFinCopies));
                 }
                 softmax_bar_sync();
             }
@@ -790,7 +784,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                 if (fin_idx >= 0) publish_counter(sync.fin_done + sync.parity);
             }
         }
-        if (!ok) { atomicOr(args.status, kStatTimeout); *abort_flag = 1; }
+        if (!ok) { atomicOr(args.status, timeout_bits(kSiteSoftmax)); *abort_flag = 1; }
     }
 
     // ---- teardown -------------------------------------------------------------------------------
