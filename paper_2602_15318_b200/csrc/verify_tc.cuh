@@ -104,6 +104,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+// Non-blocking probe of a phase.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
 // Bounded wait: false when the phase did not complete within kSpinLimit polls.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
 {
@@ -291,15 +302,24 @@ __device__ __forceinline__ bool softmax_bar_or(bool pred)
 // only after its last O += P V, so the K stream runs ahead of the V stream.
 struct Bars {
     uint32_t base;
+    // at most 3 stages and 3 S blocks: 28 slots in all
     __device__ __forceinline__ uint32_t k_full(int i) const { return base + 8u * (uint32_t)i; }
-    __device__ __forceinline__ uint32_t k_empty(int i) const { return base + 32u + 8u * (uint32_t)i; }
-    __device__ __forceinline__ uint32_t v_full(int i) const { return base + 64u + 8u * (uint32_t)i; }
-    __device__ __forceinline__ uint32_t v_empty(int i) const { return base + 96u + 8u * (uint32_t)i; }
-    __device__ __forceinline__ uint32_t s_full(int i) const { return base + 128u + 8u * (uint32_t)i; }   // <= 4 S blocks
-    __device__ __forceinline__ uint32_t p_full(int i) const { return base + 160u + 8u * (uint32_t)i; }
-    __device__ __forceinline__ uint32_t o_done(int i) const { return base + 192u + 8u * (uint32_t)i; }   // per row block
-    __device__ __forceinline__ uint32_t q_full() const { return base + 208u; }
-    __device__ __forceinline__ uint32_t fin() const { return base + 216u; }       // finishers' bulk copies
+    __device__ __forceinline__ uint32_t k_empty(int i) const { return base + 24u + 8u * (uint32_t)i; }
+    __device__ __forceinline__ uint32_t v_full(int i) const { return base + 48u + 8u * (uint32_t)i; }
+    __device__ __forceinline__ uint32_t v_empty(int i) const { return base + 72u + 8u * (uint32_t)i; }
+    __device__ __forceinline__ uint32_t s_full(int i) const { return base + 96u + 8u * (uint32_t)i; }
+    __device__ __forceinline__ uint32_t p_full(int i) const { return base + 120u + 8u * (uint32_t)i; }
+    __device__ __forceinline__ uint32_t q_full() const { return base + 144u; }
+    __device__ __forceinline__ uint32_t fin() const { return base + 152u; }       // finishers' bulk copies
+    // Completion of O += P V of key tile j on row block blk: a ring of four barriers per block,
+    // tile j on barrier j % 4 with phase parity (j / 4) & 1.  The softmax only looks at it when a
+    // row maximum moves and in the epilogue, asking for tile j - 1 while it works on tile j.  A
+    // parity wait is only meaningful for the phase in progress or the one just completed; here the
+    // barrier is in exactly that state: its previous use (tile j - 5) completed before the scores
+    // of tile j, which the warp has seen (the tensor pipe completes in issue order and the scores
+    // of tile j were issued after the product of tile j - 3), and its next use (tile j + 3) needs
+    // this warp's P of that tile.
+    __device__ __forceinline__ uint32_t o_done(int blk, int j) const { return base + 160u + 32u * (uint32_t)blk + 8u * (uint32_t)(j & 3); }
 };
 
 template <int NB>
@@ -361,11 +381,11 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_q) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_k) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_v) : "memory");
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < 3; ++i) {
             mbar_init(B.k_full(i), 1); mbar_init(B.k_empty(i), 1); mbar_init(B.v_full(i), 1); mbar_init(B.v_empty(i), 1);
             mbar_init(B.s_full(i), 1); mbar_init(B.p_full(i), 256);
         }
-        for (int i = 0; i < 2; ++i) mbar_init(B.o_done(i), 1);
+        for (int i = 0; i < 4; ++i) { mbar_init(B.o_done(0, i), 1); mbar_init(B.o_done(1, i), 1); }
         mbar_init(B.q_full(), 1);
         mbar_init(B.fin(), 1);
         *abort_flag = 0;
@@ -454,7 +474,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                 for (int kk = 0; kk < 8; ++kk)
                     mma_ts(tmem + kOCol + blk * 128, tmem + sb * 128 + kk * 8, vd + (uint64_t)((kk * 2048) >> 4),
                            idesc_pv, (n >= NB || kk > 0) ? 1u : 0u);
-                tc_commit(B.o_done(blk));
+                tc_commit(B.o_done(blk, j));
                 if (blk == NB - 1) tc_commit(B.v_empty(st));
                 if (n + NSB < n_jobs) ok = issue_qk(n + NSB);             // its S block was job n's
             }
@@ -472,19 +492,24 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
         bool row_ok[NB];
         unsigned long long anc[NB];
         float m_ref[NB], l_run[NB];
-        // Phases of o_done[blk] observed so far.  A parity wait is only meaningful for the phase in
-        // progress or the one just completed, and the softmax runs ahead of the P V products, so
-        // every job observes the previous job's phase before it releases its own P (which the next
-        // phase needs): o_seen never lags the barrier by more than one phase.
-        int o_seen[NB];
         #pragma unroll
         for (int blk = 0; blk < NB; ++blk) {
             t_row[blk] = (block0 + blk) * kTokPerBlock + row_local / kGroup;
             row_ok[blk] = row_local < kTokPerBlock * kGroup && t_row[blk] < T;
             anc[blk] = (row_ok[blk] && it.key_end > kv_len) ? anc_s[t_row[blk]] : 0ull;
-            m_ref[blk] = -INFINITY; l_run[blk] = 0.f; o_seen[blk] = 0;
+            m_ref[blk] = -INFINITY; l_run[blk] = 0.f;
         }
         bool ok = true;
+
+        // The scores of a job are requested from TMEM at the end of the job before it, ahead of the
+        // wait for that job's P stores, so the two latencies overlap; whether those scores are there
+        // is probed before the exponentials and only waited for if the probe said no.
+        float x0[32], x1[32];
+        if (n_jobs > 0) {
+            ok = mbar_wait_warp(B.s_full(0), 0);
+            tc_fence_after();
+            if (ok) { tmem_ld32(lane_addr + 64 * wg, x0); tmem_ld32(lane_addr + 64 * wg + 32, x1); }
+        }
 
         #pragma unroll 1
         for (int j = 0; j < n_tiles && ok; ++j) {
@@ -494,12 +519,6 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
             #pragma unroll
             for (int blk = 0; blk < NB; ++blk) {
                 const int n = j * NB + blk, sb = n % NSB;
-                const uint32_t s_addr = lane_addr + sb * 128 + 64 * wg;
-                if (!mbar_wait_warp(B.s_full(sb), (n / NSB) & 1)) { ok = false; break; }
-                tc_fence_after();
-                float x0[32], x1[32];
-                tmem_ld32(s_addr, x0);
-                tmem_ld32(s_addr + 32, x1);
                 // Visibility word of this row for the thread's 64 columns (all ones away from the
                 // draft block and the end of the key range).
                 const bool boundary = j0 + 64 > it.key_end || j0 + 64 > kv_len;
@@ -547,8 +566,8 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                         l_run[blk] *= alpha;
                     }
                     if (j > 0 && __any_sync(0xffffffffu, cand > -INFINITY)) {     // O holds earlier tiles: rescale this half of it
-                        for (; ok && o_seen[blk] < j; ++o_seen[blk]) ok = mbar_wait_warp(B.o_done(blk), o_seen[blk] & 1);
-                        if (!ok) break;
+                        // every earlier tile's product has been added (they complete in order)
+                        if (!mbar_wait_warp(B.o_done(blk, j - 1), ((j - 1) >> 2) & 1)) { ok = false; break; }
                         tc_fence_after();
                         const uint32_t o_addr = lane_addr + kOCol + blk * 128 + 64 * wg;
                         #pragma unroll 1
@@ -564,6 +583,13 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                     }
                 }
 
+                // are the next job's scores there already?  (asked now, used after the exponentials)
+                const bool has_next = n + 1 < n_jobs;
+                const int sb_next = (n + 1) % NSB;
+                const uint32_t par_next = (uint32_t)((n + 1) / NSB) & 1u;
+                uint32_t next_ready = 0;
+                if (has_next && lane == 0) next_ready = mbar_test_wait(B.s_full(sb_next), par_next) ? 1u : 0u;
+
                 // p = 2^(s c2 - m c2), row sum from the unrounded p, P (bf16) over the S block: this
                 // thread's 64 keys land on columns [32 wg, 32 wg + 32) of the block.
                 const float mc = (m_ref[blk] == -INFINITY) ? 0.f : m_ref[blk] * c2;
@@ -572,14 +598,21 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                 exp_chunk(x0, c2, mc, sum4, p_addr);
                 exp_chunk(x1, c2, mc, sum4, p_addr + 16);
                 l_run[blk] += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
-                // Observe the previous tile's P V (long done) BEFORE handing over this tile's P: the
-                // next phase of o_done cannot complete without this warp's arrival below, so the
-                // barrier never gets two phases ahead of a warp that has yet to look at it.
-                for (; ok && o_seen[blk] < j; ++o_seen[blk]) ok = mbar_wait_warp(B.o_done(blk), o_seen[blk] & 1);
-                if (!ok) break;
-                tmem_wait_st();
+
+                if (has_next) {                                            // request the next job's scores
+                    if (__shfl_sync(0xffffffffu, next_ready, 0) == 0u && !mbar_wait_warp(B.s_full(sb_next), par_next)) {
+                        ok = false;
+                    } else {
+                        tc_fence_after();
+                        const uint32_t s_next = lane_addr + sb_next * 128 + 64 * wg;
+                        tmem_ld32(s_next, x0);
+                        tmem_ld32(s_next + 32, x1);
+                    }
+                }
+                tmem_wait_st();                                            // this job's P is in TMEM
                 tc_fence_before();
                 mbar_arrive(B.p_full(sb));
+                if (!ok) break;
             }
         }
 
@@ -602,7 +635,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
         }
         #pragma unroll
         for (int blk = 0; blk < NB; ++blk) {
-            for (; ok && o_seen[blk] < n_tiles; ++o_seen[blk]) ok = mbar_wait_warp(B.o_done(blk), o_seen[blk] & 1);
+            if (ok) ok = mbar_wait_warp(B.o_done(blk, n_tiles - 1), ((n_tiles - 1) >> 2) & 1);    // the last product is in
             tc_fence_after();
             // the two halves' sums meet (the maxima are already the same)
             xch[wg * 128 + row_local] = l_run[blk];
