@@ -268,6 +268,9 @@ def main():
         torch.cuda.synchronize()
 
     # -- device-resident throughput: whole calls ------------------------------------------------
+    # The timed stream is thousands of independent calls queued back to back, which is what the
+    # planner's throughput policy is for; the other policies are timed below and reported beside it.
+    ctx.set_plan_policy(B.PLAN_THROUGHPUT)
     time_calls(ctx, batch, warmup, B, torch)
     sampler = ClockSampler(local_rank)
     barrier()
@@ -288,8 +291,19 @@ def main():
         clocks["note"] = f"timed region shorter than the sampling period: {continued} more untimed calls of the same workload kept the load up while sampling"
     us_call = max_over_ranks(us_call, dist, dev)
 
-    # -- latency of an isolated call (cold cache: the rotation continues) ------------------------
-    us_isolated = time_isolated_calls(ctx, cases, outs, lses, 300, B, torch)
+    # -- every policy: sustained stream and isolated call (cold cache: the rotation continues) ---
+    policies = {}
+    for name, pol in POLICIES(B):
+        ctx.set_plan_policy(pol)
+        if pol == B.PLAN_THROUGHPUT:
+            us_stream = us_call
+        else:
+            time_calls(ctx, batch, 200, B, torch)
+            us_stream = max_over_ranks(time_calls(ctx, batch, max(200, steps // 4), B, torch), dist, dev)
+        policies[name] = {"target_items": ctx.plan_target_items(), "us_per_call_stream": us_stream,
+                          "us_per_call_isolated": time_isolated_calls(ctx, cases, outs, lses, 300, B, torch)}
+    us_isolated = policies["latency"]["us_per_call_isolated"]
+    ctx.set_plan_policy(B.PLAN_THROUGHPUT)
 
     # -- L2-warm figure (one cache, labelled as such) --------------------------------------------
     warm = B.VerifyBatch([(cases[0].q, cases[0].k, cases[0].v, cases[0].kv_len, cases[0].parents,
@@ -309,6 +323,8 @@ def main():
     h2d = q_h.numel() * 2 + k_new.numel() * 2 + v_new.numel() * 2 + par_h.numel() * 4
     d2h = out_h.numel() * 2 + lse_h.numel() * 4
     e2e_steps = max(10, min(steps // 20, 5000))
+
+    ctx.set_plan_policy(B.PLAN_LATENCY)          # every step is synchronised: nothing to overlap with
 
     def e2e_loop(n):
         for i in range(n):
@@ -340,11 +356,14 @@ def main():
         "config": {"workload": WORKLOAD, "l2_policy": f"rotation over {n_caches} distinct K/V caches "
                    f"({n_caches * kv_bytes / 1e6:.0f} MB > 4 x L2 {l2 / 1e6:.0f} MB)",
                    "launch": "plain stream launches enqueued from C (sparrow_verify_attn_batch)",
+                   "plan_policy": "throughput (sparrow_set_plan_policy; the default is balanced)",
                    "parallelism": "replicas only" if world > 1 else "1 GPU"},
         "hbm_gbs_per_call": alg_bytes / (us_call * 1e-6) / 1e9,
         "pct_of_8tbs_nominal": 100.0 * alg_bytes / (us_call * 1e-6) / 8e12,
         "tflops_per_call": flops / (us_call * 1e-6) / 1e12,
         "us_per_call_isolated": us_isolated,
+        "us_per_call_isolated_what": "one call on an idle GPU under the latency policy, events around the call, median",
+        "policies": policies,
         "us_per_call_l2_warm": us_warm,
         "calls_per_s_all_gpus": world * 1e6 / us_call,
         "roofline": {"bound": "hbm", "kernel": "verify_tc_kernel<1> (the only kernel of a step: split-KV pass with the combine "
@@ -357,7 +376,7 @@ def main():
         "e2e": {"value": us_e2e, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": e2e_steps,
                 "what": "sparrow_verify_step_host: pinned host q / new K,V rows / parents in, out + lse back, "
-                        "stream synchronised every step; the committed KV prefix stays resident"},
+                        "stream synchronised every step (latency policy); the committed KV prefix stays resident"},
         "gpu_launches": launches_timed,
     }
     if rank == 0 and not args.no_cpu_baseline and world == 1:
@@ -379,6 +398,10 @@ def main():
         dist.destroy_process_group()
 
 
+def POLICIES(B):
+    return (("throughput", B.PLAN_THROUGHPUT), ("balanced", B.PLAN_BALANCED), ("latency", B.PLAN_LATENCY))
+
+
 def extra_configs(W, B, torch, dev, l2, peak):
     """Times C1, C3, C4 and the 28-layer C5 step; one JSON line each on stderr."""
     def emit(d):
@@ -388,12 +411,15 @@ def extra_configs(W, B, torch, dev, l2, peak):
         probe = W.make_config(ci, "cpu")
         n_caches = max(4, -(-4 * l2 // probe.kv_bytes()))
         cases, ctx, outs, lses, batch = build_rotation(W, B, torch, dev, ci, n_caches)
-        time_calls(ctx, batch, 500, B, torch)
-        us = time_calls(ctx, batch, 20000, B, torch)
         by = probe.kv_bytes() + probe.io_bytes()
-        emit({"config": name, "workload": probe.name, "us_per_call": us, "hbm_gbs": by / us / 1e3,
-              "pct_of_measured_hbm": 100 * by / us / 1e3 / peak, "tflops": probe.flops() / us / 1e6,
-              "rotation": n_caches})
+        for pname, pol in POLICIES(B):
+            ctx.set_plan_policy(pol)
+            time_calls(ctx, batch, 500, B, torch)
+            us = time_calls(ctx, batch, 20000, B, torch)
+            emit({"config": name, "workload": probe.name, "plan_policy": pname, "us_per_call": us, "hbm_gbs": by / us / 1e3,
+                  "pct_of_measured_hbm": 100 * by / us / 1e3 / peak, "tflops": probe.flops() / us / 1e6,
+                  "us_per_call_isolated": time_isolated_calls(ctx, cases, outs, lses, 200, B, torch),
+                  "rotation": n_caches})
         del cases, ctx, outs, lses, batch
         torch.cuda.empty_cache()
     # C4: anchored mode, rotate over full-length buffers
@@ -419,13 +445,16 @@ def extra_configs(W, B, torch, dev, l2, peak):
     outs = [torch.empty_like(c.q) for c in layers]
     lses = [torch.empty((c.B, W.HQ, c.T), dtype=torch.float32, device=dev) for c in layers]
     batch = B.VerifyBatch([(c.q, c.k, c.v, c.kv_len, c.parents, c.T, o, l) for c, o, l in zip(layers, outs, lses)])
-    time_calls(ctx, batch, 28 * 5, B, torch)
-    us = time_calls(ctx, batch, 28 * 50, B, torch)
     by = sum(c.kv_bytes() + c.io_bytes() for c in layers)
     fl = sum(c.flops() for c in layers)
-    emit({"config": "C5", "workload": "batch 8 ragged, T=32 tree, 28 layers per step", "us_per_step": us * 28,
-          "us_per_layer": us, "hbm_gbs": by / (us * 28) / 1e3, "pct_of_measured_hbm": 100 * by / (us * 28) / 1e3 / peak,
-          "tflops": fl / (us * 28) / 1e6, "kv_len": layers[0].kv_len})
+    for pname, pol in POLICIES(B):
+        ctx.set_plan_policy(pol)
+        time_calls(ctx, batch, 28 * 5, B, torch)
+        us = time_calls(ctx, batch, 28 * 50, B, torch)
+        emit({"config": "C5", "workload": "batch 8 ragged, T=32 tree, 28 layers per step", "plan_policy": pname,
+              "us_per_step": us * 28, "us_per_layer": us, "hbm_gbs": by / (us * 28) / 1e3,
+              "pct_of_measured_hbm": 100 * by / (us * 28) / 1e3 / peak, "tflops": fl / (us * 28) / 1e6,
+              "kv_len": layers[0].kv_len})
 
 
 if __name__ == "__main__":

@@ -76,6 +76,31 @@ typedef struct sparrow_ctx sparrow_ctx;
 sparrow_status sparrow_create(sparrow_ctx** ctx, const sparrow_layout* layout, int device);
 sparrow_status sparrow_destroy(sparrow_ctx* ctx);
 
+/* How sparrow_verify_attn() cuts the key range into work items (one CTA each; the paper says
+ * nothing about scheduling, this is a property of this implementation).  Calls in fused mode
+ * overlap their neighbours in the stream, so the number of items trades single-call latency
+ * against sustained throughput of a stream of calls:
+ *   LATENCY     one wave over all SMs (about n_sm items): shortest time for a call on an idle GPU;
+ *   BALANCED    about 3/8 n_sm items (the default);
+ *   THROUGHPUT  about n_sm / 7 items: longest pieces, several calls resident at once; best when
+ *               many independent calls are queued back to back (one per layer or per request).
+ * Results differ between policies only by the rounding order of the split-KV merge.  Calls that
+ * cannot overlap (stream-ordered mode, graph capture, sparrow_anchor_attn,
+ * sparrow_verify_attn_static) always use one wave over all SMs. */
+typedef enum {
+    SPARROW_PLAN_LATENCY    = 0,
+    SPARROW_PLAN_BALANCED   = 1,
+    SPARROW_PLAN_THROUGHPUT = 2
+} sparrow_plan_policy;
+
+/* Sets the policy for later calls (host state only; may be changed between any two calls).
+ * SPARROW_ERR_SHAPE for an unknown value. */
+sparrow_status sparrow_set_plan_policy(sparrow_ctx* ctx, int32_t policy);
+
+/* Work items the planner currently aims for in fused mode (pass it to sparrow_plan_splits() as
+ * n_sm to see the schedule of a call).  0 when ctx is NULL. */
+int32_t sparrow_plan_target_items(const sparrow_ctx* ctx);
+
 /* Bytes of device scratch the calls need for draft blocks of up to max_T tokens (split-KV partial
  * outputs, the device status word, staging for the host-buffer entry point).  0 on bad arguments. */
 size_t sparrow_workspace_bytes(const sparrow_ctx* ctx, int32_t max_T);
@@ -209,7 +234,8 @@ sparrow_status sparrow_debug_ancestor_masks_device(sparrow_ctx* ctx, const int32
                                                    int32_t T, uint64_t* masks_dev, void* stream);
 
 /* Host-side split schedule, exported for inspection (pure host code, needs no GPU): for `batch`
- * sequences of n_keys[b] keys, draft blocks of T tokens and a device with n_sm SMs, writes
+ * sequences of n_keys[b] keys, draft blocks of T tokens and a target of n_sm work items (the SM
+ * count, or sparrow_plan_target_items() for calls in fused mode), writes
  * splits_out[b] = key-range pieces per (sequence, KV head, row group) and the total number of
  * work items.  Piece s of n covers keys [n_keys*s/n, n_keys*(s+1)/n). */
 sparrow_status sparrow_plan_splits(int32_t n_sm, int32_t batch, int32_t n_kv_heads,

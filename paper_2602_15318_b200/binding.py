@@ -25,7 +25,11 @@ EXPORTS = ["sparrow_create", "sparrow_destroy", "sparrow_workspace_bytes", "spar
            "sparrow_build_ancestor_masks", "sparrow_build_anchor_idx",
            "sparrow_debug_ancestor_masks_device", "sparrow_debug_wait_counter", "sparrow_plan_splits",
            "sparrow_last_device_status", "sparrow_debug_status_word", "sparrow_launch_count",
+           "sparrow_set_plan_policy", "sparrow_plan_target_items",
            "sparrow_status_string"]
+
+
+PLAN_LATENCY, PLAN_BALANCED, PLAN_THROUGHPUT = 0, 1, 2
 
 
 class SparrowError(RuntimeError):
@@ -69,6 +73,9 @@ def lib():
         L.sparrow_debug_wait_counter.argtypes = [vp, ctypes.c_uint32, vp]
         L.sparrow_plan_splits.argtypes = [i32, i32, i32, vp, i32, vp, vp]
         L.sparrow_last_device_status.argtypes = [vp, vp]
+        L.sparrow_set_plan_policy.argtypes = [vp, i32]
+        L.sparrow_plan_target_items.argtypes = [vp]
+        L.sparrow_plan_target_items.restype = i32
         L.sparrow_debug_status_word.argtypes = [vp]
         L.sparrow_debug_status_word.restype = ctypes.c_uint32
         L.sparrow_launch_count.argtypes = [vp]
@@ -77,7 +84,7 @@ def lib():
         L.sparrow_status_string.restype = ctypes.c_char_p
         for name in EXPORTS:
             if name not in ("sparrow_workspace_bytes", "sparrow_launch_count", "sparrow_status_string",
-                            "sparrow_debug_status_word"):
+                            "sparrow_debug_status_word", "sparrow_plan_target_items"):
                 getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -143,6 +150,12 @@ class Context:
 
     def last_device_status(self, stream=None) -> int:
         return int(lib().sparrow_last_device_status(self.handle, _stream_handle(stream)))
+
+    def set_plan_policy(self, policy: int):
+        _chk(lib().sparrow_set_plan_policy(self.handle, int(policy)), "sparrow_set_plan_policy")
+
+    def plan_target_items(self) -> int:
+        return int(lib().sparrow_plan_target_items(self.handle))
 
     def status_word(self) -> int:
         """Raw status word read by the last last_device_status() call (wait-site bits above bit 8)."""

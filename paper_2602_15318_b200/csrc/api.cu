@@ -41,7 +41,8 @@ struct sparrow_ctx {
     sparrow_layout layout;
     int device;
     int n_sm;
-    int target_items;                        // work items the split plan aims for (<= n_sm)
+    int plan_policy;                         // sparrow_plan_policy
+    int target_override;                     // > 0: SPARROW_TARGET_ITEMS (diagnosis), replaces the policy's target
     unsigned char* ws;
     size_t ws_bytes;
     std::atomic<long long> launches;
@@ -156,15 +157,41 @@ __half* o_part_ptr(const sparrow_ctx* c, int parity)
 // Ordering arguments of the next call and, once it is enqueued, the advance of the host mirror.
 // Calls that are being captured into a graph, or made with programmatic launch switched off, or
 // served by the gathered kernel run in stream-ordered mode: their kernels touch no counter.
-SyncArgs next_sync(const sparrow_ctx* c, const SplitPlan& p, cudaStream_t st, bool fused_kernel)
+// Will this call run in fused mode, i.e. may it overlap its neighbours in the stream?  Not while the
+// stream is being captured, not with programmatic launch switched off, not on the gathered kernel.
+bool call_overlaps(const sparrow_ctx* c, cudaStream_t st, bool fused_kernel)
+{
+    if (!fused_kernel || !c->use_pdl) return false;
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) { cudaGetLastError(); return false; }
+    return cap == cudaStreamCaptureStatusNone;
+}
+
+// Work items a policy aims for.  Fewer, longer pieces leave SMs free for the next calls in the
+// stream, which then overlap this one: better sustained throughput, longer single-call latency.
+int policy_target(int n_sm, int policy)
+{
+    switch (policy) {
+        case SPARROW_PLAN_THROUGHPUT: return n_sm / 7 > 1 ? n_sm / 7 : 1;
+        case SPARROW_PLAN_BALANCED: return (3 * n_sm) / 8 > 1 ? (3 * n_sm) / 8 : 1;
+        default: return n_sm;
+    }
+}
+
+// Calls that cannot overlap others always get one wave over all SMs.
+int plan_target(const sparrow_ctx* c, bool overlaps)
+{
+    if (!overlaps) return c->n_sm;
+    return c->target_override > 0 ? c->target_override : policy_target(c->n_sm, c->plan_policy);
+}
+
+SyncArgs next_sync(const sparrow_ctx* c, const SplitPlan& p, bool overlaps)
 {
     SyncArgs sy;
-    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
-    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) { cudaGetLastError(); cap = cudaStreamCaptureStatusActive; }
     const int parity = (int)(c->seq & 1u);
     sy.arrivals = reinterpret_cast<unsigned*>(c->ws + kArrivalsOffset);
     sy.fin_done = reinterpret_cast<unsigned*>(c->ws + kFinDoneOffset);
-    sy.enabled = (fused_kernel && c->use_pdl && cap == cudaStreamCaptureStatusNone) ? 1 : 0;
+    sy.enabled = overlaps ? 1 : 0;
     sy.parity = parity;
     sy.slot = (int)(c->seq & 3u);
     int n_arrive = 0;
@@ -392,10 +419,11 @@ sparrow_status sparrow_create(sparrow_ctx** out, const sparrow_layout* L, int de
     c->layout = *L;
     c->device = device;
     c->n_sm = prop.multiProcessorCount;
-    c->target_items = c->n_sm;
+    c->plan_policy = SPARROW_PLAN_BALANCED;
+    c->target_override = 0;
     if (const char* ti = std::getenv("SPARROW_TARGET_ITEMS")) {
         const int v = std::atoi(ti);
-        if (v >= 1 && v <= c->n_sm) c->target_items = v;
+        if (v >= 1 && v <= c->n_sm) c->target_override = v;
     }
     c->ws = nullptr;
     c->ws_bytes = 0;
@@ -470,16 +498,17 @@ sparrow_status sparrow_verify_attn(sparrow_ctx* c, const void* q, const void* k,
         if (kv_len[b] < 0 || (int64_t)kv_len[b] + T > c->layout.kv_capacity) return SPARROW_ERR_SHAPE;
         n_keys[b] = kv_len[b] + T;
     }
-    SplitPlan plan;
-    const int nb = c->verify_on_gather ? 1 : blocks_per_group_tc(T);
-    sparrow_status s = make_plan(c->target_items, c->layout.batch, c->layout.n_kv_heads, n_keys, T, nb, &plan);
-    if (s != SPARROW_OK) return s;
-    for (int b = 0; b < c->layout.batch; ++b) plan.seq[b].kv_len = kv_len[b];
-    if ((s = check_ws(c, plan)) != SPARROW_OK) return s;
     DeviceGuard guard(c->device);
     if (!guard.ok) return SPARROW_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const SyncArgs sy = next_sync(c, plan, st, !c->verify_on_gather);
+    const bool overlaps = call_overlaps(c, st, !c->verify_on_gather);
+    SplitPlan plan;
+    const int nb = c->verify_on_gather ? 1 : blocks_per_group_tc(T);
+    sparrow_status s = make_plan(plan_target(c, overlaps), c->layout.batch, c->layout.n_kv_heads, n_keys, T, nb, &plan);
+    if (s != SPARROW_OK) return s;
+    for (int b = 0; b < c->layout.batch; ++b) plan.seq[b].kv_len = kv_len[b];
+    if ((s = check_ws(c, plan)) != SPARROW_OK) return s;
+    const SyncArgs sy = next_sync(c, plan, overlaps);
     s = c->verify_on_gather ? launch_split_gather(c, plan, sy, q, k, v, parents, nullptr, 0, 0, out, lse, st)
                             : launch_verify_tc(c, plan, sy, q, k, v, parents, out, lse, st);
     if (s != SPARROW_OK) return s;
@@ -555,7 +584,8 @@ sparrow_status sparrow_verify_attn_static(const sparrow_layout* L, const void* q
         c->layout = *L;
         c->device = device;
         c->n_sm = prop.multiProcessorCount;
-        c->target_items = c->n_sm;
+        c->plan_policy = SPARROW_PLAN_LATENCY;
+        c->target_override = 0;
         c->ws = static_cast<unsigned char*>(scratch);
         c->ws_bytes = SPARROW_STATIC_SCRATCH_BYTES;
         c->launches.store(0);
@@ -578,7 +608,7 @@ sparrow_status sparrow_verify_attn_static(const sparrow_layout* L, const void* q
             n_keys[b] = kv_len[b] + T;
         }
         SplitPlan plan;
-        if (lens_ok && make_plan(c->target_items, L->batch, L->n_kv_heads, n_keys, T, blocks_per_group_tc(T), &plan) == SPARROW_OK &&
+        if (lens_ok && make_plan(c->n_sm, L->batch, L->n_kv_heads, n_keys, T, blocks_per_group_tc(T), &plan) == SPARROW_OK &&
             check_ws(c, plan) != SPARROW_OK)
             return SPARROW_ERR_WORKSPACE;
     }
@@ -610,13 +640,13 @@ sparrow_status sparrow_anchor_attn(sparrow_ctx* c, const void* q, const void* k,
     int32_t n_keys[kMaxBatch];
     for (int b = 0; b < c->layout.batch; ++b) n_keys[b] = n_anchor;
     SplitPlan plan;
-    sparrow_status s = make_plan(c->target_items, c->layout.batch, c->layout.n_kv_heads, n_keys, T, 1, &plan);
+    sparrow_status s = make_plan(c->n_sm, c->layout.batch, c->layout.n_kv_heads, n_keys, T, 1, &plan);
     if (s != SPARROW_OK) return s;
     if ((s = check_ws(c, plan)) != SPARROW_OK) return s;
     DeviceGuard guard(c->device);
     if (!guard.ok) return SPARROW_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const SyncArgs sy = next_sync(c, plan, st, false);
+    const SyncArgs sy = next_sync(c, plan, false);
     if ((s = launch_split_gather(c, plan, sy, q, k, v, nullptr, anchor_idx, n_anchor, window, out, lse, st)) != SPARROW_OK) return s;
     return launch_combine(c, plan, sy, out, lse, st);
 }
@@ -751,6 +781,17 @@ sparrow_status sparrow_last_device_status(sparrow_ctx* c, void* stream)
     if (word & kStatAnchor) return SPARROW_ERR_ANCHOR;
     return SPARROW_OK;
 }
+
+sparrow_status sparrow_set_plan_policy(sparrow_ctx* c, int32_t policy)
+{
+    if (!c) return SPARROW_ERR_NULL;
+    if (policy != SPARROW_PLAN_LATENCY && policy != SPARROW_PLAN_BALANCED && policy != SPARROW_PLAN_THROUGHPUT)
+        return SPARROW_ERR_SHAPE;
+    c->plan_policy = policy;
+    return SPARROW_OK;
+}
+
+int32_t sparrow_plan_target_items(const sparrow_ctx* c) { return c ? plan_target(c, c->use_pdl) : 0; }
 
 uint32_t sparrow_debug_status_word(const sparrow_ctx* c) { return c ? c->last_status_word : 0u; }
 

@@ -11,8 +11,10 @@ TOL_OUT = 1e-2      # max |out_gpu - out_oracle|   (bf16 inputs, fp32 accumulati
 TOL_LSE = 1e-3      # max |lse_gpu - lse_oracle|
 
 
-def run_verify(case: W.VerifyCase, ctx=None):
+def run_verify(case: W.VerifyCase, ctx=None, policy=None):
     ctx = ctx or B.Context.for_cache(case.k, W.SCALE)
+    if policy is not None:
+        ctx.set_plan_policy(policy)
     out = torch.full_like(case.q, float("nan"))
     lse = torch.full((case.B, W.HQ, case.T), float("nan"), dtype=torch.float32, device=case.q.device)
     B.sparrow_verify_attn(ctx, case.q, case.k, case.v, case.kv_len, case.parents, case.T, out, lse)

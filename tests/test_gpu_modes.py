@@ -126,6 +126,38 @@ def test_bounded_wait_gives_up_and_context_survives():
     B.sparrow_debug_wait_counter(ctx, 5)                  # nothing will ever bump the counter that far
     torch.cuda.synchronize()
     assert ctx.last_device_status() == 7                  # SPARROW_ERR_TIMEOUT, then cleared
+    assert ctx.status_word() == 4 | (1 << 16)             # timeout bit + the debug wait's site bit
     assert ctx.last_device_status() == 0
     out2, lse2, _ = run_verify(case, ctx)
     check(out2, lse2, *oracle_verify(case))
+
+
+def test_plan_policy_changes_between_calls():
+    """The policy only changes how the key range is cut: every policy meets the tolerances, the
+    policy may change between two calls of a stream without any synchronisation, and a long
+    stream of calls with few, long pieces (many calls resident at once) keeps every result apart."""
+    cap = 9000 + 64
+    cases = [W.make_verify_case(700 + i, kv, T, tree, DEV, capacity=cap)
+             for i, (kv, T, tree) in enumerate([([9000], 16, "chain"), ([5000], 30, "random"), ([7000], 8, "chain")])]
+    refs = [oracle_verify(c) for c in cases]
+    ctx = B.Context.for_cache(cases[0].k, W.SCALE)
+    n_sm = torch.cuda.get_device_properties(0).multi_processor_count
+    targets = {}
+    for pol in (B.PLAN_LATENCY, B.PLAN_BALANCED, B.PLAN_THROUGHPUT):
+        ctx.set_plan_policy(pol)
+        targets[pol] = ctx.plan_target_items()
+    assert targets[B.PLAN_LATENCY] == n_sm
+    assert targets[B.PLAN_LATENCY] > targets[B.PLAN_BALANCED] > targets[B.PLAN_THROUGHPUT] >= 1
+    with pytest.raises(B.SparrowError):
+        ctx.set_plan_policy(17)
+    results = []
+    for rep in range(40):
+        ctx.set_plan_policy((B.PLAN_THROUGHPUT, B.PLAN_LATENCY, B.PLAN_THROUGHPUT, B.PLAN_BALANCED)[rep % 4])
+        for c in cases:
+            out, lse = _new(c)
+            B.sparrow_verify_attn(ctx, c.q, c.k, c.v, c.kv_len, c.parents, c.T, out, lse)
+            results.append((out, lse))
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == 0
+    for i, (out, lse) in enumerate(results):
+        check(out, lse, *refs[i % len(cases)])

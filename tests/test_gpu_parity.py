@@ -190,18 +190,23 @@ def test_config1_full():
     check(out, lse, ref_out, ref_lse)
 
 
-def test_config2_sampled_rows():
+POLICIES = [B.PLAN_LATENCY, B.PLAN_BALANCED, B.PLAN_THROUGHPUT]
+
+
+@pytest.mark.parametrize("policy", POLICIES)
+def test_config2_sampled_rows(policy):
     case = W.make_config(1, DEV)
-    out, lse, _ = run_verify(case)
+    out, lse, _ = run_verify(case, policy=policy)
     rows = sample_rows(2, 1, case.T, 48)
     ref_out, ref_lse = oracle_verify(case, rows)
     check(out, lse, ref_out, ref_lse, rows)
     assert torch.isfinite(out.float()).all() and torch.isfinite(lse).all()
 
 
-def test_config3_sampled_rows():
+@pytest.mark.parametrize("policy", POLICIES)
+def test_config3_sampled_rows(policy):
     case = W.make_config(2, DEV)
-    out, lse, _ = run_verify(case)
+    out, lse, _ = run_verify(case, policy=policy)
     rows = sample_rows(3, 1, case.T, 64)
     ref_out, ref_lse = oracle_verify(case, rows)
     check(out, lse, ref_out, ref_lse, rows)
@@ -216,10 +221,10 @@ def test_config4_full():
     check(out, lse, ref_out, ref_lse)
 
 
-@pytest.mark.parametrize("layer", [0, 13, 27])
-def test_config5_layer_sampled_rows(layer):
+@pytest.mark.parametrize("layer,policy", [(0, B.PLAN_BALANCED), (13, B.PLAN_THROUGHPUT), (27, B.PLAN_LATENCY)])
+def test_config5_layer_sampled_rows(layer, policy):
     case = W.make_config(4, DEV, layer=layer)
-    out, lse, _ = run_verify(case)
+    out, lse, _ = run_verify(case, policy=policy)
     rows = sample_rows(5 + layer, 8, case.T, 40)
     ref_out, ref_lse = oracle_verify(case, rows)
     check(out, lse, ref_out, ref_lse, rows)
