@@ -126,8 +126,10 @@ sparrow_status sparrow_set_workspace(sparrow_ctx* ctx, void* dev_ptr, size_t byt
  * pieces by log-sum-exp.  Consecutive calls on one stream overlap: the kernel is launched with
  * programmatic stream serialisation and starts reading q / k_cache / v_cache / parents while the
  * previous kernel in the stream is finishing, as soon as that kernel lets its dependents launch
- * (the library's own kernels do; an ordinary kernel never does before it completes).  Writes of
- * consecutive calls are ordered through counters in the workspace.  While a stream is being
+ * (the library's own kernels do; an ordinary kernel never does before it completes).  So the
+ * inputs of a call must not be the out / lse of the library call enqueued directly before it on
+ * the same stream; anything else in between (another kernel, a copy) restores plain stream order.
+ * Writes of consecutive calls are ordered through counters in the workspace.  While a stream is being
  * captured into a graph, or with SPARROW_NO_PDL=1 in the environment when the context is created,
  * a call is two ordinary launches (split-KV pass, combine) ordered by the stream alone.
  * Results are deterministic for fixed arguments. */
