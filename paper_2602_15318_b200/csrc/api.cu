@@ -51,6 +51,11 @@ struct sparrow_ctx {
     // of the fused calls and, per call parity, the cumulative number of finishers launched so far.
     uint32_t seq;
     uint32_t fin_total[2];
+    uint32_t fin_before_last[2];             // fin_total[p] as it was before the last call of parity p
+    // Memory the previous fused call touches (out, lse, q, parents, k, v), as [begin, end) addresses:
+    // a call whose outputs overlap none of it need not wait for that call's merge.
+    uintptr_t prev_ranges[6][2];
+    bool prev_valid;
     uint32_t last_status_word;   // raw word read by the last sparrow_last_device_status()
 };
 
@@ -185,7 +190,44 @@ int plan_target(const sparrow_ctx* c, bool overlaps)
     return c->target_override > 0 ? c->target_override : policy_target(c->n_sm, c->plan_policy);
 }
 
-SyncArgs next_sync(const sparrow_ctx* c, const SplitPlan& p, bool overlaps)
+struct CallRanges {
+    uintptr_t r[6][2];               // out, lse (written), q, parents, k, v (read)
+};
+
+CallRanges call_ranges(const sparrow_ctx* c, const void* q, const void* k, const void* v, const int32_t* parents, int T,
+                       const void* out, const float* lse)
+{
+    const sparrow_layout& L = c->layout;
+    const size_t tok_bytes = (size_t)L.batch * T * L.n_q_heads * kD * 2;
+    const size_t kv_bytes = ((size_t)(L.batch - 1) * L.kv_stride_batch + (size_t)(L.n_kv_heads - 1) * L.kv_stride_head +
+                             (size_t)L.kv_capacity * kD) * 2;
+    CallRanges cr;
+    auto set = [&](int i, const void* p, size_t n) {
+        cr.r[i][0] = reinterpret_cast<uintptr_t>(p);
+        cr.r[i][1] = cr.r[i][0] + n;
+    };
+    set(0, out, tok_bytes);
+    set(1, lse, (size_t)L.batch * L.n_q_heads * T * 4);
+    set(2, q, tok_bytes);
+    set(3, parents, (size_t)L.batch * T * 4);
+    set(4, k, kv_bytes);
+    set(5, v, kv_bytes);
+    return cr;
+}
+
+// Do this call's outputs overlap anything the previous fused call reads or writes?
+bool outputs_touch_previous(const sparrow_ctx* c, const CallRanges& cr)
+{
+    if (!c->prev_valid) return false;
+    for (int o = 0; o < 2; ++o)
+        for (int i = 0; i < 6; ++i)
+            if (cr.r[o][0] < c->prev_ranges[i][1] && c->prev_ranges[i][0] < cr.r[o][1]) return true;
+    return false;
+}
+
+// `after_previous`: the call's final results must wait for the previous fused call as a whole (its
+// outputs overlap that call's memory); otherwise they only wait for the calls before that one.
+SyncArgs next_sync(const sparrow_ctx* c, const SplitPlan& p, bool overlaps, bool after_previous)
 {
     SyncArgs sy;
     const int parity = (int)(c->seq & 1u);
@@ -200,13 +242,14 @@ SyncArgs next_sync(const sparrow_ctx* c, const SplitPlan& p, bool overlaps)
     sy.n_arrive = n_arrive;
     sy.n_fin = n_arrive == 0 ? 0 : (p.n_items < kFinisherCtas ? p.n_items : kFinisherCtas);
     sy.fin_wait_same = c->fin_total[parity];
-    sy.fin_wait_other = c->fin_total[parity ^ 1];
+    sy.fin_wait_other = after_previous ? c->fin_total[parity ^ 1] : c->fin_before_last[parity ^ 1];
     return sy;
 }
 
 void advance_sync(sparrow_ctx* c, const SplitPlan& p, const SyncArgs& sy)
 {
     if (!sy.enabled) return;         // stream-ordered calls leave the fused sequence where it is
+    c->fin_before_last[sy.parity] = c->fin_total[sy.parity];
     c->fin_total[sy.parity] += (uint32_t)(p.n_items - sy.n_arrive + sy.n_fin);    // single-piece items + finishers
     c->seq += 1;
 }
@@ -432,6 +475,8 @@ sparrow_status sparrow_create(sparrow_ctx** out, const sparrow_layout* L, int de
     c->use_pdl = !(e && e[0] == '1');
     c->seq = 0;
     c->fin_total[0] = c->fin_total[1] = 0;
+    c->fin_before_last[0] = c->fin_before_last[1] = 0;
+    c->prev_valid = false;
     c->last_status_word = 0;
     *out = c;
     return SPARROW_OK;
@@ -470,6 +515,8 @@ sparrow_status sparrow_set_workspace(sparrow_ctx* c, void* p, size_t bytes)
     c->ws_bytes = bytes;
     c->seq = 0;
     c->fin_total[0] = c->fin_total[1] = 0;
+    c->fin_before_last[0] = c->fin_before_last[1] = 0;
+    c->prev_valid = false;
     return SPARROW_OK;
 }
 
@@ -508,11 +555,16 @@ sparrow_status sparrow_verify_attn(sparrow_ctx* c, const void* q, const void* k,
     if (s != SPARROW_OK) return s;
     for (int b = 0; b < c->layout.batch; ++b) plan.seq[b].kv_len = kv_len[b];
     if ((s = check_ws(c, plan)) != SPARROW_OK) return s;
-    const SyncArgs sy = next_sync(c, plan, overlaps);
+    const CallRanges cr = call_ranges(c, q, k, v, parents, T, out, lse);
+    const SyncArgs sy = next_sync(c, plan, overlaps, outputs_touch_previous(c, cr));
     s = c->verify_on_gather ? launch_split_gather(c, plan, sy, q, k, v, parents, nullptr, 0, 0, out, lse, st)
                             : launch_verify_tc(c, plan, sy, q, k, v, parents, out, lse, st);
     if (s != SPARROW_OK) return s;
     advance_sync(c, plan, sy);
+    if (sy.enabled) {
+        std::memcpy(c->prev_ranges, cr.r, sizeof(cr.r));
+        c->prev_valid = true;
+    }
     return sy.enabled ? SPARROW_OK : launch_combine(c, plan, sy, out, lse, st);    // fused mode combines in the kernel
 }
 
@@ -592,6 +644,8 @@ sparrow_status sparrow_verify_attn_static(const sparrow_layout* L, const void* q
         c->use_pdl = false;                    // stream-ordered mode: no counters live in the shared array
         c->seq = 0;
         c->fin_total[0] = c->fin_total[1] = 0;
+    c->fin_before_last[0] = c->fin_before_last[1] = 0;
+    c->prev_valid = false;
         c->last_status_word = 0;
         slot.ready = true;
     }
@@ -646,7 +700,7 @@ sparrow_status sparrow_anchor_attn(sparrow_ctx* c, const void* q, const void* k,
     DeviceGuard guard(c->device);
     if (!guard.ok) return SPARROW_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const SyncArgs sy = next_sync(c, plan, false);
+    const SyncArgs sy = next_sync(c, plan, false, true);
     if ((s = launch_split_gather(c, plan, sy, q, k, v, nullptr, anchor_idx, n_anchor, window, out, lse, st)) != SPARROW_OK) return s;
     return launch_combine(c, plan, sy, out, lse, st);
 }
