@@ -211,6 +211,16 @@ __device__ __forceinline__ float ex2(float x)
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+__device__ __forceinline__ float lds_f32(uint32_t addr)
+{
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void lds_v4(uint32_t addr, uint32_t (&v)[4])
+{
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]) : "r"(addr));
+}
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 {
     uint32_t r;
@@ -776,34 +786,35 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                                     const int t = (grp * NB + bk) * kTokPerBlock + r / kGroup;
                                     if (t >= T) continue;
                                     const uint32_t pstride = (uint32_t)n_here * kRowBytes;     // bytes between pieces
-                                    const unsigned char* row0 = kv_sm + (uint32_t)i * kRowBytes;
+                                    const uint32_t row_sm = smem_u32(kv_sm) + (uint32_t)i * kRowBytes;
                                     float mxl = -INFINITY;
                                     #pragma unroll 4
-                                    for (uint32_t sp = 0, off = 2 * kD; sp < (uint32_t)ns; ++sp, off += pstride)
-                                        mxl = fmaxf(mxl, *reinterpret_cast<const float*>(row0 + off));
+                                    for (uint32_t sp = 0, a_l = row_sm + 2 * kD; sp < (uint32_t)ns; ++sp, a_l += pstride)
+                                        mxl = fmaxf(mxl, lds_f32(a_l));
                                     const bool any = mxl != -INFINITY;
+                                    const float mx2 = any ? mxl * 1.4426950408889634f : 0.f;
                                     float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
                                     float suml = 0.f;
-                                    const unsigned char* src = row0 + c * 16;
-                                    #pragma unroll 2
-                                    for (uint32_t sp = 0, off = 0; sp < (uint32_t)ns; ++sp, off += pstride) {
-                                        const float ws = any ? __expf(*reinterpret_cast<const float*>(row0 + off + 2 * kD) - mxl) : 0.f;
-                                        const uint4 raw = *reinterpret_cast<const uint4*>(src + off);
-                                        const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
+                                    #pragma unroll 4
+                                    for (uint32_t sp = 0, a_l = row_sm + 2 * kD, a_o = row_sm + c * 16; sp < (uint32_t)ns;
+                                         ++sp, a_l += pstride, a_o += pstride) {
+                                        const float ws = ex2(fmaf(lds_f32(a_l), 1.4426950408889634f, -mx2));   // exp(lse_s - max); 0 for -inf
+                                        uint32_t raw[4];
+                                        lds_v4(a_o, raw);
                                         suml += ws;
                                         #pragma unroll
                                         for (int q = 0; q < 4; ++q) {
-                                            const float2 f = __half22float2(h2[q]);
+                                            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&raw[q]));
                                             acc[2 * q] = fmaf(ws, f.x, acc[2 * q]); acc[2 * q + 1] = fmaf(ws, f.y, acc[2 * q + 1]);
                                         }
                                     }
-                                    const float inv = any ? 1.f / suml : 0.f;
+                                    const float inv = suml > 0.f ? __fdividef(1.f, suml) : 0.f;
                                     const int h = kvh * kGroup + r % kGroup;
                                     uint4 pk;
                                     pk.x = pack_bf16x2(acc[0] * inv, acc[1] * inv); pk.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
                                     pk.z = pack_bf16x2(acc[4] * inv, acc[5] * inv); pk.w = pack_bf16x2(acc[6] * inv, acc[7] * inv);
                                     *reinterpret_cast<uint4*>(args.out + (((size_t)b * T + t) * args.n_q_heads + h) * kD + c * 8) = pk;
-                                    if (c == 0) args.lse[((size_t)b * args.n_q_heads + h) * T + t] = any ? mxl + logf(suml) : -INFINITY;
+                                    if (c == 0) args.lse[((size_t)b * args.n_q_heads + h) * T + t] = any ? mxl + __logf(suml) : -INFINITY;
                                 }
                             }
                         }

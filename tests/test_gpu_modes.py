@@ -161,3 +161,35 @@ def test_plan_policy_changes_between_calls():
     assert ctx.last_device_status() == 0
     for i, (out, lse) in enumerate(results):
         check(out, lse, *refs[i % len(cases)])
+
+
+@pytest.mark.parametrize("policy", [B.PLAN_LATENCY, B.PLAN_BALANCED, B.PLAN_THROUGHPUT])
+def test_long_stream_is_bitwise_reproducible(policy):
+    """Thousands of calls queued back to back over rotating caches, several calls resident at
+    once: every call must reproduce, bit for bit, what the same call gave when it ran alone (any
+    ordering mistake between overlapping calls shows up as a changed bit or a timeout)."""
+    cap = 20000 + 32
+    cases = [W.make_verify_case(800 + i, [20000 - 37 * i], 16, "chain", DEV, capacity=cap) for i in range(3)]
+    ctx = B.Context.for_cache(cases[0].k, W.SCALE)
+    ctx.set_plan_policy(policy)
+    alone = []
+    for c in cases:
+        out, lse = _new(c)
+        B.sparrow_verify_attn(ctx, c.q, c.k, c.v, c.kv_len, c.parents, c.T, out, lse)
+        torch.cuda.synchronize()
+        alone.append((out, lse))
+    check(alone[0][0], alone[0][1], *oracle_verify(cases[0]))
+    n_slots = 12                                   # output buffers in rotation: more than the calls in flight
+    outs = [[_new(c) for _ in range(n_slots)] for c in cases]
+    batch = B.VerifyBatch([(c.q, c.k, c.v, c.kv_len, c.parents, c.T, outs[i][s][0], outs[i][s][1])
+                           for s in range(n_slots) for i, c in enumerate(cases)])
+    for rep in range(60):                          # 60 x 36 calls
+        B.sparrow_verify_attn_batch(ctx, batch)
+        if rep % 20 == 19:
+            torch.cuda.synchronize()
+            for i in range(len(cases)):
+                for s in range(n_slots):
+                    assert torch.equal(outs[i][s][0], alone[i][0]) and torch.equal(outs[i][s][1], alone[i][1])
+                    outs[i][s][0].zero_()
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == 0
