@@ -254,7 +254,8 @@ void advance_sync(sparrow_ctx* c, const SplitPlan& p, const SyncArgs& sy)
     c->seq += 1;
 }
 
-sparrow_status launch_combine(sparrow_ctx* c, const SplitPlan& plan, const SyncArgs& sy, void* out, float* lse, cudaStream_t st)
+sparrow_status launch_combine(sparrow_ctx* c, const SplitPlan& plan, const SyncArgs& sy, void* out, float* lse, cudaStream_t st,
+                              bool programmatic = false)
 {
     CombineArgs ca;
     ca.o_part = o_part_ptr(c, sy.parity);
@@ -264,15 +265,24 @@ sparrow_status launch_combine(sparrow_ctx* c, const SplitPlan& plan, const SyncA
     const int rows = plan.batch * plan.n_kv_heads * plan.M;
     int ctas = (rows + combine::kWarps - 1) / combine::kWarps;
     if (ctas > 8 * c->n_sm) ctas = 8 * c->n_sm;
-    combine::combine_kernel<<<ctas, combine::kWarps * 32, 0, st>>>(plan, ca);
-    if (cudaGetLastError() != cudaSuccess) return SPARROW_ERR_CUDA;
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(ctas);
+    cfg.blockDim = dim3(combine::kWarps * 32);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = programmatic ? 1 : 0;       // its CTAs become resident while the split-KV pass runs and wait for it
+    if (cudaLaunchKernelEx(&cfg, combine::combine_kernel, plan, ca) != cudaSuccess) { cudaGetLastError(); return SPARROW_ERR_CUDA; }
     c->launches.fetch_add(1);
     return SPARROW_OK;
 }
 
 sparrow_status launch_split_gather(sparrow_ctx* c, const SplitPlan& plan, const SyncArgs& sy, const void* q, const void* k, const void* v,
                                    const int32_t* parents, const int32_t* anchor_idx, int n_anchor, int window,
-                                   void* out, float* lse, cudaStream_t st)
+                                   void* out, float* lse, cudaStream_t st, bool early_dependents = false)
 {
     SplitArgs a;
     a.q = static_cast<const __nv_bfloat16*>(q);
@@ -291,6 +301,7 @@ sparrow_status launch_split_gather(sparrow_ctx* c, const SplitPlan& plan, const 
     a.out = static_cast<__nv_bfloat16*>(out);
     a.lse = lse;
     a.status = reinterpret_cast<unsigned*>(c->ws);
+    a.early_dependents = early_dependents ? 1 : 0;
     gather::split_gather_kernel<<<plan.n_items, gather::kThreads, gather::kSmemBytes, st>>>(plan, a);
     if (cudaGetLastError() != cudaSuccess) return SPARROW_ERR_CUDA;
     c->launches.fetch_add(1);
@@ -701,8 +712,12 @@ sparrow_status sparrow_anchor_attn(sparrow_ctx* c, const void* q, const void* k,
     if (!guard.ok) return SPARROW_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const SyncArgs sy = next_sync(c, plan, false, true);
-    if ((s = launch_split_gather(c, plan, sy, q, k, v, nullptr, anchor_idx, n_anchor, window, out, lse, st)) != SPARROW_OK) return s;
-    return launch_combine(c, plan, sy, out, lse, st);
+    // the two kernels of the call are chained programmatically unless the stream is being captured
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) { cudaGetLastError(); cap = cudaStreamCaptureStatusActive; }
+    const bool chained = c->use_pdl && cap == cudaStreamCaptureStatusNone;
+    if ((s = launch_split_gather(c, plan, sy, q, k, v, nullptr, anchor_idx, n_anchor, window, out, lse, st, chained)) != SPARROW_OK) return s;
+    return launch_combine(c, plan, sy, out, lse, st, chained);
 }
 
 sparrow_status sparrow_verify_step_host(sparrow_ctx* c, const void* q_host, const void* k_new_host,

@@ -141,10 +141,13 @@ __device__ __forceinline__ void combine_row(const SplitPlan& plan, const Combine
 }
 
 // The stand-alone combine kernel of the stream-ordered mode: grid-stride over the rows, one warp
-// per row.  It is an ordinary launch behind the split-KV kernel.
+// per row, launched behind the split-KV kernel (ordinarily, or programmatically in anchored mode).
 __global__ void __launch_bounds__(kWarps * 32)
 combine_kernel(const __grid_constant__ SplitPlan plan, const __grid_constant__ CombineArgs args)
 {
+    // Launched programmatically behind the split-KV kernel it may start early: wait for that grid
+    // to complete (with its writes visible).  Without a programmatic dependency this returns at once.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rows_total = plan.batch * plan.n_kv_heads * plan.M;
     for (int row_id = blockIdx.x * kWarps + warp; row_id < rows_total; row_id += gridDim.x * kWarps) {

@@ -34,6 +34,7 @@ struct SplitArgs {
     __nv_bfloat16* out;          // final output, written directly for sequences with one piece
     float* lse;
     unsigned* status;
+    int32_t early_dependents;    // the next kernel in the stream is this call's combine step, launched programmatically
 };
 
 namespace gather {
@@ -89,6 +90,8 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
     int32_t* qpos_s = reinterpret_cast<int32_t*>(smem + 4 * kStageBytes + kMaxT * 8);
     int32_t* apos_s = qpos_s + kMaxT;                                // [2][kTile] gathered row ids
 
+    // The combine kernel may be scheduled now: it waits for this grid as a whole before it reads.
+    if (args.early_dependents) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g4 = lane >> 2, c4 = lane & 3;
     const Item it = decode_item(plan, blockIdx.x);
