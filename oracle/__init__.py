@@ -176,3 +176,46 @@ def anchor_attn(q, k, v, idx, window, scale, rows=None, n_threads=None):
                                   n_threads or host_threads(), _p(out), _p(lse)),
          "oracle_anchor_attn")
     return out, lse
+
+
+def anchor_tree_visibility(idx, window: int, parents, T_new: int) -> np.ndarray:
+    """Visibility of text-anchored attention whose draft tokens form a tree (the paper drafts a
+    dynamic tree, Section 4 "Implementation"; Eq. 2 itself is written for one chain step).
+
+    idx int32 [n_anchor], strictly increasing; its last T_tree = len(parents) entries are the rows
+    of the tree's nodes, node i at idx[n_anchor - T_tree + i].  The queries are the last T_new
+    nodes.  Query node i (row qpos) sees
+      * a text anchor p (any of the first n_anchor - T_tree entries) iff p <= qpos and
+        (window <= 0 or qpos - window < p): the rule of the chain mode;
+      * a tree node a iff a == i or a is an ancestor of i.
+    Returns uint8 [T_new, n_anchor].  Written out directly from this definition (numpy loops)."""
+    idx = _c(idx, np.int32)
+    parents = _c(parents, np.int32)
+    n, Tt = idx.shape[0], parents.shape[0]
+    assert 1 <= T_new <= Tt <= n
+    anc = ancestor_masks(parents)
+    first = n - Tt
+    vis = np.zeros((T_new, n), dtype=np.uint8)
+    for t in range(T_new):
+        node = Tt - T_new + t
+        qpos = int(idx[first + node])
+        for j in range(first):
+            p = int(idx[j])
+            vis[t, j] = 1 if (p <= qpos and (window <= 0 or qpos - window < p)) else 0
+        for a in range(Tt):
+            vis[t, first + a] = (int(anc[node]) >> a) & 1
+    return vis
+
+
+def anchor_attn_tree(q, k, v, idx, window, parents, scale, rows=None, n_threads=None):
+    """Text-anchored attention with tree-structured draft tokens.  q uint16 [B,T_new,Hq,D];
+    idx int32 [B,n_anchor]; parents int32 [B,T_tree].  The definition of the attention itself is
+    the core's (Eq. 2 on the gathered rows); only the visibility differs from anchor_attn()."""
+    q = _c(q, np.uint16)
+    idx = _c(idx, np.int32)
+    parents = _c(parents, np.int32)
+    B, T_new = q.shape[0], q.shape[1]
+    assert idx.shape[0] == B and parents.shape[0] == B
+    vis = np.stack([anchor_tree_visibility(idx[b], window, parents[b], T_new) for b in range(B)])
+    return attention(q, k, v, vis, np.full(B, idx.shape[1], dtype=np.int32), scale, key_rows=idx,
+                     rows=rows, n_threads=n_threads)

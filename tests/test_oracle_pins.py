@@ -386,3 +386,68 @@ def test_pins_detect_planted_mistakes():
     assert _differs(o[0], ref_o) and _differs(l[0], ref_l)
     o, l = run(q[::-1].copy(), k, v, kv_len, scale)          # token order reversed
     assert _differs(o[0], ref_o) and _differs(l[0], ref_l)
+
+
+# ---- tree-structured draft tokens in the anchored mode ------------------------------------------
+
+def _walk_is_ancestor_or_self(parents, i, a):
+    while i >= 0:
+        if i == a:
+            return True
+        i = parents[i]
+    return False
+
+
+def test_anchor_tree_visibility_chain_reduces_to_chain_mode():
+    idx = np.array([3, 4, 9, 40, 41, 77, 100, 101, 102, 103, 104], dtype=np.int32)
+    T = 5
+    chain = np.arange(-1, T - 1, dtype=np.int32)
+    for window in (0, 64, 1000):          # windows wider than the draft block: the two rules coincide
+        assert np.array_equal(oracle.anchor_tree_visibility(idx, window, chain, T),
+                              oracle.anchor_visibility(idx, window, T))
+
+
+def test_anchor_tree_visibility_brute_force():
+    rng = np.random.default_rng(5)
+    for trial in range(30):
+        Tt = int(rng.integers(1, 13))
+        T_new = int(rng.integers(1, Tt + 1))
+        n_text = int(rng.integers(0, 20))
+        rows = np.sort(rng.choice(500, size=n_text, replace=False)).astype(np.int32)
+        idx = np.concatenate([rows, 600 + np.arange(Tt, dtype=np.int32)])
+        parents = np.array([int(rng.integers(-1, i)) for i in range(Tt)], dtype=np.int32)
+        window = int(rng.choice([0, 50, 300]))
+        vis = oracle.anchor_tree_visibility(idx, window, parents, T_new)
+        for t in range(T_new):
+            node = Tt - T_new + t
+            qpos = 600 + node
+            for j in range(n_text):
+                expect = rows[j] <= qpos and (window <= 0 or rows[j] > qpos - window)
+                assert vis[t, j] == int(expect)
+            for a in range(Tt):
+                assert vis[t, n_text + a] == int(_walk_is_ancestor_or_self(parents.tolist(), node, a))
+
+
+def test_anchor_tree_on_contiguous_rows_equals_verification():
+    """With every row an anchor and no window, the anchored mode with a tree is the verification
+    mode (whole prefix + ancestors): pins the tree variant to the oracle of mode (a), including the
+    node offset when only the last nodes are queries."""
+    case = W.make_verify_case(77, [37, 20], 9, "random", "cpu")
+    q, k, v = W.bf16_bits(case.q), W.bf16_bits(case.k), W.bf16_bits(case.v)
+    par = case.parents.numpy()
+    ref_out, ref_lse = oracle.verify_attn(q, k, v, case.kv_len, par, W.SCALE)
+    for b in range(case.B):
+        n = case.kv_len[b] + case.T
+        idx = np.arange(n, dtype=np.int32)[None]
+        for T_new in (case.T, 4, 1):
+            qb = q[b:b + 1, case.T - T_new:]
+            out, lse = oracle.anchor_attn_tree(qb, k[b:b + 1], v[b:b + 1], idx, 0, par[b:b + 1], W.SCALE)
+            assert np.allclose(out[0], ref_out[b, case.T - T_new:], atol=1e-12)
+            assert np.allclose(lse[0], ref_lse[b][:, case.T - T_new:], atol=1e-12)
+
+
+def test_anchor_tree_forest_of_roots_sees_text_and_itself_only():
+    idx = np.array([1, 2, 5, 50, 51, 52], dtype=np.int32)
+    vis = oracle.anchor_tree_visibility(idx, 0, np.array([-1, -1, -1], dtype=np.int32), 3)
+    assert np.array_equal(vis[:, :3], np.ones((3, 3), dtype=np.uint8))
+    assert np.array_equal(vis[:, 3:], np.eye(3, dtype=np.uint8))
