@@ -169,6 +169,24 @@ sparrow_status sparrow_anchor_attn(sparrow_ctx* ctx, const void* q, const void* 
                                    const int32_t* anchor_idx, int32_t n_anchor, int32_t window,
                                    int32_t T, void* out, float* lse, void* stream);
 
+/* (b) with tree-structured draft tokens (the paper drafts a dynamic tree, Section 4; Eq. 2 is
+ * written for one chain step, so the visibility among draft tokens is this library's reading).
+ * The last T_tree entries of anchor_idx are the rows of the draft tree's nodes, node i at
+ * anchor_idx[n_anchor - T_tree + i]; the queries are the last T_new nodes (T_new = T_tree: the
+ * whole tree; T_new < T_tree: only the nodes added by the latest drafting step).
+ *   parents   DEV int32 [batch][T_tree], -1 = root, parents[i] < i (as in (a))
+ *   q, out    DEV bf16 [batch][T_new][n_q_heads][128];  lse DEV fp32 [batch][n_q_heads][T_new]
+ * A query node at row qpos sees a text anchor p (one of the first n_anchor - T_tree entries) iff
+ * p <= qpos and (window <= 0 or qpos - window < p), and a tree node iff it is the query itself or
+ * one of its ancestors.  With parents = chain and a window wider than the draft block this equals
+ * sparrow_anchor_attn().  SPARROW_ERR_SHAPE unless 1 <= T_new <= T_tree <= SPARROW_MAX_T,
+ * SPARROW_ERR_ANCHOR unless T_tree <= n_anchor <= kv_capacity; a malformed device-side parent
+ * array sets the tree status bit (the node counts as a root). */
+sparrow_status sparrow_anchor_attn_tree(sparrow_ctx* ctx, const void* q, const void* k, const void* v,
+                                        const int32_t* anchor_idx, int32_t n_anchor, int32_t window,
+                                        const int32_t* parents, int32_t T_tree, int32_t T_new,
+                                        void* out, float* lse, void* stream);
+
 /* Verification step with HOST buffers (what a caller without device-side glue uses): copies q,
  * the T new K/V rows per (batch, KV head) and parents to the device, writes the new rows into
  * cache rows [kv_len[b], kv_len[b]+T), runs (a), copies out / lse back and synchronises `stream`.

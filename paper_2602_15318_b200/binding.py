@@ -25,7 +25,7 @@ EXPORTS = ["sparrow_create", "sparrow_destroy", "sparrow_workspace_bytes", "spar
            "sparrow_build_ancestor_masks", "sparrow_build_anchor_idx",
            "sparrow_debug_ancestor_masks_device", "sparrow_debug_wait_counter", "sparrow_plan_splits",
            "sparrow_last_device_status", "sparrow_debug_status_word", "sparrow_launch_count",
-           "sparrow_set_plan_policy", "sparrow_plan_target_items",
+           "sparrow_set_plan_policy", "sparrow_plan_target_items", "sparrow_anchor_attn_tree",
            "sparrow_status_string"]
 
 
@@ -66,6 +66,7 @@ def lib():
         L.sparrow_verify_attn_batch.argtypes = [vp, vp, i32, vp]
         L.sparrow_verify_attn_static.argtypes = [ctypes.POINTER(Layout), vp, vp, vp, vp, vp, i32, vp, vp, vp]
         L.sparrow_anchor_attn.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp]
+        L.sparrow_anchor_attn_tree.argtypes = [vp, vp, vp, vp, vp, i32, i32, vp, i32, i32, vp, vp, vp]
         L.sparrow_verify_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp]
         L.sparrow_build_ancestor_masks.argtypes = [vp, i32, vp]
         L.sparrow_build_anchor_idx.argtypes = [i32, vp, i32, i32, i32, vp, vp]
@@ -227,6 +228,14 @@ def sparrow_anchor_attn(ctx: Context, q, k, v, anchor_idx, n_anchor: int, window
     _chk(lib().sparrow_anchor_attn(ctx.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(anchor_idx), n_anchor,
                                    window, T, _ptr(out), _ptr(lse), _stream_handle(stream)),
          "sparrow_anchor_attn")
+
+
+def sparrow_anchor_attn_tree(ctx: Context, q, k, v, anchor_idx, n_anchor: int, window: int, parents, T_tree: int,
+                             T_new: int, out, lse, stream=None):
+    _chk(lib().sparrow_anchor_attn_tree(ctx.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(anchor_idx), n_anchor,
+                                        window, _ptr(parents), T_tree, T_new, _ptr(out), _ptr(lse),
+                                        _stream_handle(stream)),
+         "sparrow_anchor_attn_tree")
 
 
 def sparrow_verify_step_host(ctx: Context, q_host, k_new_host, v_new_host, k_cache, v_cache,

@@ -282,7 +282,7 @@ sparrow_status launch_combine(sparrow_ctx* c, const SplitPlan& plan, const SyncA
 
 sparrow_status launch_split_gather(sparrow_ctx* c, const SplitPlan& plan, const SyncArgs& sy, const void* q, const void* k, const void* v,
                                    const int32_t* parents, const int32_t* anchor_idx, int n_anchor, int window,
-                                   void* out, float* lse, cudaStream_t st, bool early_dependents = false)
+                                   void* out, float* lse, cudaStream_t st, bool early_dependents = false, int tree_nodes = 0)
 {
     SplitArgs a;
     a.q = static_cast<const __nv_bfloat16*>(q);
@@ -292,6 +292,7 @@ sparrow_status launch_split_gather(sparrow_ctx* c, const SplitPlan& plan, const 
     a.anchor_idx = anchor_idx;
     a.n_anchor = n_anchor;
     a.window = window;
+    a.tree_nodes = tree_nodes;
     a.n_q_heads = c->layout.n_q_heads;
     a.kv_capacity = c->layout.kv_capacity;
     a.kv_stride_batch = c->layout.kv_stride_batch;
@@ -694,9 +695,13 @@ sparrow_status sparrow_verify_attn_batch(sparrow_ctx* c, const sparrow_verify_ca
     return SPARROW_OK;
 }
 
-sparrow_status sparrow_anchor_attn(sparrow_ctx* c, const void* q, const void* k, const void* v,
-                                   const int32_t* anchor_idx, int32_t n_anchor, int32_t window, int32_t T,
-                                   void* out, float* lse, void* stream)
+}  // extern "C"
+
+namespace {
+// Both anchored entry points: parents == nullptr / tree_nodes == 0 is the chain rule.
+sparrow_status anchor_call(sparrow_ctx* c, const void* q, const void* k, const void* v, const int32_t* anchor_idx,
+                           int32_t n_anchor, int32_t window, const int32_t* parents, int32_t tree_nodes, int32_t T,
+                           void* out, float* lse, void* stream)
 {
     if (!c || !q || !k || !v || !anchor_idx || !out || !lse) return SPARROW_ERR_NULL;
     if (T < 1 || T > kMaxT) return SPARROW_ERR_SHAPE;
@@ -716,8 +721,31 @@ sparrow_status sparrow_anchor_attn(sparrow_ctx* c, const void* q, const void* k,
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
     if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) { cudaGetLastError(); cap = cudaStreamCaptureStatusActive; }
     const bool chained = c->use_pdl && cap == cudaStreamCaptureStatusNone;
-    if ((s = launch_split_gather(c, plan, sy, q, k, v, nullptr, anchor_idx, n_anchor, window, out, lse, st, chained)) != SPARROW_OK) return s;
+    if ((s = launch_split_gather(c, plan, sy, q, k, v, parents, anchor_idx, n_anchor, window, out, lse, st, chained,
+                                 tree_nodes)) != SPARROW_OK)
+        return s;
     return launch_combine(c, plan, sy, out, lse, st, chained);
+}
+}  // namespace
+
+extern "C" {
+
+sparrow_status sparrow_anchor_attn(sparrow_ctx* c, const void* q, const void* k, const void* v,
+                                   const int32_t* anchor_idx, int32_t n_anchor, int32_t window, int32_t T,
+                                   void* out, float* lse, void* stream)
+{
+    return anchor_call(c, q, k, v, anchor_idx, n_anchor, window, nullptr, 0, T, out, lse, stream);
+}
+
+sparrow_status sparrow_anchor_attn_tree(sparrow_ctx* c, const void* q, const void* k, const void* v,
+                                        const int32_t* anchor_idx, int32_t n_anchor, int32_t window,
+                                        const int32_t* parents, int32_t T_tree, int32_t T_new, void* out, float* lse,
+                                        void* stream)
+{
+    if (!parents) return SPARROW_ERR_NULL;
+    if (T_tree < 1 || T_tree > kMaxT || T_new < 1 || T_new > T_tree) return SPARROW_ERR_SHAPE;
+    if (n_anchor < T_tree) return SPARROW_ERR_ANCHOR;
+    return anchor_call(c, q, k, v, anchor_idx, n_anchor, window, parents, T_tree, T_new, out, lse, stream);
 }
 
 sparrow_status sparrow_verify_step_host(sparrow_ctx* c, const void* q_host, const void* k_new_host,

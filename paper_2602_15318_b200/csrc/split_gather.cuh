@@ -21,10 +21,12 @@ struct SplitArgs {
     const __nv_bfloat16* q;
     const __nv_bfloat16* k;
     const __nv_bfloat16* v;
-    const int32_t* parents;      // verification: DEV [B][T]; nullptr in anchored mode
+    const int32_t* parents;      // verification: DEV [B][T]; anchored: DEV [B][tree_nodes] or nullptr (chain)
     const int32_t* anchor_idx;   // anchored: DEV [B][n_anchor]; nullptr in verification mode
     int32_t n_anchor;
     int32_t window;
+    int32_t tree_nodes;          // anchored mode with a draft tree: its nodes are the last tree_nodes anchors, the
+                                 // queries the last T of them; 0 = chain rule for every anchor
     int32_t n_q_heads;
     int32_t kv_capacity;
     int64_t kv_stride_batch;
@@ -101,6 +103,7 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
     const int32_t* aidx = anchored ? args.anchor_idx + (size_t)it.b * args.n_anchor : nullptr;
 
     // ---- prologue: masks / query positions, packed Q block -> registers --------------------
+    const int tree_nodes = anchored ? args.tree_nodes : 0;
     if (tid < T) {
         if (anchored) {
             int p = aidx[args.n_anchor - T + tid];
@@ -110,6 +113,8 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
             anc_s[tid] = ancestor_word(args.parents + (size_t)it.b * T, T, tid, args.status);
         }
     }
+    if (tid < tree_nodes)
+        anc_s[tid] = ancestor_word(args.parents + (size_t)it.b * tree_nodes, tree_nodes, tid, args.status);
     {
         constexpr int kChunksPerThread = kRows * 16 / kThreads;      // 8: all loads first, then the stores
         uint4 val[kChunksPerThread];
@@ -146,7 +151,7 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
         row_t[rr] = it.group * kTokPerBlock + lr / kGroup;
         row_ok[rr] = lr < kTokPerBlock * kGroup && row_t[rr] < T;
         const int t = row_ok[rr] ? row_t[rr] : 0;
-        row_anc[rr] = anchored ? 0ull : anc_s[t];
+        row_anc[rr] = anchored ? (tree_nodes > 0 ? anc_s[tree_nodes - T + t] : 0ull) : anc_s[t];
         row_qpos[rr] = anchored ? qpos_s[t] : 0;
     }
     __syncthreads();                      // Q staging area is reused by the K/V ring from here on
@@ -230,7 +235,11 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
                         if (anchored) {
                             const int p = apos_s[stage * kTile + col];
                             const int qp = row_qpos[rr];
-                            vis = p >= 0 && qp >= 0 && p <= qp && (args.window <= 0 || qp - args.window < p);
+                            const int node = j - (args.n_anchor - tree_nodes);     // >= 0: a node of the draft tree
+                            if (tree_nodes > 0 && node >= 0)
+                                vis = p >= 0 && qp >= 0 && ((row_anc[rr] >> node) & 1ull);
+                            else
+                                vis = p >= 0 && qp >= 0 && p <= qp && (args.window <= 0 || qp - args.window < p);
                         } else if (j >= kv_len) {
                             vis = (row_anc[rr] >> (j - kv_len)) & 1ull;
                         }

@@ -277,3 +277,60 @@ def test_argument_errors_launch_nothing():
     with pytest.raises(B.SparrowError):
         B.Context(1, 100, 51200, 12800, W.SCALE, head_dim=64, n_q_heads=28)
     assert ctx.launch_count() == n0
+
+
+# ---- anchored mode with tree-structured draft tokens ---------------------------------------------
+
+def _run_anchor_tree(ac, parents, T_tree, T_new, ctx=None):
+    ctx = ctx or B.Context.for_cache(ac.k, W.SCALE)
+    q = ac.q[:, T_tree - T_new:].contiguous()
+    out = torch.full_like(q, float("nan"))
+    lse = torch.full((ac.B, W.HQ, T_new), float("nan"), dtype=torch.float32, device=DEV)
+    B.sparrow_anchor_attn_tree(ctx, q, ac.k, ac.v, ac.anchor_idx, ac.n_anchor, ac.window, parents, T_tree, T_new,
+                               out, lse)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == 0
+    ref_out, ref_lse = oracle.anchor_attn_tree(W.bf16_bits(q), W.bf16_bits(ac.k), W.bf16_bits(ac.v),
+                                               ac.anchor_idx.cpu().numpy(), ac.window, parents.cpu().numpy(), W.SCALE)
+    return out, lse, ref_out, ref_lse
+
+
+@pytest.mark.parametrize("seq_len,spans,window,T_tree,T_new,batch", [
+    (1500, [[32, 1300]], 0, 12, 12, 1),          # whole tree, no window
+    (1500, [[32, 1300]], 128, 12, 5, 2),         # only the nodes of the latest step are queries
+    (5000, [[100, 4200]], 600, 40, 8, 1),        # many text anchors: several pieces, tree inside the last tile
+    (900, [[0, 850]], 0, 64, 64, 1),             # largest tree: four row blocks' worth of query rows
+    (300, [], 0, 9, 1, 3),                       # no visual span, a single query node
+])
+def test_anchor_tree_small(seq_len, spans, window, T_tree, T_new, batch):
+    ac = W.make_anchor_case(4100 + T_tree, seq_len, spans, window, T_tree, batch, DEV)
+    parents = torch.tensor([W.random_tree_parents(4200 + 31 * b + T_tree, 99, T_tree) for b in range(batch)],
+                           dtype=torch.int32, device=DEV)
+    out, lse, ref_out, ref_lse = _run_anchor_tree(ac, parents, T_tree, T_new)
+    check(out, lse, ref_out, ref_lse)
+
+
+def test_anchor_tree_with_chain_parents_is_the_chain_mode():
+    ac = W.make_anchor_case(4300, 2000, [[64, 1700]], 512, 10, 2, DEV)
+    chain = torch.tensor([list(range(-1, 9))] * 2, dtype=torch.int32, device=DEV)
+    ctx = B.Context.for_cache(ac.k, W.SCALE)
+    out_c, lse_c, _ = run_anchor(ac, ctx)
+    out_t, lse_t, _, _ = _run_anchor_tree(ac, chain, 10, 10, ctx)
+    assert torch.equal(out_c, out_t) and torch.equal(lse_c, lse_t)
+
+
+def test_anchor_tree_argument_errors():
+    ac = W.make_anchor_case(4400, 500, [[10, 400]], 0, 8, 1, DEV)
+    par = torch.tensor([[-1, 0, 0, 1, 1, 2, 3, 3]], dtype=torch.int32, device=DEV)
+    ctx = B.Context.for_cache(ac.k, W.SCALE)
+    out = torch.empty_like(ac.q); lse = torch.empty((1, W.HQ, 8), dtype=torch.float32, device=DEV)
+    n0 = ctx.launch_count()
+    for T_tree, T_new, n_anchor in ((8, 9, ac.n_anchor), (0, 1, ac.n_anchor), (65, 8, ac.n_anchor), (8, 8, 5)):
+        with pytest.raises(B.SparrowError):
+            B.sparrow_anchor_attn_tree(ctx, ac.q, ac.k, ac.v, ac.anchor_idx, n_anchor, 0, par, T_tree, T_new, out, lse)
+    assert ctx.launch_count() == n0
+    bad = torch.tensor([[-1, 0, 5, 1, 1, 2, 3, 3]], dtype=torch.int32, device=DEV)      # parents[2] = 5 > 2
+    B.sparrow_anchor_attn_tree(ctx, ac.q, ac.k, ac.v, ac.anchor_idx, ac.n_anchor, 0, bad, 8, 8, out, lse)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == 3          # SPARROW_ERR_TREE, reported, nothing read out of bounds
+    assert torch.isfinite(out.float()).all()
