@@ -437,7 +437,39 @@ def extra_configs(W, B, torch, dev, l2, peak):
     torch.cuda.synchronize(); ev0.record(); anchor_loop(5000); ev1.record(); torch.cuda.synchronize()
     emit({"config": "C4", "workload": ac[0].name, "us_per_call": ev0.elapsed_time(ev1) * 1e3 / 5000,
           "gathered_bytes": ac[0].kv_bytes(), "note": "launched from Python; latency-bound"})
-    del ac, actx
+    # the same call on a compacted cache: rows gathered once, then the tensor-core kernel on a contiguous stream
+    cap_c = ac[0].n_anchor
+    kc = [torch.empty((1, W.HKV, cap_c, W.D), dtype=torch.bfloat16, device=dev) for _ in ac]
+    vc = [torch.empty_like(x) for x in kc]
+    for c, kk, vv in zip(ac, kc, vc):
+        B.sparrow_compact_anchors(actx, c.k, c.v, c.anchor_idx, c.n_anchor, kk, vv, cap_c, 0)
+    cctx = B.Context.for_cache(kc[0], W.SCALE)
+    cctx.set_plan_policy(B.PLAN_LATENCY)
+    chain = torch.arange(-1, ac[0].T - 1, dtype=torch.int32, device=dev)[None].contiguous()
+    cbatch = B.VerifyBatch([(c.q, kk, vv, [c.n_anchor - c.T], chain, c.T, aout, alse) for c, kk, vv in zip(ac, kc, vc)])
+    time_calls(cctx, cbatch, 200, B, torch)
+    emit({"config": "C4-compact", "workload": "C4 on the compacted anchor rows (sparrow_compact_anchors once, then sparrow_verify_attn)",
+          "us_per_call": time_calls(cctx, cbatch, 5000, B, torch), "note": "enqueued from C; contiguous TMA stream, no gather"})
+    del kc, vc, cctx, cbatch
+    # the same anchors with a 32-node draft tree behind them, queries = its last 8 nodes
+    T_tree, T_new = 32, 8
+    tc_ = [W.make_anchor_case(W.config_seed(3, 100 + r), 26112, [[64, 25664]], 1024, T_tree, 1, dev) for r in range(8)]
+    par = torch.tensor([W.random_tree_parents(W.config_seed(3, 0), 77, T_tree)], dtype=torch.int32, device=dev)
+    tctx = B.Context.for_cache(tc_[0].k, W.SCALE)
+    tq = [c.q[:, T_tree - T_new:].contiguous() for c in tc_]
+    tout = torch.empty_like(tq[0])
+    tlse = torch.empty((1, W.HQ, T_new), dtype=torch.float32, device=dev)
+
+    def tree_loop(n):
+        for i in range(n):
+            c = tc_[i % len(tc_)]
+            B.sparrow_anchor_attn_tree(tctx, tq[i % len(tc_)], c.k, c.v, c.anchor_idx, c.n_anchor, c.window, par,
+                                       T_tree, T_new, tout, tlse)
+    tree_loop(200)
+    torch.cuda.synchronize(); ev0.record(); tree_loop(5000); ev1.record(); torch.cuda.synchronize()
+    emit({"config": "C4-tree", "workload": "anchored, 448 text anchors + 32-node draft tree, 8 query nodes",
+          "us_per_call": ev0.elapsed_time(ev1) * 1e3 / 5000, "note": "launched from Python; latency-bound"})
+    del ac, actx, tc_, tctx
     torch.cuda.empty_cache()
     # C5: 28 layers, each with its own cache (about 15 GB resident)
     layers = [W.make_config(4, dev, layer=l) for l in range(28)]

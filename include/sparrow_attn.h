@@ -187,6 +187,32 @@ sparrow_status sparrow_anchor_attn_tree(sparrow_ctx* ctx, const void* q, const v
                                         const int32_t* parents, int32_t T_tree, int32_t T_new,
                                         void* out, float* lse, void* stream);
 
+/* Row movers (Section 3.1: the draft model keeps the text-anchored states and discards the visual
+ * KV cache; the paper gives no procedure, these two calls are this library's).  Both are plain
+ * copies, bit-exact, one ordinary kernel each, ordered by the stream like any other kernel.
+ *
+ * sparrow_kv_append: writes the T new rows of every (sequence, KV head) into cache rows
+ * [kv_len[b], kv_len[b] + T) -- what sparrow_verify_attn() expects to find there.
+ *   k_new, v_new  DEV bf16 [batch][n_kv_heads][T][128], contiguous
+ *   k_cache, v_cache  DEV, the context's layout;  kv_len HOST int32 [batch]
+ * SPARROW_ERR_SHAPE unless 1 <= T <= SPARROW_MAX_T and kv_len[b] + T <= kv_capacity.
+ *
+ * sparrow_compact_anchors: copies rows anchor_idx[b][0 .. n_anchor) of k / v (the context's layout)
+ * to rows [dst_row, dst_row + n_anchor) of a compact cache laid out
+ * [batch][n_kv_heads][compact_capacity][128], contiguous.  On the compact cache the anchored mode
+ * without a lower window bound is sparrow_verify_attn() with kv_len = (anchors before the draft
+ * block): a contiguous stream for the tensor-core kernel instead of a gather.
+ *   anchor_idx  DEV int32 [batch][n_anchor]; an entry outside [0, kv_capacity) is not read: its
+ *               row is written as zeros and the anchor status bit is set.
+ * SPARROW_ERR_ANCHOR unless 1 <= n_anchor <= kv_capacity; SPARROW_ERR_SHAPE unless
+ * 0 <= dst_row and dst_row + n_anchor <= compact_capacity.  Both need a workspace (status word). */
+sparrow_status sparrow_kv_append(sparrow_ctx* ctx, const void* k_new, const void* v_new, void* k_cache,
+                                 void* v_cache, const int32_t* kv_len, int32_t T, void* stream);
+sparrow_status sparrow_compact_anchors(sparrow_ctx* ctx, const void* k, const void* v,
+                                       const int32_t* anchor_idx, int32_t n_anchor, void* k_compact,
+                                       void* v_compact, int32_t compact_capacity, int32_t dst_row,
+                                       void* stream);
+
 /* Verification step with HOST buffers (what a caller without device-side glue uses): copies q,
  * the T new K/V rows per (batch, KV head) and parents to the device, writes the new rows into
  * cache rows [kv_len[b], kv_len[b]+T), runs (a), copies out / lse back and synchronises `stream`.

@@ -25,7 +25,7 @@ EXPORTS = ["sparrow_create", "sparrow_destroy", "sparrow_workspace_bytes", "spar
            "sparrow_build_ancestor_masks", "sparrow_build_anchor_idx",
            "sparrow_debug_ancestor_masks_device", "sparrow_debug_wait_counter", "sparrow_plan_splits",
            "sparrow_last_device_status", "sparrow_debug_status_word", "sparrow_launch_count",
-           "sparrow_set_plan_policy", "sparrow_plan_target_items", "sparrow_anchor_attn_tree",
+           "sparrow_set_plan_policy", "sparrow_plan_target_items", "sparrow_anchor_attn_tree", "sparrow_kv_append", "sparrow_compact_anchors",
            "sparrow_status_string"]
 
 
@@ -66,6 +66,8 @@ def lib():
         L.sparrow_verify_attn_batch.argtypes = [vp, vp, i32, vp]
         L.sparrow_verify_attn_static.argtypes = [ctypes.POINTER(Layout), vp, vp, vp, vp, vp, i32, vp, vp, vp]
         L.sparrow_anchor_attn.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp]
+        L.sparrow_kv_append.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp]
+        L.sparrow_compact_anchors.argtypes = [vp, vp, vp, vp, i32, vp, vp, i32, i32, vp]
         L.sparrow_anchor_attn_tree.argtypes = [vp, vp, vp, vp, vp, i32, i32, vp, i32, i32, vp, vp, vp]
         L.sparrow_verify_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp]
         L.sparrow_build_ancestor_masks.argtypes = [vp, i32, vp]
@@ -236,6 +238,18 @@ def sparrow_anchor_attn_tree(ctx: Context, q, k, v, anchor_idx, n_anchor: int, w
                                         window, _ptr(parents), T_tree, T_new, _ptr(out), _ptr(lse),
                                         _stream_handle(stream)),
          "sparrow_anchor_attn_tree")
+
+
+def sparrow_kv_append(ctx: Context, k_new, v_new, k_cache, v_cache, kv_len: Sequence[int], T: int, stream=None):
+    _chk(lib().sparrow_kv_append(ctx.handle, _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache),
+                                 _i32_array(kv_len), T, _stream_handle(stream)), "sparrow_kv_append")
+
+
+def sparrow_compact_anchors(ctx: Context, k, v, anchor_idx, n_anchor: int, k_compact, v_compact,
+                            compact_capacity: int, dst_row: int = 0, stream=None):
+    _chk(lib().sparrow_compact_anchors(ctx.handle, _ptr(k), _ptr(v), _ptr(anchor_idx), n_anchor, _ptr(k_compact),
+                                       _ptr(v_compact), compact_capacity, dst_row, _stream_handle(stream)),
+         "sparrow_compact_anchors")
 
 
 def sparrow_verify_step_host(ctx: Context, q_host, k_new_host, v_new_host, k_cache, v_cache,

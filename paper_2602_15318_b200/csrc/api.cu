@@ -16,6 +16,7 @@
 
 #include "combine.cuh"
 #include "common.cuh"
+#include "kv_rows.cuh"
 #include "split_gather.cuh"
 #include "verify_tc.cuh"
 
@@ -746,6 +747,81 @@ sparrow_status sparrow_anchor_attn_tree(sparrow_ctx* c, const void* q, const voi
     if (T_tree < 1 || T_tree > kMaxT || T_new < 1 || T_new > T_tree) return SPARROW_ERR_SHAPE;
     if (n_anchor < T_tree) return SPARROW_ERR_ANCHOR;
     return anchor_call(c, q, k, v, anchor_idx, n_anchor, window, parents, T_tree, T_new, out, lse, stream);
+}
+
+sparrow_status sparrow_kv_append(sparrow_ctx* c, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                                 const int32_t* kv_len, int32_t T, void* stream)
+{
+    if (!c || !k_new || !v_new || !k_cache || !v_cache || !kv_len) return SPARROW_ERR_NULL;
+    if (T < 1 || T > kMaxT) return SPARROW_ERR_SHAPE;
+    if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(k_cache) || !aligned16(v_cache)) return SPARROW_ERR_SHAPE;
+    if (!c->ws) return SPARROW_ERR_WORKSPACE;
+    const sparrow_layout& L = c->layout;
+    RowMoveArgs a;
+    std::memset(&a, 0, sizeof a);
+    for (int b = 0; b < L.batch; ++b) {
+        if (kv_len[b] < 0 || (int64_t)kv_len[b] + T > L.kv_capacity) return SPARROW_ERR_SHAPE;
+        a.dst_row0[b] = kv_len[b];
+    }
+    a.k_src = static_cast<const __nv_bfloat16*>(k_new);
+    a.v_src = static_cast<const __nv_bfloat16*>(v_new);
+    a.k_dst = static_cast<__nv_bfloat16*>(k_cache);
+    a.v_dst = static_cast<__nv_bfloat16*>(v_cache);
+    a.src_rows = nullptr;
+    a.n_rows = T;
+    a.batch = L.batch;
+    a.n_kv_heads = L.n_kv_heads;
+    a.src_capacity = T;
+    a.src_stride_head = (int64_t)T * kD;
+    a.src_stride_batch = a.src_stride_head * L.n_kv_heads;
+    a.dst_stride_batch = L.kv_stride_batch;
+    a.dst_stride_head = L.kv_stride_head;
+    a.status = reinterpret_cast<unsigned*>(c->ws);
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return SPARROW_ERR_CUDA;
+    const long long threads = (long long)L.batch * L.n_kv_heads * T * 16;
+    move_rows_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(a);
+    if (cudaGetLastError() != cudaSuccess) return SPARROW_ERR_CUDA;
+    c->launches.fetch_add(1);
+    return SPARROW_OK;
+}
+
+sparrow_status sparrow_compact_anchors(sparrow_ctx* c, const void* k, const void* v, const int32_t* anchor_idx,
+                                       int32_t n_anchor, void* k_compact, void* v_compact, int32_t compact_capacity,
+                                       int32_t dst_row, void* stream)
+{
+    if (!c || !k || !v || !anchor_idx || !k_compact || !v_compact) return SPARROW_ERR_NULL;
+    if (!aligned16(k) || !aligned16(v) || !aligned16(k_compact) || !aligned16(v_compact)) return SPARROW_ERR_SHAPE;
+    if (n_anchor < 1 || n_anchor > c->layout.kv_capacity) return SPARROW_ERR_ANCHOR;
+    if (compact_capacity < 1 || dst_row < 0 || (int64_t)dst_row + n_anchor > compact_capacity) return SPARROW_ERR_SHAPE;
+    if (!c->ws) return SPARROW_ERR_WORKSPACE;
+    const sparrow_layout& L = c->layout;
+    RowMoveArgs a;
+    std::memset(&a, 0, sizeof a);
+    for (int b = 0; b < L.batch; ++b) a.dst_row0[b] = dst_row;
+    a.k_src = static_cast<const __nv_bfloat16*>(k);
+    a.v_src = static_cast<const __nv_bfloat16*>(v);
+    a.k_dst = static_cast<__nv_bfloat16*>(k_compact);
+    a.v_dst = static_cast<__nv_bfloat16*>(v_compact);
+    a.src_rows = anchor_idx;
+    a.n_rows = n_anchor;
+    a.batch = L.batch;
+    a.n_kv_heads = L.n_kv_heads;
+    a.src_capacity = L.kv_capacity;
+    a.src_stride_batch = L.kv_stride_batch;
+    a.src_stride_head = L.kv_stride_head;
+    a.dst_stride_head = (int64_t)compact_capacity * kD;
+    a.dst_stride_batch = a.dst_stride_head * L.n_kv_heads;
+    a.status = reinterpret_cast<unsigned*>(c->ws);
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return SPARROW_ERR_CUDA;
+    const long long threads = (long long)L.batch * L.n_kv_heads * n_anchor * 16;
+    long long blocks = (threads + 255) / 256;
+    if (blocks > 8LL * c->n_sm) blocks = 8LL * c->n_sm;
+    move_rows_kernel<<<(unsigned)blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(a);
+    if (cudaGetLastError() != cudaSuccess) return SPARROW_ERR_CUDA;
+    c->launches.fetch_add(1);
+    return SPARROW_OK;
 }
 
 sparrow_status sparrow_verify_step_host(sparrow_ctx* c, const void* q_host, const void* k_new_host,

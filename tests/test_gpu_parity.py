@@ -334,3 +334,66 @@ def test_anchor_tree_argument_errors():
     torch.cuda.synchronize()
     assert ctx.last_device_status() == 3          # SPARROW_ERR_TREE, reported, nothing read out of bounds
     assert torch.isfinite(out.float()).all()
+
+
+# ---- row movers: append of the draft rows, compaction of the anchored rows -------------------
+
+def test_kv_append_is_a_bit_exact_copy_into_the_right_rows():
+    case = W.make_verify_case(4500, [300, 77], 6, "chain", DEV, capacity=400)
+    ctx = B.Context.for_cache(case.k, W.SCALE)
+    k0, v0 = case.k.clone(), case.v.clone()
+    k_new = W.normal_bf16(4501, 40, (2, W.HKV, 6, W.D), DEV)
+    v_new = W.normal_bf16(4501, 41, (2, W.HKV, 6, W.D), DEV)
+    B.sparrow_kv_append(ctx, k_new, v_new, case.k, case.v, case.kv_len, 6)
+    torch.cuda.synchronize()
+    for b, n in enumerate(case.kv_len):
+        assert torch.equal(case.k[b, :, n:n + 6], k_new[b]) and torch.equal(case.v[b, :, n:n + 6], v_new[b])
+        k0[b, :, n:n + 6] = k_new[b]
+        v0[b, :, n:n + 6] = v_new[b]
+    assert torch.equal(case.k, k0) and torch.equal(case.v, v0)          # nothing else was touched
+    with pytest.raises(B.SparrowError):
+        B.sparrow_kv_append(ctx, k_new, v_new, case.k, case.v, [396, 10], 6)     # 396 + 6 > capacity
+
+
+def test_compacted_anchors_are_a_bit_exact_gather_and_serve_the_verify_kernel():
+    """Compacting the anchored rows and running the verification kernel on the short cache is the
+    anchored mode without a lower window bound: same oracle, contiguous stream instead of a gather."""
+    T = 10
+    ac = W.make_anchor_case(4600, 3000, [[40, 2600]], 0, T, 2, DEV)
+    ctx = B.Context.for_cache(ac.k, W.SCALE)
+    cap_c = ac.n_anchor + 7
+    kc = torch.zeros((2, W.HKV, cap_c, W.D), dtype=torch.bfloat16, device=DEV)
+    vc = torch.zeros_like(kc)
+    B.sparrow_compact_anchors(ctx, ac.k, ac.v, ac.anchor_idx, ac.n_anchor, kc, vc, cap_c, 0)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == 0
+    rows = ac.anchor_idx[0].long()
+    assert torch.equal(kc[:, :, :ac.n_anchor], ac.k[:, :, rows]) and torch.equal(vc[:, :, :ac.n_anchor], ac.v[:, :, rows])
+    assert not kc[:, :, ac.n_anchor:].any()
+    # tree among the draft rows, all text anchors visible: the verification kernel on the compact cache
+    parents = torch.tensor([W.random_tree_parents(4601 + b, 99, T) for b in range(2)], dtype=torch.int32, device=DEV)
+    cctx = B.Context.for_cache(kc, W.SCALE)
+    out = torch.full_like(ac.q, float("nan"))
+    lse = torch.full((2, W.HQ, T), float("nan"), dtype=torch.float32, device=DEV)
+    B.sparrow_verify_attn(cctx, ac.q, kc, vc, [ac.n_anchor - T] * 2, parents, T, out, lse)
+    torch.cuda.synchronize()
+    assert cctx.last_device_status() == 0
+    ref_out, ref_lse = oracle.anchor_attn_tree(W.bf16_bits(ac.q), W.bf16_bits(ac.k), W.bf16_bits(ac.v),
+                                               ac.anchor_idx.cpu().numpy(), 0, parents.cpu().numpy(), W.SCALE)
+    check(out, lse, ref_out, ref_lse)
+
+
+def test_compact_anchors_reports_a_bad_index_and_writes_zeros():
+    ac = W.make_anchor_case(4700, 600, [[10, 500]], 0, 4, 1, DEV)
+    ctx = B.Context.for_cache(ac.k, W.SCALE)
+    idx = ac.anchor_idx.clone()
+    idx[0, 3] = ac.capacity + 5
+    kc = torch.ones((1, W.HKV, ac.n_anchor, W.D), dtype=torch.bfloat16, device=DEV)
+    vc = torch.ones_like(kc)
+    B.sparrow_compact_anchors(ctx, ac.k, ac.v, idx, ac.n_anchor, kc, vc, ac.n_anchor, 0)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == 4                      # SPARROW_ERR_ANCHOR
+    assert not kc[:, :, 3].any() and not vc[:, :, 3].any()
+    assert torch.equal(kc[:, :, 4], ac.k[:, :, int(idx[0, 4])])
+    with pytest.raises(B.SparrowError):
+        B.sparrow_compact_anchors(ctx, ac.k, ac.v, idx, ac.n_anchor, kc, vc, ac.n_anchor, 1)     # does not fit
