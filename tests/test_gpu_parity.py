@@ -41,6 +41,34 @@ def test_verify_small(kv_len, T, tree):
     check(out, lse, ref_out, ref_lse)
 
 
+@pytest.mark.parametrize("T", [17, 18, 19, 35, 36, 37, 54, 55, 63])
+@pytest.mark.parametrize("policy", [B.PLAN_LATENCY, B.PLAN_THROUGHPUT])
+def test_verify_row_block_boundaries(T, policy):
+    """Draft blocks around the 18-token row blocks and 36-token row groups, random trees, a key
+    count that ends inside a tile; one wave of pieces and a few long ones."""
+    case = W.make_verify_case(3000 + T, [2300 - T, 700], T, "random", DEV)
+    out, lse, _ = run_verify(case, policy=policy)
+    ref_out, ref_lse = oracle_verify(case)
+    check(out, lse, ref_out, ref_lse)
+
+
+@pytest.mark.parametrize("n_keys", [127, 128, 129, 255, 256, 257, 384])
+def test_verify_key_counts_around_tile_boundaries(n_keys):
+    T = 6
+    case = W.make_verify_case(3100 + n_keys, [n_keys - T], T, "chain", DEV)
+    out, lse, _ = run_verify(case)
+    ref_out, ref_lse = oracle_verify(case)
+    check(out, lse, ref_out, ref_lse)
+
+
+def test_verify_largest_batch():
+    lens = [(37 * i) % 300 for i in range(64)]
+    case = W.make_verify_case(3200, lens, 5, "random", DEV)
+    out, lse, _ = run_verify(case)
+    ref_out, ref_lse = oracle_verify(case)
+    check(out, lse, ref_out, ref_lse)
+
+
 def test_verify_capacity_larger_than_used_and_garbage_tail():
     """Rows past kv_len+T may hold anything, NaN and Inf patterns included."""
     case = W.make_verify_case(77, [200, 333], 6, "random", DEV, capacity=700)
