@@ -219,3 +219,40 @@ def anchor_attn_tree(q, k, v, idx, window, parents, scale, rows=None, n_threads=
     vis = np.stack([anchor_tree_visibility(idx[b], window, parents[b], T_new) for b in range(B)])
     return attention(q, k, v, vis, np.full(B, idx.shape[1], dtype=np.int32), scale, key_rows=idx,
                      rows=rows, n_threads=n_threads)
+
+
+def greedy_accept(draft_tokens, parents, target_next):
+    """Greedy (temperature 0) verification of a draft tree (Appendix A, "Speculative Decoding": the
+    target checks the candidates of the tree in one forward pass and keeps what it would have
+    produced itself, which is what makes the method lossless).
+
+    draft_tokens int [T]; parents int [T] (-1 = root, parents[i] < i); target_next int [T + 1]:
+    target_next[0] is the target's own next token after the committed prefix, target_next[1 + i]
+    its next token after node i.  A node is accepted iff its token is what the target produces
+    after its parent (after the prefix, for a root) and its parent is accepted.  Returns
+    (path, bonus): the nodes of the deepest accepted chain from its root down (ties: the chain
+    whose last node has the smallest index) and the target's token after the chain's last node
+    (target_next[0] when nothing is accepted).  Plain loops, straight from this definition."""
+    tok = [int(x) for x in draft_tokens]
+    par = [int(x) for x in parents]
+    nxt = [int(x) for x in target_next]
+    T = len(tok)
+    assert len(par) == T and len(nxt) == T + 1
+    accepted, depth = [False] * T, [0] * T
+    for i in range(T):
+        p = par[i]
+        assert -1 <= p < i
+        ok_parent = True if p < 0 else accepted[p]
+        accepted[i] = ok_parent and tok[i] == nxt[p + 1]
+        depth[i] = (0 if p < 0 else depth[p]) + 1 if accepted[i] else 0
+    best = -1
+    for i in range(T):
+        if accepted[i] and (best < 0 or depth[i] > depth[best]):
+            best = i
+    path = []
+    i = best
+    while i >= 0:
+        path.append(i)
+        i = par[i]
+    path.reverse()
+    return path, nxt[best + 1]

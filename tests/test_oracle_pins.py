@@ -451,3 +451,50 @@ def test_anchor_tree_forest_of_roots_sees_text_and_itself_only():
     vis = oracle.anchor_tree_visibility(idx, 0, np.array([-1, -1, -1], dtype=np.int32), 3)
     assert np.array_equal(vis[:, :3], np.ones((3, 3), dtype=np.uint8))
     assert np.array_equal(vis[:, 3:], np.eye(3, dtype=np.uint8))
+
+
+# ---- greedy acceptance of a draft tree -----------------------------------------------------------
+
+def _accepted_paths_brute_force(tok, par, nxt):
+    """Every node whose whole chain from its root matches the target, found by walking up from the
+    node and checking each step on its own (independent of the oracle's forward recurrence)."""
+    good = []
+    for i in range(len(tok)):
+        chain, n = [], i
+        while n >= 0:
+            chain.append(n)
+            n = par[n]
+        chain.reverse()
+        if all(tok[c] == nxt[par[c] + 1] for c in chain):
+            good.append(chain)
+    return good
+
+
+def test_greedy_accept_brute_force_on_random_trees():
+    rng = np.random.default_rng(11)
+    for trial in range(300):
+        T = int(rng.integers(1, 12))
+        par = [int(rng.integers(-1, i)) for i in range(T)]
+        nxt = [int(rng.integers(0, 3)) for _ in range(T + 1)]
+        tok = [int(rng.integers(0, 3)) for _ in range(T)]
+        path, bonus = oracle.greedy_accept(tok, par, nxt)
+        good = _accepted_paths_brute_force(tok, par, nxt)
+        if not good:
+            assert path == [] and bonus == nxt[0]
+            continue
+        longest = max(len(c) for c in good)
+        expect = min((c for c in good if len(c) == longest), key=lambda c: c[-1])
+        assert path == expect and bonus == nxt[expect[-1] + 1]
+
+
+def test_greedy_accept_closed_forms():
+    chain = [-1, 0, 1, 2, 3]
+    nxt = [7, 8, 9, 10, 11, 12]
+    assert oracle.greedy_accept([7, 8, 9, 10, 11], chain, nxt) == ([0, 1, 2, 3, 4], 12)     # everything matches
+    assert oracle.greedy_accept([7, 8, 0, 10, 11], chain, nxt) == ([0, 1], 9)               # first mismatch cuts the chain
+    assert oracle.greedy_accept([0, 8, 9, 10, 11], chain, nxt) == ([], 7)                   # nothing accepted: the target's own token
+    # two roots, the second one right; its two children compete, the deeper branch wins
+    par = [-1, -1, 1, 1, 3]
+    assert oracle.greedy_accept([5, 7, 8, 8, 4], par, [7, 0, 8, 0, 4, 6]) == ([1, 3, 4], 6)
+    # equal depth: the chain ending at the smaller index
+    assert oracle.greedy_accept([5, 7, 8, 8, 1], par, [7, 0, 8, 0, 4, 6]) == ([1, 2], 0)
