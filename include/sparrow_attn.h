@@ -213,6 +213,34 @@ sparrow_status sparrow_compact_anchors(sparrow_ctx* ctx, const void* k, const vo
                                        void* v_compact, int32_t compact_capacity, int32_t dst_row,
                                        void* stream);
 
+/* After the verification pass (Appendix A, "Speculative Decoding": the target keeps exactly what it
+ * would have produced itself; the paper relies on the standard procedure and does not restate it).
+ *
+ * sparrow_accept_greedy: temperature-0 acceptance of a draft tree.
+ *   draft_tokens DEV int32 [batch][T]      token of every draft node
+ *   parents      DEV int32 [batch][T]      as in (a)
+ *   target_next  DEV int32 [batch][T + 1]  [0]: the target's next token after the committed prefix,
+ *                                          [1 + i]: its next token after node i (argmax of the logits
+ *                                          the verification pass produced at that node)
+ *   path_out     DEV int32 [batch][T]      nodes of the deepest accepted chain, root first, then -1
+ *   n_accept_out DEV int32 [batch]         its length (0 .. T)
+ *   bonus_out    DEV int32 [batch]         the target's token after the chain's last node
+ * A node is accepted iff its token equals target_next[parent + 1] and its parent is accepted (a
+ * root: iff it equals target_next[0]); among chains of equal depth the one ending at the smallest
+ * node index wins.  A malformed parent sets the tree status bit and counts as a root.
+ *
+ * sparrow_kv_keep_accepted: moves the K/V rows of the accepted nodes, rows kv_len[b] + path[i], to
+ * rows kv_len[b] + i (i < n_accept[b]) of one cache pair, in place; afterwards the committed
+ * length is kv_len[b] + n_accept[b].  One call per layer.  kv_len is HOST, path / n_accept are the
+ * device arrays sparrow_accept_greedy() wrote.
+ * Both: SPARROW_ERR_SHAPE unless 1 <= T <= SPARROW_MAX_T (and kv_len[b] + T <= kv_capacity). */
+sparrow_status sparrow_accept_greedy(sparrow_ctx* ctx, const int32_t* draft_tokens, const int32_t* parents,
+                                     const int32_t* target_next, int32_t T, int32_t* path_out,
+                                     int32_t* n_accept_out, int32_t* bonus_out, void* stream);
+sparrow_status sparrow_kv_keep_accepted(sparrow_ctx* ctx, void* k_cache, void* v_cache,
+                                        const int32_t* kv_len, const int32_t* path,
+                                        const int32_t* n_accept, int32_t T, void* stream);
+
 /* Verification step with HOST buffers (what a caller without device-side glue uses): copies q,
  * the T new K/V rows per (batch, KV head) and parents to the device, writes the new rows into
  * cache rows [kv_len[b], kv_len[b]+T), runs (a), copies out / lse back and synchronises `stream`.

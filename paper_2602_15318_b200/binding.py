@@ -26,6 +26,7 @@ EXPORTS = ["sparrow_create", "sparrow_destroy", "sparrow_workspace_bytes", "spar
            "sparrow_debug_ancestor_masks_device", "sparrow_debug_wait_counter", "sparrow_plan_splits",
            "sparrow_last_device_status", "sparrow_debug_status_word", "sparrow_launch_count",
            "sparrow_set_plan_policy", "sparrow_plan_target_items", "sparrow_anchor_attn_tree", "sparrow_kv_append", "sparrow_compact_anchors",
+           "sparrow_accept_greedy", "sparrow_kv_keep_accepted",
            "sparrow_status_string"]
 
 
@@ -66,6 +67,8 @@ def lib():
         L.sparrow_verify_attn_batch.argtypes = [vp, vp, i32, vp]
         L.sparrow_verify_attn_static.argtypes = [ctypes.POINTER(Layout), vp, vp, vp, vp, vp, i32, vp, vp, vp]
         L.sparrow_anchor_attn.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp]
+        L.sparrow_accept_greedy.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp]
+        L.sparrow_kv_keep_accepted.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp]
         L.sparrow_kv_append.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp]
         L.sparrow_compact_anchors.argtypes = [vp, vp, vp, vp, i32, vp, vp, i32, i32, vp]
         L.sparrow_anchor_attn_tree.argtypes = [vp, vp, vp, vp, vp, i32, i32, vp, i32, i32, vp, vp, vp]
@@ -250,6 +253,19 @@ def sparrow_compact_anchors(ctx: Context, k, v, anchor_idx, n_anchor: int, k_com
     _chk(lib().sparrow_compact_anchors(ctx.handle, _ptr(k), _ptr(v), _ptr(anchor_idx), n_anchor, _ptr(k_compact),
                                        _ptr(v_compact), compact_capacity, dst_row, _stream_handle(stream)),
          "sparrow_compact_anchors")
+
+
+def sparrow_accept_greedy(ctx: Context, draft_tokens, parents, target_next, T: int, path_out, n_accept_out,
+                          bonus_out, stream=None):
+    _chk(lib().sparrow_accept_greedy(ctx.handle, _ptr(draft_tokens), _ptr(parents), _ptr(target_next), T,
+                                     _ptr(path_out), _ptr(n_accept_out), _ptr(bonus_out), _stream_handle(stream)),
+         "sparrow_accept_greedy")
+
+
+def sparrow_kv_keep_accepted(ctx: Context, k_cache, v_cache, kv_len: Sequence[int], path, n_accept, T: int,
+                             stream=None):
+    _chk(lib().sparrow_kv_keep_accepted(ctx.handle, _ptr(k_cache), _ptr(v_cache), _i32_array(kv_len), _ptr(path),
+                                        _ptr(n_accept), T, _stream_handle(stream)), "sparrow_kv_keep_accepted")
 
 
 def sparrow_verify_step_host(ctx: Context, q_host, k_new_host, v_new_host, k_cache, v_cache,

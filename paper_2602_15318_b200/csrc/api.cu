@@ -16,6 +16,7 @@
 
 #include "combine.cuh"
 #include "common.cuh"
+#include "accept.cuh"
 #include "kv_rows.cuh"
 #include "split_gather.cuh"
 #include "verify_tc.cuh"
@@ -819,6 +820,52 @@ sparrow_status sparrow_compact_anchors(sparrow_ctx* c, const void* k, const void
     long long blocks = (threads + 255) / 256;
     if (blocks > 8LL * c->n_sm) blocks = 8LL * c->n_sm;
     move_rows_kernel<<<(unsigned)blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(a);
+    if (cudaGetLastError() != cudaSuccess) return SPARROW_ERR_CUDA;
+    c->launches.fetch_add(1);
+    return SPARROW_OK;
+}
+
+sparrow_status sparrow_accept_greedy(sparrow_ctx* c, const int32_t* draft_tokens, const int32_t* parents,
+                                     const int32_t* target_next, int32_t T, int32_t* path_out, int32_t* n_accept_out,
+                                     int32_t* bonus_out, void* stream)
+{
+    if (!c || !draft_tokens || !parents || !target_next || !path_out || !n_accept_out || !bonus_out) return SPARROW_ERR_NULL;
+    if (T < 1 || T > kMaxT) return SPARROW_ERR_SHAPE;
+    if (!c->ws) return SPARROW_ERR_WORKSPACE;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return SPARROW_ERR_CUDA;
+    accept_greedy_kernel<<<1, kMaxBatch, 0, static_cast<cudaStream_t>(stream)>>>(
+        draft_tokens, parents, target_next, c->layout.batch, T, path_out, n_accept_out, bonus_out,
+        reinterpret_cast<unsigned*>(c->ws));
+    if (cudaGetLastError() != cudaSuccess) return SPARROW_ERR_CUDA;
+    c->launches.fetch_add(1);
+    return SPARROW_OK;
+}
+
+sparrow_status sparrow_kv_keep_accepted(sparrow_ctx* c, void* k_cache, void* v_cache, const int32_t* kv_len,
+                                        const int32_t* path, const int32_t* n_accept, int32_t T, void* stream)
+{
+    if (!c || !k_cache || !v_cache || !kv_len || !path || !n_accept) return SPARROW_ERR_NULL;
+    if (T < 1 || T > kMaxT) return SPARROW_ERR_SHAPE;
+    if (!aligned16(k_cache) || !aligned16(v_cache)) return SPARROW_ERR_SHAPE;
+    const sparrow_layout& L = c->layout;
+    KeepArgs a;
+    std::memset(&a, 0, sizeof a);
+    for (int b = 0; b < L.batch; ++b) {
+        if (kv_len[b] < 0 || (int64_t)kv_len[b] + T > L.kv_capacity) return SPARROW_ERR_SHAPE;
+        a.kv_len[b] = kv_len[b];
+    }
+    a.k = static_cast<__nv_bfloat16*>(k_cache);
+    a.v = static_cast<__nv_bfloat16*>(v_cache);
+    a.path = path;
+    a.n_accept = n_accept;
+    a.T = T;
+    a.n_kv_heads = L.n_kv_heads;
+    a.stride_batch = L.kv_stride_batch;
+    a.stride_head = L.kv_stride_head;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return SPARROW_ERR_CUDA;
+    keep_accepted_rows_kernel<<<L.batch * L.n_kv_heads, 256, (size_t)2 * T * 256, static_cast<cudaStream_t>(stream)>>>(a);
     if (cudaGetLastError() != cudaSuccess) return SPARROW_ERR_CUDA;
     c->launches.fetch_add(1);
     return SPARROW_OK;
