@@ -193,3 +193,55 @@ def test_long_stream_is_bitwise_reproducible(policy):
                     outs[i][s][0].zero_()
     torch.cuda.synchronize()
     assert ctx.last_device_status() == 0
+
+
+def test_whole_step_in_one_stream_without_synchronisation():
+    """Append draft rows, verify, accept, keep the accepted rows, append the next draft block and
+    verify again -- everything enqueued on one stream with no host synchronisation in between.
+    The second verification must see the cache exactly as the row moves left it (fused calls
+    overlap their neighbours; the plain kernels in between must still be ordered)."""
+    import oracle
+    T, kv0 = 12, 3000
+    case = W.make_verify_case(900, [kv0], T, "random", DEV, capacity=kv0 + 3 * T)
+    ctx = B.Context.for_cache(case.k, W.SCALE)
+    ctx.set_plan_policy(B.PLAN_THROUGHPUT)
+    d = lambda x: torch.tensor(x, dtype=torch.int32, device=DEV)
+    par = case.parents[0].tolist()
+    # synthetic tokens: the chain 0 -> first child -> ... is "right", everything else wrong
+    nxt = [100 + i for i in range(T + 1)]
+    tok = [nxt[par[i] + 1] if (par[i] == -1 or i == min(c for c in range(T) if par[c] == par[i])) else -5 for i in range(T)]
+    ref_path, _ = oracle.greedy_accept(tok, par, nxt)
+    assert len(ref_path) >= 2
+    k_new = W.normal_bf16(901, 40, (1, W.HKV, T, W.D), DEV)
+    v_new = W.normal_bf16(901, 41, (1, W.HKV, T, W.D), DEV)
+    k_new2 = W.normal_bf16(902, 40, (1, W.HKV, T, W.D), DEV)
+    v_new2 = W.normal_bf16(902, 41, (1, W.HKV, T, W.D), DEV)
+    q2 = W.normal_bf16(903, 42, (1, T, W.HQ, W.D), DEV)
+    out1, lse1 = _new(case)
+    out2, lse2 = _new(case)
+    path = torch.empty((1, T), dtype=torch.int32, device=DEV)
+    n_acc = torch.empty((1,), dtype=torch.int32, device=DEV)
+    bonus = torch.empty((1,), dtype=torch.int32, device=DEV)
+    kv1 = kv0 + len(ref_path)                    # (known here because the tokens are synthetic)
+    B.sparrow_kv_append(ctx, k_new, v_new, case.k, case.v, [kv0], T)
+    B.sparrow_verify_attn(ctx, case.q, case.k, case.v, [kv0], case.parents, T, out1, lse1)
+    B.sparrow_accept_greedy(ctx, d([tok]), case.parents, d([nxt]), T, path, n_acc, bonus)
+    B.sparrow_kv_keep_accepted(ctx, case.k, case.v, [kv0], path, n_acc, T)
+    B.sparrow_kv_append(ctx, k_new2, v_new2, case.k, case.v, [kv1], T)
+    B.sparrow_verify_attn(ctx, q2, case.k, case.v, [kv1], case.parents, T, out2, lse2)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == 0
+    assert int(n_acc[0]) == len(ref_path) and path[0, :len(ref_path)].tolist() == ref_path
+    # the same sequence of cache states on the host
+    host = W.make_verify_case(900, [kv0], T, "random", "cpu", capacity=kv0 + 3 * T)
+    k_ref, v_ref = host.k.clone(), host.v.clone()
+    k_ref[0, :, kv0:kv0 + T] = k_new[0].cpu(); v_ref[0, :, kv0:kv0 + T] = v_new[0].cpu()
+    r1 = oracle.verify_attn(W.bf16_bits(case.q), W.bf16_bits(k_ref), W.bf16_bits(v_ref), [kv0], [par], W.SCALE)
+    check(out1, lse1, *r1)
+    k_old, v_old = k_ref.clone(), v_ref.clone()
+    for i, node in enumerate(ref_path):
+        k_ref[0, :, kv0 + i] = k_old[0, :, kv0 + node]; v_ref[0, :, kv0 + i] = v_old[0, :, kv0 + node]
+    k_ref[0, :, kv1:kv1 + T] = k_new2[0].cpu(); v_ref[0, :, kv1:kv1 + T] = v_new2[0].cpu()
+    assert torch.equal(case.k[0, :, :kv1 + T].cpu(), k_ref[0, :, :kv1 + T])
+    r2 = oracle.verify_attn(W.bf16_bits(q2), W.bf16_bits(k_ref), W.bf16_bits(v_ref), [kv1], [par], W.SCALE)
+    check(out2, lse2, *r2)
