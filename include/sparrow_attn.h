@@ -311,10 +311,14 @@ sparrow_status sparrow_debug_ancestor_masks_device(sparrow_ctx* ctx, const int32
  * sequences of n_keys[b] keys, draft blocks of T tokens and a target of n_sm work items (the SM
  * count, or sparrow_plan_target_items() for calls in fused mode), writes
  * splits_out[b] = key-range pieces per (sequence, KV head, row group) and the total number of
- * work items.  Piece s of n covers keys [n_keys*s/n, n_keys*(s+1)/n). */
+ * work items.  Pieces are whole 128-key tiles, as even as whole tiles allow (the last one takes
+ * the ragged end): sparrow_plan_piece_range() gives the keys [begin, end) of piece `piece` of
+ * `n_splits`; SPARROW_ERR_SHAPE unless 0 <= piece < n_splits <= ceil(n_keys / 128). */
 sparrow_status sparrow_plan_splits(int32_t n_sm, int32_t batch, int32_t n_kv_heads,
                                    const int32_t* n_keys, int32_t T, int32_t* splits_out,
                                    int32_t* n_items_out);
+sparrow_status sparrow_plan_piece_range(int32_t n_keys, int32_t n_splits, int32_t piece,
+                                        int32_t* begin_out, int32_t* end_out);
 
 /* Exercises the bounded device-side wait the kernels use between consecutive calls: enqueues a
  * one-thread kernel that waits until the finisher counter of even calls reaches its current

@@ -26,7 +26,7 @@ EXPORTS = ["sparrow_create", "sparrow_destroy", "sparrow_workspace_bytes", "spar
            "sparrow_debug_ancestor_masks_device", "sparrow_debug_wait_counter", "sparrow_plan_splits",
            "sparrow_last_device_status", "sparrow_debug_status_word", "sparrow_launch_count",
            "sparrow_set_plan_policy", "sparrow_plan_target_items", "sparrow_anchor_attn_tree", "sparrow_kv_append", "sparrow_compact_anchors",
-           "sparrow_accept_greedy", "sparrow_kv_keep_accepted",
+           "sparrow_accept_greedy", "sparrow_kv_keep_accepted", "sparrow_plan_piece_range",
            "sparrow_status_string"]
 
 
@@ -67,6 +67,7 @@ def lib():
         L.sparrow_verify_attn_batch.argtypes = [vp, vp, i32, vp]
         L.sparrow_verify_attn_static.argtypes = [ctypes.POINTER(Layout), vp, vp, vp, vp, vp, i32, vp, vp, vp]
         L.sparrow_anchor_attn.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp]
+        L.sparrow_plan_piece_range.argtypes = [i32, i32, i32, vp, vp]
         L.sparrow_accept_greedy.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp]
         L.sparrow_kv_keep_accepted.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp]
         L.sparrow_kv_append.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp]
@@ -315,6 +316,13 @@ def sparrow_plan_splits(n_sm: int, n_kv_heads: int, n_keys: Sequence[int], T: in
     _chk(lib().sparrow_plan_splits(n_sm, len(n_keys), n_kv_heads, nk, T, splits, ctypes.byref(n_items)),
          "sparrow_plan_splits")
     return [int(x) for x in splits], int(n_items.value)
+
+
+def sparrow_plan_piece_range(n_keys: int, n_splits: int, piece: int):
+    b, e = ctypes.c_int32(0), ctypes.c_int32(0)
+    _chk(lib().sparrow_plan_piece_range(n_keys, n_splits, piece, ctypes.byref(b), ctypes.byref(e)),
+         "sparrow_plan_piece_range")
+    return b.value, e.value
 
 
 def sparrow_status_string(status: int) -> str:

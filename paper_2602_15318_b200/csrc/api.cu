@@ -547,6 +547,18 @@ sparrow_status sparrow_plan_splits(int32_t n_sm, int32_t batch, int32_t n_kv_hea
     return SPARROW_OK;
 }
 
+sparrow_status sparrow_plan_piece_range(int32_t n_keys, int32_t n_splits, int32_t piece, int32_t* begin_out, int32_t* end_out)
+{
+    if (!begin_out || !end_out) return SPARROW_ERR_NULL;
+    if (n_keys < 1 || n_splits < 1 || piece < 0 || piece >= n_splits || n_splits > (n_keys + kKeyTile - 1) / kKeyTile)
+        return SPARROW_ERR_SHAPE;
+    int b, e;
+    piece_range(n_keys, n_splits, piece, &b, &e);
+    *begin_out = b;
+    *end_out = e;
+    return SPARROW_OK;
+}
+
 sparrow_status sparrow_verify_attn(sparrow_ctx* c, const void* q, const void* k, const void* v,
                                    const int32_t* kv_len, const int32_t* parents, int32_t T, void* out,
                                    float* lse, void* stream)

@@ -13,6 +13,7 @@ constexpr int kMaxT = 64;
 constexpr int kMaxBatch = 64;
 constexpr int kTokPerBlock = 18;  // draft tokens per 128-row block: 18 x 7 = 126 rows, 2 rows of padding
 constexpr int kBlockRows = 128;
+constexpr int kKeyTile = 128;      // keys per tile of the tensor-core kernel; pieces of the key range are whole tiles
 
 // device status bits (sticky, OR-ed into the first word of the workspace)
 constexpr unsigned kStatTree = 1u;
@@ -134,6 +135,17 @@ struct Item {
     int b, kvh, group, split, key_begin, key_end;
 };
 
+// Key range of piece `split` of `ns` over `n_keys` keys: pieces are whole 128-key tiles (the
+// tensor-core kernel's unit of work), as even as whole tiles allow; the last piece takes the
+// ragged end.  Needs ns <= number of tiles, which the planner guarantees (pieces of >= 128 keys).
+__host__ __device__ __forceinline__ void piece_range(int n_keys, int ns, int split, int* begin, int* end)
+{
+    const long long n_tiles = (n_keys + kKeyTile - 1) / kKeyTile;
+    const long long b = n_tiles * split / ns * kKeyTile, e = n_tiles * (split + 1) / ns * kKeyTile;
+    *begin = (int)b;
+    *end = (int)(e < n_keys ? e : n_keys);
+}
+
 __device__ __forceinline__ Item decode_item(const SplitPlan& p, int item)
 {
     int b = 0;
@@ -146,9 +158,7 @@ __device__ __forceinline__ Item decode_item(const SplitPlan& p, int item)
     const int unit = local / ns;
     it.group = unit % p.n_groups;
     it.kvh = unit / p.n_groups;
-    const long long nk = p.seq[b].n_keys;
-    it.key_begin = (int)(nk * it.split / ns);
-    it.key_end = (int)(nk * (it.split + 1) / ns);
+    piece_range(p.seq[b].n_keys, ns, it.split, &it.key_begin, &it.key_end);
     return it;
 }
 

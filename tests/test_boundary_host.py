@@ -68,11 +68,23 @@ def test_split_plan_properties():
             assert all(1 <= s <= n for s, n in zip(splits, n_keys))
             units = 4 * groups * len(n_keys)
             assert n_items <= max(n_sm, units)
-            # pieces tile the key range exactly
+            # pieces tile the key range exactly, in whole 128-key tiles, sizes within one tile of each other
             for s, n in zip(splits, n_keys):
-                edges = [n * i // s for i in range(s + 1)]
-                assert edges[0] == 0 and edges[-1] == n and all(a < b for a, b in zip(edges, edges[1:]))
+                ranges = [B.sparrow_plan_piece_range(n, s, i) for i in range(s)]
+                assert ranges[0][0] == 0 and ranges[-1][1] == n
+                assert all(a[1] == b[0] for a, b in zip(ranges, ranges[1:]))
+                assert all(b < e and b % 128 == 0 for b, e in ranges)
+                assert all(e % 128 == 0 for _, e in ranges[:-1])
+                tiles = [-(-(e - b) // 128) for b, e in ranges]
+                assert max(tiles) - min(tiles) <= 1
     assert B.sparrow_plan_splits(148, 4, [26128], 16) == ([37], 148)
+
+
+def test_piece_range_rejects_bad_arguments():
+    for args in ((0, 1, 0), (100, 2, 0), (1000, 3, 3), (1000, 0, 0), (1000, 3, -1)):
+        with pytest.raises(B.SparrowError):
+            B.sparrow_plan_piece_range(*args)
+    assert B.sparrow_plan_piece_range(1000, 3, 2) == (640, 1000)
 
 
 def test_plan_rejects_bad_arguments():
