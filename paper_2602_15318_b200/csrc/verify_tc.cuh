@@ -31,9 +31,9 @@
 // whole.  All reads of q / k / v / parents are issued as soon as the CTA starts, so the K/V stream
 // of this call overlaps the tail of the previous one; in front of its first global write a CTA
 // waits on the finisher counters.  After storing its partials a CTA publishes its item; the last
-// pieces of each unit merge the unit's pieces by log-sum-exp (combine_row) and write out / lse,
-// the others exit at once.  In stream-ordered mode the kernel only writes partials and a separate
-// combine kernel follows.
+// CTAs of the grid (the finishers) wait for the call's arrivals, share the call's rows among them,
+// merge each row's pieces by log-sum-exp and write out / lse; the others exit at once.  In
+// stream-ordered mode the kernel only writes partials and a separate combine kernel follows.
 //
 // Every wait is bounded; a wait that gives up sets the timeout status bit and the CTA drains and
 // exits.  TMEM is always released.
