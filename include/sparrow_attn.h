@@ -10,7 +10,10 @@
  *       is lossless, i.e. this is the target's ordinary softmax attention under the tree mask.
  *   (b) text-anchored window attention -- Eq. 2 (Section 3.1, VATA): Softmax(Q_t K_T^T/sqrt(d)) V_T
  *       with K_T, V_T restricted to the text-anchored positions T; the visual KV rows are never
- *       touched.
+ *       touched.  sparrow_anchor_attn_tree() is the same for a draft tree.
+ * Around them, for a whole speculative step on the device: sparrow_kv_append(),
+ * sparrow_compact_anchors() (row movers), sparrow_accept_greedy(), sparrow_kv_keep_accepted()
+ * (temperature-0 acceptance of the draft tree and the move of the accepted rows).
  *
  * For every batch entry b, query head h (KV head h / 7), draft token t and visible key set Vis:
  *     s_j = softmax_scale * <q[b,t,h,:], k[b,h/7,j,:]>,   lse = log sum_{j in Vis} exp(s_j),
