@@ -132,7 +132,10 @@ sparrow_status sparrow_set_workspace(sparrow_ctx* ctx, void* dev_ptr, size_t byt
  * (the library's own kernels do; an ordinary kernel never does before it completes).  So the
  * inputs of a call must not be the out / lse of the library call enqueued directly before it on
  * the same stream; anything else in between (another kernel, a copy) restores plain stream order.
- * Writes of consecutive calls are ordered through counters in the workspace.  While a stream is being
+ * Writes of consecutive calls of one context are ordered through counters in its workspace; a
+ * call that follows a call of another context takes plain stream order.  All fused calls of a
+ * context belong on one stream (or must be kept from running concurrently by events): the
+ * counters assume that calls run in the order they were enqueued.  While a stream is being
  * captured into a graph, or with SPARROW_NO_PDL=1 in the environment when the context is created,
  * a call is two ordinary launches (split-KV pass, combine) ordered by the stream alone.
  * Results are deterministic for fixed arguments. */

@@ -256,6 +256,9 @@ void advance_sync(sparrow_ctx* c, const SplitPlan& p, const SyncArgs& sy)
     c->seq += 1;
 }
 
+// Context of the most recent fused launch in this process (any stream): see launch_verify_tc().
+std::atomic<sparrow_ctx*> g_last_fused_ctx{nullptr};
+
 sparrow_status launch_combine(sparrow_ctx* c, const SplitPlan& plan, const SyncArgs& sy, void* out, float* lse, cudaStream_t st,
                               bool programmatic = false)
 {
@@ -375,7 +378,11 @@ sparrow_status launch_verify_tc(sparrow_ctx* c, const SplitPlan& plan, const Syn
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = sy.enabled ? 1 : 0;
+    // The early start only reaches back to the kernel launched directly before this one.  The
+    // counters order this context's own calls; if that kernel may belong to another context (whose
+    // writes these counters know nothing about), this launch takes plain stream order instead.
+    const bool same_ctx_before = g_last_fused_ctx.exchange(c) == c;
+    cfg.numAttrs = (sy.enabled && same_ctx_before) ? 1 : 0;
     const cudaError_t e = nb == 1 ? cudaLaunchKernelEx(&cfg, tc::verify_tc_kernel<1>, a, sy, plan, *mq, *mk, *mv)
                                   : cudaLaunchKernelEx(&cfg, tc::verify_tc_kernel<2>, a, sy, plan, *mq, *mk, *mv);
     if (e != cudaSuccess) return SPARROW_ERR_CUDA;
@@ -499,6 +506,8 @@ sparrow_status sparrow_create(sparrow_ctx** out, const sparrow_layout* L, int de
 sparrow_status sparrow_destroy(sparrow_ctx* c)
 {
     if (!c) return SPARROW_ERR_NULL;
+    sparrow_ctx* expected = c;
+    g_last_fused_ctx.compare_exchange_strong(expected, nullptr);      // a later context may reuse the address
     delete c;
     return SPARROW_OK;
 }

@@ -245,3 +245,26 @@ def test_whole_step_in_one_stream_without_synchronisation():
     assert torch.equal(case.k[0, :, :kv1 + T].cpu(), k_ref[0, :, :kv1 + T])
     r2 = oracle.verify_attn(W.bf16_bits(q2), W.bf16_bits(k_ref), W.bf16_bits(v_ref), [kv1], [par], W.SCALE)
     check(out2, lse2, *r2)
+
+
+def test_calls_of_two_contexts_on_one_stream_take_stream_order():
+    """A call that follows a call of ANOTHER context must not start early (the other context's
+    writes are invisible to this context's counters): here its queries are the other call's output."""
+    T = 16
+    a = W.make_verify_case(950, [9000], T, "chain", DEV)
+    b = W.make_verify_case(951, [7000], T, "random", DEV)
+    ctx_a = B.Context.for_cache(a.k, W.SCALE)
+    ctx_b = B.Context.for_cache(b.k, W.SCALE)
+    out_a, lse_a = _new(a)
+    out_b, lse_b = _new(b)
+    for _ in range(5):
+        out_a.fill_(float("nan"))
+        B.sparrow_verify_attn(ctx_a, a.q, a.k, a.v, a.kv_len, a.parents, T, out_a, lse_a)
+        B.sparrow_verify_attn(ctx_b, out_a, b.k, b.v, b.kv_len, b.parents, T, out_b, lse_b)     # q = the other call's out
+        torch.cuda.synchronize()
+        again, lse_again = _new(b)
+        B.sparrow_verify_attn(ctx_b, out_a, b.k, b.v, b.kv_len, b.parents, T, again, lse_again)
+        torch.cuda.synchronize()
+        assert torch.isfinite(out_b.float()).all()
+        assert torch.equal(out_b, again) and torch.equal(lse_b, lse_again)
+    assert ctx_a.last_device_status() == 0 and ctx_b.last_device_status() == 0
