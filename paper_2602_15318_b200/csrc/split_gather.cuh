@@ -104,17 +104,18 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
 
     // ---- prologue: masks / query positions, packed Q block -> registers --------------------
     const int tree_nodes = anchored ? args.tree_nodes : 0;
-    if (tid < T) {
-        if (anchored) {
-            int p = aidx[args.n_anchor - T + tid];
-            if (p < 0 || p >= args.kv_capacity) { atomicOr(args.status, kStatAnchor); p = -1; }
-            qpos_s[tid] = p;
-        } else {
-            anc_s[tid] = ancestor_word(args.parents + (size_t)it.b * T, T, tid, args.status);
-        }
+    // The parent array is staged in shared memory first: the walk up the tree is a chain of
+    // dependent reads, one memory round trip each if it went to global memory.
+    __shared__ int32_t par_s[kMaxT];
+    const int n_par = anchored ? tree_nodes : T;
+    if (tid < n_par) par_s[tid] = __ldg(args.parents + (size_t)it.b * n_par + tid);
+    if (anchored && tid < T) {
+        int p = aidx[args.n_anchor - T + tid];
+        if (p < 0 || p >= args.kv_capacity) { atomicOr(args.status, kStatAnchor); p = -1; }
+        qpos_s[tid] = p;
     }
-    if (tid < tree_nodes)
-        anc_s[tid] = ancestor_word(args.parents + (size_t)it.b * tree_nodes, tree_nodes, tid, args.status);
+    __syncthreads();
+    if (tid < n_par) anc_s[tid] = ancestor_word(par_s, n_par, tid, args.status);
     {
         constexpr int kChunksPerThread = kRows * 16 / kThreads;      // 8: all loads first, then the stores
         uint4 val[kChunksPerThread];
