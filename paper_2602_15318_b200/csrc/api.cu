@@ -67,6 +67,9 @@ constexpr size_t kStatusBytes = 1024;      // word 0: sticky status; words 16, 1
 constexpr size_t kFinDoneOffset = 64;
 constexpr size_t kArrivalsOffset = 128;     // words 32..35: arrival words of the four call slots
 constexpr int kMinPieceKeys = 128;
+// The gathered kernel works on 64-key tiles and is bound by its per-tile arithmetic (legacy
+// mma.sync): short anchor lists are cut down to single tiles.
+constexpr int kMinGatherPieceKeys = 64;
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -97,7 +100,7 @@ int max_items(int n_sm, int batch, int n_kv_heads, int n_groups)
 // Chooses the number of key-range pieces per sequence so that the total number of work items is
 // close to (and not above) the SM count while every item streams about the same number of keys.
 sparrow_status make_plan(int n_sm, int batch, int n_kv_heads, const int32_t* n_keys, int T, int blocks_per_group,
-                         SplitPlan* p)
+                         SplitPlan* p, int min_piece_keys = kMinPieceKeys)
 {
     if (batch < 1 || batch > kMaxBatch || T < 1 || T > kMaxT || n_kv_heads < 1 || n_sm < 1) return SPARROW_ERR_SHAPE;
     std::memset(p, 0, sizeof(*p));
@@ -107,6 +110,7 @@ sparrow_status make_plan(int n_sm, int batch, int n_kv_heads, const int32_t* n_k
     p->blocks_per_group = blocks_per_group;
     p->n_groups = (T + kTokPerBlock * blocks_per_group - 1) / (kTokPerBlock * blocks_per_group);
     p->n_kv_heads = n_kv_heads;
+    p->piece_tile = min_piece_keys < kKeyTile ? min_piece_keys : kKeyTile;
     p->part_rows = blocks_per_group * kBlockRows + 1;    // odd pitch: partial rows of successive pieces must not share L2 sets
     const int units = n_kv_heads * p->n_groups;
     int max_keys = 1;
@@ -119,7 +123,7 @@ sparrow_status make_plan(int n_sm, int batch, int n_kv_heads, const int32_t* n_k
         for (int b = 0; b < batch; ++b) n += (long long)units * ((n_keys[b] + L - 1) / L);
         return n;
     };
-    long long lo = kMinPieceKeys, hi = max_keys > kMinPieceKeys ? max_keys : kMinPieceKeys;
+    long long lo = min_piece_keys, hi = max_keys > min_piece_keys ? max_keys : min_piece_keys;
     if (items_for(lo) > n_sm) {                 // smallest piece length that fits the SM count
         while (lo < hi) {
             const long long mid = (lo + hi) / 2;
@@ -562,7 +566,7 @@ sparrow_status sparrow_plan_piece_range(int32_t n_keys, int32_t n_splits, int32_
     if (n_keys < 1 || n_splits < 1 || piece < 0 || piece >= n_splits || n_splits > (n_keys + kKeyTile - 1) / kKeyTile)
         return SPARROW_ERR_SHAPE;
     int b, e;
-    piece_range(n_keys, n_splits, piece, &b, &e);
+    piece_range(n_keys, n_splits, piece, kKeyTile, &b, &e);
     *begin_out = b;
     *end_out = e;
     return SPARROW_OK;
@@ -733,7 +737,7 @@ sparrow_status anchor_call(sparrow_ctx* c, const void* q, const void* k, const v
     int32_t n_keys[kMaxBatch];
     for (int b = 0; b < c->layout.batch; ++b) n_keys[b] = n_anchor;
     SplitPlan plan;
-    sparrow_status s = make_plan(c->n_sm, c->layout.batch, c->layout.n_kv_heads, n_keys, T, 1, &plan);
+    sparrow_status s = make_plan(c->n_sm, c->layout.batch, c->layout.n_kv_heads, n_keys, T, 1, &plan, kMinGatherPieceKeys);
     if (s != SPARROW_OK) return s;
     if ((s = check_ws(c, plan)) != SPARROW_OK) return s;
     DeviceGuard guard(c->device);

@@ -48,6 +48,7 @@ struct SplitPlan {
     int32_t n_groups;             // ceil(T / (18 * blocks_per_group))
     int32_t n_kv_heads;
     int32_t part_rows;            // row pitch of one item's partial block in the workspace
+    int32_t piece_tile;           // pieces of the key range are whole tiles of this many keys (128 or 64)
     SeqPlan seq[kMaxBatch];
 };
 
@@ -135,13 +136,14 @@ struct Item {
     int b, kvh, group, split, key_begin, key_end;
 };
 
-// Key range of piece `split` of `ns` over `n_keys` keys: pieces are whole 128-key tiles (the
-// tensor-core kernel's unit of work), as even as whole tiles allow; the last piece takes the
-// ragged end.  Needs ns <= number of tiles, which the planner guarantees (pieces of >= 128 keys).
-__host__ __device__ __forceinline__ void piece_range(int n_keys, int ns, int split, int* begin, int* end)
+// Key range of piece `split` of `ns` over `n_keys` keys: pieces are whole tiles of `tile` keys (the
+// kernel's unit of work: 128 on the tensor-core path, 64 on the gathered one), as even as whole
+// tiles allow; the last piece takes the ragged end.  Needs ns <= number of tiles, which the
+// planner guarantees (pieces of at least one tile).
+__host__ __device__ __forceinline__ void piece_range(int n_keys, int ns, int split, int tile, int* begin, int* end)
 {
-    const long long n_tiles = (n_keys + kKeyTile - 1) / kKeyTile;
-    const long long b = n_tiles * split / ns * kKeyTile, e = n_tiles * (split + 1) / ns * kKeyTile;
+    const long long n_tiles = (n_keys + tile - 1) / tile;
+    const long long b = n_tiles * split / ns * tile, e = n_tiles * (split + 1) / ns * tile;
     *begin = (int)b;
     *end = (int)(e < n_keys ? e : n_keys);
 }
@@ -158,7 +160,7 @@ __device__ __forceinline__ Item decode_item(const SplitPlan& p, int item)
     const int unit = local / ns;
     it.group = unit % p.n_groups;
     it.kvh = unit / p.n_groups;
-    piece_range(p.seq[b].n_keys, ns, it.split, &it.key_begin, &it.key_end);
+    piece_range(p.seq[b].n_keys, ns, it.split, p.piece_tile, &it.key_begin, &it.key_end);
     return it;
 }
 

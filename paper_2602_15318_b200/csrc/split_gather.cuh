@@ -88,6 +88,7 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
 {
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* kv_smem = smem;                                   // [2 stages][K 16K | V 16K]
+    unsigned char* q_stage = smem + 2 * kStageBytes;                 // stage 1 doubles as the staging area of the Q block
     unsigned long long* anc_s = reinterpret_cast<unsigned long long*>(smem + 4 * kStageBytes);
     int32_t* qpos_s = reinterpret_cast<int32_t*>(smem + 4 * kStageBytes + kMaxT * 8);
     int32_t* apos_s = qpos_s + kMaxT;                                // [2][kTile] gathered row ids
@@ -101,6 +102,41 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
     const bool anchored = args.anchor_idx != nullptr;
     const int kv_len = anchored ? 0 : plan.seq[it.b].kv_len;
     const int32_t* aidx = anchored ? args.anchor_idx + (size_t)it.b * args.n_anchor : nullptr;
+
+    const __nv_bfloat16* kbase = args.k + (size_t)it.b * args.kv_stride_batch + (size_t)it.kvh * args.kv_stride_head;
+    const __nv_bfloat16* vbase = args.v + (size_t)it.b * args.kv_stride_batch + (size_t)it.kvh * args.kv_stride_head;
+    const int n_tiles = (it.key_end - it.key_begin + kTile - 1) / kTile;
+
+    auto load_tile = [&](int stage, int tile) {
+        unsigned char* ks = kv_smem + stage * 2 * kStageBytes;
+        unsigned char* vs = ks + kStageBytes;
+        #pragma unroll
+        for (int i = 0; i < (kTile * 16) / kThreads; ++i) {
+            const int idx = tid + i * kThreads;
+            const int r = idx >> 4, c = idx & 15;
+            const int j = it.key_begin + tile * kTile + r;
+            int row = -1;
+            if (j < it.key_end) {
+                if (anchored) {
+                    row = __ldg(aidx + j);
+                    if (row < 0 || row >= args.kv_capacity) { atomicOr(args.status, kStatAnchor); row = -1; }
+                } else {
+                    row = j;
+                }
+            }
+            if (anchored && c == 0) apos_s[stage * kTile + r] = row;
+            const size_t off = (size_t)(row < 0 ? 0 : row) * kD + c * 8;
+            const int bytes = row < 0 ? 0 : 16;          // 0 -> the 16 bytes are zero-filled
+            cp_async16(smem_u32(ks + swz(r, c)), kbase + off, bytes);
+            cp_async16(smem_u32(vs + swz(r, c)), vbase + off, bytes);
+        }
+    };
+
+    // Tile 0 is requested before anything else: its two dependent round trips (anchor indices,
+    // then the rows) overlap the loads of the prologue.  It lands in stage 0; the packed Q block is
+    // staged in stage 1, which the ring only reuses after Q has moved to registers.
+    if (n_tiles > 0) { load_tile(0, 0); }
+    cp_async_commit();
 
     // ---- prologue: masks / query positions, packed Q block -> registers --------------------
     const int tree_nodes = anchored ? args.tree_nodes : 0;
@@ -133,7 +169,7 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
         #pragma unroll
         for (int u = 0; u < kChunksPerThread; ++u) {
             const int i = tid + u * kThreads;
-            *reinterpret_cast<uint4*>(kv_smem + swz(i >> 4, i & 15)) = val[u];
+            *reinterpret_cast<uint4*>(q_stage + swz(i >> 4, i & 15)) = val[u];
         }
     }
     __syncthreads();
@@ -142,7 +178,7 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
         const int r = warp * 16 + (lane & 15);
         #pragma unroll
         for (int ks = 0; ks < 8; ++ks)
-            ldsm_x4(smem_u32(kv_smem + swz(r, ks * 2 + (lane >> 4))), qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
+            ldsm_x4(smem_u32(q_stage + swz(r, ks * 2 + (lane >> 4))), qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
     }
     // per-thread row state: rows lr0 = warp*16+g4 and lr0+8
     int row_t[2]; bool row_ok[2]; unsigned long long row_anc[2]; int row_qpos[2];
@@ -155,36 +191,8 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
         row_anc[rr] = anchored ? (tree_nodes > 0 ? anc_s[tree_nodes - T + t] : 0ull) : anc_s[t];
         row_qpos[rr] = anchored ? qpos_s[t] : 0;
     }
+    const bool warp_has_rows = __any_sync(0xffffffffu, row_ok[0] || row_ok[1]);
     __syncthreads();                      // Q staging area is reused by the K/V ring from here on
-
-    const __nv_bfloat16* kbase = args.k + (size_t)it.b * args.kv_stride_batch + (size_t)it.kvh * args.kv_stride_head;
-    const __nv_bfloat16* vbase = args.v + (size_t)it.b * args.kv_stride_batch + (size_t)it.kvh * args.kv_stride_head;
-    const int n_tiles = (it.key_end - it.key_begin + kTile - 1) / kTile;
-
-    auto load_tile = [&](int stage, int tile) {
-        unsigned char* ks = kv_smem + stage * 2 * kStageBytes;
-        unsigned char* vs = ks + kStageBytes;
-        #pragma unroll
-        for (int i = 0; i < (kTile * 16) / kThreads; ++i) {
-            const int idx = tid + i * kThreads;
-            const int r = idx >> 4, c = idx & 15;
-            const int j = it.key_begin + tile * kTile + r;
-            int row = -1;
-            if (j < it.key_end) {
-                if (anchored) {
-                    row = __ldg(aidx + j);
-                    if (row < 0 || row >= args.kv_capacity) { atomicOr(args.status, kStatAnchor); row = -1; }
-                } else {
-                    row = j;
-                }
-            }
-            if (anchored && c == 0) apos_s[stage * kTile + r] = row;
-            const size_t off = (size_t)(row < 0 ? 0 : row) * kD + c * 8;
-            const int bytes = row < 0 ? 0 : 16;          // 0 -> the 16 bytes are zero-filled
-            cp_async16(smem_u32(ks + swz(r, c)), kbase + off, bytes);
-            cp_async16(smem_u32(vs + swz(r, c)), vbase + off, bytes);
-        }
-    };
 
     float o[16][4];
     #pragma unroll
@@ -193,8 +201,6 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
     float l_run[2] = {0.f, 0.f};
     const float c2 = args.scale_log2e;
 
-    if (n_tiles > 0) { load_tile(0, 0); }
-    cp_async_commit();
     for (int tile = 0; tile < n_tiles; ++tile) {
         const int stage = tile & 1;
         if (tile + 1 < n_tiles) load_tile(stage ^ 1, tile + 1);
@@ -204,6 +210,10 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
         const unsigned char* ks = kv_smem + stage * 2 * kStageBytes;
         const unsigned char* vs = ks + kStageBytes;
 
+        // A warp whose 16 rows are all padding (fewer than 126 packed rows in this block) has no
+        // arithmetic to do: it only takes part in the loads and the barriers.  (mma.sync is the
+        // legacy tensor path here, a fraction of the tcgen05 rate: idle rows are not free.)
+        if (warp_has_rows) {
         // S = Q K^T for 16 rows x 64 keys
         float s[8][4];
         #pragma unroll
@@ -295,6 +305,7 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
                 mma_bf16(o[2 * dn + 1], a, b2, b3);
             }
         }
+        }   // warp_has_rows
         __syncthreads();                  // this stage is refilled by the next iteration's loads
     }
     cp_async_wait<0>();
