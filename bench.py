@@ -311,6 +311,29 @@ def main():
     time_calls(ctx, warm, 50, B, torch)
     us_warm = time_calls(ctx, warm, max(1, steps // 10), B, torch)
 
+    # -- the same rotation replayed from a CUDA graph (captured calls run in stream-ordered mode:
+    #    split-KV kernel, then combine kernel, one wave of pieces) -------------------------------
+    us_graph = None
+    try:
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            B.sparrow_verify_attn_batch(ctx, batch, stream=side)
+            side.synchronize()
+            with torch.cuda.graph(graph, stream=side):
+                B.sparrow_verify_attn_batch(ctx, batch, stream=side)
+            graph.replay(); side.synchronize()
+            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            n_rep = max(5, min(200, steps // len(cases)))
+            g0.record(side)
+            for _ in range(n_rep):
+                graph.replay()
+            g1.record(side); side.synchronize()
+        us_graph = g0.elapsed_time(g1) * 1e3 / (n_rep * len(cases))
+        del graph
+    except Exception as e:                                   # reported, never fatal for the headline
+        us_graph = f"unavailable: {type(e).__name__}"
+
     # -- end to end through the host-buffer entry point -----------------------------------------
     c0 = cases[0]
     T = c0.T
@@ -345,6 +368,10 @@ def main():
         raise SystemExit(f"device status {status} (word {ctx.status_word():#x}) after the timed region")
 
     peak, peak_kind, peaks = measured_peaks()
+    # overhead outside the algorithmic bytes: partial rows (272 B) written once and read once through L2
+    tgt = policies["throughput"]["target_items"]
+    splits, n_items = B.sparrow_plan_splits(tgt, W.HKV, [n + cases[0].T for n in cases[0].kv_len], cases[0].T)
+    partial_bytes = 2 * n_items * 7 * cases[0].T * 272
     alg_bytes = kv_bytes + io_bytes
     achieved = alg_bytes / (us_call * 1e-6) / 1e9
     traffic = profiled_traffic()
@@ -361,6 +388,11 @@ def main():
         "hbm_gbs_per_call": alg_bytes / (us_call * 1e-6) / 1e9,
         "pct_of_8tbs_nominal": 100.0 * alg_bytes / (us_call * 1e-6) / 8e12,
         "tflops_per_call": flops / (us_call * 1e-6) / 1e12,
+        "pct_of_bf16_burst_peak": (100.0 * flops / (us_call * 1e-6) / 1e12 / peaks["bf16_tflops"]) if peaks.get("bf16_tflops") else None,
+        "pct_of_bf16_sustained_peak": (100.0 * flops / (us_call * 1e-6) / 1e12 / peaks["bf16_tflops_sustained"])
+        if peaks.get("bf16_tflops_sustained") else None,
+        "us_per_call_graph_replay": us_graph,
+        "partials_bytes_per_call": partial_bytes,
         "us_per_call_isolated": us_isolated,
         "us_per_call_isolated_what": "one call on an idle GPU under the latency policy, events around the call, median",
         "policies": policies,

@@ -259,6 +259,21 @@ def test_config5_layer_sampled_rows(layer, policy):
     assert torch.isfinite(out.float()).all() and torch.isfinite(lse).all()
 
 
+def test_config5_every_layer_sampled_rows():
+    """All 28 per-layer caches of the batched step, one after the other (generate, run, check a few
+    rows of every sequence against the oracle), the planner policy changing from layer to layer."""
+    ctx = None
+    for layer in range(28):
+        case = W.make_config(4, DEV, layer=layer)
+        ctx = ctx or B.Context.for_cache(case.k, W.SCALE)
+        out, lse, _ = run_verify(case, ctx, policy=POLICIES[layer % 3])
+        rows = sample_rows(500 + layer, 8, case.T, 12)
+        ref_out, ref_lse = oracle_verify(case, rows)
+        check(out, lse, ref_out, ref_lse, rows)
+        del case, out, lse
+        torch.cuda.empty_cache()
+
+
 # ---- host-buffer entry point and argument errors --------------------------------------------
 
 def test_verify_step_host_matches_device_call():
