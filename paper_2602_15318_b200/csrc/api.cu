@@ -67,8 +67,9 @@ constexpr size_t kStatusBytes = 1024;      // word 0: sticky status; words 16, 1
 constexpr size_t kFinDoneOffset = 64;
 constexpr size_t kArrivalsOffset = 128;     // words 32..35: arrival words of the four call slots
 constexpr int kMinPieceKeys = 128;
-// The gathered kernel works on 64-key tiles and is bound by its per-tile arithmetic (legacy
-// mma.sync): short anchor lists are cut down to single tiles.
+// The gathered kernel works on 64-key tiles and pays two dependent memory round trips per tile
+// (anchor indices, then the rows), which a CTA with several tiles takes one after the other: short
+// anchor lists are cut down to single tiles, one CTA each.
 constexpr int kMinGatherPieceKeys = 64;
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

@@ -211,8 +211,7 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
         const unsigned char* vs = ks + kStageBytes;
 
         // A warp whose 16 rows are all padding (fewer than 126 packed rows in this block) has no
-        // arithmetic to do: it only takes part in the loads and the barriers.  (mma.sync is the
-        // legacy tensor path here, a fraction of the tcgen05 rate: idle rows are not free.)
+        // arithmetic to do: it only takes part in the loads and the barriers.
         if (warp_has_rows) {
         // S = Q K^T for 16 rows x 64 keys
         float s[8][4];
