@@ -107,22 +107,32 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
     const __nv_bfloat16* vbase = args.v + (size_t)it.b * args.kv_stride_batch + (size_t)it.kvh * args.kv_stride_head;
     const int n_tiles = (it.key_end - it.key_begin + kTile - 1) / kTile;
 
-    auto load_tile = [&](int stage, int tile) {
+    // Row indices of a tile, four per thread (one per 16-byte chunk this thread copies).  In anchored
+    // mode they come from the anchor list: a memory round trip that the row copies depend on, so
+    // the indices of a tile are fetched one whole tile ahead of its copies.
+    constexpr int kAbsent = -2147483647 - 1;                 // key past the end of the piece
+    constexpr int kPerThread = (kTile * 16) / kThreads;      // 4
+    auto fetch_rows = [&](int tile, int (&rows)[kPerThread]) {
+        #pragma unroll
+        for (int i = 0; i < kPerThread; ++i) {
+            const int r = (tid + i * kThreads) >> 4;
+            const int j = it.key_begin + tile * kTile + r;
+            rows[i] = j < it.key_end ? (anchored ? __ldg(aidx + j) : j) : kAbsent;
+        }
+    };
+    auto issue_tile = [&](int stage, const int (&rows)[kPerThread]) {
         unsigned char* ks = kv_smem + stage * 2 * kStageBytes;
         unsigned char* vs = ks + kStageBytes;
         #pragma unroll
-        for (int i = 0; i < (kTile * 16) / kThreads; ++i) {
+        for (int i = 0; i < kPerThread; ++i) {
             const int idx = tid + i * kThreads;
             const int r = idx >> 4, c = idx & 15;
-            const int j = it.key_begin + tile * kTile + r;
-            int row = -1;
-            if (j < it.key_end) {
-                if (anchored) {
-                    row = __ldg(aidx + j);
-                    if (row < 0 || row >= args.kv_capacity) { atomicOr(args.status, kStatAnchor); row = -1; }
-                } else {
-                    row = j;
-                }
+            int row = rows[i];
+            if (row == kAbsent) {
+                row = -1;
+            } else if (row < 0 || row >= args.kv_capacity) {
+                atomicOr(args.status, kStatAnchor);
+                row = -1;
             }
             if (anchored && c == 0) apos_s[stage * kTile + r] = row;
             const size_t off = (size_t)(row < 0 ? 0 : row) * kD + c * 8;
@@ -131,12 +141,14 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
             cp_async16(smem_u32(vs + swz(r, c)), vbase + off, bytes);
         }
     };
+    int rows_next[kPerThread];
 
     // Tile 0 is requested before anything else: its two dependent round trips (anchor indices,
     // then the rows) overlap the loads of the prologue.  It lands in stage 0; the packed Q block is
     // staged in stage 1, which the ring only reuses after Q has moved to registers.
-    if (n_tiles > 0) { load_tile(0, 0); }
+    if (n_tiles > 0) { fetch_rows(0, rows_next); issue_tile(0, rows_next); }
     cp_async_commit();
+    if (n_tiles > 1) fetch_rows(1, rows_next);
 
     // ---- prologue: masks / query positions, packed Q block -> registers --------------------
     const int tree_nodes = anchored ? args.tree_nodes : 0;
@@ -203,8 +215,9 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
 
     for (int tile = 0; tile < n_tiles; ++tile) {
         const int stage = tile & 1;
-        if (tile + 1 < n_tiles) load_tile(stage ^ 1, tile + 1);
+        if (tile + 1 < n_tiles) issue_tile(stage ^ 1, rows_next);
         cp_async_commit();
+        if (tile + 2 < n_tiles) fetch_rows(tile + 2, rows_next);     // arrives while this tile is being worked on
         cp_async_wait<1>();
         __syncthreads();
         const unsigned char* ks = kv_smem + stage * 2 * kStageBytes;
