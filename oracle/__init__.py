@@ -256,3 +256,98 @@ def greedy_accept(draft_tokens, parents, target_next):
         i = par[i]
     path.reverse()
     return path, nxt[best + 1]
+
+
+# ---------------------------------------------------------------------------------------------
+# Acceptance at temperature 1 (speculative sampling over a draft tree).
+#
+# Appendix A ("Speculative Decoding") states that verification keeps the target model's output
+# distribution exactly and Section 4 reports every result at temperature 0 and 1; the paper relies
+# on the standard procedure without restating it.  The reading taken here is the usual multi-round
+# rejection rule for a tree whose sibling candidates were drawn without replacement from the
+# draft distribution: at the current node, with target distribution p and draft distribution q,
+# the children are tried in index order; a child with token x is accepted with probability
+# min(1, p(x) / q(x)); after a rejection p becomes the normalised positive part of (p - q) and q
+# loses x and is renormalised; when no child is accepted the next token is drawn from what p has
+# become.  Accepting a child moves to it, with that node's own p and q.
+#
+# The result is a set of integers (accepted path, bonus token), so the arithmetic that decides
+# them is fixed to something every implementation reproduces bit for bit: probabilities are
+# rounded once to 30-bit fixed point and everything after that is integer arithmetic, whose sums
+# do not depend on the order of summation.
+# ---------------------------------------------------------------------------------------------
+
+PROB_BITS = 30
+
+
+def fixed_point_probs(p) -> np.ndarray:
+    """float32 probabilities -> int64 fixed point: floor(p * 2^30 + 1/2), evaluated in float64
+    (exact for float32 inputs in [0, 1])."""
+    p = np.asarray(p, dtype=np.float32).astype(np.float64)
+    assert np.all(p >= 0.0) and np.all(p <= 1.0)
+    return np.floor(p * float(1 << PROB_BITS) + 0.5).astype(np.int64)
+
+
+def sample_accept(draft_tokens, parents, p_target, p_draft, u_node, u_bonus):
+    """Temperature-1 verification of one draft tree.
+
+    draft_tokens int [T]; parents int [T] (-1 = root, parents[i] < i);
+    p_target, p_draft float32 [T + 1][V]: row 0 belongs to the committed prefix, row 1 + i to node
+    i -- the target's next-token distribution there, and the draft distribution that node's
+    children were drawn from (without replacement, in index order);
+    u_node uint32 [T]: the uniform that decides node i's acceptance test;
+    u_bonus uint32 [T + 1]: row r's uniform for the token drawn when the walk stops at row r.
+    Returns (path, bonus): accepted nodes from the root down, and the token emitted after them.
+
+    With P, Q the fixed-point rows (int), A = sum P, B = sum Q and r = u_node[c] in [0, 2^32):
+      accept child c (token x)  iff  Q[x] > 0 and r * Q[x] * A < P[x] * B * 2^32
+                                     (i.e. r / 2^32 < (P[x] / A) / (Q[x] / B));
+      after a rejection         P <- max(B * P - A * Q, 0) >> 30  (element-wise; left as it is when B == 0),
+                                A <- sum P,  B <- B - Q[x],  Q[x] <- 0;
+      bonus                     the smallest v with P[0] + ... + P[v] > (u_bonus[row] * A) >> 32,
+                                P being the row's original target row again if A == 0.
+    """
+    tok = [int(x) for x in draft_tokens]
+    par = [int(x) for x in parents]
+    T = len(tok)
+    p_target = np.asarray(p_target, dtype=np.float32)
+    p_draft = np.asarray(p_draft, dtype=np.float32)
+    assert p_target.shape == p_draft.shape and p_target.shape[0] == T + 1
+    assert len(par) == T and len(u_node) == T and len(u_bonus) == T + 1
+    children = {i: [] for i in range(-1, T)}
+    for i, p in enumerate(par):
+        assert -1 <= p < i
+        children[p].append(i)
+    cur, path = -1, []
+    while True:
+        row = cur + 1
+        P = fixed_point_probs(p_target[row])
+        Q = fixed_point_probs(p_draft[row])
+        A, B = int(P.sum()), int(Q.sum())
+        taken = None
+        for c in children[cur]:
+            x, r = tok[c], int(u_node[c])
+            assert 0 <= x < P.shape[0] and 0 <= r < (1 << 32)
+            if int(Q[x]) > 0 and r * int(Q[x]) * A < int(P[x]) * B * (1 << 32):
+                taken = c
+                break
+            if B > 0:
+                P = np.maximum(B * P - A * Q, 0) >> PROB_BITS
+                A = int(P.sum())
+            B -= int(Q[x])
+            Q[x] = 0
+        if taken is None:
+            if A == 0:
+                P = fixed_point_probs(p_target[row])
+                A = int(P.sum())
+            assert A > 0, "a target row without any probability mass"
+            t = (int(u_bonus[row]) * A) >> 32
+            acc, bonus = 0, None
+            for v in range(P.shape[0]):
+                acc += int(P[v])
+                if acc > t:
+                    bonus = v
+                    break
+            return path, bonus
+        path.append(taken)
+        cur = taken

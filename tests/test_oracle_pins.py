@@ -334,6 +334,19 @@ def test_verify_visibility_layout():
                             [1, 1, 1, 1, 0, 1, 0], [1, 1, 1, 1, 0, 1, 1]]
 
 
+def _brute_force_anchor_list(seq_len, vis_spans, window, T):
+    """Eq. 2's index set under the window reading, filtered position by position: every position of
+    [0, seq_len) that lies in no visual span and within the last `window` positions (window <= 0:
+    no limit), then the T draft rows."""
+    keep = []
+    for p in range(seq_len):
+        visual = any(a <= p < e for a, e in vis_spans)
+        recent = window <= 0 or p >= seq_len - window
+        if recent and not visual:
+            keep.append(p)
+    return keep + [seq_len + t for t in range(T)]
+
+
 def test_anchor_idx_brute_force_and_c4_closed_form():
     rng = np.random.default_rng(20)
     for _ in range(30):
@@ -341,7 +354,7 @@ def test_anchor_idx_brute_force_and_c4_closed_form():
         cuts = sorted(rng.integers(0, L + 1, size=4).tolist())
         spans = [[cuts[0], cuts[1]], [cuts[2], cuts[3]]]
         Wn = int(rng.integers(0, 80)); T = int(rng.integers(0, 9))
-        want = W.text_anchor_list(L, spans, Wn, T)
+        want = _brute_force_anchor_list(L, spans, Wn, T)
         assert oracle.anchor_idx(L, spans, Wn, T).tolist() == want
     got = oracle.anchor_idx(26112, [[64, 25664]], 1024, 8)
     assert got.tolist() == list(range(25664, 26112)) + list(range(26112, 26120))
@@ -498,3 +511,142 @@ def test_greedy_accept_closed_forms():
     assert oracle.greedy_accept([5, 7, 8, 8, 4], par, [7, 0, 8, 0, 4, 6]) == ([1, 3, 4], 6)
     # equal depth: the chain ending at the smaller index
     assert oracle.greedy_accept([5, 7, 8, 8, 1], par, [7, 0, 8, 0, 4, 6]) == ([1, 2], 0)
+
+
+# ---------------------------------------------------------------- acceptance at temperature 1 ----
+# Pinned by what speculative sampling must satisfy whatever the implementation: identical draft and
+# target distributions accept everything, disjoint supports accept nothing, a one-hot target is
+# the greedy rule, and the emitted tokens follow the target distribution exactly (checked
+# empirically with siblings drawn without replacement from the draft distribution).
+
+def _rows(rng, n_rows, V, conc=1.0):
+    return rng.dirichlet([conc] * V, size=n_rows).astype(np.float32)
+
+
+def _uniforms(rng, n):
+    return rng.integers(0, 1 << 32, size=n, dtype=np.uint64)
+
+
+def test_sample_accept_identical_distributions_accept_the_first_child_chain():
+    rng = np.random.default_rng(41)
+    for _ in range(20):
+        T, V = int(rng.integers(1, 12)), 17
+        par = W.random_tree_parents(int(rng.integers(1 << 30)), 3, T)
+        p = _rows(rng, T + 1, V)
+        # any token with draft probability > 0 is accepted, whatever the uniform says
+        tok = [int(rng.choice(np.flatnonzero(p[par[i] + 1] > 1e-6))) for i in range(T)]
+        path, bonus = oracle.sample_accept(tok, par, p, p, _uniforms(rng, T), _uniforms(rng, T + 1))
+        want, cur = [], -1
+        while True:
+            kids = [i for i in range(T) if par[i] == cur]
+            if not kids:
+                break
+            cur = kids[0]
+            want.append(cur)
+        assert path == want and 0 <= bonus < V
+
+
+def test_sample_accept_disjoint_supports_accept_nothing_and_emit_from_the_target():
+    rng = np.random.default_rng(42)
+    V, T, n = 8, 3, 4000
+    p = np.zeros((T + 1, V), np.float32); q = np.zeros_like(p)
+    p[:, :4] = _rows(rng, T + 1, 4); q[:, 4:] = _rows(rng, T + 1, 4)
+    counts = np.zeros(V)
+    for _ in range(n):
+        tok = [int(rng.integers(4, 8)) for _ in range(T)]
+        path, bonus = oracle.sample_accept(tok, [-1, -1, 0], p, q, _uniforms(rng, T), _uniforms(rng, T + 1))
+        assert path == []
+        counts[bonus] += 1
+    assert counts[4:].sum() == 0
+    expect = p[0].astype(np.float64) * n
+    assert np.all(np.abs(counts[:4] - expect[:4]) < 5 * np.sqrt(expect[:4] + 1))
+
+
+def test_sample_accept_with_one_hot_target_is_the_greedy_rule():
+    rng = np.random.default_rng(43)
+    for _ in range(30):
+        T, V = int(rng.integers(1, 14)), 6
+        par = W.random_tree_parents(int(rng.integers(1 << 30)), 5, T)
+        nxt = rng.integers(0, V, size=T + 1)
+        p = np.zeros((T + 1, V), np.float32)
+        p[np.arange(T + 1), nxt] = 1.0
+        q = _rows(rng, T + 1, V) * 0.98 + 0.02 / V           # every token has draft mass
+        tok = []
+        for i in range(T):                                   # siblings carry distinct tokens
+            used = {tok[j] for j in range(i) if par[j] == par[i]}
+            tok.append(int(rng.choice([v for v in range(V) if v not in used])))
+        path, bonus = oracle.sample_accept(tok, par, p, q, _uniforms(rng, T), _uniforms(rng, T + 1))
+        g_path, g_bonus = oracle.greedy_accept(tok, par, nxt)
+        # the walk follows accepted children, so it is the greedy chain whenever that chain is unique
+        # (distinct sibling tokens: at most one child of a node can match the target's token)
+        assert path == g_path and bonus == g_bonus
+
+
+def _draw_children_without_replacement(rng, q_row, k):
+    q = q_row.astype(np.float64).copy()
+    out = []
+    for _ in range(k):
+        q /= q.sum()
+        x = int(rng.choice(len(q), p=q))
+        out.append(x)
+        q[x] = 0.0
+    return out
+
+
+def test_sample_accept_emits_the_target_distribution():
+    """Root level with up to 3 sibling candidates drawn without replacement from q, then one more
+    level below the first candidate: the first and the second emitted token must be distributed as
+    the target rows say, although target and draft differ a lot."""
+    rng = np.random.default_rng(44)
+    V, n = 4, 30000
+    par = [-1, -1, -1, 0, 0]
+    p = np.array([[0.55, 0.05, 0.30, 0.10], [0.10, 0.60, 0.10, 0.20], [0.25, 0.25, 0.25, 0.25],
+                  [0.70, 0.10, 0.10, 0.10], [0.40, 0.30, 0.20, 0.10], [0.10, 0.20, 0.30, 0.40]], np.float32)
+    q = np.array([[0.10, 0.40, 0.20, 0.30], [0.30, 0.20, 0.40, 0.10], [0.25, 0.25, 0.25, 0.25],
+                  [0.25, 0.25, 0.25, 0.25], [0.25, 0.25, 0.25, 0.25], [0.25, 0.25, 0.25, 0.25]], np.float32)
+    first = np.zeros(V)
+    second_after_node0 = np.zeros(V)
+    n_node0 = 0
+    for _ in range(n):
+        roots = _draw_children_without_replacement(rng, q[0], 3)
+        kids = _draw_children_without_replacement(rng, q[1], 2)
+        tok = roots + kids
+        path, bonus = oracle.sample_accept(tok, par, p, q, _uniforms(rng, 5), _uniforms(rng, 6))
+        emitted = [tok[i] for i in path] + [bonus]
+        first[emitted[0]] += 1
+        if path and path[0] == 0:                           # the walk went through node 0: row 1 is next
+            n_node0 += 1
+            second_after_node0[emitted[1]] += 1
+    e1 = p[0].astype(np.float64) * n
+    assert np.all(np.abs(first - e1) < 4.5 * np.sqrt(e1)), (first, e1)
+    assert n_node0 > 2000
+    # the token after node 0 follows the target row of node 0 whatever token node 0 carried
+    e2 = p[1].astype(np.float64) * n_node0
+    assert np.all(np.abs(second_after_node0 - e2) < 4.5 * np.sqrt(e2)), (second_after_node0, e2)
+
+
+def test_sample_accept_pin_detects_a_planted_mistake():
+    """The distribution pin bites: leaving the draft distribution untouched after a rejection (the
+    with-replacement rule applied to candidates drawn without replacement) shifts the output."""
+    rng = np.random.default_rng(45)
+    V, n = 4, 30000
+    p = np.array([[0.55, 0.05, 0.30, 0.10]] * 4, np.float32)
+    q = np.array([[0.10, 0.40, 0.20, 0.30]] * 4, np.float32)
+
+    def wrong(tok, u_node, u_bonus):                        # the oracle's steps with the planted mistake
+        P, Q = oracle.fixed_point_probs(p[0]), oracle.fixed_point_probs(q[0])
+        A, Bq = int(P.sum()), int(Q.sum())
+        for c, x in enumerate(tok):
+            if int(u_node[c]) * int(Q[x]) * A < int(P[x]) * Bq * (1 << 32):
+                return x
+            P = np.maximum(Bq * P - A * Q, 0) >> 30
+            A = int(P.sum())                                # Q keeps x: the mistake
+        t = (int(u_bonus[0]) * A) >> 32
+        return int(np.searchsorted(np.cumsum(P), t, side="right"))
+
+    counts = np.zeros(V)
+    for _ in range(n):
+        tok = _draw_children_without_replacement(rng, q[0], 3)
+        counts[wrong(tok, _uniforms(rng, 3), _uniforms(rng, 1))] += 1
+    e = p[0].astype(np.float64) * n
+    assert np.any(np.abs(counts - e) > 6 * np.sqrt(e))
