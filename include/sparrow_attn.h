@@ -12,8 +12,9 @@
  *       with K_T, V_T restricted to the text-anchored positions T; the visual KV rows are never
  *       touched.  sparrow_anchor_attn_tree() is the same for a draft tree.
  * Around them, for a whole speculative step on the device: sparrow_kv_append(),
- * sparrow_compact_anchors() (row movers), sparrow_accept_greedy(), sparrow_kv_keep_accepted()
- * (temperature-0 acceptance of the draft tree and the move of the accepted rows).
+ * sparrow_compact_anchors() (row movers), sparrow_accept_greedy(), sparrow_accept_sample(),
+ * sparrow_kv_keep_accepted() (acceptance of the draft tree at temperature 0 and 1, and the move of
+ * the accepted rows).
  *
  * For every batch entry b, query head h (KV head h / 7), draft token t and visible key set Vis:
  *     s_j = softmax_scale * <q[b,t,h,:], k[b,h/7,j,:]>,   lse = log sum_{j in Vis} exp(s_j),
@@ -100,6 +101,10 @@ typedef enum {
  * SPARROW_ERR_SHAPE for an unknown value. */
 sparrow_status sparrow_set_plan_policy(sparrow_ctx* ctx, int32_t policy);
 
+/* enable != 0: single sparrow_verify_attn() calls of this context may start early too (see the
+ * ordering rules at sparrow_verify_attn()).  Off by default.  Host state only. */
+sparrow_status sparrow_set_call_overlap(sparrow_ctx* ctx, int32_t enable);
+
 /* Work items the planner currently aims for in fused mode (pass it to sparrow_plan_splits() as
  * n_sm to see the schedule of a call).  0 when ctx is NULL. */
 int32_t sparrow_plan_target_items(const sparrow_ctx* ctx);
@@ -126,28 +131,78 @@ sparrow_status sparrow_set_workspace(sparrow_ctx* ctx, void* dev_ptr, size_t byt
  *   lse      DEV fp32 [batch][n_q_heads][T], natural log of the softmax normaliser
  *   stream   cudaStream_t (NULL = default stream)
  * One kernel per call: a split-KV pass over ~one work item per SM whose last CTAs merge the
- * pieces by log-sum-exp.  Consecutive calls on one stream overlap: the kernel is launched with
- * programmatic stream serialisation and starts reading q / k_cache / v_cache / parents while the
- * previous kernel in the stream is finishing, as soon as that kernel lets its dependents launch
- * (the library's own kernels do; an ordinary kernel never does before it completes).  So the
- * inputs of a call must not be the out / lse of the library call enqueued directly before it on
- * the same stream; anything else in between (another kernel, a copy) restores plain stream order.
- * Writes of consecutive calls of one context are ordered through counters in its workspace; a
- * call that follows a call of another context takes plain stream order.  All fused calls of a
- * context belong on one stream (or must be kept from running concurrently by events): the
- * counters assume that calls run in the order they were enqueued.  While a stream is being
- * captured into a graph, or with SPARROW_NO_PDL=1 in the environment when the context is created,
- * a call is two ordinary launches (split-KV pass, combine) ordered by the stream alone.
+ * pieces by log-sum-exp.
+ *
+ * Ordering.  By default a call is an ordinary launch: it starts after everything enqueued before
+ * it on `stream` has finished.  Where the library knows that the kernel directly before a call in
+ * the stream is this context's previous verification call, the call starts early (programmatic
+ * stream serialisation): it reads q / k_cache / v_cache / parents while that call is still
+ * finishing, and several calls can be resident at once.  That is the case
+ *   - for the second and later calls of one sparrow_verify_attn_batch(), and
+ *   - for every call after sparrow_set_call_overlap(ctx, 1), by which the caller vouches that
+ *     whatever it enqueues on the stream between two calls of this context either is an ordinary
+ *     kernel / copy (which completes before its successors start) or writes none of the next
+ *     call's inputs.  (A kernel that lets its dependents launch early -- many library GEMM, norm
+ *     and RoPE kernels do -- and then writes q or the new K/V rows is what must not sit there.)
+ * A call that would start early but reads memory that one of this context's calls which may
+ * still be running writes (its out / lse) is launched in plain stream order instead, as is a call
+ * that follows a call of another context.  Writes of consecutive calls of one context are ordered
+ * through counters in its workspace.  All calls of a context belong on one stream (or must be kept
+ * from running concurrently by events): the counters assume that calls run in the order they were
+ * enqueued.  While a stream is being captured into a graph, or with SPARROW_NO_PDL=1 in the
+ * environment when the context is created, a call is two ordinary launches (split-KV pass,
+ * combine) ordered by the stream alone.
  * Results are deterministic for fixed arguments. */
 sparrow_status sparrow_verify_attn(sparrow_ctx* ctx, const void* q, const void* k_cache,
                                    const void* v_cache, const int32_t* kv_len,
                                    const int32_t* parents, int32_t T, void* out, float* lse,
                                    void* stream);
 
+/* (a) generalised for the draft model's attention on a COMPACTED text-anchored cache (Eq. 2,
+ * Section 3.1; sparrow_compact_anchors() builds such a cache): the text-anchored window mode as a
+ * contiguous stream for the tensor-core kernel.
+ *   - The draft block holds the T_tree nodes of the draft tree (rows [kv_len[b], kv_len[b] +
+ *     T_tree), parents DEV int32 [batch][T_tree]); the queries are its last T_new nodes
+ *     (q, out: [batch][T_new][n_q_heads][128]; lse: [batch][n_q_heads][T_new]).  T_new = T_tree
+ *     is sparrow_verify_attn().
+ *   - first_visible  DEV int32 [batch][T_new] or NULL: query t sees prefix key j only if
+ *     j >= first_visible[b][t] (values above kv_len[b] count as kv_len[b]); the draft block is
+ *     governed by the tree alone.  With anchors in increasing order the window rule of
+ *     sparrow_anchor_attn() ("qpos - window < p") selects exactly such a run of compact rows;
+ *     sparrow_window_first_visible() / _device() compute the index.
+ *   - first_visible_min  HOST int32 [batch] or NULL: a lower bound of first_visible[b][*] that the
+ *     caller knows on the host (0 <= value <= kv_len[b]); keys left of it (rounded down to a
+ *     128-key tile) are not streamed at all.  A device-side bound below it is reported through
+ *     the anchor status bit and treated as the first streamed key.
+ * Ordering, errors and everything else as for sparrow_verify_attn(); SPARROW_ERR_SHAPE unless
+ * 1 <= T_new <= T_tree <= SPARROW_MAX_T and kv_len[b] + T_tree <= kv_capacity. */
+sparrow_status sparrow_verify_attn_window(sparrow_ctx* ctx, const void* q, const void* k_cache,
+                                          const void* v_cache, const int32_t* kv_len,
+                                          const int32_t* parents, int32_t T_tree, int32_t T_new,
+                                          const int32_t* first_visible, const int32_t* first_visible_min,
+                                          void* out, float* lse, void* stream);
+
+/* The window rule of mode (b) on a compacted cache.  anchor_idx: n_anchor strictly increasing
+ * rows, the last T_tree of them the draft tree's nodes, the queries its last T_new nodes (as in
+ * sparrow_anchor_attn_tree()); compact row j holds anchor j.  first_visible[t] = the first text
+ * anchor j (j < n_anchor - T_tree) with anchor_idx[j] > qpos_t - window, qpos_t = the query's own
+ * row; n_anchor - T_tree if there is none; 0 when window <= 0.
+ * Host version: one sequence, HOST arrays, also returns the smallest of them (may be NULL);
+ * SPARROW_ERR_ANCHOR unless the list is strictly increasing and n_anchor >= T_tree.
+ * Device version: DEV anchor_idx [batch][n_anchor] -> DEV first_visible [batch][T_new], one small
+ * kernel on `stream` (a binary search per query). */
+sparrow_status sparrow_window_first_visible(const int32_t* anchor_idx, int32_t n_anchor, int32_t window,
+                                            int32_t T_tree, int32_t T_new, int32_t* first_visible,
+                                            int32_t* first_visible_min);
+sparrow_status sparrow_window_first_visible_device(sparrow_ctx* ctx, const int32_t* anchor_idx,
+                                                   int32_t n_anchor, int32_t window, int32_t T_tree,
+                                                   int32_t T_new, int32_t* first_visible, void* stream);
+
 /* Several verification calls enqueued back to back on one stream -- e.g. the layers of one
  * decode step, each with its own KV cache (Section 4: the target verifies the draft tree in one
- * forward pass, i.e. one such call per decoder layer).  Equivalent to calling
- * sparrow_verify_attn() n_calls times; stops at the first error.  `calls` is HOST memory. */
+ * forward pass, i.e. one such call per decoder layer).  Same results as calling
+ * sparrow_verify_attn() n_calls times; the calls after the first start early (nothing can sit
+ * between them in the stream).  Stops at the first error.  `calls` is HOST memory. */
 typedef struct {
     const void*    q;
     const void*    k_cache;
@@ -206,8 +261,8 @@ sparrow_status sparrow_anchor_attn_tree(sparrow_ctx* ctx, const void* q, const v
  * sparrow_compact_anchors: copies rows anchor_idx[b][0 .. n_anchor) of k / v (the context's layout)
  * to rows [dst_row, dst_row + n_anchor) of a compact cache laid out
  * [batch][n_kv_heads][compact_capacity][128], contiguous.  On the compact cache the anchored mode
- * without a lower window bound is sparrow_verify_attn() with kv_len = (anchors before the draft
- * block): a contiguous stream for the tensor-core kernel instead of a gather.
+ * is sparrow_verify_attn_window() with kv_len = (anchors before the draft block): a contiguous
+ * stream for the tensor-core kernel instead of a gather.
  *   anchor_idx  DEV int32 [batch][n_anchor]; an entry outside [0, kv_capacity) is not read: its
  *               row is written as zeros and the anchor status bit is set.
  * SPARROW_ERR_ANCHOR unless 1 <= n_anchor <= kv_capacity; SPARROW_ERR_SHAPE unless
@@ -242,6 +297,35 @@ sparrow_status sparrow_compact_anchors(sparrow_ctx* ctx, const void* k, const vo
  * Both: SPARROW_ERR_SHAPE unless 1 <= T <= SPARROW_MAX_T (and kv_len[b] + T <= kv_capacity). */
 sparrow_status sparrow_accept_greedy(sparrow_ctx* ctx, const int32_t* draft_tokens, const int32_t* parents,
                                      const int32_t* target_next, int32_t T, int32_t* path_out,
+                                     int32_t* n_accept_out, int32_t* bonus_out, void* stream);
+/* sparrow_accept_sample: temperature-1 acceptance of a draft tree by multi-round rejection sampling
+ * (Appendix A: the verification keeps the target's output distribution exactly; Section 4 reports
+ * every result at temperature 0 and 1.  The paper relies on the standard procedure; the reading
+ * taken here: at the current node, with target distribution p and draft distribution q, the
+ * children are tried in index order; a child with token x is accepted with probability
+ * min(1, p(x) / q(x)); after a rejection p becomes the normalised positive part of (p - q) and q
+ * loses x, the siblings having been drawn without replacement; when no child is accepted the
+ * next token is drawn from what p has become.)
+ *   draft_tokens DEV int32 [batch][T];  parents DEV int32 [batch][T] as in (a)
+ *   p_target,
+ *   p_draft      DEV fp32 [batch][T + 1][vocab]: row 0 belongs to the committed prefix, row 1 + i to
+ *                node i -- the target's next-token distribution there and the draft distribution
+ *                that node's children were drawn from; entries in [0, 1]
+ *   u_node       DEV uint32 [batch][T]      the uniform of node i's acceptance test
+ *   u_bonus      DEV uint32 [batch][T + 1]  the uniform of the token drawn when the walk stops at a row
+ *   path_out, n_accept_out, bonus_out as for sparrow_accept_greedy (the accepted chain, its length,
+ *                the token emitted after it); sparrow_kv_keep_accepted() takes them as they are.
+ * The outputs are integers, so the arithmetic is fixed: P = floor(p 2^30 + 1/2) (likewise Q), and
+ * with A = sum P, B = sum Q, r the node's uniform: accept iff Q[x] > 0 and r Q[x] A < P[x] B 2^32;
+ * after a rejection P <- max(B P - A Q, 0) >> 30 (unless B == 0), A <- sum P, B <- B - Q[x],
+ * Q[x] <- 0; the bonus token is the smallest v with P[0] + ... + P[v] > (u_bonus A) >> 32, P
+ * being the row's original target row again if A == 0.  Integer sums: the result does not depend
+ * on how the reduction is parallelised.  A token outside [0, vocab) is never accepted and sets
+ * the tree status bit, as does a malformed parent (which counts as a root).
+ * SPARROW_ERR_SHAPE unless 1 <= T <= SPARROW_MAX_T and vocab >= 1. */
+sparrow_status sparrow_accept_sample(sparrow_ctx* ctx, const int32_t* draft_tokens, const int32_t* parents,
+                                     const float* p_target, const float* p_draft, const uint32_t* u_node,
+                                     const uint32_t* u_bonus, int32_t vocab, int32_t T, int32_t* path_out,
                                      int32_t* n_accept_out, int32_t* bonus_out, void* stream);
 sparrow_status sparrow_kv_keep_accepted(sparrow_ctx* ctx, void* k_cache, void* v_cache,
                                         const int32_t* kv_len, const int32_t* path,
@@ -281,8 +365,11 @@ sparrow_status sparrow_verify_step_host(sparrow_ctx* ctx, const void* q_host,
  *   - First call on a device: one-time set-up (device query, kernel attributes, address of the
  *     scratch array, clearing its header with a synchronising cudaMemset).  Make that first call
  *     outside any stream capture.
- *   - SPARROW_ERR_WORKSPACE when the layout / T need more scratch than the array holds (on a
- *     148-SM part: blocks of more than 36 draft tokens, or large batches); nothing is launched then.
+ *   - Argument errors are reported as by sparrow_verify_attn(), before anything is enqueued.
+ *     SPARROW_ERR_WORKSPACE when the split-KV partials of the call do not fit the array behind its
+ *     1 KiB header: a call has max(SM count, batch x KV heads x row groups) work items of at most
+ *     70 KB each, so on a 148-SM part everything fits except very large batches of draft blocks
+ *     longer than 18 tokens (e.g. 32 sequences x 64 tokens); nothing is enqueued then either.
  *   - The call always runs in the stream-ordered mode: two ordinary kernel launches on `stream`.
  *   - All calls on a device share the one array, which keeps the previous call's contents.  What
  *     must start clean (the status word) is cleared on `stream` at the start of every call;
@@ -332,6 +419,13 @@ sparrow_status sparrow_plan_piece_range(int32_t n_keys, int32_t n_splits, int32_
  * ahead > 0 nothing will ever satisfy it, the wait gives up after about one second, the kernel
  * sets the timeout status bit and ends -- the context stays usable. */
 sparrow_status sparrow_debug_wait_counter(sparrow_ctx* ctx, uint32_t ahead, void* stream);
+
+/* Test aid for the ordering rules of sparrow_verify_attn(): enqueues a small kernel that lets its
+ * dependents launch at once, idles for about delay_us microseconds (at most 10 ms) and only then
+ * copies `bytes` (a multiple of 16, both pointers 16-byte aligned, DEV) from src to dst -- the
+ * behaviour of a foreign kernel with an early launch trigger in front of a verification call. */
+sparrow_status sparrow_debug_early_trigger_copy(sparrow_ctx* ctx, const void* src, void* dst, size_t bytes,
+                                               uint32_t delay_us, void* stream);
 
 /* Synchronises `stream`, returns the sticky device status (SPARROW_OK, SPARROW_ERR_TREE,
  * SPARROW_ERR_ANCHOR or SPARROW_ERR_TIMEOUT) and clears it.  Not for the hot path. */

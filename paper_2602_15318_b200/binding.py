@@ -25,8 +25,10 @@ EXPORTS = ["sparrow_create", "sparrow_destroy", "sparrow_workspace_bytes", "spar
            "sparrow_build_ancestor_masks", "sparrow_build_anchor_idx",
            "sparrow_debug_ancestor_masks_device", "sparrow_debug_wait_counter", "sparrow_plan_splits",
            "sparrow_last_device_status", "sparrow_debug_status_word", "sparrow_launch_count",
-           "sparrow_set_plan_policy", "sparrow_plan_target_items", "sparrow_anchor_attn_tree", "sparrow_kv_append", "sparrow_compact_anchors",
-           "sparrow_accept_greedy", "sparrow_kv_keep_accepted", "sparrow_plan_piece_range",
+           "sparrow_set_plan_policy", "sparrow_set_call_overlap", "sparrow_debug_early_trigger_copy",
+           "sparrow_verify_attn_window", "sparrow_window_first_visible", "sparrow_window_first_visible_device",
+           "sparrow_plan_target_items", "sparrow_anchor_attn_tree", "sparrow_kv_append", "sparrow_compact_anchors",
+           "sparrow_accept_greedy", "sparrow_accept_sample", "sparrow_kv_keep_accepted", "sparrow_plan_piece_range",
            "sparrow_status_string"]
 
 
@@ -65,10 +67,14 @@ def lib():
         L.sparrow_set_workspace.argtypes = [vp, vp, ctypes.c_size_t]
         L.sparrow_verify_attn.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp, vp, vp]
         L.sparrow_verify_attn_batch.argtypes = [vp, vp, i32, vp]
+        L.sparrow_verify_attn_window.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp]
+        L.sparrow_window_first_visible.argtypes = [vp, i32, i32, i32, i32, vp, vp]
+        L.sparrow_window_first_visible_device.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp]
         L.sparrow_verify_attn_static.argtypes = [ctypes.POINTER(Layout), vp, vp, vp, vp, vp, i32, vp, vp, vp]
         L.sparrow_anchor_attn.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp]
         L.sparrow_plan_piece_range.argtypes = [i32, i32, i32, vp, vp]
         L.sparrow_accept_greedy.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp]
+        L.sparrow_accept_sample.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp]
         L.sparrow_kv_keep_accepted.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp]
         L.sparrow_kv_append.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp]
         L.sparrow_compact_anchors.argtypes = [vp, vp, vp, vp, i32, vp, vp, i32, i32, vp]
@@ -81,6 +87,8 @@ def lib():
         L.sparrow_plan_splits.argtypes = [i32, i32, i32, vp, i32, vp, vp]
         L.sparrow_last_device_status.argtypes = [vp, vp]
         L.sparrow_set_plan_policy.argtypes = [vp, i32]
+        L.sparrow_set_call_overlap.argtypes = [vp, i32]
+        L.sparrow_debug_early_trigger_copy.argtypes = [vp, vp, vp, ctypes.c_size_t, ctypes.c_uint32, vp]
         L.sparrow_plan_target_items.argtypes = [vp]
         L.sparrow_plan_target_items.restype = i32
         L.sparrow_debug_status_word.argtypes = [vp]
@@ -161,6 +169,10 @@ class Context:
     def set_plan_policy(self, policy: int):
         _chk(lib().sparrow_set_plan_policy(self.handle, int(policy)), "sparrow_set_plan_policy")
 
+    def set_call_overlap(self, enable: bool):
+        """Single sparrow_verify_attn calls may start early behind this context's previous call."""
+        _chk(lib().sparrow_set_call_overlap(self.handle, 1 if enable else 0), "sparrow_set_call_overlap")
+
     def plan_target_items(self) -> int:
         return int(lib().sparrow_plan_target_items(self.handle))
 
@@ -187,6 +199,35 @@ def sparrow_verify_attn(ctx: Context, q, k_cache, v_cache, kv_len: Sequence[int]
     kl = _i32_array(kv_len)
     _chk(lib().sparrow_verify_attn(ctx.handle, _ptr(q), _ptr(k_cache), _ptr(v_cache), kl, _ptr(parents),
                                    T, _ptr(out), _ptr(lse), _stream_handle(stream)), "sparrow_verify_attn")
+
+
+def sparrow_verify_attn_window(ctx: Context, q, k_cache, v_cache, kv_len: Sequence[int], parents, T_tree: int,
+                               T_new: int, first_visible, first_visible_min: Optional[Sequence[int]], out, lse,
+                               stream=None):
+    """Verification kernel on a compacted anchored cache: queries = the last T_new of T_tree draft
+    nodes; first_visible: CUDA int32 [B,T_new] or None; first_visible_min: host ints or None."""
+    kl = _i32_array(kv_len)
+    fm = _i32_array(first_visible_min) if first_visible_min is not None else None
+    _chk(lib().sparrow_verify_attn_window(ctx.handle, _ptr(q), _ptr(k_cache), _ptr(v_cache), kl, _ptr(parents),
+                                          T_tree, T_new, _ptr(first_visible), fm, _ptr(out), _ptr(lse),
+                                          _stream_handle(stream)), "sparrow_verify_attn_window")
+
+
+def sparrow_window_first_visible(anchor_idx: Sequence[int], window: int, T_tree: int, T_new: int):
+    """Host helper: (first_visible list of T_new ints, their minimum)."""
+    idx = _i32_array(anchor_idx)
+    first = (ctypes.c_int32 * T_new)()
+    lowest = ctypes.c_int32(0)
+    _chk(lib().sparrow_window_first_visible(idx, len(anchor_idx), window, T_tree, T_new, first, ctypes.byref(lowest)),
+         "sparrow_window_first_visible")
+    return [int(x) for x in first], int(lowest.value)
+
+
+def sparrow_window_first_visible_device(ctx: Context, anchor_idx, n_anchor: int, window: int, T_tree: int, T_new: int,
+                                        first_visible, stream=None):
+    _chk(lib().sparrow_window_first_visible_device(ctx.handle, _ptr(anchor_idx), n_anchor, window, T_tree, T_new,
+                                                   _ptr(first_visible), _stream_handle(stream)),
+         "sparrow_window_first_visible_device")
 
 
 def sparrow_verify_attn_static(layout: Layout, q, k_cache, v_cache, kv_len: Sequence[int], parents, T: int,
@@ -263,6 +304,15 @@ def sparrow_accept_greedy(ctx: Context, draft_tokens, parents, target_next, T: i
          "sparrow_accept_greedy")
 
 
+def sparrow_accept_sample(ctx: Context, draft_tokens, parents, p_target, p_draft, u_node, u_bonus, vocab: int, T: int,
+                          path_out, n_accept_out, bonus_out, stream=None):
+    """Temperature-1 acceptance.  p_target / p_draft: CUDA fp32 [B, T+1, vocab]; u_node: CUDA int32
+    [B, T] and u_bonus: CUDA int32 [B, T+1] holding the bit patterns of 32-bit unsigned uniforms."""
+    _chk(lib().sparrow_accept_sample(ctx.handle, _ptr(draft_tokens), _ptr(parents), _ptr(p_target), _ptr(p_draft),
+                                     _ptr(u_node), _ptr(u_bonus), vocab, T, _ptr(path_out), _ptr(n_accept_out),
+                                     _ptr(bonus_out), _stream_handle(stream)), "sparrow_accept_sample")
+
+
 def sparrow_kv_keep_accepted(ctx: Context, k_cache, v_cache, kv_len: Sequence[int], path, n_accept, T: int,
                              stream=None):
     _chk(lib().sparrow_kv_keep_accepted(ctx.handle, _ptr(k_cache), _ptr(v_cache), _i32_array(kv_len), _ptr(path),
@@ -307,6 +357,11 @@ def sparrow_debug_ancestor_masks_device(ctx: Context, parents_dev: torch.Tensor,
 
 def sparrow_debug_wait_counter(ctx: Context, ahead: int, stream=None):
     _chk(lib().sparrow_debug_wait_counter(ctx.handle, ahead, _stream_handle(stream)), "sparrow_debug_wait_counter")
+
+
+def sparrow_debug_early_trigger_copy(ctx: Context, src, dst, nbytes: int, delay_us: int, stream=None):
+    _chk(lib().sparrow_debug_early_trigger_copy(ctx.handle, _ptr(src), _ptr(dst), nbytes, delay_us,
+                                                _stream_handle(stream)), "sparrow_debug_early_trigger_copy")
 
 
 def sparrow_plan_splits(n_sm: int, n_kv_heads: int, n_keys: Sequence[int], T: int):

@@ -17,9 +17,11 @@
 #include "combine.cuh"
 #include "common.cuh"
 #include "accept.cuh"
+#include "accept_sample.cuh"
 #include "kv_rows.cuh"
 #include "split_gather.cuh"
 #include "verify_tc.cuh"
+#include "window.cuh"
 
 using namespace sparrow;
 
@@ -28,36 +30,50 @@ typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint3
                                       CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 struct TensorMapEntry {
-    const void* base;
+    const void* base;        // nullptr: free slot
     int tag;                 // 0: K/V cache map; n > 0: Q map for n = batch * T tokens
     CUtensorMap map;
 };
-constexpr int kMapCacheSize = 128;
+// Hashed by (base pointer, tag), a bucket being kMapWays consecutive slots: room for the q / K / V
+// buffers of a few hundred layers or rotation slots before anything is encoded twice.
+constexpr int kMapCacheSize = 1024;
+constexpr int kMapWays = 8;
+
+// Fused calls that can still be resident on the GPU when a new one starts: each has at least one
+// CTA on an SM of its own, so there are fewer of them than SMs.
+constexpr int kRecentCalls = 192;
+struct RecentCall {
+    uintptr_t out[2], lse[2];    // [begin, end) of what the call writes
+};
 
 struct sparrow_ctx {
     TensorMapEntry maps[kMapCacheSize];      // Q / K / V tensor maps, keyed by base pointer (and token count)
-    int n_maps;
-    int next_evict;
+    unsigned evict_tick;
     TensorMapEncodeFn encode;
-    bool verify_on_gather;                   // bring-up aid: route verification through the gather kernel
     sparrow_layout layout;
     int device;
     int n_sm;
     int plan_policy;                         // sparrow_plan_policy
-    int target_override;                     // > 0: SPARROW_TARGET_ITEMS (diagnosis), replaces the policy's target
     unsigned char* ws;
     size_t ws_bytes;
+    size_t part_offset;                      // first byte of the split-KV partials in the workspace
+    int part_buffers;                        // 2: alternate by call parity (fused mode); 1: stream-ordered calls only
     std::atomic<long long> launches;
     bool use_pdl;
+    bool overlap_single_calls;               // sparrow_set_call_overlap()
+    bool chain_next;                         // the call being enqueued directly follows this context's previous fused call
     // Host mirror of the ordering counters in the workspace (see SyncArgs): call sequence number
     // of the fused calls and, per call parity, the cumulative number of finishers launched so far.
     uint32_t seq;
     uint32_t fin_total[2];
     uint32_t fin_before_last[2];             // fin_total[p] as it was before the last call of parity p
-    // Memory the previous fused call touches (out, lse, q, parents, k, v), as [begin, end) addresses:
+    // Memory the previous fused call touches (out, lse, q, parents, k, v, window bounds), as [begin, end) addresses:
     // a call whose outputs overlap none of it need not wait for that call's merge.
-    uintptr_t prev_ranges[6][2];
+    uintptr_t prev_ranges[7][2];
     bool prev_valid;
+    // Outputs of the fused calls launched since this context's last launch in plain stream order.
+    RecentCall recent[kRecentCalls];
+    int n_recent, recent_head;
     uint32_t last_status_word;   // raw word read by the last sparrow_last_device_status()
 };
 
@@ -66,6 +82,7 @@ namespace {
 constexpr size_t kStatusBytes = 1024;      // word 0: sticky status; words 16, 17: finisher counters
 constexpr size_t kFinDoneOffset = 64;
 constexpr size_t kArrivalsOffset = 128;     // words 32..35: arrival words of the four call slots
+constexpr size_t kSerialOffset = 192;       // words 48, 49: arrival / exit words of a call that runs alone (serial mode)
 constexpr int kMinPieceKeys = 128;
 // The gathered kernel works on 64-key tiles and pays two dependent memory round trips per tile
 // (anchor indices, then the rows), which a CTA with several tiles takes one after the other: short
@@ -100,13 +117,15 @@ int max_items(int n_sm, int batch, int n_kv_heads, int n_groups)
 
 // Chooses the number of key-range pieces per sequence so that the total number of work items is
 // close to (and not above) the SM count while every item streams about the same number of keys.
+// key0 (optional): per sequence, the first key that is streamed at all (a multiple of 128).
 sparrow_status make_plan(int n_sm, int batch, int n_kv_heads, const int32_t* n_keys, int T, int blocks_per_group,
-                         SplitPlan* p, int min_piece_keys = kMinPieceKeys)
+                         SplitPlan* p, int min_piece_keys = kMinPieceKeys, const int32_t* key0 = nullptr)
 {
     if (batch < 1 || batch > kMaxBatch || T < 1 || T > kMaxT || n_kv_heads < 1 || n_sm < 1) return SPARROW_ERR_SHAPE;
     std::memset(p, 0, sizeof(*p));
     p->batch = batch;
     p->T = T;
+    p->T_tree = T;
     p->M = kGroup * T;
     p->blocks_per_group = blocks_per_group;
     p->n_groups = (T + kTokPerBlock * blocks_per_group - 1) / (kTokPerBlock * blocks_per_group);
@@ -115,13 +134,16 @@ sparrow_status make_plan(int n_sm, int batch, int n_kv_heads, const int32_t* n_k
     p->part_rows = blocks_per_group * kBlockRows + 1;    // odd pitch: partial rows of successive pieces must not share L2 sets
     const int units = n_kv_heads * p->n_groups;
     int max_keys = 1;
+    int32_t streamed[kMaxBatch];                  // keys each sequence streams
     for (int b = 0; b < batch; ++b) {
-        if (n_keys[b] < 1) return SPARROW_ERR_SHAPE;
-        if (n_keys[b] > max_keys) max_keys = n_keys[b];
+        const int32_t k0 = key0 ? key0[b] : 0;
+        if (n_keys[b] < 1 || k0 < 0 || k0 >= n_keys[b] || (k0 % kKeyTile) != 0) return SPARROW_ERR_SHAPE;
+        streamed[b] = n_keys[b] - k0;
+        if (streamed[b] > max_keys) max_keys = streamed[b];
     }
     auto items_for = [&](long long L) {
         long long n = 0;
-        for (int b = 0; b < batch; ++b) n += (long long)units * ((n_keys[b] + L - 1) / L);
+        for (int b = 0; b < batch; ++b) n += (long long)units * ((streamed[b] + L - 1) / L);
         return n;
     };
     long long lo = min_piece_keys, hi = max_keys > min_piece_keys ? max_keys : min_piece_keys;
@@ -134,7 +156,8 @@ sparrow_status make_plan(int n_sm, int batch, int n_kv_heads, const int32_t* n_k
     int total = 0;
     for (int b = 0; b < batch; ++b) {
         p->seq[b].n_keys = n_keys[b];
-        p->seq[b].n_splits = (int)((n_keys[b] + lo - 1) / lo);
+        p->seq[b].key0 = key0 ? key0[b] : 0;
+        p->seq[b].n_splits = (int)((streamed[b] + lo - 1) / lo);
         p->seq[b].item_begin = total;
         total += units * p->seq[b].n_splits;
     }
@@ -147,12 +170,11 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 size_t fixed_bytes(const sparrow_layout& L) { return kStatusBytes + staging_layout(L).total; }
 size_t part_bytes(size_t rows) { return align_up(rows * kPartRowHalves * sizeof(__half), 256); }
 
-// The partial outputs are double-buffered by call parity: buffer p is the p-th half of what
-// follows the header and the staging area.
+// The partial outputs start at part_offset (behind the header and, for a caller-provided
+// workspace, the staging area) and are double-buffered by call parity where calls can overlap.
 size_t part_half_bytes(const sparrow_ctx* c)
 {
-    const size_t fixed = fixed_bytes(c->layout);
-    return c->ws_bytes > fixed ? ((c->ws_bytes - fixed) / 2) & ~(size_t)255 : 0;
+    return c->ws_bytes > c->part_offset ? ((c->ws_bytes - c->part_offset) / c->part_buffers) & ~(size_t)255 : 0;
 }
 
 sparrow_status check_ws(const sparrow_ctx* c, const SplitPlan& p)
@@ -163,7 +185,7 @@ sparrow_status check_ws(const sparrow_ctx* c, const SplitPlan& p)
 
 __half* o_part_ptr(const sparrow_ctx* c, int parity)
 {
-    return reinterpret_cast<__half*>(c->ws + fixed_bytes(c->layout) + parity * part_half_bytes(c));
+    return reinterpret_cast<__half*>(c->ws + c->part_offset + (c->part_buffers > 1 ? parity : 0) * part_half_bytes(c));
 }
 
 // Ordering arguments of the next call and, once it is enqueued, the advance of the host mirror.
@@ -193,16 +215,16 @@ int policy_target(int n_sm, int policy)
 // Calls that cannot overlap others always get one wave over all SMs.
 int plan_target(const sparrow_ctx* c, bool overlaps)
 {
-    if (!overlaps) return c->n_sm;
-    return c->target_override > 0 ? c->target_override : policy_target(c->n_sm, c->plan_policy);
+    return overlaps ? policy_target(c->n_sm, c->plan_policy) : c->n_sm;
 }
 
+constexpr int kCallRanges = 7;
 struct CallRanges {
-    uintptr_t r[6][2];               // out, lse (written), q, parents, k, v (read)
+    uintptr_t r[kCallRanges][2];     // out, lse (written), q, parents, k, v, window bounds (read)
 };
 
-CallRanges call_ranges(const sparrow_ctx* c, const void* q, const void* k, const void* v, const int32_t* parents, int T,
-                       const void* out, const float* lse)
+CallRanges call_ranges(const sparrow_ctx* c, const void* q, const void* k, const void* v, const int32_t* parents, int T_tree,
+                       int T, const int32_t* first_visible, const void* out, const float* lse)
 {
     const sparrow_layout& L = c->layout;
     const size_t tok_bytes = (size_t)L.batch * T * L.n_q_heads * kD * 2;
@@ -216,9 +238,10 @@ CallRanges call_ranges(const sparrow_ctx* c, const void* q, const void* k, const
     set(0, out, tok_bytes);
     set(1, lse, (size_t)L.batch * L.n_q_heads * T * 4);
     set(2, q, tok_bytes);
-    set(3, parents, (size_t)L.batch * T * 4);
+    set(3, parents, (size_t)L.batch * T_tree * 4);
     set(4, k, kv_bytes);
     set(5, v, kv_bytes);
+    set(6, first_visible, first_visible ? (size_t)L.batch * T * 4 : 0);
     return cr;
 }
 
@@ -227,19 +250,57 @@ bool outputs_touch_previous(const sparrow_ctx* c, const CallRanges& cr)
 {
     if (!c->prev_valid) return false;
     for (int o = 0; o < 2; ++o)
-        for (int i = 0; i < 6; ++i)
+        for (int i = 0; i < kCallRanges; ++i)
             if (cr.r[o][0] < c->prev_ranges[i][1] && c->prev_ranges[i][0] < cr.r[o][1]) return true;
     return false;
 }
 
+// Does this call read (q, parents, k, v) anything that a fused call which may still be running
+// writes?  Such a call must not start early: it is launched in plain stream order.
+bool inputs_touch_recent_outputs(const sparrow_ctx* c, const CallRanges& cr)
+{
+    uintptr_t lo = cr.r[2][0], hi = cr.r[2][1];
+    for (int i = 3; i < kCallRanges; ++i) {
+        if (cr.r[i][0] == cr.r[i][1]) continue;            // absent
+        if (cr.r[i][0] < lo) lo = cr.r[i][0];
+        if (cr.r[i][1] > hi) hi = cr.r[i][1];
+    }
+    for (int n = 0; n < c->n_recent; ++n) {
+        const RecentCall& rc = c->recent[n];
+        const uintptr_t w_lo = rc.out[0] < rc.lse[0] ? rc.out[0] : rc.lse[0];
+        const uintptr_t w_hi = rc.out[1] > rc.lse[1] ? rc.out[1] : rc.lse[1];
+        if (hi <= w_lo || w_hi <= lo) continue;            // nothing of this call near what that one writes
+        for (int i = 2; i < kCallRanges; ++i)
+            if ((cr.r[i][0] < rc.out[1] && rc.out[0] < cr.r[i][1]) || (cr.r[i][0] < rc.lse[1] && rc.lse[0] < cr.r[i][1]))
+                return true;
+    }
+    return false;
+}
+
+// Book-keeping after a fused launch.  A launch in plain stream order follows everything enqueued
+// before it, so the calls before it cannot be running beside any later call; otherwise the list
+// keeps the last kRecentCalls calls, which is more than can be resident at once.
+void note_fused_launch(sparrow_ctx* c, const CallRanges& cr, bool launched_early)
+{
+    if (!launched_early) c->n_recent = c->recent_head = 0;
+    RecentCall& rc = c->recent[c->recent_head];
+    rc.out[0] = cr.r[0][0]; rc.out[1] = cr.r[0][1];
+    rc.lse[0] = cr.r[1][0]; rc.lse[1] = cr.r[1][1];
+    c->recent_head = (c->recent_head + 1) % kRecentCalls;
+    if (c->n_recent < kRecentCalls) ++c->n_recent;
+}
+
 // `after_previous`: the call's final results must wait for the previous fused call as a whole (its
 // outputs overlap that call's memory); otherwise they only wait for the calls before that one.
-SyncArgs next_sync(const sparrow_ctx* c, const SplitPlan& p, bool overlaps, bool after_previous)
+// `self_merging`: the kernel merges its own partials (the tensor-core kernel); a call of it that
+// cannot overlap its neighbours runs in serial mode.
+SyncArgs next_sync(const sparrow_ctx* c, const SplitPlan& p, bool overlaps, bool after_previous, bool self_merging)
 {
     SyncArgs sy;
     const int parity = (int)(c->seq & 1u);
     sy.arrivals = reinterpret_cast<unsigned*>(c->ws + kArrivalsOffset);
     sy.fin_done = reinterpret_cast<unsigned*>(c->ws + kFinDoneOffset);
+    sy.serial_words = reinterpret_cast<unsigned*>(c->ws + kSerialOffset);
     sy.enabled = overlaps ? 1 : 0;
     sy.parity = parity;
     sy.slot = (int)(c->seq & 3u);
@@ -247,7 +308,12 @@ SyncArgs next_sync(const sparrow_ctx* c, const SplitPlan& p, bool overlaps, bool
     for (int b = 0; b < p.batch; ++b)
         if (p.seq[b].n_splits > 1) n_arrive += p.n_kv_heads * p.n_groups * p.seq[b].n_splits;
     sy.n_arrive = n_arrive;
-    sy.n_fin = n_arrive == 0 ? 0 : (p.n_items < kFinisherCtas ? p.n_items : kFinisherCtas);
+    sy.serial = (!overlaps && self_merging && n_arrive > 0) ? 1 : 0;
+    // Finishers wait, holding their SM, until the call's last piece is in: few of them where later
+    // calls should move in beside this one, all CTAs where the call has the GPU to itself anyway
+    // (serial mode, and the one-wave latency policy).
+    const bool all_finish = sy.serial || (overlaps && c->plan_policy == SPARROW_PLAN_LATENCY);
+    sy.n_fin = n_arrive == 0 ? 0 : ((all_finish || p.n_items < kFinisherCtas) ? p.n_items : kFinisherCtas);
     sy.fin_wait_same = c->fin_total[parity];
     sy.fin_wait_other = after_previous ? c->fin_total[parity ^ 1] : c->fin_before_last[parity ^ 1];
     return sy;
@@ -324,15 +390,21 @@ sparrow_status launch_split_gather(sparrow_ctx* c, const SplitPlan& plan, const 
 // query tensor [n_tok][KV heads][7][128], boxes of 64 dims x 7 heads x 18 tokens, which land in
 // shared memory as the rows (t * 7 + g) of a K-major operand block; tokens past n_tok read as zero.
 // Both use the 128-byte swizzle.
-const CUtensorMap* tensor_map_for(sparrow_ctx* c, const void* base, int tag)
+bool tensor_map_for(sparrow_ctx* c, const void* base, int tag, CUtensorMap* out)
 {
-    for (int i = 0; i < c->n_maps; ++i)
-        if (c->maps[i].base == base && c->maps[i].tag == tag) return &c->maps[i].map;
-    if (!c->encode) return nullptr;
+    // The map is copied out: a later lookup of the same call may evict the slot it came from.
+    size_t h = reinterpret_cast<uintptr_t>(base) >> 8;
+    h = (h ^ (h >> 11) ^ ((size_t)tag * 0x9E3779B1u)) * 0x9E3779B97F4A7C15ull;
+    const int bucket = (int)((h >> 40) % (kMapCacheSize / kMapWays)) * kMapWays;
+    int free_slot = -1;
+    for (int w = 0; w < kMapWays; ++w) {
+        TensorMapEntry& e = c->maps[bucket + w];
+        if (e.base == base && e.tag == tag) { *out = e.map; return true; }
+        if (!e.base && free_slot < 0) free_slot = bucket + w;
+    }
+    if (!c->encode) return false;
     const sparrow_layout& L = c->layout;
-    int slot;
-    if (c->n_maps < kMapCacheSize) slot = c->n_maps++;
-    else { slot = c->next_evict; c->next_evict = (c->next_evict + 1) % kMapCacheSize; }
+    const int slot = free_slot >= 0 ? free_slot : bucket + (int)(c->evict_tick++ % kMapWays);
     const cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r;
     if (tag == 0) {
@@ -340,33 +412,41 @@ const CUtensorMap* tensor_map_for(sparrow_ctx* c, const void* base, int tag)
         const cuuint64_t batch_stride = L.batch > 1 ? (cuuint64_t)L.kv_stride_batch : (cuuint64_t)L.kv_stride_head * L.n_kv_heads;
         const cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)L.kv_stride_head * 2, batch_stride * 2};
         const cuuint32_t box[4] = {64, 128, 1, 1};
-        r = c->encode(&c->maps[slot].map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
+        r = c->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
                       estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     } else {
         const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)kGroup, (cuuint64_t)L.n_kv_heads, (cuuint64_t)tag};
         const cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)kGroup * kD * 2, (cuuint64_t)L.n_q_heads * kD * 2};
         const cuuint32_t box[4] = {64, (cuuint32_t)kGroup, 1, (cuuint32_t)kTokPerBlock};
-        r = c->encode(&c->maps[slot].map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
+        r = c->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
                       estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     }
-    if (r != CUDA_SUCCESS) { c->maps[slot].base = nullptr; if (slot == c->n_maps - 1) --c->n_maps; return nullptr; }
+    if (r != CUDA_SUCCESS) return false;
     c->maps[slot].base = base;
     c->maps[slot].tag = tag;
-    return &c->maps[slot].map;
+    c->maps[slot].map = *out;
+    return true;
+}
+
+void clear_tensor_maps(sparrow_ctx* c)
+{
+    for (int i = 0; i < kMapCacheSize; ++i) c->maps[i].base = nullptr;
+    c->evict_tick = 0;
 }
 
 sparrow_status launch_verify_tc(sparrow_ctx* c, const SplitPlan& plan, const SyncArgs& sy, const void* q, const void* k, const void* v,
-                                const int32_t* parents, void* out, float* lse, cudaStream_t st)
+                                const int32_t* parents, const int32_t* first_visible, void* out, float* lse, cudaStream_t st,
+                                bool may_start_early, bool* started_early)
 {
-    const CUtensorMap* mq = tensor_map_for(c, q, plan.batch * plan.T);
-    const CUtensorMap* mk = tensor_map_for(c, k, 0);
-    const CUtensorMap* mv = tensor_map_for(c, v, 0);
-    if (!mq || !mk || !mv) return SPARROW_ERR_CUDA;
+    CUtensorMap mq, mk, mv;
+    if (!tensor_map_for(c, q, plan.batch * plan.T, &mq) || !tensor_map_for(c, k, 0, &mk) || !tensor_map_for(c, v, 0, &mv))
+        return SPARROW_ERR_CUDA;
     const int nb = plan.blocks_per_group;
     TcArgs a;
     a.parents = parents;
+    a.first_visible = first_visible;
     a.n_q_heads = c->layout.n_q_heads;
     a.scale_log2e = c->layout.softmax_scale * 1.4426950408889634f;
     a.o_part = o_part_ptr(c, sy.parity);
@@ -383,13 +463,18 @@ sparrow_status launch_verify_tc(sparrow_ctx* c, const SplitPlan& plan, const Syn
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    // The early start only reaches back to the kernel launched directly before this one.  The
-    // counters order this context's own calls; if that kernel may belong to another context (whose
-    // writes these counters know nothing about), this launch takes plain stream order instead.
+    // The early start reaches back to the kernel launched directly before this one in the stream,
+    // whatever it is, so it is only taken where that kernel is known: this context's previous
+    // fused call (the counters order this context's own calls and know nothing about another
+    // context's writes), with nothing enqueued in between as far as the library can tell -- the
+    // calls after the first of sparrow_verify_attn_batch(), or any call once the caller has vouched
+    // for the stream with sparrow_set_call_overlap().  Every other launch takes plain stream order.
     const bool same_ctx_before = g_last_fused_ctx.exchange(c) == c;
-    cfg.numAttrs = (sy.enabled && same_ctx_before) ? 1 : 0;
-    const cudaError_t e = nb == 1 ? cudaLaunchKernelEx(&cfg, tc::verify_tc_kernel<1>, a, sy, plan, *mq, *mk, *mv)
-                                  : cudaLaunchKernelEx(&cfg, tc::verify_tc_kernel<2>, a, sy, plan, *mq, *mk, *mv);
+    const bool early = sy.enabled && same_ctx_before && may_start_early;
+    cfg.numAttrs = early ? 1 : 0;
+    if (started_early) *started_early = early;
+    const cudaError_t e = nb == 1 ? cudaLaunchKernelEx(&cfg, tc::verify_tc_kernel<1>, a, sy, plan, mq, mk, mv)
+                                  : cudaLaunchKernelEx(&cfg, tc::verify_tc_kernel<2>, a, sy, plan, mq, mk, mv);
     if (e != cudaSuccess) return SPARROW_ERR_CUDA;
     c->launches.fetch_add(1);
     return SPARROW_OK;
@@ -405,6 +490,16 @@ __global__ void ancestor_masks_kernel(const int32_t* parents, int T, unsigned lo
 __global__ void wait_counter_kernel(const unsigned* counter, unsigned target, unsigned* status)
 {
     if (!wait_counter(counter, target)) atomicOr(status, timeout_bits(kSiteDebug));
+}
+
+// A stand-in for a foreign kernel that lets its dependents launch early and only then produces
+// its output (as many library GEMM / norm kernels do): see sparrow_debug_early_trigger_copy().
+__global__ void early_trigger_copy_kernel(const uint4* src, uint4* dst, size_t n_vec, unsigned delay_us)
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (delay_us > 10000u) delay_us = 10000u;
+    for (unsigned i = 0; i < delay_us; ++i) __nanosleep(1000);
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec; i += (size_t)gridDim.x * blockDim.x) dst[i] = src[i];
 }
 
 struct DeviceGuard {
@@ -425,6 +520,51 @@ sparrow_status check_tree_host(const int32_t* parents, int T)
     for (int i = 0; i < T; ++i)
         if (parents[i] < -1 || parents[i] >= i) return SPARROW_ERR_TREE;
     return SPARROW_OK;
+}
+
+// One verification call: T query tokens, the last T of the T_tree nodes whose K/V rows sit at
+// [kv_len, kv_len + T_tree); optional per-token lower window bound over the prefix keys.
+sparrow_status verify_call(sparrow_ctx* c, const void* q, const void* k, const void* v, const int32_t* kv_len,
+                           const int32_t* parents, int32_t T_tree, int32_t T, const int32_t* first_visible,
+                           const int32_t* first_visible_min, void* out, float* lse, void* stream)
+{
+    if (!c || !q || !k || !v || !kv_len || !parents || !out || !lse) return SPARROW_ERR_NULL;
+    if (T < 1 || T > T_tree || T_tree > kMaxT) return SPARROW_ERR_SHAPE;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return SPARROW_ERR_SHAPE;
+    int32_t n_keys[kMaxBatch], key0[kMaxBatch];
+    for (int b = 0; b < c->layout.batch; ++b) {
+        if (kv_len[b] < 0 || (int64_t)kv_len[b] + T_tree > c->layout.kv_capacity) return SPARROW_ERR_SHAPE;
+        n_keys[b] = kv_len[b] + T_tree;
+        key0[b] = 0;
+        if (first_visible_min) {                 // nothing left of every row's bound is streamed
+            if (first_visible_min[b] < 0 || first_visible_min[b] > kv_len[b]) return SPARROW_ERR_SHAPE;
+            key0[b] = first_visible_min[b] / kKeyTile * kKeyTile;
+        }
+    }
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return SPARROW_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool overlaps = call_overlaps(c, st, true);
+    SplitPlan plan;
+    sparrow_status s = make_plan(plan_target(c, overlaps), c->layout.batch, c->layout.n_kv_heads, n_keys, T,
+                                 blocks_per_group_tc(T), &plan, kMinPieceKeys, key0);
+    if (s != SPARROW_OK) return s;
+    plan.T_tree = T_tree;
+    for (int b = 0; b < c->layout.batch; ++b) plan.seq[b].kv_len = kv_len[b];
+    if ((s = check_ws(c, plan)) != SPARROW_OK) return s;
+    const CallRanges cr = call_ranges(c, q, k, v, parents, T_tree, T, first_visible, out, lse);
+    const SyncArgs sy = next_sync(c, plan, overlaps, outputs_touch_previous(c, cr), true);
+    const bool may_start_early = overlaps && (c->chain_next || c->overlap_single_calls) && !inputs_touch_recent_outputs(c, cr);
+    bool started_early = false;
+    if ((s = launch_verify_tc(c, plan, sy, q, k, v, parents, first_visible, out, lse, st, may_start_early, &started_early)) != SPARROW_OK)
+        return s;
+    advance_sync(c, plan, sy);
+    if (sy.enabled) {
+        std::memcpy(c->prev_ranges, cr.r, sizeof(cr.r));
+        c->prev_valid = true;
+        note_fused_launch(c, cr, started_early);
+    }
+    return SPARROW_OK;                                       // the kernel merges its own partials in either mode
 }
 
 }  // namespace
@@ -480,25 +620,23 @@ sparrow_status sparrow_create(sparrow_ctx** out, const sparrow_layout* L, int de
         return SPARROW_ERR_CUDA;
     sparrow_ctx* c = new (std::nothrow) sparrow_ctx();
     if (!c) return SPARROW_ERR_CUDA;
-    c->n_maps = 0;
-    c->next_evict = 0;
+    clear_tensor_maps(c);
     c->encode = reinterpret_cast<TensorMapEncodeFn>(fn);
-    const char* eg = std::getenv("SPARROW_VERIFY_GATHER");
-    c->verify_on_gather = eg && eg[0] == '1';
     c->layout = *L;
     c->device = device;
     c->n_sm = prop.multiProcessorCount;
     c->plan_policy = SPARROW_PLAN_BALANCED;
-    c->target_override = 0;
-    if (const char* ti = std::getenv("SPARROW_TARGET_ITEMS")) {
-        const int v = std::atoi(ti);
-        if (v >= 1 && v <= c->n_sm) c->target_override = v;
-    }
     c->ws = nullptr;
     c->ws_bytes = 0;
+    c->part_offset = fixed_bytes(*L);
+    c->part_buffers = 2;
     c->launches.store(0);
     const char* e = std::getenv("SPARROW_NO_PDL");
-    c->use_pdl = !(e && e[0] == '1');
+    // more SMs than the list of possibly-resident calls can hold: calls never start early
+    c->use_pdl = !(e && e[0] == '1') && c->n_sm < kRecentCalls;
+    c->overlap_single_calls = false;
+    c->chain_next = false;
+    c->n_recent = c->recent_head = 0;
     c->seq = 0;
     c->fin_total[0] = c->fin_total[1] = 0;
     c->fin_before_last[0] = c->fin_before_last[1] = 0;
@@ -545,6 +683,7 @@ sparrow_status sparrow_set_workspace(sparrow_ctx* c, void* p, size_t bytes)
     c->fin_total[0] = c->fin_total[1] = 0;
     c->fin_before_last[0] = c->fin_before_last[1] = 0;
     c->prev_valid = false;
+    c->n_recent = c->recent_head = 0;
     return SPARROW_OK;
 }
 
@@ -577,35 +716,16 @@ sparrow_status sparrow_verify_attn(sparrow_ctx* c, const void* q, const void* k,
                                    const int32_t* kv_len, const int32_t* parents, int32_t T, void* out,
                                    float* lse, void* stream)
 {
-    if (!c || !q || !k || !v || !kv_len || !parents || !out || !lse) return SPARROW_ERR_NULL;
-    if (T < 1 || T > kMaxT) return SPARROW_ERR_SHAPE;
-    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return SPARROW_ERR_SHAPE;
-    int32_t n_keys[kMaxBatch];
-    for (int b = 0; b < c->layout.batch; ++b) {
-        if (kv_len[b] < 0 || (int64_t)kv_len[b] + T > c->layout.kv_capacity) return SPARROW_ERR_SHAPE;
-        n_keys[b] = kv_len[b] + T;
-    }
-    DeviceGuard guard(c->device);
-    if (!guard.ok) return SPARROW_ERR_CUDA;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const bool overlaps = call_overlaps(c, st, !c->verify_on_gather);
-    SplitPlan plan;
-    const int nb = c->verify_on_gather ? 1 : blocks_per_group_tc(T);
-    sparrow_status s = make_plan(plan_target(c, overlaps), c->layout.batch, c->layout.n_kv_heads, n_keys, T, nb, &plan);
-    if (s != SPARROW_OK) return s;
-    for (int b = 0; b < c->layout.batch; ++b) plan.seq[b].kv_len = kv_len[b];
-    if ((s = check_ws(c, plan)) != SPARROW_OK) return s;
-    const CallRanges cr = call_ranges(c, q, k, v, parents, T, out, lse);
-    const SyncArgs sy = next_sync(c, plan, overlaps, outputs_touch_previous(c, cr));
-    s = c->verify_on_gather ? launch_split_gather(c, plan, sy, q, k, v, parents, nullptr, 0, 0, out, lse, st)
-                            : launch_verify_tc(c, plan, sy, q, k, v, parents, out, lse, st);
-    if (s != SPARROW_OK) return s;
-    advance_sync(c, plan, sy);
-    if (sy.enabled) {
-        std::memcpy(c->prev_ranges, cr.r, sizeof(cr.r));
-        c->prev_valid = true;
-    }
-    return sy.enabled ? SPARROW_OK : launch_combine(c, plan, sy, out, lse, st);    // fused mode combines in the kernel
+    return verify_call(c, q, k, v, kv_len, parents, T, T, nullptr, nullptr, out, lse, stream);
+}
+
+sparrow_status sparrow_verify_attn_window(sparrow_ctx* c, const void* q, const void* k, const void* v,
+                                          const int32_t* kv_len, const int32_t* parents, int32_t T_tree, int32_t T_new,
+                                          const int32_t* first_visible, const int32_t* first_visible_min, void* out,
+                                          float* lse, void* stream)
+{
+    if (T_tree < 1 || T_tree > kMaxT || T_new < 1 || T_new > T_tree) return SPARROW_ERR_SHAPE;
+    return verify_call(c, q, k, v, kv_len, parents, T_tree, T_new, first_visible, first_visible_min, out, lse, stream);
 }
 
 }  // extern "C"  (closed for the file-scope objects of the no-allocation entry point)
@@ -636,7 +756,8 @@ sparrow_status sparrow_verify_attn_static(const sparrow_layout* L, const void* q
                                           const int32_t* kv_len, const int32_t* parents, int32_t T, void* out,
                                           float* lse, void* stream)
 {
-    if (!L) return SPARROW_ERR_NULL;
+    // every argument check comes first: a refused call has not touched the GPU
+    if (!L || !q || !k || !v || !kv_len || !parents || !out || !lse) return SPARROW_ERR_NULL;
     if (L->batch < 1 || L->batch > kMaxBatch || L->head_dim != kD || L->n_kv_heads < 1 ||
         L->n_q_heads != kGroup * L->n_kv_heads || L->kv_capacity < 1 ||
         !(L->softmax_scale > 0.f) || !std::isfinite(L->softmax_scale) ||
@@ -644,6 +765,13 @@ sparrow_status sparrow_verify_attn_static(const sparrow_layout* L, const void* q
         (L->kv_stride_batch % 8) != 0 ||
         (L->batch > 1 && L->kv_stride_batch < L->kv_stride_head * (int64_t)L->n_kv_heads))
         return SPARROW_ERR_SHAPE;
+    if (T < 1 || T > kMaxT) return SPARROW_ERR_SHAPE;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return SPARROW_ERR_SHAPE;
+    int32_t n_keys[kMaxBatch];
+    for (int b = 0; b < L->batch; ++b) {
+        if (kv_len[b] < 0 || (int64_t)kv_len[b] + T > L->kv_capacity) return SPARROW_ERR_SHAPE;
+        n_keys[b] = kv_len[b] + T;
+    }
     int device = -1;
     if (cudaGetDevice(&device) != cudaSuccess) { cudaGetLastError(); return SPARROW_ERR_CUDA; }
     if (device < 0 || device >= kMaxStaticDevices) return SPARROW_ERR_SHAPE;
@@ -669,45 +797,42 @@ sparrow_status sparrow_verify_attn_static(const sparrow_layout* L, const void* q
         void* scratch = nullptr;               // the array's device address on THIS device
         if (cudaGetSymbolAddress(&scratch, g_static_scratch) != cudaSuccess || !scratch) return SPARROW_ERR_CUDA;
         if (cudaMemset(scratch, 0, kStatusBytes) != cudaSuccess) return SPARROW_ERR_CUDA;
-        c->n_maps = 0;
-        c->next_evict = 0;
+        clear_tensor_maps(c);
         c->encode = reinterpret_cast<TensorMapEncodeFn>(fn);
-        c->verify_on_gather = false;
         c->layout = *L;
         c->device = device;
         c->n_sm = prop.multiProcessorCount;
         c->plan_policy = SPARROW_PLAN_LATENCY;
-        c->target_override = 0;
         c->ws = static_cast<unsigned char*>(scratch);
         c->ws_bytes = SPARROW_STATIC_SCRATCH_BYTES;
+        // Stream-ordered calls only: no counters live in the shared array, nothing is double-buffered,
+        // and there is no staging area -- the partials take everything behind the 1 KiB header.
+        c->part_offset = kStatusBytes;
+        c->part_buffers = 1;
         c->launches.store(0);
-        c->use_pdl = false;                    // stream-ordered mode: no counters live in the shared array
+        c->use_pdl = false;
+        c->overlap_single_calls = false;
+        c->chain_next = false;
+        c->n_recent = c->recent_head = 0;
         c->seq = 0;
         c->fin_total[0] = c->fin_total[1] = 0;
-    c->fin_before_last[0] = c->fin_before_last[1] = 0;
-    c->prev_valid = false;
+        c->fin_before_last[0] = c->fin_before_last[1] = 0;
+        c->prev_valid = false;
         c->last_status_word = 0;
         slot.ready = true;
     }
     if (!same_layout(c->layout, *L)) {         // tensor maps depend on the layout
         c->layout = *L;
-        c->n_maps = 0;
-        c->next_evict = 0;
+        clear_tensor_maps(c);
     }
-    if (T >= 1 && T <= kMaxT && kv_len) {      // refuse what does not fit the array before touching the GPU
-        int32_t n_keys[kMaxBatch];
-        bool lens_ok = true;
-        for (int b = 0; b < L->batch; ++b) {
-            lens_ok = lens_ok && kv_len[b] >= 0 && (int64_t)kv_len[b] + T <= L->kv_capacity;
-            n_keys[b] = kv_len[b] + T;
-        }
-        SplitPlan plan;
-        if (lens_ok && make_plan(c->n_sm, L->batch, L->n_kv_heads, n_keys, T, blocks_per_group_tc(T), &plan) == SPARROW_OK &&
-            check_ws(c, plan) != SPARROW_OK)
-            return SPARROW_ERR_WORKSPACE;
-    }
+    // refuse what does not fit the array before anything is enqueued
+    SplitPlan plan;
+    if (make_plan(c->n_sm, L->batch, L->n_kv_heads, n_keys, T, blocks_per_group_tc(T), &plan) != SPARROW_OK) return SPARROW_ERR_SHAPE;
+    if (check_ws(c, plan) != SPARROW_OK) return SPARROW_ERR_WORKSPACE;
     // the status word is the one thing that must start clean
-    if (cudaMemsetAsync(c->ws, 0, sizeof(unsigned), static_cast<cudaStream_t>(stream)) != cudaSuccess) return SPARROW_ERR_CUDA;
+    // the status word must start clean, and so must the two words of the serial merge (an earlier call that gave up
+    // on a wait may have left them behind)
+    if (cudaMemsetAsync(c->ws, 0, 256, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SPARROW_ERR_CUDA;
     return sparrow_verify_attn(c, q, k, v, kv_len, parents, T, out, lse, stream);
 }
 
@@ -717,7 +842,10 @@ sparrow_status sparrow_verify_attn_batch(sparrow_ctx* c, const sparrow_verify_ca
     if (n_calls < 0) return SPARROW_ERR_SHAPE;
     for (int i = 0; i < n_calls; ++i) {
         const sparrow_verify_call& k = calls[i];
+        // from the second call on, the kernel directly before this one in the stream is the previous call's
+        c->chain_next = i > 0;
         const sparrow_status s = sparrow_verify_attn(c, k.q, k.k_cache, k.v_cache, k.kv_len, k.parents, k.T, k.out, k.lse, stream);
+        c->chain_next = false;
         if (s != SPARROW_OK) return s;
     }
     return SPARROW_OK;
@@ -744,7 +872,7 @@ sparrow_status anchor_call(sparrow_ctx* c, const void* q, const void* k, const v
     DeviceGuard guard(c->device);
     if (!guard.ok) return SPARROW_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const SyncArgs sy = next_sync(c, plan, false, true);
+    const SyncArgs sy = next_sync(c, plan, false, true, false);
     // the two kernels of the call are chained programmatically unless the stream is being captured
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
     if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) { cudaGetLastError(); cap = cudaStreamCaptureStatusActive; }
@@ -851,6 +979,42 @@ sparrow_status sparrow_compact_anchors(sparrow_ctx* c, const void* k, const void
     return SPARROW_OK;
 }
 
+sparrow_status sparrow_window_first_visible(const int32_t* anchor_idx, int32_t n_anchor, int32_t window, int32_t T_tree,
+                                            int32_t T_new, int32_t* first_visible, int32_t* first_visible_min)
+{
+    if (!anchor_idx || !first_visible) return SPARROW_ERR_NULL;
+    if (T_tree < 1 || T_tree > kMaxT || T_new < 1 || T_new > T_tree) return SPARROW_ERR_SHAPE;
+    if (n_anchor < T_tree) return SPARROW_ERR_ANCHOR;
+    for (int j = 1; j < n_anchor; ++j)
+        if (anchor_idx[j] <= anchor_idx[j - 1]) return SPARROW_ERR_ANCHOR;
+    const int n_text = n_anchor - T_tree;
+    int32_t lowest = n_text;
+    for (int t = 0; t < T_new; ++t) {
+        int32_t f = 0;
+        if (window > 0) f = first_anchor_above(anchor_idx, n_text, (long long)anchor_idx[n_anchor - T_new + t] - window);
+        first_visible[t] = f;
+        if (f < lowest) lowest = f;
+    }
+    if (first_visible_min) *first_visible_min = lowest;
+    return SPARROW_OK;
+}
+
+sparrow_status sparrow_window_first_visible_device(sparrow_ctx* c, const int32_t* anchor_idx, int32_t n_anchor, int32_t window,
+                                                   int32_t T_tree, int32_t T_new, int32_t* first_visible, void* stream)
+{
+    if (!c || !anchor_idx || !first_visible) return SPARROW_ERR_NULL;
+    if (T_tree < 1 || T_tree > kMaxT || T_new < 1 || T_new > T_tree) return SPARROW_ERR_SHAPE;
+    if (n_anchor < T_tree) return SPARROW_ERR_ANCHOR;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return SPARROW_ERR_CUDA;
+    const int n = c->layout.batch * T_new;
+    window_bounds_kernel<<<(n + 127) / 128, 128, 0, static_cast<cudaStream_t>(stream)>>>(anchor_idx, n_anchor, window, T_tree, T_new,
+                                                                                         c->layout.batch, first_visible);
+    if (cudaGetLastError() != cudaSuccess) return SPARROW_ERR_CUDA;
+    c->launches.fetch_add(1);
+    return SPARROW_OK;
+}
+
 sparrow_status sparrow_accept_greedy(sparrow_ctx* c, const int32_t* draft_tokens, const int32_t* parents,
                                      const int32_t* target_next, int32_t T, int32_t* path_out, int32_t* n_accept_out,
                                      int32_t* bonus_out, void* stream)
@@ -862,6 +1026,24 @@ sparrow_status sparrow_accept_greedy(sparrow_ctx* c, const int32_t* draft_tokens
     if (!guard.ok) return SPARROW_ERR_CUDA;
     accept_greedy_kernel<<<1, kMaxBatch, 0, static_cast<cudaStream_t>(stream)>>>(
         draft_tokens, parents, target_next, c->layout.batch, T, path_out, n_accept_out, bonus_out,
+        reinterpret_cast<unsigned*>(c->ws));
+    if (cudaGetLastError() != cudaSuccess) return SPARROW_ERR_CUDA;
+    c->launches.fetch_add(1);
+    return SPARROW_OK;
+}
+
+sparrow_status sparrow_accept_sample(sparrow_ctx* c, const int32_t* draft_tokens, const int32_t* parents, const float* p_target,
+                                     const float* p_draft, const uint32_t* u_node, const uint32_t* u_bonus, int32_t vocab,
+                                     int32_t T, int32_t* path_out, int32_t* n_accept_out, int32_t* bonus_out, void* stream)
+{
+    if (!c || !draft_tokens || !parents || !p_target || !p_draft || !u_node || !u_bonus || !path_out || !n_accept_out || !bonus_out)
+        return SPARROW_ERR_NULL;
+    if (T < 1 || T > kMaxT || vocab < 1) return SPARROW_ERR_SHAPE;
+    if (!c->ws) return SPARROW_ERR_WORKSPACE;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return SPARROW_ERR_CUDA;
+    sample::accept_sample_kernel<<<c->layout.batch, sample::kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        draft_tokens, parents, p_target, p_draft, u_node, u_bonus, T, vocab, path_out, n_accept_out, bonus_out,
         reinterpret_cast<unsigned*>(c->ws));
     if (cudaGetLastError() != cudaSuccess) return SPARROW_ERR_CUDA;
     c->launches.fetch_add(1);
@@ -1010,6 +1192,20 @@ sparrow_status sparrow_debug_wait_counter(sparrow_ctx* c, uint32_t ahead, void* 
     return SPARROW_OK;
 }
 
+sparrow_status sparrow_debug_early_trigger_copy(sparrow_ctx* c, const void* src, void* dst, size_t bytes,
+                                               uint32_t delay_us, void* stream)
+{
+    if (!c || !src || !dst) return SPARROW_ERR_NULL;
+    if (!aligned16(src) || !aligned16(dst) || (bytes & 15u) != 0) return SPARROW_ERR_SHAPE;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return SPARROW_ERR_CUDA;
+    early_trigger_copy_kernel<<<8, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint4*>(src), static_cast<uint4*>(dst), bytes / 16, delay_us);
+    if (cudaGetLastError() != cudaSuccess) return SPARROW_ERR_CUDA;
+    c->launches.fetch_add(1);
+    return SPARROW_OK;
+}
+
 sparrow_status sparrow_last_device_status(sparrow_ctx* c, void* stream)
 {
     if (!c) return SPARROW_ERR_NULL;
@@ -1022,6 +1218,15 @@ sparrow_status sparrow_last_device_status(sparrow_ctx* c, void* stream)
     if (cudaMemsetAsync(c->ws, 0, sizeof word, st) != cudaSuccess) return SPARROW_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return SPARROW_ERR_CUDA;
     c->last_status_word = word;
+    if (word & kStatTimeout) {
+        // A wait that gave up leaves the ordering counters in an unknown state: start them over.
+        if (cudaMemsetAsync(c->ws, 0, kStatusBytes, st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess) return SPARROW_ERR_CUDA;
+        c->seq = 0;
+        c->fin_total[0] = c->fin_total[1] = 0;
+        c->fin_before_last[0] = c->fin_before_last[1] = 0;
+        c->prev_valid = false;
+        c->n_recent = c->recent_head = 0;
+    }
     if (word & kStatTimeout) return SPARROW_ERR_TIMEOUT;
     if (word & kStatTree) return SPARROW_ERR_TREE;
     if (word & kStatAnchor) return SPARROW_ERR_ANCHOR;
@@ -1034,6 +1239,13 @@ sparrow_status sparrow_set_plan_policy(sparrow_ctx* c, int32_t policy)
     if (policy != SPARROW_PLAN_LATENCY && policy != SPARROW_PLAN_BALANCED && policy != SPARROW_PLAN_THROUGHPUT)
         return SPARROW_ERR_SHAPE;
     c->plan_policy = policy;
+    return SPARROW_OK;
+}
+
+sparrow_status sparrow_set_call_overlap(sparrow_ctx* c, int32_t enable)
+{
+    if (!c) return SPARROW_ERR_NULL;
+    c->overlap_single_calls = enable != 0;
     return SPARROW_OK;
 }
 

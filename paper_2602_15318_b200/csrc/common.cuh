@@ -34,15 +34,17 @@ enum WaitSite { kSiteProducer = 0, kSiteMma = 1, kSiteSoftmax = 2, kSiteWriteSam
 struct SeqPlan {                  // per sequence
     int32_t item_begin;           // first work item of the sequence
     int32_t n_splits;             // key-range pieces per unit
-    int32_t n_keys;               // kv_len + T (verify) or n_anchor (anchored)
+    int32_t n_keys;               // kv_len + draft-tree nodes (verify) or n_anchor (anchored)
     int32_t kv_len;               // verify mode only
+    int32_t key0;                 // first key that is streamed at all (a multiple of the tile; 0 unless a window cuts the prefix)
 };
 // Scalars first and the per-sequence entries as an array of structs: what a CTA reads of the plan
 // then sits in one or two lines of the constant bank the kernel parameters live in.
 struct SplitPlan {
     int32_t n_items;
     int32_t batch;
-    int32_t T;                    // draft tokens
+    int32_t T;                    // query tokens
+    int32_t T_tree;               // nodes of the draft tree = rows of the draft block; the queries are its last T nodes
     int32_t M;                    // query rows per KV head = 7*T
     int32_t blocks_per_group;     // 128-row blocks one work item handles (1 or 2)
     int32_t n_groups;             // ceil(T / (18 * blocks_per_group))
@@ -86,7 +88,9 @@ constexpr int kPartRowHalves = 136;
 struct SyncArgs {
     unsigned* arrivals;      // [4]
     unsigned* fin_done;      // [2]
-    int32_t enabled;
+    unsigned* serial_words;  // [2] serial mode: arrivals of the running call, CTAs that have left it
+    int32_t enabled;         // overlapped mode
+    int32_t serial;          // serial mode: the call runs alone between its neighbours in the stream, and merges its own partials
     int32_t parity;          // n % 2
     int32_t slot;            // n % 4
     int32_t n_arrive;        // items of this call that store partials
@@ -160,7 +164,10 @@ __device__ __forceinline__ Item decode_item(const SplitPlan& p, int item)
     const int unit = local / ns;
     it.group = unit % p.n_groups;
     it.kvh = unit / p.n_groups;
-    piece_range(p.seq[b].n_keys, ns, it.split, p.piece_tile, &it.key_begin, &it.key_end);
+    const int key0 = p.seq[b].key0;
+    piece_range(p.seq[b].n_keys - key0, ns, it.split, p.piece_tile, &it.key_begin, &it.key_end);
+    it.key_begin += key0;
+    it.key_end += key0;
     return it;
 }
 

@@ -112,15 +112,19 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
     // the indices of a tile are fetched one whole tile ahead of its copies.
     constexpr int kAbsent = -2147483647 - 1;                 // key past the end of the piece
     constexpr int kPerThread = (kTile * 16) / kThreads;      // 4
-    auto fetch_rows = [&](int tile, int (&rows)[kPerThread]) {
+    // The thread that owns chunk 0 of a row also fetches the anchor before it: the list must be
+    // strictly increasing (the window rule and the position of the tree nodes rely on it).
+    const bool checks_order = anchored && (tid & 15) == 0;
+    auto fetch_rows = [&](int tile, int (&rows)[kPerThread], int (&before)[kPerThread]) {
         #pragma unroll
         for (int i = 0; i < kPerThread; ++i) {
             const int r = (tid + i * kThreads) >> 4;
             const int j = it.key_begin + tile * kTile + r;
             rows[i] = j < it.key_end ? (anchored ? __ldg(aidx + j) : j) : kAbsent;
+            before[i] = (checks_order && j > 0 && j < it.key_end) ? __ldg(aidx + j - 1) : kAbsent;
         }
     };
-    auto issue_tile = [&](int stage, const int (&rows)[kPerThread]) {
+    auto issue_tile = [&](int stage, const int (&rows)[kPerThread], const int (&before)[kPerThread]) {
         unsigned char* ks = kv_smem + stage * 2 * kStageBytes;
         unsigned char* vs = ks + kStageBytes;
         #pragma unroll
@@ -128,6 +132,7 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
             const int idx = tid + i * kThreads;
             const int r = idx >> 4, c = idx & 15;
             int row = rows[i];
+            if (checks_order && row != kAbsent && before[i] != kAbsent && row <= before[i]) atomicOr(args.status, kStatAnchor);
             if (row == kAbsent) {
                 row = -1;
             } else if (row < 0 || row >= args.kv_capacity) {
@@ -141,14 +146,14 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
             cp_async16(smem_u32(vs + swz(r, c)), vbase + off, bytes);
         }
     };
-    int rows_next[kPerThread];
+    int rows_next[kPerThread], before_next[kPerThread];
 
     // Tile 0 is requested before anything else: its two dependent round trips (anchor indices,
     // then the rows) overlap the loads of the prologue.  It lands in stage 0; the packed Q block is
     // staged in stage 1, which the ring only reuses after Q has moved to registers.
-    if (n_tiles > 0) { fetch_rows(0, rows_next); issue_tile(0, rows_next); }
+    if (n_tiles > 0) { fetch_rows(0, rows_next, before_next); issue_tile(0, rows_next, before_next); }
     cp_async_commit();
-    if (n_tiles > 1) fetch_rows(1, rows_next);
+    if (n_tiles > 1) fetch_rows(1, rows_next, before_next);
 
     // ---- prologue: masks / query positions, packed Q block -> registers --------------------
     const int tree_nodes = anchored ? args.tree_nodes : 0;
@@ -215,9 +220,9 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
 
     for (int tile = 0; tile < n_tiles; ++tile) {
         const int stage = tile & 1;
-        if (tile + 1 < n_tiles) issue_tile(stage ^ 1, rows_next);
+        if (tile + 1 < n_tiles) issue_tile(stage ^ 1, rows_next, before_next);
         cp_async_commit();
-        if (tile + 2 < n_tiles) fetch_rows(tile + 2, rows_next);     // arrives while this tile is being worked on
+        if (tile + 2 < n_tiles) fetch_rows(tile + 2, rows_next, before_next);     // arrives while this tile is being worked on
         cp_async_wait<1>();
         __syncthreads();
         const unsigned char* ks = kv_smem + stage * 2 * kStageBytes;

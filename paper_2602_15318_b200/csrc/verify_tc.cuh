@@ -47,7 +47,8 @@
 namespace sparrow {
 
 struct TcArgs {
-    const int32_t* parents;      // DEV [B][T]
+    const int32_t* parents;      // DEV [B][T_tree]
+    const int32_t* first_visible;   // DEV [B][T] or nullptr: query t sees prefix key j only if j >= first_visible[b][t]
     int32_t n_q_heads;
     float scale_log2e;           // softmax_scale * log2(e)
     __half* o_part;              // [n_items][part_rows] partial rows: 128 fp16 outputs + fp32 LSE (kPartRowHalves)
@@ -58,10 +59,10 @@ struct TcArgs {
 
 namespace tc {
 
-constexpr int kThreads = 320;                    // 8 softmax warps, producer, MMA issuer
-// Declared thread bound: caps the kernel at 65536 / 512 = 128 registers per thread.
-constexpr int kBoundThreads = 512;
-constexpr int kProducerWarp = 8, kMmaWarp = 9;
+constexpr int kThreads = 352;                    // 8 softmax warps, producer, MMA issuer, gatekeeper
+// Declared thread bound: caps the kernel at 65536 / 384 = 170 registers per thread.
+constexpr int kBoundThreads = 384;
+constexpr int kProducerWarp = 8, kMmaWarp = 9, kGateWarp = 10;
 constexpr int kTile = 128;                       // keys per stage and per job
 constexpr int kSubTileBytes = 128 * 64 * 2;      // one 128 x 64 bf16 box: 16 KB
 constexpr int kQBlockBytes = 2 * kSubTileBytes;  // 128 rows x 128 dims: 32 KB
@@ -73,7 +74,8 @@ constexpr float kRescaleLog2 = 8.0f;             // lazy-max threshold in log2 u
 
 __host__ __device__ constexpr int smem_bytes(int n_blocks, int n_stages)
 {
-    return 1024 /*alignment slack*/ + n_blocks * kQBlockBytes + n_stages * kStageBytes + kMiscBytes;
+    // two row blocks: 1 KB more for the per-row results the two warpgroups hand each other
+    return 1024 /*alignment slack*/ + n_blocks * kQBlockBytes + n_stages * kStageBytes + kMiscBytes + (n_blocks == 2 ? 1024 : 0);
 }
 // S blocks (score tiles in flight) for a given number of row blocks; TMEM: S blocks first, then
 // one 128-column O accumulator per row block, 512 columns in all.
@@ -145,6 +147,9 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// Orders generic-proxy accesses to global memory that this thread has observed before its later
+// async-proxy (bulk copy) accesses to it.
+__device__ __forceinline__ void fence_proxy_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar)
@@ -153,6 +158,8 @@ __device__ __forceinline__ void tc_commit(uint32_t bar)
 }
 // barrier among the 256 softmax threads only (id 1; id 0 is __syncthreads)
 __device__ __forceinline__ void softmax_bar_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+// barrier among the 128 threads of one softmax warpgroup (ids 3 and 4)
+__device__ __forceinline__ void warpgroup_bar_sync(int wg) { asm volatile("bar.sync %0, 128;" ::"r"(3 + wg) : "memory"); }
 // D[tmem] (+)= A[smem] * B[smem]
 __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
 {
@@ -254,10 +261,10 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
     d |= (uint64_t)2 << 61;          // SWIZZLE_128B
     return d;
 }
-// Instruction descriptor, kind::f16: D fp32, A/B bf16, A K-major, M = 128, N = 128.
-__host__ __device__ constexpr uint32_t idesc_bf16(bool b_mn_major)
+// Instruction descriptor, kind::f16: D fp32, A/B bf16, A K-major, M = 128, N = n (128 or 64).
+__host__ __device__ constexpr uint32_t idesc_bf16(bool b_mn_major, uint32_t n = 128u)
 {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((n >> 3) << 17) | ((128u >> 4) << 24);
 }
 
 // ---- softmax helpers on a 32-column chunk of one score row ---------------------------------------
@@ -317,8 +324,9 @@ struct Bars {
     __device__ __forceinline__ uint32_t k_empty(int i) const { return base + 24u + 8u * (uint32_t)i; }
     __device__ __forceinline__ uint32_t v_full(int i) const { return base + 48u + 8u * (uint32_t)i; }
     __device__ __forceinline__ uint32_t v_empty(int i) const { return base + 72u + 8u * (uint32_t)i; }
-    __device__ __forceinline__ uint32_t s_full(int i) const { return base + 96u + 8u * (uint32_t)i; }
-    __device__ __forceinline__ uint32_t p_full(int i) const { return base + 120u + 8u * (uint32_t)i; }
+    // (a fourth score / P slot, used with two row blocks, sits behind the other barriers)
+    __device__ __forceinline__ uint32_t s_full(int i) const { return i < 3 ? base + 96u + 8u * (uint32_t)i : base + 240u; }
+    __device__ __forceinline__ uint32_t p_full(int i) const { return i < 3 ? base + 120u + 8u * (uint32_t)i : base + 248u; }
     __device__ __forceinline__ uint32_t q_full() const { return base + 144u; }
     __device__ __forceinline__ uint32_t fin() const { return base + 152u; }       // finishers' bulk copies
     // Completion of O += P V of key tile j on row block blk: a ring of four barriers per block,
@@ -353,7 +361,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
     volatile uint32_t* write_ok = reinterpret_cast<volatile uint32_t*>(misc + 232);   // the counters allow global writes
     volatile int32_t* fin_go = reinterpret_cast<volatile int32_t*>(misc + 236);       // finishers: their waits succeeded
     unsigned long long* anc_s = reinterpret_cast<unsigned long long*>(misc + 256);   // [64]
-    int32_t* par_s = reinterpret_cast<int32_t*>(misc + 768);                          // [64], prologue only
+    int32_t* par_s = reinterpret_cast<int32_t*>(misc + 768);                          // [64]: parents in the prologue, then the rows' first visible keys
     float* xch = reinterpret_cast<float*>(misc + 1024);                               // [2][128] maxima / sums exchange
 
     Bars B;
@@ -391,14 +399,14 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_q) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_k) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_v) : "memory");
-        for (int i = 0; i < 3; ++i) {
-            mbar_init(B.k_full(i), 1); mbar_init(B.k_empty(i), 1); mbar_init(B.v_full(i), 1); mbar_init(B.v_empty(i), 1);
-            mbar_init(B.s_full(i), 1); mbar_init(B.p_full(i), 256);
-        }
+        for (int i = 0; i < 3; ++i) { mbar_init(B.k_full(i), 1); mbar_init(B.k_empty(i), 1); mbar_init(B.v_full(i), 1); mbar_init(B.v_empty(i), 1); }
+        // one row block: a P block comes from all 256 softmax threads; two: from the block's own warpgroup
+        for (int i = 0; i < 4; ++i) { mbar_init(B.s_full(i), 1); mbar_init(B.p_full(i), NB == 1 ? 256 : 128); }
         for (int i = 0; i < 4; ++i) { mbar_init(B.o_done(0, i), 1); mbar_init(B.o_done(1, i), 1); }
         mbar_init(B.q_full(), 1);
         mbar_init(B.fin(), 1);
         *abort_flag = 0;
+        *write_ok = sync.enabled ? 0u : 1u;
         fence_barrier_init();
         // Q first (the first S = Q K^T needs it and it is small), then K and V tiles in the order
         // they are consumed.  Nothing here depends on the previous kernel in the stream.
@@ -416,12 +424,27 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    if (warp == 0 && it.key_end > kv_len) {          // this piece reaches the draft block: it needs the tree
-        const int32_t* par_g = args.parents + (size_t)it.b * T;
-        if (lane < T) par_s[lane] = __ldg(par_g + lane);
-        if (lane + 32 < T) par_s[lane + 32] = __ldg(par_g + lane + 32);
-        __syncwarp();
-        for (int i = lane; i < T; i += 32) anc_s[i] = ancestor_word(par_s, T, i, args.status);
+    if (warp == 0) {
+        const int Tt = plan.T_tree;
+        if (it.key_end > kv_len) {                   // this piece reaches the draft block: it needs the tree
+            const int32_t* par_g = args.parents + (size_t)it.b * Tt;
+            if (lane < Tt) par_s[lane] = __ldg(par_g + lane);
+            if (lane + 32 < Tt) par_s[lane + 32] = __ldg(par_g + lane + 32);
+            __syncwarp();
+            for (int i = lane; i < Tt; i += 32) anc_s[i] = ancestor_word(par_s, Tt, i, args.status);
+            __syncwarp();
+        }
+        // Lower window bound of every query token, clamped to what this call streams: a bound
+        // left of the first streamed key cannot be honoured (the keys in between were not planned)
+        // and is reported.
+        for (int t = lane; t < T; t += 32) {
+            int lo = args.first_visible ? __ldg(args.first_visible + (size_t)it.b * T + t) : 0;
+            if (lo < plan.seq[it.b].key0) {
+                if (args.first_visible) atomicOr(args.status, kStatAnchor);
+                lo = plan.seq[it.b].key0;
+            }
+            par_s[t] = lo < kv_len ? lo : kv_len;
+        }
     }
     tc_fence_before();
     __syncthreads();
@@ -447,13 +470,58 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
     } else if (warp == kMmaWarp) {
         // ================= MMA issuer =================
         if (lane == 0) {
-            constexpr uint32_t idesc_qk = idesc_bf16(false);
-            constexpr uint32_t idesc_pv = idesc_bf16(true);
             // descriptors differ from job to job only in their 14-bit address field
             const uint64_t q_desc0 = smem_desc(smem_u32(q_sm), 16, 1024);
             const uint64_t k_desc0 = smem_desc(smem_u32(kv_sm), 16, 1024);
             const uint64_t v_desc0 = smem_desc(smem_u32(kv_sm) + 2 * kSubTileBytes, kSubTileBytes, 1024);
             bool ok = mbar_wait(B.q_full(), 0);
+            if constexpr (NB == 2) {
+                // Two row blocks, each with its own softmax warpgroup.  A job is HALF a key tile
+                // (64 keys) against one row block: job n = (half-tile h = n / 2, block b = n % 2),
+                // key tile j = h / 2.  Block b owns TMEM columns [128 b, 128 b + 128): two score
+                // slots of 64 fp32 columns (slot h % 2), the P of a slot (bf16, 32 columns) written
+                // over the slot's upper half; the accumulators follow at 256 + 128 b.  Four slots in
+                // all keep the scores two half-tiles ahead of each warpgroup, so the tensor pipe
+                // has S = Q K^T work queued while it waits for a P.
+                constexpr uint32_t idesc_qk64 = idesc_bf16(false, 64);
+                constexpr uint32_t idesc_pv = idesc_bf16(true);
+                const int n_half_jobs = 4 * n_tiles;
+                auto issue_qk64 = [&](int m) -> bool {
+                    const int h = m >> 1, b = m & 1, hh = h & 1, j = h >> 1, st = j % NS;
+                    if (b == 0 && hh == 0) {                                  // first use of this K tile
+                        if (!mbar_wait(B.k_full(st), (j / NS) & 1)) return false;
+                        tc_fence_after();
+                    }
+                    const uint64_t qd = q_desc0 + (uint64_t)((b * kQBlockBytes) >> 4);
+                    const uint64_t kd = k_desc0 + (uint64_t)((st * kStageBytes + hh * 64 * 128) >> 4);   // keys [64 hh, 64 hh + 64) of the tile
+                    #pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint32_t off = ((ks >> 2) * kSubTileBytes + (ks & 3) * 32) >> 4;
+                        mma_ss(tmem + b * 128 + hh * 64, qd + off, kd + off, idesc_qk64, ks > 0);
+                    }
+                    tc_commit(B.s_full(2 * b + hh));
+                    if (b == 1 && hh == 1) tc_commit(B.k_empty(st));          // last use of the tile
+                    return true;
+                };
+                for (int m = 0; m < 4 && m < n_half_jobs && ok; ++m) ok = issue_qk64(m);
+                #pragma unroll 1
+                for (int n = 0; n < n_half_jobs && ok; ++n) {
+                    const int h = n >> 1, b = n & 1, hh = h & 1, j = h >> 1, st = j % NS;
+                    if (b == 0 && hh == 0 && !mbar_wait(B.v_full(st), (j / NS) & 1)) { ok = false; break; }
+                    if (!mbar_wait(B.p_full(2 * b + hh), j & 1)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint64_t vd = v_desc0 + (uint64_t)((st * kStageBytes) >> 4);
+                    #pragma unroll
+                    for (int i = 0; i < 4; ++i)                               // keys [64 hh + 16 i, + 16) of the tile
+                        mma_ts(tmem + 256 + b * 128, tmem + b * 128 + hh * 64 + 32 + i * 8,
+                               vd + (uint64_t)(((4 * hh + i) * 2048) >> 4), idesc_pv, (h > 0 || i > 0) ? 1u : 0u);
+                    tc_commit(B.o_done(b, h));
+                    if (b == 1 && hh == 1) tc_commit(B.v_empty(st));
+                    if (n + 4 < n_half_jobs) ok = issue_qk64(n + 4);          // the slot this job's scores were in
+                }
+            } else {
+            constexpr uint32_t idesc_qk = idesc_bf16(false);
+            constexpr uint32_t idesc_pv = idesc_bf16(true);
             // S = Q K^T of job m into S block m % NSB
             auto issue_qk = [&](int m) -> bool {
                 const int j = m / NB, blk = m % NB, sb = m % NSB, st = j % NS;
@@ -488,7 +556,23 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                 if (blk == NB - 1) tc_commit(B.v_empty(st));
                 if (n + NSB < n_jobs) ok = issue_qk(n + NSB);             // its S block was job n's
             }
+            }
             if (!ok) { atomicOr(args.status, timeout_bits(kSiteMma)); *abort_flag = 1; }
+        }
+    } else if (warp == kGateWarp) {
+        if (lane == 0 && sync.enabled) {
+            // Overlapped mode: whoever read this parity's partial buffer two calls ago must be done
+            // before this CTA's first global write, and final results may only follow every earlier
+            // call's.  Waiting here, beside the main loop, keeps the round trip to the counters off the
+            // epilogue's critical path.  1 = go, 2 = a wait gave up.
+            bool go = wait_counter(sync.fin_done + sync.parity, sync.fin_wait_same);
+            if (!go) atomicOr(args.status, timeout_bits(kSiteWriteSame));
+            if (go && plan.seq[it.b].n_splits == 1) {
+                go = wait_counter(sync.fin_done + (sync.parity ^ 1), sync.fin_wait_other);
+                if (!go) atomicOr(args.status, timeout_bits(kSiteWriteOther));
+            }
+            __threadfence_block();
+            *write_ok = go ? 1u : 2u;
         }
     } else if (warp < 8) {
         // ================= softmax =================
@@ -498,7 +582,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
         const float c2 = args.scale_log2e;
         const float thr = kRescaleLog2 / c2;             // threshold in raw score units
         const int g_row = row_local % kGroup;
-        int t_row[NB];
+        int t_row[NB], lo_row[NB];
         bool row_ok[NB];
         unsigned long long anc[NB];
         float m_ref[NB], l_run[NB];
@@ -506,11 +590,102 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
         for (int blk = 0; blk < NB; ++blk) {
             t_row[blk] = (block0 + blk) * kTokPerBlock + row_local / kGroup;
             row_ok[blk] = row_local < kTokPerBlock * kGroup && t_row[blk] < T;
-            anc[blk] = (row_ok[blk] && it.key_end > kv_len) ? anc_s[t_row[blk]] : 0ull;
+            // the queries are the last T nodes of the tree
+            anc[blk] = (row_ok[blk] && it.key_end > kv_len) ? anc_s[plan.T_tree - T + t_row[blk]] : 0ull;
+            lo_row[blk] = row_ok[blk] ? par_s[t_row[blk]] : 0;
             m_ref[blk] = -INFINITY; l_run[blk] = 0.f;
         }
         bool ok = true;
 
+        float my_m = -INFINITY, my_l = 0.f;       // two row blocks: the state of this warpgroup's own block
+        if constexpr (NB == 2) {
+            // ---- two row blocks: warpgroup g owns block g, one thread per query row, and works
+            // through the block's half-tile jobs on its own -- no exchange with the other warpgroup,
+            // whose exponentials fill the gaps this one leaves while it waits for the tensor pipe.
+            const int blk = wg;
+            const int n_half = 2 * n_tiles;
+            // this warpgroup's block, in scalars (indexing the per-block arrays with wg would put them in local memory)
+            const unsigned long long my_anc = wg ? anc[NB - 1] : anc[0];
+            const int my_lo = wg ? lo_row[NB - 1] : lo_row[0];
+            const bool my_ok = wg ? row_ok[NB - 1] : row_ok[0];
+            float x0[32], x1[32];
+            #pragma unroll 1
+            for (int h = 0; h < n_half && ok; ++h) {
+                const int hh = h & 1, j = h >> 1, st = j % NS;
+                const int tile0 = it.key_begin + j * kTile;
+                const int j0 = tile0 + 64 * hh;                      // first key of this half-tile
+                const uint32_t s_addr = lane_addr + blk * 128 + hh * 64;
+                if (!mbar_wait_warp(B.s_full(2 * blk + hh), j & 1)) { ok = false; break; }
+                tc_fence_after();
+                tmem_ld32(s_addr, x0);
+                tmem_ld32(s_addr + 32, x1);
+                const bool boundary = j0 + 64 > it.key_end || j0 + 64 > kv_len || j0 < my_lo;
+                unsigned long long vis = ~0ull;
+                if (boundary) {
+                    const int d0 = kv_len - j0;                             // column of draft token 0 (any sign)
+                    const int nval = it.key_end - j0;                       // valid columns (may be <= 0)
+                    if (d0 >= 64) vis = ~0ull;
+                    else if (d0 > 0) vis = ((1ull << d0) - 1ull) | (my_anc << d0);
+                    else if (d0 > -64) vis = my_anc >> (-d0);
+                    else vis = 0ull;
+                    if (nval <= 0) vis = 0ull;
+                    else if (nval < 64) vis &= (1ull << nval) - 1ull;
+                    const int cut = my_lo - j0;
+                    if (cut >= 64) vis = 0ull;
+                    else if (cut > 0) vis &= ~((1ull << cut) - 1ull);
+                }
+                // V rows past the end of the sequence may hold anything: zero them so 0 * x stays 0
+                // (once per tile, by the threads of the first block, thread r taking key row r)
+                if (blk == 0 && hh == 0 && tile0 + kTile > n_keys_seq && tile0 + row_local >= n_keys_seq) {
+                    mbar_wait(B.v_full(st), (j / NS) & 1);
+                    unsigned char* vrow = kv_sm + st * kStageBytes + 2 * kSubTileBytes + row_local * 128;
+                    #pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        *reinterpret_cast<uint4*>(vrow + c * 16) = make_uint4(0, 0, 0, 0);
+                        *reinterpret_cast<uint4*>(vrow + kSubTileBytes + c * 16) = make_uint4(0, 0, 0, 0);
+                    }
+                    fence_proxy_async();
+                }
+                tmem_wait_ld();
+                if (boundary) { mask_chunk(x0, (uint32_t)vis); mask_chunk(x1, (uint32_t)(vis >> 32)); }
+                const float mx = fmaxf(chunk_max(x0), chunk_max(x1));
+                // lazy reference maximum, per row; the accumulator is rescaled by the whole warp (the
+                // TMEM accesses are warp-wide) whenever one of its rows moved
+                const bool need = my_ok && (mx > my_m + thr || (my_m == -INFINITY && mx > -INFINITY));
+                if (__any_sync(0xffffffffu, need)) {
+                    float alpha = 1.f;
+                    if (need) {
+                        alpha = (my_m == -INFINITY) ? 0.f : ex2((my_m - mx) * c2);
+                        my_m = mx;
+                        my_l *= alpha;
+                    }
+                    if (h > 0) {                                            // O holds earlier half-tiles
+                        if (!mbar_wait_warp(B.o_done(blk, h - 1), ((h - 1) >> 2) & 1)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t o_addr = lane_addr + kOCol + blk * 128;
+                        #pragma unroll 1
+                        for (int ch = 0; ch < 4; ++ch) {
+                            float o[32];
+                            tmem_ld32(o_addr + ch * 32, o);
+                            tmem_wait_ld();
+                            #pragma unroll
+                            for (int c = 0; c < 32; ++c) o[c] *= alpha;
+                            tmem_st32(o_addr + ch * 32, reinterpret_cast<uint32_t*>(o));
+                        }
+                        tmem_wait_st();
+                    }
+                }
+                // p = 2^(s c2 - m c2), row sum from the unrounded p, P (bf16) over the slot's upper half
+                const float mc = (my_m == -INFINITY) ? 0.f : my_m * c2;
+                float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+                exp_chunk(x0, c2, mc, sum4, s_addr + 32);
+                exp_chunk(x1, c2, mc, sum4, s_addr + 48);
+                my_l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+                tmem_wait_st();                                            // this job's P is in TMEM
+                tc_fence_before();
+                mbar_arrive(B.p_full(2 * blk + hh));
+            }
+        } else {
         // The scores of a job are requested from TMEM at the end of the job before it, ahead of the
         // wait for that job's P stores, so the two latencies overlap; whether those scores are there
         // is probed before the exponentials and only waited for if the probe said no.
@@ -531,7 +706,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                 const int n = j * NB + blk, sb = n % NSB;
                 // Visibility word of this row for the thread's 64 columns (all ones away from the
                 // draft block and the end of the key range).
-                const bool boundary = j0 + 64 > it.key_end || j0 + 64 > kv_len;
+                const bool boundary = j0 + 64 > it.key_end || j0 + 64 > kv_len || j0 < lo_row[blk];
                 unsigned long long vis = ~0ull;
                 if (boundary) {
                     // prefix columns, then the ancestor word shifted to the draft block's column, cut
@@ -544,6 +719,11 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                     else vis = 0ull;
                     if (nval <= 0) vis = 0ull;
                     else if (nval < 64) vis &= (1ull << nval) - 1ull;
+                    // prefix keys left of the row's window (the bound never exceeds kv_len, so
+                    // the draft block's columns are not touched)
+                    const int cut = lo_row[blk] - j0;
+                    if (cut >= 64) vis = 0ull;
+                    else if (cut > 0) vis &= ~((1ull << cut) - 1ull);
                 }
                 // V rows past the end of the sequence may hold anything: zero them so 0 * x stays 0
                 // (once per tile, by the threads of the first half, thread r taking key row r).
@@ -626,35 +806,44 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
             }
         }
 
+        }
         // ---- epilogue: normalised partial output + natural-log LSE -------------------------------
         const bool direct = plan.seq[it.b].n_splits == 1;                  // the only piece: write the final result
         if (tid == 0) {
-            // global writes start below: whoever read this parity's partial buffer two calls ago must
-            // be done, and final results may only follow every earlier call's
-            bool go = true;
-            if (sync.enabled) {
-                go = wait_counter(sync.fin_done + sync.parity, sync.fin_wait_same);
-                if (!go) atomicOr(args.status, timeout_bits(kSiteWriteSame));
-                if (go && direct) {
-                    go = wait_counter(sync.fin_done + (sync.parity ^ 1), sync.fin_wait_other);
-                    if (!go) atomicOr(args.status, timeout_bits(kSiteWriteOther));
-                }
-                if (go && blockIdx.x == 0) sync.arrivals[(sync.slot + 2) & 3] = 0u;   // the call after next: unused by now
-            }
-            *write_ok = go ? 1u : 0u;
+            // Global writes start below.  In overlapped mode a lane of the MMA warp has been waiting,
+            // since the kernel started, for the counters that allow them (see there).
+            uint32_t w = *write_ok;
+            for (uint32_t i = 0; w == 0u && i < (1u << 26); ++i) { __nanosleep(20); w = *write_ok; }
+            __threadfence_block();
+            if (w == 1u && sync.enabled && blockIdx.x == 0) sync.arrivals[(sync.slot + 2) & 3] = 0u;   // the call after next: unused by now
+            *write_ok = w == 1u ? 1u : 2u;
+        }
+        float* xch2 = reinterpret_cast<float*>(misc + kMiscBytes);         // [2][128], two row blocks only
+        if constexpr (NB == 2) {
+            // each warpgroup hands over its block's per-row results: both warpgroups store both blocks
+            xch[wg * 128 + row_local] = my_l > 0.f ? 1.f / my_l : 0.f;
+            xch2[wg * 128 + row_local] = my_l > 0.f ? (my_m * c2 + log2f(my_l)) * 0.6931471805599453f : -INFINITY;
+            softmax_bar_sync();
         }
         #pragma unroll
         for (int blk = 0; blk < NB; ++blk) {
-            if (ok) ok = mbar_wait_warp(B.o_done(blk, n_tiles - 1), ((n_tiles - 1) >> 2) & 1);    // the last product is in
+            const int last_product = NB == 2 ? 2 * n_tiles - 1 : n_tiles - 1;
+            if (ok) ok = mbar_wait_warp(B.o_done(blk, last_product), (last_product >> 2) & 1);    // the last product is in
             tc_fence_after();
-            // the two halves' sums meet (the maxima are already the same)
-            xch[wg * 128 + row_local] = l_run[blk];
-            softmax_bar_sync();
-            const float l_all = l_run[blk] + xch[(wg ^ 1) * 128 + row_local];
-            softmax_bar_sync();                                        // xch is reused by the next block
-            ok = ok && *write_ok != 0;                                 // (thread 0 wrote it before the barriers above)
-            const float inv = l_all > 0.f ? 1.f / l_all : 0.f;
-            const float lse_val = l_all > 0.f ? (m_ref[blk] * c2 + log2f(l_all)) * 0.6931471805599453f : -INFINITY;
+            float inv, lse_val;
+            if constexpr (NB == 2) {
+                inv = xch[blk * 128 + row_local];
+                lse_val = xch2[blk * 128 + row_local];
+            } else {
+                // the two halves' sums meet (the maxima are already the same)
+                xch[wg * 128 + row_local] = l_run[blk];
+                softmax_bar_sync();
+                const float l_all = l_run[blk] + xch[(wg ^ 1) * 128 + row_local];
+                softmax_bar_sync();                                    // xch is reused by the next block
+                inv = l_all > 0.f ? 1.f / l_all : 0.f;
+                lse_val = l_all > 0.f ? (m_ref[blk] * c2 + log2f(l_all)) * 0.6931471805599453f : -INFINITY;
+            }
+            ok = ok && *write_ok == 1u;                                // (thread 0 settled it before the barriers above)
             const int h_row = it.kvh * kGroup + g_row;
             // Staging area for coalesced stores: the Q block (every MMA has completed by now).  Row r
             // holds 16 chunks of 16 bytes (128 halves), chunk c stored at position c ^ (r & 15).
@@ -707,62 +896,79 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
             }
         }
 
-        // ---- fused mode: publish this item; the grid's last CTAs merge the call's partials -----------
-        if (sync.enabled) {
+        // ---- publish this item; the call's finisher CTAs merge its partials ---------------------------
+        // Overlapped mode (sync.enabled): arrival words and finisher counters as described at SyncArgs.
+        // Serial mode (sync.serial; the call runs alone between its neighbours in the stream): one
+        // arrival word and one exit word that start at zero; the CTA that exits last puts both back.
+        if (sync.enabled || sync.serial) {
             const int fin_idx = (int)blockIdx.x - (plan.n_items - sync.n_fin);     // >= 0: this CTA is a finisher
+            constexpr int kRowsPerBlock = kTokPerBlock * kGroup;       // 126
+            constexpr int kRowBytes = kPartRowHalves * 2;              // 272
+            // The call's row list: for every unit (sequence, KV head, row group) with several pieces,
+            // its valid query rows (7 per draft token).  Finisher f takes rows [f chunk, (f + 1) chunk).
+            int total = 0;
+            for (int b = 0; b < plan.batch; ++b)
+                if (plan.seq[b].n_splits > 1) total += plan.n_kv_heads * kGroup * T;
+            const int chunk = sync.n_fin > 0 ? (total + sync.n_fin - 1) / sync.n_fin : 0;
+            const int my_begin = fin_idx >= 0 ? min(total, fin_idx * chunk) : 0;
+            const int my_end = fin_idx >= 0 ? min(total, my_begin + chunk) : 0;
+            const bool merges = my_begin < my_end;
+            unsigned* arrive_word = sync.enabled ? sync.arrivals + sync.slot : sync.serial_words;
             softmax_bar_sync();                                        // every global store of this CTA has been issued
             if (tid == 0) {
-                if (!direct) publish_counter(sync.arrivals + sync.slot);
-                if (fin_idx >= 0) {
-                    // every partial of the call in place, and the previous call's final results written
-                    bool go = wait_equal(sync.arrivals + sync.slot, (unsigned)sync.n_arrive);
+                if (!direct) publish_counter(arrive_word);
+                if (merges) {
+                    // every partial of the call in place, and (overlapped mode) the previous call's final results written
+                    bool go = wait_equal(arrive_word, (unsigned)sync.n_arrive);
                     if (!go) atomicOr(args.status, timeout_bits(kSiteArrivals));
-                    if (go) {
+                    if (go && sync.enabled) {
                         go = wait_counter(sync.fin_done + (sync.parity ^ 1), sync.fin_wait_other);
                         if (!go) atomicOr(args.status, timeout_bits(kSiteFinOther));
                     }
                     *fin_go = go ? 1 : 0;
                 }
             }
-            if (fin_idx >= 0) {
+            if (merges) {
                 softmax_bar_sync();
                 if (*fin_go) {
-                    // The call's row list: for every unit with several pieces, its (block, r) rows,
-                    // r < 126.  This finisher takes a contiguous chunk of the list.  Per unit, the
-                    // pieces' rows are copied into the (idle) K/V ring in bulk -- per piece one copy per
-                    // block touched, one memory round trip for a whole batch -- and merged from
-                    // there, one warp per row, lane l owning output dims [4 l, 4 l + 4).
-                    constexpr int kRowsPerBlock = kTokPerBlock * kGroup;       // 126
-                    constexpr int kRowBytes = kPartRowHalves * 2;              // 272
-                    constexpr int kBatchRowsMax = 64;                          // rows merged at once
-                    const int list_len = NB * kRowsPerBlock;                   // rows per unit
-                    int n_units = 0;
-                    for (int b = 0; b < plan.batch; ++b)
-                        if (plan.seq[b].n_splits > 1) n_units += plan.n_kv_heads * plan.n_groups;
-                    const int total = n_units * list_len;
-                    const int chunk = (total + sync.n_fin - 1) / sync.n_fin;
-                    const int my_begin = fin_idx * chunk, my_end = min(total, my_begin + chunk);
+                    // Per unit, the pieces' rows are copied into the (idle) K/V ring in bulk -- per piece
+                    // one copy per block touched, one memory round trip for a whole batch of R rows --
+                    // and merged from there by 16 R G threads: thread (row i, 16-byte chunk c, piece
+                    // group g) takes pieces g, g + G, ...; the groups' partial maxima, sums and weighted
+                    // outputs meet in shared memory (the Q blocks, idle by now).
+                    float* red = reinterpret_cast<float*>(q_sm);                // [256][9] partial sums, then [256] maxima
+                    float* red_max = red + 256 * 9;
                     bool fin_ok = true;
                     int phase = 0, ubase = 0;
                     #pragma unroll 1
                     for (int b = 0; b < plan.batch; ++b) {
                         const int ns = plan.seq[b].n_splits;
                         if (ns == 1) continue;
-                        int batch_rows = (NS * kStageBytes) / (ns * kRowBytes);    // rows whose pieces fit the ring at once
-                        if (batch_rows > kBatchRowsMax) batch_rows = kBatchRowsMax;
+                        // rows per batch: a power of two, no more than this finisher has, than fit the ring
+                        // with all their pieces, or than 16
+                        int R = 1;
+                        while (R < 16 && R < chunk) R <<= 1;
+                        while (R > 1 && R * ns * kRowBytes > NS * kStageBytes) R >>= 1;
+                        const int G = 16 / R;                                   // piece groups
+                        const int c16 = tid & 15, grp_p = (tid >> 4) % G, row_i = tid / (16 * G);
                         #pragma unroll 1
-                        for (int u = 0; u < plan.n_kv_heads * plan.n_groups; ++u, ubase += list_len) {
-                            const int row_begin = max(my_begin, ubase) - ubase, row_end = min(my_end, ubase + list_len) - ubase;
-                            if (row_begin >= row_end) continue;                    // (the same in every thread of the CTA)
+                        for (int u = 0; u < plan.n_kv_heads * plan.n_groups; ++u) {
                             const int kvh = u / plan.n_groups, grp = u - kvh * plan.n_groups;
+                            const int tok0 = grp * NB * kTokPerBlock;                        // first token of this row group
+                            const int list_len = kGroup * min(NB * kTokPerBlock, T - tok0);  // its valid rows
+                            const int row_begin = max(my_begin, ubase) - ubase, row_end = min(my_end, ubase + list_len) - ubase;
+                            ubase += list_len;
+                            if (row_begin >= row_end) continue;                    // (the same in every thread of the CTA)
                             const size_t item0 = (size_t)plan.seq[b].item_begin + (size_t)u * ns;
                             #pragma unroll 1
-                            for (int r0 = row_begin; r0 < row_end; r0 += batch_rows, phase ^= 1) {
-                                const int n_here = min(batch_rows, row_end - r0);
+                            for (int r0 = row_begin; r0 < row_end; r0 += R, phase ^= 1) {
+                                const int n_here = min(R, row_end - r0);
                                 // the batch may straddle the two blocks: rows [r0, split) and [split, r0 + n_here)
                                 const int split = (r0 < kRowsPerBlock && r0 + n_here > kRowsPerBlock) ? kRowsPerBlock : r0 + n_here;
                                 if (tid == 0) mbar_expect_tx(B.fin(), (uint32_t)(n_here * ns * kRowBytes));
                                 softmax_bar_sync();                                // previous batch consumed, byte count posted
+                                // the partial rows were written with ordinary stores; the bulk copies read them through the async proxy
+                                if (tid < ns) fence_proxy_async_global();
                                 for (int sp = tid; sp < ns; sp += 256) {           // shared memory: [piece][row of the batch][272 bytes]
                                     const __half* piece = args.o_part + (item0 + sp) * plan.part_rows * kPartRowHalves;
                                     const uint32_t dst = smem_u32(kv_sm + (size_t)sp * n_here * kRowBytes);
@@ -774,30 +980,31 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                                                   (uint32_t)(r0 + n_here - split) * kRowBytes, B.fin());
                                 }
                                 fin_ok = fin_ok && mbar_wait_warp(B.fin(), phase);
-                                // One thread per (row, 8 output dims), all rows of the batch at once.  Every
-                                // thread of a row scans the row's piece LSEs itself (broadcast reads): a first
-                                // pass for the maximum, a second that accumulates exp(lse_s - max) and the
-                                // weighted outputs; normalising by the sum at the end gives the merged row.
-                                #pragma unroll 1
-                                for (int e = tid; e < n_here * 16 && fin_ok; e += 256) {
-                                    const int i = e >> 4, c = e & 15;
-                                    const int idx = r0 + i;
-                                    const int bk = idx / kRowsPerBlock, r = idx - bk * kRowsPerBlock;
-                                    const int t = (grp * NB + bk) * kTokPerBlock + r / kGroup;
-                                    if (t >= T) continue;
-                                    const uint32_t pstride = (uint32_t)n_here * kRowBytes;     // bytes between pieces
-                                    const uint32_t row_sm = smem_u32(kv_sm) + (uint32_t)i * kRowBytes;
-                                    float mxl = -INFINITY;
+                                const bool active = fin_ok && row_i < n_here;
+                                const uint32_t pstride = (uint32_t)n_here * kRowBytes;     // bytes between pieces
+                                const uint32_t row_sm = smem_u32(kv_sm) + (uint32_t)row_i * kRowBytes;
+                                // pass 1: the row's largest piece LSE
+                                float mxl = -INFINITY;
+                                if (active) {
                                     #pragma unroll 4
-                                    for (uint32_t sp = 0, a_l = row_sm + 2 * kD; sp < (uint32_t)ns; ++sp, a_l += pstride)
+                                    for (uint32_t sp = grp_p, a_l = row_sm + 2 * kD + grp_p * pstride; sp < (uint32_t)ns; sp += G, a_l += G * pstride)
                                         mxl = fmaxf(mxl, lds_f32(a_l));
-                                    const bool any = mxl != -INFINITY;
-                                    const float mx2 = any ? mxl * 1.4426950408889634f : 0.f;
-                                    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-                                    float suml = 0.f;
+                                }
+                                if (G > 1) {
+                                    red_max[tid] = mxl;
+                                    softmax_bar_sync();
+                                    const int base = tid - grp_p * 16;
+                                    for (int g2 = 0; g2 < G; ++g2) mxl = fmaxf(mxl, red_max[base + g2 * 16]);
+                                }
+                                // pass 2: weights exp(lse_s - max), their sum, the weighted outputs of this thread's 8 dims
+                                const bool any = mxl != -INFINITY;
+                                const float mx2 = any ? mxl * 1.4426950408889634f : 0.f;
+                                float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                                float suml = 0.f;
+                                if (active) {
                                     #pragma unroll 4
-                                    for (uint32_t sp = 0, a_l = row_sm + 2 * kD, a_o = row_sm + c * 16; sp < (uint32_t)ns;
-                                         ++sp, a_l += pstride, a_o += pstride) {
+                                    for (uint32_t sp = grp_p, a_l = row_sm + 2 * kD + grp_p * pstride, a_o = row_sm + c16 * 16 + grp_p * pstride;
+                                         sp < (uint32_t)ns; sp += G, a_l += G * pstride, a_o += G * pstride) {
                                         const float ws = ex2(fmaf(lds_f32(a_l), 1.4426950408889634f, -mx2));   // exp(lse_s - max); 0 for -inf
                                         uint32_t raw[4];
                                         lds_v4(a_o, raw);
@@ -808,13 +1015,31 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                                             acc[2 * q] = fmaf(ws, f.x, acc[2 * q]); acc[2 * q + 1] = fmaf(ws, f.y, acc[2 * q + 1]);
                                         }
                                     }
+                                }
+                                if (G > 1) {
+                                    #pragma unroll
+                                    for (int q = 0; q < 8; ++q) red[tid * 9 + q] = acc[q];
+                                    red[tid * 9 + 8] = suml;
+                                    softmax_bar_sync();
+                                    if (grp_p == 0) {
+                                        for (int g2 = 1; g2 < G; ++g2) {
+                                            const float* o = red + (tid + g2 * 16) * 9;
+                                            #pragma unroll
+                                            for (int q = 0; q < 8; ++q) acc[q] += o[q];
+                                            suml += o[8];
+                                        }
+                                    }
+                                }
+                                if (active && grp_p == 0) {
+                                    const int idx = r0 + row_i;                            // row of the unit's list: token idx / 7, head idx % 7
+                                    const int t = tok0 + idx / kGroup;
+                                    const int h = kvh * kGroup + idx % kGroup;
                                     const float inv = suml > 0.f ? __fdividef(1.f, suml) : 0.f;
-                                    const int h = kvh * kGroup + r % kGroup;
                                     uint4 pk;
                                     pk.x = pack_bf16x2(acc[0] * inv, acc[1] * inv); pk.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
                                     pk.z = pack_bf16x2(acc[4] * inv, acc[5] * inv); pk.w = pack_bf16x2(acc[6] * inv, acc[7] * inv);
-                                    *reinterpret_cast<uint4*>(args.out + (((size_t)b * T + t) * args.n_q_heads + h) * kD + c * 8) = pk;
-                                    if (c == 0) args.lse[((size_t)b * args.n_q_heads + h) * T + t] = any ? mxl + __logf(suml) : -INFINITY;
+                                    *reinterpret_cast<uint4*>(args.out + (((size_t)b * T + t) * args.n_q_heads + h) * kD + c16 * 8) = pk;
+                                    if (c16 == 0) args.lse[((size_t)b * args.n_q_heads + h) * T + t] = any ? mxl + __logf(suml) : -INFINITY;
                                 }
                             }
                         }
@@ -824,8 +1049,17 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                 softmax_bar_sync();
             }
             if (tid == 0) {
-                if (direct) publish_counter(sync.fin_done + sync.parity);
-                if (fin_idx >= 0) publish_counter(sync.fin_done + sync.parity);
+                if (sync.enabled) {
+                    if (direct) publish_counter(sync.fin_done + sync.parity);
+                    if (fin_idx >= 0) publish_counter(sync.fin_done + sync.parity);
+                } else {
+                    // serial mode: the last CTA to leave puts the two words back to zero for the next call
+                    __threadfence();
+                    if (atomicAdd(sync.serial_words + 1, 1u) == (unsigned)plan.n_items - 1u) {
+                        sync.serial_words[0] = 0u;
+                        sync.serial_words[1] = 0u;
+                    }
+                }
             }
         }
         if (!ok) { atomicOr(args.status, timeout_bits(kSiteSoftmax)); *abort_flag = 1; }

@@ -16,7 +16,7 @@ from __future__ import annotations
 
 import math
 from dataclasses import dataclass, field
-from typing import List, Optional
+from typing import List, Optional, Sequence
 
 import numpy as np
 import torch
@@ -184,8 +184,6 @@ class AnchorCase:
     window: int
     T: int
     capacity: int
-    seq_len: int
-    vis_spans: List[List[int]]
     name: str = ""
 
     @property
@@ -235,26 +233,29 @@ def make_verify_case(seed: int, kv_len: List[int], T: int, tree: str = "chain", 
                       name=name)
 
 
-def text_anchor_list(seq_len: int, vis_spans, window: int, T: int) -> List[int]:
-    """Workload-side construction of the anchor list (plain filter; the library and the oracle
-    each have their own)."""
-    idx = [p for p in range(seq_len)
-           if not any(a <= p < e for a, e in vis_spans) and (window <= 0 or p >= seq_len - window)]
-    return idx + [seq_len + t for t in range(T)]
-
-
-def make_anchor_case(seed: int, seq_len: int, vis_spans, window: int, T: int, B: int = 1,
+def make_anchor_case(seed: int, anchor_list: Sequence[int], window: int, T: int, B: int = 1,
                      device="cpu", capacity: Optional[int] = None, name: str = "") -> AnchorCase:
-    cap = capacity if capacity is not None else seq_len + T
-    assert cap >= seq_len + T
+    """Inputs of one anchored-mode call.  ``anchor_list`` is the caller's list of anchored rows
+    (strictly increasing, the last T entries being the draft tokens' rows); which rows are anchors
+    is decided by the caller -- this module only draws the tensors."""
+    idx = [int(x) for x in anchor_list]
+    cap = capacity if capacity is not None else idx[-1] + 1
+    assert len(idx) >= T and cap > idx[-1]
     q = normal_bf16(seed, _TID_Q, (B, T, HQ, D), device)
     k = normal_bf16(seed, _TID_K, (B, HKV, cap, D), device)
     v = normal_bf16(seed, _TID_V, (B, HKV, cap, D), device)
-    idx = text_anchor_list(seq_len, vis_spans, window, T)
     anchor = torch.tensor([idx] * B, dtype=torch.int32, device=device)
     return AnchorCase(q=q, k=k, v=v, anchor_idx=anchor, n_anchor=len(idx), window=window, T=T,
-                      capacity=cap, seq_len=seq_len, vis_spans=[list(s) for s in vis_spans],
-                      name=name)
+                      capacity=cap, name=name)
+
+
+# The anchored configuration, written out: 26,112 positions, visual span [64, 25,664), the text
+# rows inside the last 1024 positions (25,664 .. 26,111: 448 of them), then the draft rows.
+C4_SEQ_LEN, C4_VIS_SPANS, C4_WINDOW = 26112, [[64, 25664]], 1024
+
+
+def c4_anchor_list(T: int) -> List[int]:
+    return list(range(25664, 26112)) + list(range(26112, 26112 + T))
 
 
 # ---- the five benchmark configurations --------------------------------------------------------
@@ -274,7 +275,7 @@ def make_config(c: int, device="cpu", layer: int = 0):
     if c == 2:
         return make_verify_case(s, [16384], 64, "random", device, name="C3 verify kv16384 T64 tree")
     if c == 3:
-        return make_anchor_case(s, 26112, [[64, 25664]], 1024, 8, 1, device,
+        return make_anchor_case(s, c4_anchor_list(8), C4_WINDOW, 8, 1, device,
                                 name="C4 anchor L26112 W1024 T8")
     if c == 4:
         # lengths and trees are per sequence and shared by all layers; K/V/Q differ per layer

@@ -34,6 +34,14 @@ def run_anchor(case: W.AnchorCase, ctx=None):
     return out, lse, ctx
 
 
+def anchor_case(seed, seq_len, vis_spans, window, T, batch=1, device="cuda:0", capacity=None, name=""):
+    """An anchored-mode case whose anchor list is the oracle's (Eq. 2's index set under the window
+    reading): text positions of [0, seq_len) within the last `window` positions, then the T draft rows."""
+    idx = oracle.anchor_idx(seq_len, vis_spans, window, T).tolist()
+    return W.make_anchor_case(seed, idx, window, T, batch, device,
+                              capacity=capacity if capacity is not None else seq_len + T, name=name)
+
+
 def oracle_verify(case: W.VerifyCase, rows=None):
     return oracle.verify_attn(W.bf16_bits(case.q), W.bf16_bits(case.k), W.bf16_bits(case.v),
                               case.kv_len, case.parents.cpu().numpy(), W.SCALE, rows=rows)

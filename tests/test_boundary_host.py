@@ -104,3 +104,28 @@ def test_create_without_gpu_fails_loudly():
 def test_status_strings():
     assert B.sparrow_status_string(0) == "ok"
     assert "anchor" in B.sparrow_status_string(4)
+
+
+def test_window_first_visible_matches_the_oracles_visibility():
+    """The first visible compact row per query, against the oracle's visibility matrix of the
+    anchored tree mode (the visible text anchors of a query are a contiguous run)."""
+    rng = np.random.default_rng(7)
+    for _ in range(60):
+        n_text = int(rng.integers(0, 120))
+        T_tree = int(rng.integers(1, 20)); T_new = int(rng.integers(1, T_tree + 1))
+        text = np.sort(rng.choice(2000, size=n_text, replace=False))
+        tree_rows = 2000 + int(rng.integers(0, 50)) + np.arange(T_tree)
+        idx = np.concatenate([text, tree_rows]).astype(np.int32)
+        window = int(rng.integers(-1, 2500))
+        par = W.random_tree_parents(int(rng.integers(1 << 30)), 8, T_tree)
+        vis = oracle.anchor_tree_visibility(idx, window, np.array(par, np.int32), T_new)       # [T_new, n_anchor]
+        first, lowest = B.sparrow_window_first_visible(idx.tolist(), window, T_tree, T_new)
+        for t in range(T_new):
+            row = vis[t, :n_text]
+            want = int(np.argmax(row)) if row.any() else n_text
+            assert first[t] == want
+            assert row[first[t]:].all() and not row[:first[t]].any()        # a contiguous run up to the tree
+        assert lowest == min(first)
+    with pytest.raises(B.SparrowError) as e:
+        B.sparrow_window_first_visible([1, 5, 5, 9], 3, 2, 2)
+    assert e.value.status == 4

@@ -89,3 +89,95 @@ def test_accept_greedy_reports_malformed_parents_and_argument_errors():
         B.sparrow_accept_greedy(ctx, d([[1]]), d([[-1]]), d([[1, 2]]), 0, path, n_acc, bonus)
     with pytest.raises(B.SparrowError):
         B.sparrow_kv_keep_accepted(ctx, case.k, case.v, [case.capacity], path, n_acc, 4)
+
+
+# ---- temperature 1: rejection sampling over the tree, bit-exact against the oracle --------------
+
+def _sampling_problem(seed, batch, T, vocab, sharp=1.0, same=False):
+    """Synthetic distributions (a softmax of seeded normals, sharper for the target), draft tokens
+    drawn from the draft rows without replacement among siblings, seeded 32-bit uniforms."""
+    rng = np.random.default_rng(seed)
+    par = [W.random_tree_parents(seed + 17 * b, 56, T) for b in range(batch)]
+    lt = rng.standard_normal((batch, T + 1, vocab)) * 2.0 * sharp
+    ld = lt + rng.standard_normal((batch, T + 1, vocab)) * (0.0 if same else 1.0)
+    p = np.exp(lt - lt.max(-1, keepdims=True)); p /= p.sum(-1, keepdims=True)
+    q = np.exp(ld - ld.max(-1, keepdims=True)); q /= q.sum(-1, keepdims=True)
+    p, q = p.astype(np.float32), q.astype(np.float32)
+    tok = np.zeros((batch, T), np.int64)
+    for b in range(batch):
+        for i in range(T):
+            row = q[b, par[b][i] + 1].astype(np.float64).copy()
+            for j in range(i):
+                if par[b][j] == par[b][i]:
+                    row[tok[b, j]] = 0.0
+            row /= row.sum()
+            tok[b, i] = rng.choice(vocab, p=row)
+    u_node = rng.integers(0, 1 << 32, size=(batch, T), dtype=np.uint64)
+    u_bonus = rng.integers(0, 1 << 32, size=(batch, T + 1), dtype=np.uint64)
+    return tok, par, p, q, u_node, u_bonus
+
+
+def _u32(a):
+    return torch.from_numpy(a.astype(np.uint32).view(np.int32).copy()).to(DEV)
+
+
+@pytest.mark.parametrize("batch,T,vocab,sharp,same", [
+    (1, 1, 7, 1.0, False),
+    (2, 12, 50, 1.0, False),
+    (3, 30, 1000, 0.5, False),          # flat distributions: many rejections per level
+    (2, 48, 5000, 2.0, False),          # peaked target
+    (1, 25, 151936, 1.0, False),        # a Qwen2-sized vocabulary
+    (4, 20, 300, 1.0, True),            # draft = target: everything on the first-child chain is accepted
+    (64, 5, 33, 1.0, False),
+])
+def test_accept_sample_matches_the_oracle(batch, T, vocab, sharp, same):
+    tok, par, p, q, u_node, u_bonus = _sampling_problem(9500 + batch + T, batch, T, vocab, sharp, same)
+    case = W.make_verify_case(9501, [40] * batch, T, "chain", DEV)
+    ctx = B.Context.for_cache(case.k, W.SCALE)
+    d = lambda x: torch.tensor(np.asarray(x), dtype=torch.int32, device=DEV)
+    path = torch.full((batch, T), 99, dtype=torch.int32, device=DEV)
+    n_acc = torch.full((batch,), 99, dtype=torch.int32, device=DEV)
+    bonus = torch.full((batch,), 99, dtype=torch.int32, device=DEV)
+    B.sparrow_accept_sample(ctx, d(tok), d(par), torch.from_numpy(p).to(DEV), torch.from_numpy(q).to(DEV),
+                            _u32(u_node), _u32(u_bonus), vocab, T, path, n_acc, bonus)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == 0
+    lengths = []
+    for b in range(batch):
+        ref_path, ref_bonus = oracle.sample_accept(tok[b], par[b], p[b], q[b], u_node[b], u_bonus[b])
+        assert int(n_acc[b]) == len(ref_path)
+        assert path[b].tolist() == ref_path + [-1] * (T - len(ref_path))
+        assert int(bonus[b]) == ref_bonus
+        lengths.append(len(ref_path))
+    if same:
+        assert min(lengths) >= 1
+
+
+def test_accept_sample_edge_cases():
+    """Zero draft mass on the drafted token, a target row equal to the draft row after a rejection
+    (nothing left of the residual: the original row is used), tokens outside the vocabulary."""
+    T, V = 3, 4
+    par = [[-1, -1, 0]]
+    p = np.array([[[0.5, 0.5, 0.0, 0.0]] * (T + 1)], np.float32)
+    q = np.array([[[0.5, 0.5, 0.0, 0.0]] * (T + 1)], np.float32)
+    case = W.make_verify_case(9502, [40], T, "chain", DEV)
+    ctx = B.Context.for_cache(case.k, W.SCALE)
+    d = lambda x: torch.tensor(np.asarray(x), dtype=torch.int32, device=DEV)
+    for tok, expect_status in (([[2, 3, 1]], 0), ([[2, 0, 1]], 0), ([[9, -4, 1]], 3)):
+        u_node = np.array([[7, 1 << 31, 123456]], np.uint64)
+        u_bonus = np.array([[1 << 30, 3 << 30, 5, 77]], np.uint64)
+        path = torch.full((1, T), 99, dtype=torch.int32, device=DEV)
+        n_acc = torch.full((1,), 99, dtype=torch.int32, device=DEV)
+        bonus = torch.full((1,), 99, dtype=torch.int32, device=DEV)
+        B.sparrow_accept_sample(ctx, d(tok), d(par), torch.from_numpy(p).to(DEV), torch.from_numpy(q).to(DEV),
+                                _u32(u_node), _u32(u_bonus), V, T, path, n_acc, bonus)
+        torch.cuda.synchronize()
+        assert ctx.last_device_status() == expect_status
+        if expect_status == 0:
+            ref_path, ref_bonus = oracle.sample_accept(tok[0], par[0], p[0], q[0], u_node[0], u_bonus[0])
+            assert path[0, :int(n_acc[0])].tolist() == ref_path and int(bonus[0]) == ref_bonus
+        else:
+            assert int(n_acc[0]) == 0 and 0 <= int(bonus[0]) < V
+    with pytest.raises(B.SparrowError):
+        B.sparrow_accept_sample(ctx, d([[0]]), d([[-1]]), torch.from_numpy(p).to(DEV), torch.from_numpy(q).to(DEV),
+                                _u32(np.zeros((1, 1), np.uint64)), _u32(np.zeros((1, 2), np.uint64)), 0, 1, path, n_acc, bonus)

@@ -10,10 +10,18 @@ import torch
 from paper_2602_15318_b200 import binding as B
 from paper_2602_15318_b200 import workloads as W
 
-from gpu_util import check, oracle_verify, run_verify
+from gpu_util import anchor_case, check, oracle_verify, run_verify
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
+
+
+def _overlapping_ctx(k_cache):
+    """A context whose single calls may start early behind its previous call (the tests here
+    enqueue nothing in between that could break the rule this opt-in states)."""
+    ctx = B.Context.for_cache(k_cache, W.SCALE)
+    ctx.set_call_overlap(True)
+    return ctx
 
 
 def _new(case):
@@ -31,7 +39,7 @@ def test_back_to_back_calls_keep_their_results_apart():
              for i, (kv, T, tree) in enumerate([([3000], 16, "chain"), ([90], 5, "random"), ([2500], 24, "random"),
                                                 ([1700], 8, "chain"), ([40], 19, "chain")])]
     refs = [oracle_verify(c) for c in cases]
-    ctx = B.Context.for_cache(cases[0].k, W.SCALE)
+    ctx = _overlapping_ctx(cases[0].k)
     results = []
     for rep in range(6):
         for c in cases:
@@ -49,7 +57,7 @@ def test_same_output_buffer_reused_by_consecutive_calls():
     buffers hold the last call's result."""
     a = W.make_verify_case(601, [2800], 12, "random", DEV)
     b = W.make_verify_case(602, [2800], 12, "chain", DEV)
-    ctx = B.Context.for_cache(a.k, W.SCALE)
+    ctx = _overlapping_ctx(a.k)
     out, lse = _new(a)
     for _ in range(5):
         B.sparrow_verify_attn(ctx, a.q, a.k, a.v, a.kv_len, a.parents, a.T, out, lse)
@@ -63,8 +71,8 @@ def test_same_output_buffer_reused_by_consecutive_calls():
 
 def test_anchor_and_verify_calls_interleave():
     v = W.make_verify_case(603, [2000], 8, "chain", DEV, capacity=2100)
-    a = W.make_anchor_case(604, 2000, [[50, 1800]], 0, 8, 1, DEV, capacity=2100)
-    ctx = B.Context.for_cache(v.k, W.SCALE)
+    a = anchor_case(604, 2000, [[50, 1800]], 0, 8, 1, DEV, capacity=2100)
+    ctx = _overlapping_ctx(v.k)
     outs = []
     for _ in range(3):
         ov, lv = _new(v)
@@ -82,20 +90,21 @@ def test_anchor_and_verify_calls_interleave():
 
 
 def test_stream_ordered_mode(monkeypatch):
-    """SPARROW_NO_PDL=1 at context creation: two ordinary launches per call, no counters."""
+    """SPARROW_NO_PDL=1 at context creation: every call is one ordinary launch that merges its own
+    pieces (serial mode), ordered by the stream alone."""
     monkeypatch.setenv("SPARROW_NO_PDL", "1")
     for kv, T, tree in [([3000, 1500], 12, "random"), ([129], 19, "random"), ([64], 8, "chain")]:
         case = W.make_verify_case(610 + T, kv, T, tree, DEV)
-        ctx = B.Context.for_cache(case.k, W.SCALE)
+        ctx = _overlapping_ctx(case.k)
         n0 = ctx.launch_count()
         out, lse, _ = run_verify(case, ctx)
-        assert ctx.launch_count() - n0 == 2
+        assert ctx.launch_count() - n0 == 1
         check(out, lse, *oracle_verify(case))
 
 
 def test_call_captured_into_a_graph_replays():
     case = W.make_verify_case(620, [2500, 900], 10, "random", DEV)
-    ctx = B.Context.for_cache(case.k, W.SCALE)
+    ctx = _overlapping_ctx(case.k)
     out, lse = _new(case)
     s = torch.cuda.Stream()
     s.wait_stream(torch.cuda.current_stream())
@@ -118,7 +127,7 @@ def test_call_captured_into_a_graph_replays():
 
 def test_bounded_wait_gives_up_and_context_survives():
     case = W.make_verify_case(630, [1500], 8, "chain", DEV)
-    ctx = B.Context.for_cache(case.k, W.SCALE)
+    ctx = _overlapping_ctx(case.k)
     out, lse, _ = run_verify(case, ctx)
     B.sparrow_debug_wait_counter(ctx, 0)                  # everything it waits for has happened
     torch.cuda.synchronize()
@@ -140,7 +149,7 @@ def test_plan_policy_changes_between_calls():
     cases = [W.make_verify_case(700 + i, kv, T, tree, DEV, capacity=cap)
              for i, (kv, T, tree) in enumerate([([9000], 16, "chain"), ([5000], 30, "random"), ([7000], 8, "chain")])]
     refs = [oracle_verify(c) for c in cases]
-    ctx = B.Context.for_cache(cases[0].k, W.SCALE)
+    ctx = _overlapping_ctx(cases[0].k)
     n_sm = torch.cuda.get_device_properties(0).multi_processor_count
     targets = {}
     for pol in (B.PLAN_LATENCY, B.PLAN_BALANCED, B.PLAN_THROUGHPUT):
@@ -170,7 +179,7 @@ def test_long_stream_is_bitwise_reproducible(policy):
     ordering mistake between overlapping calls shows up as a changed bit or a timeout)."""
     cap = 20000 + 32
     cases = [W.make_verify_case(800 + i, [20000 - 37 * i], 16, "chain", DEV, capacity=cap) for i in range(3)]
-    ctx = B.Context.for_cache(cases[0].k, W.SCALE)
+    ctx = _overlapping_ctx(cases[0].k)
     ctx.set_plan_policy(policy)
     alone = []
     for c in cases:
@@ -203,7 +212,7 @@ def test_whole_step_in_one_stream_without_synchronisation():
     import oracle
     T, kv0 = 12, 3000
     case = W.make_verify_case(900, [kv0], T, "random", DEV, capacity=kv0 + 3 * T)
-    ctx = B.Context.for_cache(case.k, W.SCALE)
+    ctx = _overlapping_ctx(case.k)
     ctx.set_plan_policy(B.PLAN_THROUGHPUT)
     d = lambda x: torch.tensor(x, dtype=torch.int32, device=DEV)
     par = case.parents[0].tolist()
@@ -253,8 +262,8 @@ def test_calls_of_two_contexts_on_one_stream_take_stream_order():
     T = 16
     a = W.make_verify_case(950, [9000], T, "chain", DEV)
     b = W.make_verify_case(951, [7000], T, "random", DEV)
-    ctx_a = B.Context.for_cache(a.k, W.SCALE)
-    ctx_b = B.Context.for_cache(b.k, W.SCALE)
+    ctx_a = _overlapping_ctx(a.k)
+    ctx_b = _overlapping_ctx(b.k)
     out_a, lse_a = _new(a)
     out_b, lse_b = _new(b)
     for _ in range(5):
@@ -268,3 +277,90 @@ def test_calls_of_two_contexts_on_one_stream_take_stream_order():
         assert torch.isfinite(out_b.float()).all()
         assert torch.equal(out_b, again) and torch.equal(lse_b, lse_again)
     assert ctx_a.last_device_status() == 0 and ctx_b.last_device_status() == 0
+
+
+# ---- what may start early, and what may not ---------------------------------------------------
+
+def test_call_behind_a_foreign_kernel_with_an_early_trigger_waits_for_it():
+    """A kernel that is not the library's sits between two calls; it lets its dependents launch at
+    once and writes the next call's q only much later.  The call must still see that q."""
+    T = 16
+    a = W.make_verify_case(960, [6000], T, "chain", DEV)
+    b = W.make_verify_case(961, [6000], T, "random", DEV, capacity=a.capacity)
+    ref_b = oracle_verify(b)
+    ctx = B.Context.for_cache(a.k, W.SCALE)           # default: single calls take plain stream order
+    q_live = torch.zeros_like(b.q)
+    out_a, lse_a = _new(a)
+    for delay in (0, 50, 400):
+        q_live.zero_()
+        out_b, lse_b = _new(b)
+        B.sparrow_verify_attn(ctx, a.q, a.k, a.v, a.kv_len, a.parents, T, out_a, lse_a)
+        B.sparrow_debug_early_trigger_copy(ctx, b.q, q_live, b.q.numel() * 2, delay)
+        B.sparrow_verify_attn(ctx, q_live, b.k, b.v, b.kv_len, b.parents, T, out_b, lse_b)
+        torch.cuda.synchronize()
+        check(out_b, lse_b, *ref_b)
+    assert ctx.last_device_status() == 0
+
+
+@pytest.mark.parametrize("gap", [1, 2, 5])
+@pytest.mark.parametrize("policy", [B.PLAN_LATENCY, B.PLAN_THROUGHPUT])
+def test_call_reading_an_earlier_calls_output_is_not_started_early(gap, policy):
+    """Inside one batch (calls start early behind each other) call n reads, as its q, the out of
+    call n - gap, with other calls in between: the library must notice and order that launch.
+    The result must equal, bit for bit, what the same chain gives with a synchronisation after
+    every call."""
+    T, n_calls = 16, 12
+    cases = [W.make_verify_case(970 + i, [9000 - 100 * i], T, "chain", DEV, capacity=9100) for i in range(3)]
+    ctx = B.Context.for_cache(cases[0].k, W.SCALE)
+    ctx.set_plan_policy(policy)
+
+    def run(sync_every_call):
+        outs = [_new(cases[0]) for _ in range(n_calls)]
+        calls = []
+        for n in range(n_calls):
+            c = cases[n % 3]
+            q = c.q if n < gap else outs[n - gap][0]
+            calls.append((q, c.k, c.v, c.kv_len, c.parents, T, outs[n][0], outs[n][1]))
+        if sync_every_call:
+            for call in calls:
+                B.sparrow_verify_attn_batch(ctx, B.VerifyBatch([call]))
+                torch.cuda.synchronize()
+        else:
+            B.sparrow_verify_attn_batch(ctx, B.VerifyBatch(calls))
+            torch.cuda.synchronize()
+        return outs
+
+    want = run(True)
+    for _ in range(3):
+        got = run(False)
+        for (o, l), (wo, wl) in zip(got, want):
+            assert torch.equal(o, wo) and torch.equal(l, wl)
+    assert ctx.last_device_status() == 0
+
+
+def test_many_caches_through_one_context():
+    """More distinct K / V / q buffers than the context's tensor-map cache holds, revisited in an
+    order that mixes hits with evictions: every call must use the maps of its own buffers."""
+    T, kv, n_buf = 4, 200, 1400
+    base = W.make_verify_case(980, [kv], T, "chain", DEV, capacity=256)
+    ks = W.normal_bf16(981, 2, (n_buf, W.HKV, 256, W.D), DEV)
+    vs = W.normal_bf16(981, 3, (n_buf, W.HKV, 256, W.D), DEV)
+    qs = W.normal_bf16(981, 1, (n_buf, T, W.HQ, W.D), DEV)
+    ctx = B.Context.for_cache(base.k, W.SCALE)
+    outs = torch.full((n_buf, T, W.HQ, W.D), float("nan"), dtype=torch.bfloat16, device=DEV)
+    lses = torch.full((n_buf, W.HQ, T), float("nan"), dtype=torch.float32, device=DEV)
+    order = list(range(n_buf)) + [0, 777, 1, 1399, 2, 640] + list(range(0, n_buf, 7))
+    for i in order:
+        B.sparrow_verify_attn(ctx, qs[i:i + 1], ks[i:i + 1], vs[i:i + 1], [kv], base.parents, T, outs[i:i + 1], lses[i:i + 1])
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == 0
+    import oracle
+    for i in (0, 1, 2, 640, 777, 1398, 1399):
+        ref = oracle.verify_attn(W.bf16_bits(qs[i:i + 1]), W.bf16_bits(ks[i:i + 1]), W.bf16_bits(vs[i:i + 1]), [kv],
+                                 base.parents.cpu().numpy(), W.SCALE)
+        check(outs[i:i + 1], lses[i:i + 1], *ref)
+    first = outs.clone()
+    for i in reversed(order):
+        B.sparrow_verify_attn(ctx, qs[i:i + 1], ks[i:i + 1], vs[i:i + 1], [kv], base.parents, T, outs[i:i + 1], lses[i:i + 1])
+    torch.cuda.synchronize()
+    assert torch.equal(first, outs)

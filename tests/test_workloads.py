@@ -30,7 +30,7 @@ def test_config_shapes():
     assert par[0] == -1 and all(-1 <= p < i for i, p in enumerate(par))
     lens = W.ragged_lengths(W.config_seed(4), 5, 8)
     assert all(8192 <= n <= 32768 for n in lens)
-    idx = W.text_anchor_list(26112, [[64, 25664]], 1024, 8)
+    idx = W.c4_anchor_list(8)
     assert len(idx) == 456 and idx[0] == 25664 and idx[-1] == 26119
 
 
