@@ -351,3 +351,32 @@ def sample_accept(draft_tokens, parents, p_target, p_draft, u_node, u_bonus):
             return path, bonus
         path.append(taken)
         cur = taken
+
+
+# ---------------------------------------------------------------------------------------------
+# Hidden-state reuse: the draft model's input (Section 3.1, Eq. 1)
+#     z_t = FC(e_t (+) h_t),
+# the projection FC applied to the concatenation of the token embedding e_t and the target model's
+# hidden state h_t (of its second-to-last layer, at the previous position) -- 2 d features down to
+# d.  FC is taken as an ordinary linear layer, z = W x + b with W of shape [d_out][2 d] (the layout
+# of torch.nn.Linear); the paper does not say whether it has a bias, so the bias is optional.
+# ---------------------------------------------------------------------------------------------
+
+def bf16_bits_to_f64(bits) -> np.ndarray:
+    """uint16 bf16 bit patterns -> float64, exactly (a bf16 is the top half of a float32)."""
+    b = np.ascontiguousarray(bits, dtype=np.uint16)
+    return (b.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+
+
+def hsr_fuse(e, h, w, bias=None) -> np.ndarray:
+    """e, h: uint16 bf16 bits [M][d]; w: bits [d_out][2 d]; bias: bits [d_out] or None.
+    Returns z float64 [M][d_out] = concat(e, h) @ w.T (+ bias), all in float64."""
+    E, H, Wt = bf16_bits_to_f64(e), bf16_bits_to_f64(h), bf16_bits_to_f64(w)
+    assert E.ndim == 2 and E.shape == H.shape and Wt.ndim == 2 and Wt.shape[1] == 2 * E.shape[1]
+    x = np.concatenate([E, H], axis=1)                 # e (+) h
+    z = x @ Wt.T
+    if bias is not None:
+        b = bf16_bits_to_f64(bias)
+        assert b.shape == (Wt.shape[0],)
+        z = z + b[None, :]
+    return z

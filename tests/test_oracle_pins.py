@@ -650,3 +650,50 @@ def test_sample_accept_pin_detects_a_planted_mistake():
         counts[wrong(tok, _uniforms(rng, 3), _uniforms(rng, 1))] += 1
     e = p[0].astype(np.float64) * n
     assert np.any(np.abs(counts - e) > 6 * np.sqrt(e))
+
+
+# ---------------------------------------------------------------- hidden-state reuse (Eq. 1) ----
+
+def _bits(a):
+    return W.bf16_bits(torch.tensor(np.asarray(a, dtype=np.float32)).to(torch.bfloat16))
+
+
+def test_hsr_fuse_hand_worked_example():
+    g = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "hsr_fuse_small.json")))
+    z = oracle.hsr_fuse(_bits(g["e"]), _bits(g["h"]), _bits(g["w"]), _bits(g["bias"]))
+    assert np.array_equal(z, np.array(g["z"]))
+    z0 = oracle.hsr_fuse(_bits(g["e"]), _bits(g["h"]), _bits(g["w"]))
+    assert np.array_equal(z0, np.array(g["z_without_bias"]))
+
+
+def test_hsr_fuse_selector_weights_pick_the_two_halves():
+    """W = [I | 0] returns e, W = [0 | I] returns h, W = [I | I] their sum: the concatenation puts
+    the embedding first and the hidden state second."""
+    rng = np.random.default_rng(50)
+    M, d = 5, 16
+    e, h = rand_bits(rng, (M, d)), rand_bits(rng, (M, d))
+    E, H = oracle.bf16_bits_to_f64(e), oracle.bf16_bits_to_f64(h)
+    I, Z = np.eye(d), np.zeros((d, d))
+    assert np.array_equal(oracle.hsr_fuse(e, h, _bits(np.hstack([I, Z]))), E)
+    assert np.array_equal(oracle.hsr_fuse(e, h, _bits(np.hstack([Z, I]))), H)
+    assert np.array_equal(oracle.hsr_fuse(e, h, _bits(np.hstack([I, I]))), E + H)
+    assert not np.array_equal(E, H)
+
+
+def test_hsr_fuse_brute_force_and_library_linear():
+    rng = np.random.default_rng(51)
+    M, d, n = 3, 8, 6
+    e, h, w, b = rand_bits(rng, (M, d)), rand_bits(rng, (M, d)), rand_bits(rng, (n, 2 * d)), rand_bits(rng, (n,))
+    z = oracle.hsr_fuse(e, h, w, b)
+    E, H, Wt, Bv = (oracle.bf16_bits_to_f64(a) for a in (e, h, w, b))
+    for m in range(M):                              # the definition, term by term
+        for o in range(n):
+            acc = Bv[o]
+            for k in range(d):
+                acc += E[m, k] * Wt[o, k]
+            for k in range(d):
+                acc += H[m, k] * Wt[o, d + k]
+            assert abs(z[m, o] - acc) <= 1e-12 * (1 + abs(acc))
+    lib = torch.nn.functional.linear(torch.cat([torch.from_numpy(E), torch.from_numpy(H)], dim=1),
+                                     torch.from_numpy(Wt), torch.from_numpy(Bv)).numpy()
+    assert np.max(np.abs(z - lib)) <= 1e-12
