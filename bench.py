@@ -242,6 +242,12 @@ def main():
                     help="skip the other configurations (C1, C3, C4, C5), which are otherwise timed and "
                          "reported under other_configs in the same JSON line")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--only", choices=["C1", "C2", "C3", "C5"],
+                    help="time just this configuration's stream of calls (a small run for a profiler capture): "
+                         "--steps calls after --warmup calls under --policy, one JSON line")
+    ap.add_argument("--policy", choices=["latency", "balanced", "throughput"], default="throughput")
+    ap.add_argument("--single-calls", action="store_true",
+                    help="with --only: enqueue every call on its own (plain stream order, nothing overlaps)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -268,6 +274,9 @@ def main():
 
     steps, warmup = max(1, args.steps), max(3, args.warmup)
     l2 = torch.cuda.get_device_properties(local_rank).L2_cache_size or L2_BYTES_FALLBACK
+    if args.only:
+        run_only(args, W, B, torch, dev, l2, steps, warmup)
+        return
     probe = W.make_config(1, "cpu")
     kv_bytes, io_bytes, flops = probe.kv_bytes(), probe.io_bytes(), probe.flops()
     n_caches = max(4, -(-4 * l2 // kv_bytes))                 # R * bytes >= 4 x L2
@@ -447,6 +456,35 @@ def main():
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def run_only(args, W, B, torch, dev, l2, steps, warmup):
+    """One configuration, one policy, few calls: what a profiler capture runs."""
+    ci = {"C1": 0, "C2": 1, "C3": 2, "C5": 4}[args.only]
+    probe = W.make_config(ci, "cpu")
+    n_caches = 3 if ci == 4 else max(4, -(-4 * l2 // probe.kv_bytes()))
+    cases, ctx, outs, lses, batch = build_rotation(W, B, torch, dev, ci, n_caches, calls_per_batch=max(n_caches, min(1000, steps)))
+    ctx.set_plan_policy({"latency": B.PLAN_LATENCY, "balanced": B.PLAN_BALANCED, "throughput": B.PLAN_THROUGHPUT}[args.policy])
+    if args.single_calls:
+        singles = [B.VerifyBatch([(c.q, c.k, c.v, c.kv_len, c.parents, c.T, o, l)]) for c, o, l in zip(cases, outs, lses)]
+
+        def run(n):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize(); e0.record()
+            for i in range(n):
+                B.sparrow_verify_attn_batch(ctx, singles[i % len(singles)])
+            e1.record(); torch.cuda.synchronize()
+            return e0.elapsed_time(e1) * 1e3 / n
+        run(warmup)
+        us = run(steps)
+    else:
+        time_calls(ctx, batch, warmup, B, torch)
+        us = time_calls(ctx, batch, steps, B, torch)
+    by = probe.kv_bytes() + probe.io_bytes()
+    print(json.dumps({"only": args.only, "workload": probe.name, "plan_policy": args.policy, "single_calls": bool(args.single_calls),
+                      "steps": steps, "warmup": warmup, "us_per_call": us, "algorithmic_bytes_per_call": by,
+                      "hbm_gbs": by / us / 1e3, "tflops": probe.flops() / us / 1e6, "rotation": n_caches,
+                      "target_items": ctx.plan_target_items(), "device_status": ctx.last_device_status()}), flush=True)
 
 
 def POLICIES(B):

@@ -28,7 +28,7 @@ EXPORTS = ["sparrow_create", "sparrow_destroy", "sparrow_workspace_bytes", "spar
            "sparrow_set_plan_policy", "sparrow_set_call_overlap", "sparrow_debug_early_trigger_copy",
            "sparrow_verify_attn_window", "sparrow_window_first_visible", "sparrow_window_first_visible_device",
            "sparrow_plan_target_items", "sparrow_anchor_attn_tree", "sparrow_kv_append", "sparrow_compact_anchors",
-           "sparrow_accept_greedy", "sparrow_accept_sample", "sparrow_kv_keep_accepted", "sparrow_plan_piece_range",
+           "sparrow_hsr_scratch_bytes", "sparrow_hsr_fuse", "sparrow_accept_greedy", "sparrow_accept_sample", "sparrow_kv_keep_accepted", "sparrow_plan_piece_range",
            "sparrow_status_string"]
 
 
@@ -74,6 +74,9 @@ def lib():
         L.sparrow_anchor_attn.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp]
         L.sparrow_plan_piece_range.argtypes = [i32, i32, i32, vp, vp]
         L.sparrow_accept_greedy.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp]
+        L.sparrow_hsr_scratch_bytes.argtypes = [vp, i32, i32]
+        L.sparrow_hsr_scratch_bytes.restype = ctypes.c_size_t
+        L.sparrow_hsr_fuse.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp, ctypes.c_size_t, vp, vp]
         L.sparrow_accept_sample.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp]
         L.sparrow_kv_keep_accepted.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp]
         L.sparrow_kv_append.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp]
@@ -98,7 +101,7 @@ def lib():
         L.sparrow_status_string.argtypes = [ctypes.c_int]
         L.sparrow_status_string.restype = ctypes.c_char_p
         for name in EXPORTS:
-            if name not in ("sparrow_workspace_bytes", "sparrow_launch_count", "sparrow_status_string",
+            if name not in ("sparrow_workspace_bytes", "sparrow_hsr_scratch_bytes", "sparrow_launch_count", "sparrow_status_string",
                             "sparrow_debug_status_word", "sparrow_plan_target_items"):
                 getattr(L, name).restype = ctypes.c_int
         _lib = L
@@ -302,6 +305,20 @@ def sparrow_accept_greedy(ctx: Context, draft_tokens, parents, target_next, T: i
     _chk(lib().sparrow_accept_greedy(ctx.handle, _ptr(draft_tokens), _ptr(parents), _ptr(target_next), T,
                                      _ptr(path_out), _ptr(n_accept_out), _ptr(bonus_out), _stream_handle(stream)),
          "sparrow_accept_greedy")
+
+
+def sparrow_hsr_scratch_bytes(ctx: Context, d: int, d_out: int) -> int:
+    return int(lib().sparrow_hsr_scratch_bytes(ctx.handle, d, d_out))
+
+
+def sparrow_hsr_fuse(ctx: Context, e, h, w, bias, z, scratch=None, stream=None):
+    """z = [e | h] @ w.T (+ bias).  e, h: CUDA bf16 [M, d]; w: CUDA bf16 [d_out, 2d]; bias: CUDA bf16
+    [d_out] or None; z: CUDA bf16 [M, d_out]; scratch: CUDA uint8 tensor of sparrow_hsr_scratch_bytes."""
+    M, d = e.shape
+    d_out = w.shape[0]
+    _chk(lib().sparrow_hsr_fuse(ctx.handle, _ptr(e), _ptr(h), _ptr(w), _ptr(bias), M, d, d_out, _ptr(scratch),
+                                scratch.numel() if scratch is not None else 0, _ptr(z), _stream_handle(stream)),
+         "sparrow_hsr_fuse")
 
 
 def sparrow_accept_sample(ctx: Context, draft_tokens, parents, p_target, p_draft, u_node, u_bonus, vocab: int, T: int,

@@ -21,6 +21,7 @@
 #include "kv_rows.cuh"
 #include "split_gather.cuh"
 #include "verify_tc.cuh"
+#include "hsr_fuse.cuh"
 #include "window.cuh"
 
 using namespace sparrow;
@@ -82,6 +83,8 @@ namespace {
 constexpr size_t kStatusBytes = 1024;      // word 0: sticky status; words 16, 17: finisher counters
 constexpr size_t kFinDoneOffset = 64;
 constexpr size_t kArrivalsOffset = 128;     // words 32..35: arrival words of the four call slots
+constexpr size_t kHsrCountersOffset = 256;  // words 64..255: one arrival counter per 128-feature tile of sparrow_hsr_fuse()
+constexpr int kHsrMaxFeatureTiles = 192;
 constexpr size_t kSerialOffset = 192;       // words 48, 49: arrival / exit words of a call that runs alone (serial mode)
 constexpr int kMinPieceKeys = 128;
 // The gathered kernel works on 64-key tiles and pays two dependent memory round trips per tile
@@ -1010,6 +1013,71 @@ sparrow_status sparrow_window_first_visible_device(sparrow_ctx* c, const int32_t
     const int n = c->layout.batch * T_new;
     window_bounds_kernel<<<(n + 127) / 128, 128, 0, static_cast<cudaStream_t>(stream)>>>(anchor_idx, n_anchor, window, T_tree, T_new,
                                                                                          c->layout.batch, first_visible);
+    if (cudaGetLastError() != cudaSuccess) return SPARROW_ERR_CUDA;
+    c->launches.fetch_add(1);
+    return SPARROW_OK;
+}
+
+// K-range slices per feature tile: about one work item per SM, never more slices than K tiles.
+static int hsr_slices(int n_sm, int d, int d_out)
+{
+    const int f_tiles = d_out / hsr::kFeat, k_tiles = 2 * d / hsr::kKTile;
+    int s = n_sm / f_tiles;
+    if (s < 1) s = 1;
+    if (s > k_tiles) s = k_tiles;
+    return s;
+}
+
+size_t sparrow_hsr_scratch_bytes(const sparrow_ctx* c, int32_t d, int32_t d_out)
+{
+    if (!c || d < 64 || (d % 64) != 0 || d_out < 128 || (d_out % 128) != 0) return 0;
+    return (size_t)hsr_slices(c->n_sm, d, d_out) * d_out * hsr::kTok * sizeof(float);
+}
+
+sparrow_status sparrow_hsr_fuse(sparrow_ctx* c, const void* e, const void* h, const void* w, const void* bias, int32_t M,
+                                int32_t d, int32_t d_out, void* scratch, size_t scratch_bytes, void* z, void* stream)
+{
+    if (!c || !e || !h || !w || !z) return SPARROW_ERR_NULL;
+    if (M < 1 || M > hsr::kTok || d < 64 || (d % 64) != 0 || d_out < 128 || (d_out % 128) != 0 ||
+        d_out / hsr::kFeat > kHsrMaxFeatureTiles)
+        return SPARROW_ERR_SHAPE;
+    if (!aligned16(e) || !aligned16(h) || !aligned16(w) || !aligned16(z) || (scratch && !aligned16(scratch))) return SPARROW_ERR_SHAPE;
+    if (!c->ws) return SPARROW_ERR_WORKSPACE;                       // status word and the tiles' arrival counters live there
+    const int n_slices = hsr_slices(c->n_sm, d, d_out);
+    if (n_slices > 1 && (!scratch || scratch_bytes < (size_t)n_slices * d_out * hsr::kTok * sizeof(float))) return SPARROW_ERR_WORKSPACE;
+    if (!c->encode) return SPARROW_ERR_CUDA;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return SPARROW_ERR_CUDA;
+    static bool attr_set[kMaxStaticDevices] = {};
+    if (c->device >= 0 && c->device < kMaxStaticDevices && !attr_set[c->device]) {
+        if (cudaFuncSetAttribute(hsr::hsr_fuse_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, hsr::kSmemBytes) != cudaSuccess)
+            return SPARROW_ERR_CUDA;
+        attr_set[c->device] = true;
+    }
+    // W: [d_out][2 d], boxes of 64 k x 128 features; e, h: [M][d], boxes of 64 k x 64 tokens (rows past M read as zero)
+    CUtensorMap mw, me, mh;
+    const cuuint32_t estr[2] = {1, 1};
+    auto encode2d = [&](CUtensorMap* m, const void* base, cuuint64_t cols, cuuint64_t rows, cuuint32_t box_rows) {
+        const cuuint64_t dims[2] = {cols, rows};
+        const cuuint64_t strides[1] = {cols * 2};
+        const cuuint32_t box[2] = {(cuuint32_t)hsr::kKTile, box_rows};
+        return c->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    };
+    if (!encode2d(&mw, w, (cuuint64_t)2 * d, (cuuint64_t)d_out, hsr::kFeat) || !encode2d(&me, e, (cuuint64_t)d, (cuuint64_t)M, hsr::kTok) ||
+        !encode2d(&mh, h, (cuuint64_t)d, (cuuint64_t)M, hsr::kTok))
+        return SPARROW_ERR_CUDA;
+    HsrArgs a;
+    a.bias = static_cast<const __nv_bfloat16*>(bias);
+    a.partial = static_cast<float*>(scratch);
+    a.z = static_cast<__nv_bfloat16*>(z);
+    a.counters = reinterpret_cast<unsigned*>(c->ws + kHsrCountersOffset);
+    a.status = reinterpret_cast<unsigned*>(c->ws);
+    a.M = M; a.d = d; a.d_out = d_out;
+    a.n_slices = n_slices;
+    a.k_tiles = 2 * d / hsr::kKTile;
+    hsr::hsr_fuse_kernel<<<(d_out / hsr::kFeat) * n_slices, hsr::kThreadsHsr, hsr::kSmemBytes, static_cast<cudaStream_t>(stream)>>>(a, mw, me, mh);
     if (cudaGetLastError() != cudaSuccess) return SPARROW_ERR_CUDA;
     c->launches.fetch_add(1);
     return SPARROW_OK;

@@ -476,48 +476,46 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
             const uint64_t v_desc0 = smem_desc(smem_u32(kv_sm) + 2 * kSubTileBytes, kSubTileBytes, 1024);
             bool ok = mbar_wait(B.q_full(), 0);
             if constexpr (NB == 2) {
-                // Two row blocks, each with its own softmax warpgroup.  A job is HALF a key tile
-                // (64 keys) against one row block: job n = (half-tile h = n / 2, block b = n % 2),
-                // key tile j = h / 2.  Block b owns TMEM columns [128 b, 128 b + 128): two score
-                // slots of 64 fp32 columns (slot h % 2), the P of a slot (bf16, 32 columns) written
-                // over the slot's upper half; the accumulators follow at 256 + 128 b.  Four slots in
-                // all keep the scores two half-tiles ahead of each warpgroup, so the tensor pipe
-                // has S = Q K^T work queued while it waits for a P.
-                constexpr uint32_t idesc_qk64 = idesc_bf16(false, 64);
+                // Two row blocks, each with its own softmax warpgroup.  Job n = (key tile j = n / 2,
+                // block b = n % 2).  Block b owns TMEM columns [128 b, 128 b + 128) for its scores,
+                // with its P (bf16, 64 columns) written over the upper half, and the accumulator at
+                // 256 + 128 b.  Per block the chain is scores -> softmax -> O += P V -> next scores;
+                // the two blocks' chains interleave, so the tensor pipe works for one block while
+                // the other block's warpgroup is in its exponentials.
+                constexpr uint32_t idesc_qk = idesc_bf16(false);
                 constexpr uint32_t idesc_pv = idesc_bf16(true);
-                const int n_half_jobs = 4 * n_tiles;
-                auto issue_qk64 = [&](int m) -> bool {
-                    const int h = m >> 1, b = m & 1, hh = h & 1, j = h >> 1, st = j % NS;
-                    if (b == 0 && hh == 0) {                                  // first use of this K tile
+                auto issue_qk2 = [&](int m) -> bool {
+                    const int j = m >> 1, b = m & 1, st = j % NS;
+                    if (b == 0) {                                             // first use of this K tile
                         if (!mbar_wait(B.k_full(st), (j / NS) & 1)) return false;
                         tc_fence_after();
                     }
                     const uint64_t qd = q_desc0 + (uint64_t)((b * kQBlockBytes) >> 4);
-                    const uint64_t kd = k_desc0 + (uint64_t)((st * kStageBytes + hh * 64 * 128) >> 4);   // keys [64 hh, 64 hh + 64) of the tile
+                    const uint64_t kd = k_desc0 + (uint64_t)((st * kStageBytes) >> 4);
                     #pragma unroll
                     for (int ks = 0; ks < 8; ++ks) {
                         const uint32_t off = ((ks >> 2) * kSubTileBytes + (ks & 3) * 32) >> 4;
-                        mma_ss(tmem + b * 128 + hh * 64, qd + off, kd + off, idesc_qk64, ks > 0);
+                        mma_ss(tmem + b * 128, qd + off, kd + off, idesc_qk, ks > 0);
                     }
-                    tc_commit(B.s_full(2 * b + hh));
-                    if (b == 1 && hh == 1) tc_commit(B.k_empty(st));          // last use of the tile
+                    tc_commit(B.s_full(b));
+                    if (b == 1) tc_commit(B.k_empty(st));                     // last use of the tile
                     return true;
                 };
-                for (int m = 0; m < 4 && m < n_half_jobs && ok; ++m) ok = issue_qk64(m);
+                for (int m = 0; m < 2 && m < n_jobs && ok; ++m) ok = issue_qk2(m);
                 #pragma unroll 1
-                for (int n = 0; n < n_half_jobs && ok; ++n) {
-                    const int h = n >> 1, b = n & 1, hh = h & 1, j = h >> 1, st = j % NS;
-                    if (b == 0 && hh == 0 && !mbar_wait(B.v_full(st), (j / NS) & 1)) { ok = false; break; }
-                    if (!mbar_wait(B.p_full(2 * b + hh), j & 1)) { ok = false; break; }
+                for (int n = 0; n < n_jobs && ok; ++n) {
+                    const int j = n >> 1, b = n & 1, st = j % NS;
+                    if (b == 0 && !mbar_wait(B.v_full(st), (j / NS) & 1)) { ok = false; break; }
+                    if (!mbar_wait(B.p_full(b), j & 1)) { ok = false; break; }
                     tc_fence_after();
                     const uint64_t vd = v_desc0 + (uint64_t)((st * kStageBytes) >> 4);
                     #pragma unroll
-                    for (int i = 0; i < 4; ++i)                               // keys [64 hh + 16 i, + 16) of the tile
-                        mma_ts(tmem + 256 + b * 128, tmem + b * 128 + hh * 64 + 32 + i * 8,
-                               vd + (uint64_t)(((4 * hh + i) * 2048) >> 4), idesc_pv, (h > 0 || i > 0) ? 1u : 0u);
-                    tc_commit(B.o_done(b, h));
-                    if (b == 1 && hh == 1) tc_commit(B.v_empty(st));
-                    if (n + 4 < n_half_jobs) ok = issue_qk64(n + 4);          // the slot this job's scores were in
+                    for (int kk = 0; kk < 8; ++kk)
+                        mma_ts(tmem + 256 + b * 128, tmem + b * 128 + 64 + kk * 8, vd + (uint64_t)((kk * 2048) >> 4),
+                               idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);
+                    tc_commit(B.o_done(b, j));
+                    if (b == 1) tc_commit(B.v_empty(st));
+                    if (n + 2 < n_jobs) ok = issue_qk2(n + 2);                // this block's next scores
                 }
             } else {
             constexpr uint32_t idesc_qk = idesc_bf16(false);
@@ -603,40 +601,43 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
             // through the block's half-tile jobs on its own -- no exchange with the other warpgroup,
             // whose exponentials fill the gaps this one leaves while it waits for the tensor pipe.
             const int blk = wg;
-            const int n_half = 2 * n_tiles;
             // this warpgroup's block, in scalars (indexing the per-block arrays with wg would put them in local memory)
             const unsigned long long my_anc = wg ? anc[NB - 1] : anc[0];
             const int my_lo = wg ? lo_row[NB - 1] : lo_row[0];
             const bool my_ok = wg ? row_ok[NB - 1] : row_ok[0];
+            const uint32_t s_addr = lane_addr + blk * 128;
+            // visibility word of this row for the 64 keys that start at key j0
+            auto vis_word = [&](int j0) -> unsigned long long {
+                if (!(j0 + 64 > it.key_end || j0 + 64 > kv_len || j0 < my_lo)) return ~0ull;
+                const int d0 = kv_len - j0;                                 // column of draft token 0 (any sign)
+                const int nval = it.key_end - j0;                           // valid columns (may be <= 0)
+                unsigned long long vis;
+                if (d0 >= 64) vis = ~0ull;
+                else if (d0 > 0) vis = ((1ull << d0) - 1ull) | (my_anc << d0);
+                else if (d0 > -64) vis = my_anc >> (-d0);
+                else vis = 0ull;
+                if (nval <= 0) vis = 0ull;
+                else if (nval < 64) vis &= (1ull << nval) - 1ull;
+                const int cut = my_lo - j0;
+                if (cut >= 64) vis = 0ull;
+                else if (cut > 0) vis &= ~((1ull << cut) - 1ull);
+                return vis;
+            };
             float x0[32], x1[32];
             #pragma unroll 1
-            for (int h = 0; h < n_half && ok; ++h) {
-                const int hh = h & 1, j = h >> 1, st = j % NS;
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                const int st = j % NS;
                 const int tile0 = it.key_begin + j * kTile;
-                const int j0 = tile0 + 64 * hh;                      // first key of this half-tile
-                const uint32_t s_addr = lane_addr + blk * 128 + hh * 64;
-                if (!mbar_wait_warp(B.s_full(2 * blk + hh), j & 1)) { ok = false; break; }
+                if (!mbar_wait_warp(B.s_full(blk), j & 1)) { ok = false; break; }
                 tc_fence_after();
+                // first pass over the row's 128 scores, 64 at a time: the maximum.  The upper 64 stay
+                // in registers; the lower 64 are fetched again for the second pass.
                 tmem_ld32(s_addr, x0);
                 tmem_ld32(s_addr + 32, x1);
-                const bool boundary = j0 + 64 > it.key_end || j0 + 64 > kv_len || j0 < my_lo;
-                unsigned long long vis = ~0ull;
-                if (boundary) {
-                    const int d0 = kv_len - j0;                             // column of draft token 0 (any sign)
-                    const int nval = it.key_end - j0;                       // valid columns (may be <= 0)
-                    if (d0 >= 64) vis = ~0ull;
-                    else if (d0 > 0) vis = ((1ull << d0) - 1ull) | (my_anc << d0);
-                    else if (d0 > -64) vis = my_anc >> (-d0);
-                    else vis = 0ull;
-                    if (nval <= 0) vis = 0ull;
-                    else if (nval < 64) vis &= (1ull << nval) - 1ull;
-                    const int cut = my_lo - j0;
-                    if (cut >= 64) vis = 0ull;
-                    else if (cut > 0) vis &= ~((1ull << cut) - 1ull);
-                }
+                const unsigned long long vis_lo = vis_word(tile0), vis_hi = vis_word(tile0 + 64);
                 // V rows past the end of the sequence may hold anything: zero them so 0 * x stays 0
                 // (once per tile, by the threads of the first block, thread r taking key row r)
-                if (blk == 0 && hh == 0 && tile0 + kTile > n_keys_seq && tile0 + row_local >= n_keys_seq) {
+                if (blk == 0 && tile0 + kTile > n_keys_seq && tile0 + row_local >= n_keys_seq) {
                     mbar_wait(B.v_full(st), (j / NS) & 1);
                     unsigned char* vrow = kv_sm + st * kStageBytes + 2 * kSubTileBytes + row_local * 128;
                     #pragma unroll
@@ -647,8 +648,13 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                     fence_proxy_async();
                 }
                 tmem_wait_ld();
-                if (boundary) { mask_chunk(x0, (uint32_t)vis); mask_chunk(x1, (uint32_t)(vis >> 32)); }
-                const float mx = fmaxf(chunk_max(x0), chunk_max(x1));
+                if (vis_lo != ~0ull) { mask_chunk(x0, (uint32_t)vis_lo); mask_chunk(x1, (uint32_t)(vis_lo >> 32)); }
+                float mx = fmaxf(chunk_max(x0), chunk_max(x1));
+                tmem_ld32(s_addr + 64, x0);
+                tmem_ld32(s_addr + 96, x1);
+                tmem_wait_ld();
+                if (vis_hi != ~0ull) { mask_chunk(x0, (uint32_t)vis_hi); mask_chunk(x1, (uint32_t)(vis_hi >> 32)); }
+                mx = fmaxf(mx, fmaxf(chunk_max(x0), chunk_max(x1)));
                 // lazy reference maximum, per row; the accumulator is rescaled by the whole warp (the
                 // TMEM accesses are warp-wide) whenever one of its rows moved
                 const bool need = my_ok && (mx > my_m + thr || (my_m == -INFINITY && mx > -INFINITY));
@@ -659,8 +665,8 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                         my_m = mx;
                         my_l *= alpha;
                     }
-                    if (h > 0) {                                            // O holds earlier half-tiles
-                        if (!mbar_wait_warp(B.o_done(blk, h - 1), ((h - 1) >> 2) & 1)) { ok = false; break; }
+                    if (j > 0) {                                            // O holds earlier tiles
+                        if (!mbar_wait_warp(B.o_done(blk, j - 1), ((j - 1) >> 2) & 1)) { ok = false; break; }
                         tc_fence_after();
                         const uint32_t o_addr = lane_addr + kOCol + blk * 128;
                         #pragma unroll 1
@@ -675,15 +681,23 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                         tmem_wait_st();
                     }
                 }
-                // p = 2^(s c2 - m c2), row sum from the unrounded p, P (bf16) over the slot's upper half
+                // second pass: p = 2^(s c2 - m c2), row sum from the unrounded p, P (bf16) over the upper
+                // half of the score block -- first the upper 64 keys (their scores are in registers and
+                // their columns are the ones P overwrites), then the lower 64, fetched again
                 const float mc = (my_m == -INFINITY) ? 0.f : my_m * c2;
                 float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-                exp_chunk(x0, c2, mc, sum4, s_addr + 32);
-                exp_chunk(x1, c2, mc, sum4, s_addr + 48);
+                exp_chunk(x0, c2, mc, sum4, s_addr + 64 + 32);
+                exp_chunk(x1, c2, mc, sum4, s_addr + 64 + 48);
+                tmem_ld32(s_addr, x0);
+                tmem_ld32(s_addr + 32, x1);
+                tmem_wait_ld();
+                if (vis_lo != ~0ull) { mask_chunk(x0, (uint32_t)vis_lo); mask_chunk(x1, (uint32_t)(vis_lo >> 32)); }
+                exp_chunk(x0, c2, mc, sum4, s_addr + 64);
+                exp_chunk(x1, c2, mc, sum4, s_addr + 64 + 16);
                 my_l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
                 tmem_wait_st();                                            // this job's P is in TMEM
                 tc_fence_before();
-                mbar_arrive(B.p_full(2 * blk + hh));
+                mbar_arrive(B.p_full(blk));
             }
         } else {
         // The scores of a job are requested from TMEM at the end of the job before it, ahead of the
@@ -827,7 +841,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
         }
         #pragma unroll
         for (int blk = 0; blk < NB; ++blk) {
-            const int last_product = NB == 2 ? 2 * n_tiles - 1 : n_tiles - 1;
+            const int last_product = n_tiles - 1;
             if (ok) ok = mbar_wait_warp(B.o_done(blk, last_product), (last_product >> 2) & 1);    // the last product is in
             tc_fence_after();
             float inv, lse_val;
@@ -903,7 +917,6 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
         if (sync.enabled || sync.serial) {
             const int fin_idx = (int)blockIdx.x - (plan.n_items - sync.n_fin);     // >= 0: this CTA is a finisher
             constexpr int kRowsPerBlock = kTokPerBlock * kGroup;       // 126
-            constexpr int kRowBytes = kPartRowHalves * 2;              // 272
             // The call's row list: for every unit (sequence, KV head, row group) with several pieces,
             // its valid query rows (7 per draft token).  Finisher f takes rows [f chunk, (f + 1) chunk).
             int total = 0;
@@ -919,38 +932,41 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                 if (!direct) publish_counter(arrive_word);
                 if (merges) {
                     // every partial of the call in place, and (overlapped mode) the previous call's final results written
-                    bool go = wait_equal(arrive_word, (unsigned)sync.n_arrive);
-                    if (!go) atomicOr(args.status, timeout_bits(kSiteArrivals));
-                    if (go && sync.enabled) {
-                        go = wait_counter(sync.fin_done + (sync.parity ^ 1), sync.fin_wait_other);
-                        if (!go) atomicOr(args.status, timeout_bits(kSiteFinOther));
+                    // (both words are polled in one loop: the second is usually there already)
+                    bool have_all = false, prev_done = !sync.enabled;
+                    #pragma unroll 1
+                    for (uint32_t i = 0; i < kCounterPolls && !(have_all && prev_done); ++i) {
+                        if (!have_all) have_all = ld_acquire(arrive_word) == (unsigned)sync.n_arrive;
+                        if (!prev_done) prev_done = (int32_t)(ld_acquire(sync.fin_done + (sync.parity ^ 1)) - sync.fin_wait_other) >= 0;
+                        if (!(have_all && prev_done)) __nanosleep(i < 256 ? 20 : 200);
                     }
-                    *fin_go = go ? 1 : 0;
+                    if (!have_all) atomicOr(args.status, timeout_bits(kSiteArrivals));
+                    else if (!prev_done) atomicOr(args.status, timeout_bits(kSiteFinOther));
+                    *fin_go = (have_all && prev_done) ? 1 : 0;
                 }
             }
             if (merges) {
                 softmax_bar_sync();
                 if (*fin_go) {
-                    // Per unit, the pieces' rows are copied into the (idle) K/V ring in bulk -- per piece
-                    // one copy per block touched, one memory round trip for a whole batch of R rows --
-                    // and merged from there by 16 R G threads: thread (row i, 16-byte chunk c, piece
-                    // group g) takes pieces g, g + G, ...; the groups' partial maxima, sums and weighted
-                    // outputs meet in shared memory (the Q blocks, idle by now).
-                    float* red = reinterpret_cast<float*>(q_sm);                // [256][9] partial sums, then [256] maxima
-                    float* red_max = red + 256 * 9;
-                    bool fin_ok = true;
-                    int phase = 0, ubase = 0;
+                    // 16 R G threads merge R rows at a time: thread (row i, 16-byte chunk c, piece group
+                    // g) takes pieces g, g + G, ... of its row, read straight from the workspace (L2;
+                    // thread 0's acquire and the barrier above order these loads behind the pieces'
+                    // stores), ten pieces in flight at a time (one round trip to L2 for a one-wave call), folding them into a running
+                    // (max, sum, weighted output); the groups' results meet in shared memory (the Q
+                    // blocks, idle by now).
+                    constexpr int kFold = 10;                                   // pieces a thread has in flight
+                    float* red = reinterpret_cast<float*>(q_sm);                // [256][10]: 8 outputs, sum, max
+                    int ubase = 0;
                     #pragma unroll 1
                     for (int b = 0; b < plan.batch; ++b) {
                         const int ns = plan.seq[b].n_splits;
                         if (ns == 1) continue;
-                        // rows per batch: a power of two, no more than this finisher has, than fit the ring
-                        // with all their pieces, or than 16
+                        // rows per pass: a power of two, no more than this finisher has, or than 16
                         int R = 1;
                         while (R < 16 && R < chunk) R <<= 1;
-                        while (R > 1 && R * ns * kRowBytes > NS * kStageBytes) R >>= 1;
                         const int G = 16 / R;                                   // piece groups
                         const int c16 = tid & 15, grp_p = (tid >> 4) % G, row_i = tid / (16 * G);
+                        const size_t piece_pitch = (size_t)plan.part_rows * kPartRowHalves;      // halves between pieces
                         #pragma unroll 1
                         for (int u = 0; u < plan.n_kv_heads * plan.n_groups; ++u) {
                             const int kvh = u / plan.n_groups, grp = u - kvh * plan.n_groups;
@@ -961,90 +977,85 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                             if (row_begin >= row_end) continue;                    // (the same in every thread of the CTA)
                             const size_t item0 = (size_t)plan.seq[b].item_begin + (size_t)u * ns;
                             #pragma unroll 1
-                            for (int r0 = row_begin; r0 < row_end; r0 += R, phase ^= 1) {
-                                const int n_here = min(R, row_end - r0);
-                                // the batch may straddle the two blocks: rows [r0, split) and [split, r0 + n_here)
-                                const int split = (r0 < kRowsPerBlock && r0 + n_here > kRowsPerBlock) ? kRowsPerBlock : r0 + n_here;
-                                if (tid == 0) mbar_expect_tx(B.fin(), (uint32_t)(n_here * ns * kRowBytes));
-                                softmax_bar_sync();                                // previous batch consumed, byte count posted
-                                // the partial rows were written with ordinary stores; the bulk copies read them through the async proxy
-                                if (tid < ns) fence_proxy_async_global();
-                                for (int sp = tid; sp < ns; sp += 256) {           // shared memory: [piece][row of the batch][272 bytes]
-                                    const __half* piece = args.o_part + (item0 + sp) * plan.part_rows * kPartRowHalves;
-                                    const uint32_t dst = smem_u32(kv_sm + (size_t)sp * n_here * kRowBytes);
-                                    const int bk0 = r0 / kRowsPerBlock;
-                                    bulk_load(dst, piece + (size_t)(bk0 * kBlockRows + r0 - bk0 * kRowsPerBlock) * kPartRowHalves,
-                                              (uint32_t)(split - r0) * kRowBytes, B.fin());
-                                    if (split < r0 + n_here)
-                                        bulk_load(dst + (uint32_t)(split - r0) * kRowBytes, piece + (size_t)kBlockRows * kPartRowHalves,
-                                                  (uint32_t)(r0 + n_here - split) * kRowBytes, B.fin());
-                                }
-                                fin_ok = fin_ok && mbar_wait_warp(B.fin(), phase);
-                                const bool active = fin_ok && row_i < n_here;
-                                const uint32_t pstride = (uint32_t)n_here * kRowBytes;     // bytes between pieces
-                                const uint32_t row_sm = smem_u32(kv_sm) + (uint32_t)row_i * kRowBytes;
-                                // pass 1: the row's largest piece LSE
-                                float mxl = -INFINITY;
-                                if (active) {
-                                    #pragma unroll 4
-                                    for (uint32_t sp = grp_p, a_l = row_sm + 2 * kD + grp_p * pstride; sp < (uint32_t)ns; sp += G, a_l += G * pstride)
-                                        mxl = fmaxf(mxl, lds_f32(a_l));
-                                }
-                                if (G > 1) {
-                                    red_max[tid] = mxl;
-                                    softmax_bar_sync();
-                                    const int base = tid - grp_p * 16;
-                                    for (int g2 = 0; g2 < G; ++g2) mxl = fmaxf(mxl, red_max[base + g2 * 16]);
-                                }
-                                // pass 2: weights exp(lse_s - max), their sum, the weighted outputs of this thread's 8 dims
-                                const bool any = mxl != -INFINITY;
-                                const float mx2 = any ? mxl * 1.4426950408889634f : 0.f;
+                            for (int r0 = row_begin; r0 < row_end; r0 += R) {
+                                const int idx = r0 + row_i;                            // row of the unit's list: token idx / 7, head idx % 7
+                                const bool active = idx < row_end;
+                                const int bk = idx / kRowsPerBlock;
+                                const __half* row0 = args.o_part + (item0 * plan.part_rows + (size_t)(bk * kBlockRows + idx - bk * kRowsPerBlock)) * kPartRowHalves;
+                                float m_run = -INFINITY, s_run = 0.f;                  // natural-log units
                                 float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-                                float suml = 0.f;
                                 if (active) {
-                                    #pragma unroll 4
-                                    for (uint32_t sp = grp_p, a_l = row_sm + 2 * kD + grp_p * pstride, a_o = row_sm + c16 * 16 + grp_p * pstride;
-                                         sp < (uint32_t)ns; sp += G, a_l += G * pstride, a_o += G * pstride) {
-                                        const float ws = ex2(fmaf(lds_f32(a_l), 1.4426950408889634f, -mx2));   // exp(lse_s - max); 0 for -inf
-                                        uint32_t raw[4];
-                                        lds_v4(a_o, raw);
-                                        suml += ws;
+                                    #pragma unroll 1
+                                    for (int sp0 = grp_p; sp0 < ns; sp0 += kFold * G) {
+                                        float l4[kFold];
+                                        uint4 o4[kFold];
                                         #pragma unroll
-                                        for (int q = 0; q < 4; ++q) {
-                                            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&raw[q]));
-                                            acc[2 * q] = fmaf(ws, f.x, acc[2 * q]); acc[2 * q + 1] = fmaf(ws, f.y, acc[2 * q + 1]);
+                                        for (int k = 0; k < kFold; ++k) {
+                                            const int sp = sp0 + k * G;
+                                            l4[k] = -INFINITY;
+                                            o4[k] = make_uint4(0, 0, 0, 0);
+                                            if (sp < ns) {
+                                                const __half* pr = row0 + (size_t)sp * piece_pitch;
+                                                l4[k] = __ldcg(reinterpret_cast<const float*>(pr + kD));
+                                                o4[k] = __ldcg(reinterpret_cast<const uint4*>(pr) + c16);
+                                            }
+                                        }
+                                        #pragma unroll
+                                        for (int k = 0; k < kFold; ++k) {
+                                            if (l4[k] == -INFINITY) continue;          // a piece that saw no visible key (or none at all)
+                                            const float m_new = fmaxf(m_run, l4[k]);
+                                            const float a = ex2((m_run - m_new) * 1.4426950408889634f);   // 0 for the first piece
+                                            const float w = ex2((l4[k] - m_new) * 1.4426950408889634f);
+                                            const uint32_t* raw = reinterpret_cast<const uint32_t*>(&o4[k]);
+                                            s_run = fmaf(s_run, a, w);
+                                            #pragma unroll
+                                            for (int q = 0; q < 4; ++q) {
+                                                const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&raw[q]));
+                                                acc[2 * q] = fmaf(acc[2 * q], a, w * f.x); acc[2 * q + 1] = fmaf(acc[2 * q + 1], a, w * f.y);
+                                            }
+                                            m_run = m_new;
                                         }
                                     }
                                 }
-                                if (G > 1) {
+                                if (G > 1) {                                           // (G is the same in every thread)
+                                    softmax_bar_sync();                                // the pass before has been read
                                     #pragma unroll
-                                    for (int q = 0; q < 8; ++q) red[tid * 9 + q] = acc[q];
-                                    red[tid * 9 + 8] = suml;
+                                    for (int q = 0; q < 8; ++q) red[tid * 10 + q] = acc[q];
+                                    red[tid * 10 + 8] = s_run;
+                                    red[tid * 10 + 9] = m_run;
                                     softmax_bar_sync();
                                     if (grp_p == 0) {
+                                        const float* mine = red + tid * 10;
+                                        float m_all = m_run;
+                                        for (int g2 = 1; g2 < G; ++g2) m_all = fmaxf(m_all, mine[g2 * 160 + 9]);
+                                        const float a0 = m_run == -INFINITY ? 0.f : ex2((m_run - m_all) * 1.4426950408889634f);
+                                        s_run *= a0;
+                                        #pragma unroll
+                                        for (int q = 0; q < 8; ++q) acc[q] *= a0;
                                         for (int g2 = 1; g2 < G; ++g2) {
-                                            const float* o = red + (tid + g2 * 16) * 9;
+                                            const float* o = mine + g2 * 160;
+                                            if (o[9] == -INFINITY) continue;
+                                            const float ag = ex2((o[9] - m_all) * 1.4426950408889634f);
+                                            s_run = fmaf(o[8], ag, s_run);
                                             #pragma unroll
-                                            for (int q = 0; q < 8; ++q) acc[q] += o[q];
-                                            suml += o[8];
+                                            for (int q = 0; q < 8; ++q) acc[q] = fmaf(o[q], ag, acc[q]);
                                         }
+                                        m_run = m_all;
                                     }
                                 }
                                 if (active && grp_p == 0) {
-                                    const int idx = r0 + row_i;                            // row of the unit's list: token idx / 7, head idx % 7
                                     const int t = tok0 + idx / kGroup;
                                     const int h = kvh * kGroup + idx % kGroup;
-                                    const float inv = suml > 0.f ? __fdividef(1.f, suml) : 0.f;
+                                    const float inv = s_run > 0.f ? __fdividef(1.f, s_run) : 0.f;
                                     uint4 pk;
                                     pk.x = pack_bf16x2(acc[0] * inv, acc[1] * inv); pk.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
                                     pk.z = pack_bf16x2(acc[4] * inv, acc[5] * inv); pk.w = pack_bf16x2(acc[6] * inv, acc[7] * inv);
                                     *reinterpret_cast<uint4*>(args.out + (((size_t)b * T + t) * args.n_q_heads + h) * kD + c16 * 8) = pk;
-                                    if (c16 == 0) args.lse[((size_t)b * args.n_q_heads + h) * T + t] = any ? mxl + __logf(suml) : -INFINITY;
+                                    if (c16 == 0) args.lse[((size_t)b * args.n_q_heads + h) * T + t] = s_run > 0.f ? m_run + __logf(s_run) : -INFINITY;
                                 }
                             }
                         }
                     }
-                    if (!fin_ok) atomicOr(args.status, timeout_bits(kSiteFinCopies));
                 }
                 softmax_bar_sync();
             }

@@ -1,0 +1,104 @@
+"""GPU parity of the hidden-state reuse projection z = FC(e (+) h) (Eq. 1) against the float64
+oracle.  Tolerance: fp32 accumulation of bf16 products over 2 d terms (error ~1e-6 relative to the
+accumulated magnitude) and one rounding of z to bf16 (2^-9 |z|); with weights scaled so that
+|z| stays below about 4, max |dz| <= 2e-2 holds with a wide margin and is what is asserted, together
+with the relative bound 2^-8 |z| + 1e-3 element by element."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2602_15318_b200 import binding as B
+from paper_2602_15318_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _case(seed, M, d, d_out, bias=True):
+    e = W.normal_bf16(seed, 61, (M, d), DEV)
+    h = W.normal_bf16(seed, 62, (M, d), DEV)
+    w = (W.normal_bf16(seed, 63, (d_out, 2 * d), DEV).float() / (2 * d) ** 0.5).to(torch.bfloat16)
+    b = W.normal_bf16(seed, 64, (d_out,), DEV) if bias else None
+    return e, h, w, b
+
+
+def _ctx():
+    k = torch.empty((1, W.HKV, 128, W.D), dtype=torch.bfloat16, device=DEV)
+    return B.Context.for_cache(k, W.SCALE)
+
+
+def _run(ctx, e, h, w, b):
+    M, d = e.shape
+    d_out = w.shape[0]
+    n = B.sparrow_hsr_scratch_bytes(ctx, d, d_out)
+    scratch = torch.empty(max(n, 16), dtype=torch.uint8, device=DEV)
+    z = torch.full((M, d_out), float("nan"), dtype=torch.bfloat16, device=DEV)
+    B.sparrow_hsr_fuse(ctx, e, h, w, b, z, scratch)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == 0
+    return z
+
+
+def _check(z, e, h, w, b):
+    ref = oracle.hsr_fuse(W.bf16_bits(e), W.bf16_bits(h), W.bf16_bits(w), W.bf16_bits(b) if b is not None else None)
+    got = z.double().cpu().numpy()
+    assert not np.isnan(got).any()
+    err = np.abs(got - ref)
+    assert float(err.max()) <= 2e-2
+    assert np.all(err <= 2.0 ** -8 * np.abs(ref) + 1e-3)
+
+
+@pytest.mark.parametrize("M,d,d_out,bias", [
+    (1, 64, 128, True),            # smallest shape: one feature tile, two K tiles
+    (8, 3584, 3584, True),         # one drafting step of a Qwen2-7B-shaped model (28 feature tiles x 5 K slices)
+    (48, 3584, 3584, False),       # a 48-node tree, no bias
+    (64, 3584, 3584, True),
+    (30, 1536, 1536, True),        # a smaller model: 12 feature tiles, 12 slices
+    (5, 128, 24576, True),         # more feature tiles than SMs: one slice each, no partial sums
+    (17, 4096, 512, True),         # few feature tiles, long K slices
+])
+def test_hsr_fuse_matches_the_oracle(M, d, d_out, bias):
+    e, h, w, b = _case(7000 + M + d, M, d, d_out, bias)
+    ctx = _ctx()
+    _check(_run(ctx, e, h, w, b), e, h, w, b)
+
+
+def test_hsr_fuse_repeats_bit_for_bit_and_keeps_its_counters_clean():
+    e, h, w, b = _case(7100, 25, 3584, 3584)
+    ctx = _ctx()
+    first = _run(ctx, e, h, w, b)
+    for _ in range(5):
+        assert torch.equal(_run(ctx, e, h, w, b), first)
+    e2, h2, w2, b2 = _case(7101, 3, 256, 1024)
+    _check(_run(ctx, e2, h2, w2, b2), e2, h2, w2, b2)          # other shape, same context
+    _check(_run(ctx, e, h, w, b), e, h, w, b)
+
+
+def test_hsr_fuse_selector_weights():
+    """W = [I | 0] copies e, W = [0 | I] copies h: the two halves of the K range are taken from the
+    right inputs, bit for bit."""
+    M, d = 7, 256
+    e = W.normal_bf16(7200, 61, (M, d), DEV)
+    h = W.normal_bf16(7200, 62, (M, d), DEV)
+    eye, zero = torch.eye(d, dtype=torch.bfloat16, device=DEV), torch.zeros((d, d), dtype=torch.bfloat16, device=DEV)
+    ctx = _ctx()
+    assert torch.equal(_run(ctx, e, h, torch.cat([eye, zero], 1).contiguous(), None), e)
+    assert torch.equal(_run(ctx, e, h, torch.cat([zero, eye], 1).contiguous(), None), h)
+
+
+def test_hsr_fuse_argument_errors():
+    e, h, w, b = _case(7300, 4, 128, 256)
+    ctx = _ctx()
+    z = torch.empty((4, 256), dtype=torch.bfloat16, device=DEV)
+    n0 = ctx.launch_count()
+    L = B.lib()
+    for M, d, d_out, status in ((0, 128, 256, 2), (65, 128, 256, 2), (4, 100, 256, 2), (4, 128, 200, 2)):
+        assert L.sparrow_hsr_fuse(ctx.handle, e.data_ptr(), h.data_ptr(), w.data_ptr(), None, M, d, d_out, None, 0,
+                                  z.data_ptr(), None) == status
+    assert L.sparrow_hsr_fuse(ctx.handle, None, h.data_ptr(), w.data_ptr(), None, 4, 128, 256, None, 0, z.data_ptr(), None) == 1
+    e2, h2, w2, b2 = _case(7301, 4, 3584, 3584)
+    z2 = torch.empty((4, 3584), dtype=torch.bfloat16, device=DEV)
+    assert L.sparrow_hsr_fuse(ctx.handle, e2.data_ptr(), h2.data_ptr(), w2.data_ptr(), None, 4, 3584, 3584, None, 0,
+                              z2.data_ptr(), None) == 5          # split-K partials need scratch
+    assert ctx.launch_count() == n0
