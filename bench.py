@@ -242,7 +242,7 @@ def main():
                     help="skip the other configurations (C1, C3, C4, C5), which are otherwise timed and "
                          "reported under other_configs in the same JSON line")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--only", choices=["C1", "C2", "C3", "C5"],
+    ap.add_argument("--only", choices=["C1", "C2", "C3", "C5", "HSR"],
                     help="time just this configuration's stream of calls (a small run for a profiler capture): "
                          "--steps calls after --warmup calls under --policy, one JSON line")
     ap.add_argument("--policy", choices=["latency", "balanced", "throughput"], default="throughput")
@@ -460,6 +460,30 @@ def main():
 
 def run_only(args, W, B, torch, dev, l2, steps, warmup):
     """One configuration, one policy, few calls: what a profiler capture runs."""
+    if args.only == "HSR":
+        d_model, m_tok, n_w = 3584, 48, 12
+        ws_ = [(W.normal_bf16(W.config_seed(5, r), 63, (d_model, 2 * d_model), dev).float() / (2 * d_model) ** 0.5).to(torch.bfloat16)
+               for r in range(n_w)]
+        e_ = W.normal_bf16(W.config_seed(5), 61, (m_tok, d_model), dev)
+        h_ = W.normal_bf16(W.config_seed(5), 62, (m_tok, d_model), dev)
+        z_ = torch.empty((m_tok, d_model), dtype=torch.bfloat16, device=dev)
+        hctx = B.Context.for_cache(torch.empty((1, W.HKV, 128, W.D), dtype=torch.bfloat16, device=dev), W.SCALE)
+        scratch = torch.empty(max(16, B.sparrow_hsr_scratch_bytes(hctx, d_model, d_model)), dtype=torch.uint8, device=dev)
+
+        def run(n):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize(); e0.record()
+            for i in range(n):
+                B.sparrow_hsr_fuse(hctx, e_, h_, ws_[i % n_w], None, z_, scratch)
+            e1.record(); torch.cuda.synchronize()
+            return e0.elapsed_time(e1) * 1e3 / n
+        run(warmup)
+        us = run(steps)
+        by = d_model * 2 * d_model * 2 + 3 * m_tok * d_model * 2
+        print(json.dumps({"only": "HSR", "workload": f"z = FC(e (+) h), {m_tok} tokens, d = {d_model}", "steps": steps, "warmup": warmup,
+                          "us_per_call_from_python": us, "algorithmic_bytes_per_call": by, "rotation": n_w,
+                          "device_status": hctx.last_device_status()}), flush=True)
+        return
     ci = {"C1": 0, "C2": 1, "C3": 2, "C5": 4}[args.only]
     probe = W.make_config(ci, "cpu")
     n_caches = 3 if ci == 4 else max(4, -(-4 * l2 // probe.kv_bytes()))
@@ -594,6 +618,43 @@ def extra_configs(W, B, torch, dev, l2, peak, peaks, anchored_variants):
               "us_per_call": ev0.elapsed_time(ev1) * 1e3 / 3000, "note": "launched from Python; latency-bound"})
         del tc_, tctx
     del ac, actx
+    torch.cuda.empty_cache()
+    # Draft-model input fusion z = FC(e (+) h) (Eq. 1) at a Qwen2-7B-like width: a weight-streaming GEMM,
+    # rotated over enough weight matrices to stay out of L2, replayed from a CUDA graph (the call
+    # encodes three tensor maps on the host, which a per-call launch loop would be timing instead)
+    d_model, m_tok = 3584, 48
+    n_w = max(4, -(-4 * l2 // (d_model * 2 * d_model * 2)))
+    ws_ = [(W.normal_bf16(W.config_seed(5, r), 63, (d_model, 2 * d_model), dev).float() / (2 * d_model) ** 0.5).to(torch.bfloat16)
+           for r in range(n_w)]
+    e_ = W.normal_bf16(W.config_seed(5), 61, (m_tok, d_model), dev)
+    h_ = W.normal_bf16(W.config_seed(5), 62, (m_tok, d_model), dev)
+    b_ = W.normal_bf16(W.config_seed(5), 64, (d_model,), dev)
+    z_ = torch.empty((m_tok, d_model), dtype=torch.bfloat16, device=dev)
+    hk = torch.empty((1, W.HKV, 128, W.D), dtype=torch.bfloat16, device=dev)
+    hctx = B.Context.for_cache(hk, W.SCALE)
+    scratch = torch.empty(max(16, B.sparrow_hsr_scratch_bytes(hctx, d_model, d_model)), dtype=torch.uint8, device=dev)
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        for w_ in ws_:
+            B.sparrow_hsr_fuse(hctx, e_, h_, w_, b_, z_, scratch, stream=side)
+        side.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            for w_ in ws_:
+                B.sparrow_hsr_fuse(hctx, e_, h_, w_, b_, z_, scratch, stream=side)
+        graph.replay(); side.synchronize()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record(side)
+        for _ in range(100):
+            graph.replay()
+        g1.record(side); side.synchronize()
+    us = g0.elapsed_time(g1) * 1e3 / (100 * n_w)
+    by = d_model * 2 * d_model * 2 + 2 * m_tok * d_model * 2 + d_model * 2 + m_tok * d_model * 2
+    emit({"config": "HSR", "workload": f"z = FC(e (+) h), {m_tok} tokens, d = {d_model} (weights {d_model} x {2 * d_model} bf16)",
+          "us_per_call": us, "algorithmic_bytes": by, "hbm_gbs": by / us / 1e3, "frac_of_measured_hbm": by / us / 1e3 / peak,
+          "rotation": n_w, "device_status": hctx.last_device_status(),
+          "note": "rotation over weight matrices larger than 4 x L2, calls replayed from a CUDA graph"})
+    del graph, ws_, hctx
     torch.cuda.empty_cache()
     # C5: 28 layers, each with its own cache (about 15 GB resident)
     layers = [W.make_config(4, dev, layer=l) for l in range(28)]

@@ -16,9 +16,10 @@
  * sparrow_kv_keep_accepted() (acceptance of the draft tree at temperature 0 and 1, and the move of
  * the accepted rows).
  *
- * For every batch entry b, query head h (KV head h / 7), draft token t and visible key set Vis:
- *     s_j = softmax_scale * <q[b,t,h,:], k[b,h/7,j,:]>,   lse = log sum_{j in Vis} exp(s_j),
- *     out = sum_{j in Vis} exp(s_j - lse) * v[b,h/7,j,:].
+ * For every batch entry b, query head h (KV head h / g, g = n_q_heads / n_kv_heads query heads
+ * per KV head; g = 7 for the paper's Qwen2-7B-shaped targets), draft token t and visible key set Vis:
+ *     s_j = softmax_scale * <q[b,t,h,:], k[b,h/g,j,:]>,   lse = log sum_{j in Vis} exp(s_j),
+ *     out = sum_{j in Vis} exp(s_j - lse) * v[b,h/g,j,:].
  *
  * Conventions
  *   - Every function returns a sparrow_status; nothing aborts or throws.  Argument errors are
@@ -57,14 +58,14 @@ typedef enum {
 #define SPARROW_MAX_T      64   /* draft tokens per sequence (one 64-bit ancestor word per token) */
 #define SPARROW_MAX_BATCH  64   /* sequences per call */
 #define SPARROW_HEAD_DIM   128  /* only value accepted */
-#define SPARROW_GQA_GROUP  7    /* query heads per KV head; only value accepted */
+#define SPARROW_MAX_GQA_GROUP 16 /* query heads per KV head: 1 .. 16 (7 for the paper's Qwen2-7B-shaped targets) */
 
 /* Fixed per context.  K/V buffers hold, for batch b and KV head g, `kv_capacity` rows of 128 bf16:
  * element offset of (b, g, row, d) = b*kv_stride_batch + g*kv_stride_head + row*128 + d.
  * Both strides must be multiples of 8 elements and the base pointers 16-byte aligned. */
 typedef struct {
     int32_t batch;           /* 1 .. SPARROW_MAX_BATCH */
-    int32_t n_q_heads;       /* must equal 7 * n_kv_heads */
+    int32_t n_q_heads;       /* g * n_kv_heads, 1 <= g <= SPARROW_MAX_GQA_GROUP */
     int32_t n_kv_heads;
     int32_t head_dim;        /* must be 128 */
     int32_t kv_capacity;     /* rows per (batch, KV head) */
@@ -421,13 +422,14 @@ sparrow_status sparrow_debug_ancestor_masks_device(sparrow_ctx* ctx, const int32
                                                    int32_t T, uint64_t* masks_dev, void* stream);
 
 /* Host-side split schedule, exported for inspection (pure host code, needs no GPU): for `batch`
- * sequences of n_keys[b] keys, draft blocks of T tokens and a target of n_sm work items (the SM
+ * sequences of n_keys[b] keys, gqa_group query heads per KV head, draft blocks of T tokens and a
+ * target of n_sm work items (the SM
  * count, or sparrow_plan_target_items() for calls in fused mode), writes
  * splits_out[b] = key-range pieces per (sequence, KV head, row group) and the total number of
  * work items.  Pieces are whole 128-key tiles, as even as whole tiles allow (the last one takes
  * the ragged end): sparrow_plan_piece_range() gives the keys [begin, end) of piece `piece` of
  * `n_splits`; SPARROW_ERR_SHAPE unless 0 <= piece < n_splits <= ceil(n_keys / 128). */
-sparrow_status sparrow_plan_splits(int32_t n_sm, int32_t batch, int32_t n_kv_heads,
+sparrow_status sparrow_plan_splits(int32_t n_sm, int32_t batch, int32_t n_kv_heads, int32_t gqa_group,
                                    const int32_t* n_keys, int32_t T, int32_t* splits_out,
                                    int32_t* n_items_out);
 sparrow_status sparrow_plan_piece_range(int32_t n_keys, int32_t n_splits, int32_t piece,

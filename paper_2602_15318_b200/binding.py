@@ -87,7 +87,7 @@ def lib():
         L.sparrow_build_anchor_idx.argtypes = [i32, vp, i32, i32, i32, vp, vp]
         L.sparrow_debug_ancestor_masks_device.argtypes = [vp, vp, i32, vp, vp]
         L.sparrow_debug_wait_counter.argtypes = [vp, ctypes.c_uint32, vp]
-        L.sparrow_plan_splits.argtypes = [i32, i32, i32, vp, i32, vp, vp]
+        L.sparrow_plan_splits.argtypes = [i32, i32, i32, i32, vp, i32, vp, vp]
         L.sparrow_last_device_status.argtypes = [vp, vp]
         L.sparrow_set_plan_policy.argtypes = [vp, i32]
         L.sparrow_set_call_overlap.argtypes = [vp, i32]
@@ -381,11 +381,11 @@ def sparrow_debug_early_trigger_copy(ctx: Context, src, dst, nbytes: int, delay_
                                                 _stream_handle(stream)), "sparrow_debug_early_trigger_copy")
 
 
-def sparrow_plan_splits(n_sm: int, n_kv_heads: int, n_keys: Sequence[int], T: int):
+def sparrow_plan_splits(n_sm: int, n_kv_heads: int, n_keys: Sequence[int], T: int, gqa_group: int = 7):
     nk = _i32_array(n_keys)
     splits = (ctypes.c_int32 * len(n_keys))()
     n_items = ctypes.c_int32(0)
-    _chk(lib().sparrow_plan_splits(n_sm, len(n_keys), n_kv_heads, nk, T, splits, ctypes.byref(n_items)),
+    _chk(lib().sparrow_plan_splits(n_sm, len(n_keys), n_kv_heads, gqa_group, nk, T, splits, ctypes.byref(n_items)),
          "sparrow_plan_splits")
     return [int(x) for x in splits], int(n_items.value)
 

@@ -111,7 +111,7 @@ Staging staging_layout(const sparrow_layout& L)
 }
 
 // 128-row blocks (18 draft tokens each) one work item of the tensor-core pass handles
-int blocks_per_group_tc(int T) { return T <= kTokPerBlock ? 1 : 2; }
+int blocks_per_group_tc(int T, int group) { return T <= tokens_per_block(group) ? 1 : 2; }
 
 int max_items(int n_sm, int batch, int n_kv_heads, int n_groups)
 {
@@ -121,17 +121,21 @@ int max_items(int n_sm, int batch, int n_kv_heads, int n_groups)
 // Chooses the number of key-range pieces per sequence so that the total number of work items is
 // close to (and not above) the SM count while every item streams about the same number of keys.
 // key0 (optional): per sequence, the first key that is streamed at all (a multiple of 128).
-sparrow_status make_plan(int n_sm, int batch, int n_kv_heads, const int32_t* n_keys, int T, int blocks_per_group,
+sparrow_status make_plan(int n_sm, int batch, int n_kv_heads, int group, const int32_t* n_keys, int T, int blocks_per_group,
                          SplitPlan* p, int min_piece_keys = kMinPieceKeys, const int32_t* key0 = nullptr)
 {
-    if (batch < 1 || batch > kMaxBatch || T < 1 || T > kMaxT || n_kv_heads < 1 || n_sm < 1) return SPARROW_ERR_SHAPE;
+    if (batch < 1 || batch > kMaxBatch || T < 1 || T > kMaxT || n_kv_heads < 1 || n_sm < 1 || group < 1 || group > kMaxGroup)
+        return SPARROW_ERR_SHAPE;
+    const int tpb = tokens_per_block(group);
     std::memset(p, 0, sizeof(*p));
     p->batch = batch;
     p->T = T;
     p->T_tree = T;
-    p->M = kGroup * T;
+    p->group = group;
+    p->tok_per_block = tpb;
+    p->M = group * T;
     p->blocks_per_group = blocks_per_group;
-    p->n_groups = (T + kTokPerBlock * blocks_per_group - 1) / (kTokPerBlock * blocks_per_group);
+    p->n_groups = (T + tpb * blocks_per_group - 1) / (tpb * blocks_per_group);
     p->n_kv_heads = n_kv_heads;
     p->piece_tile = min_piece_keys < kKeyTile ? min_piece_keys : kKeyTile;
     p->part_rows = blocks_per_group * kBlockRows + 1;    // odd pitch: partial rows of successive pieces must not share L2 sets
@@ -167,6 +171,13 @@ sparrow_status make_plan(int n_sm, int batch, int n_kv_heads, const int32_t* n_k
     p->n_items = total;
     return SPARROW_OK;
 }
+
+// n_q_heads = g * n_kv_heads with 1 <= g <= kMaxGroup
+bool layout_heads_ok(const sparrow_layout& L)
+{
+    return L.n_kv_heads >= 1 && L.n_q_heads >= L.n_kv_heads && L.n_q_heads % L.n_kv_heads == 0 && L.n_q_heads / L.n_kv_heads <= kMaxGroup;
+}
+int layout_group(const sparrow_layout& L) { return L.n_q_heads / L.n_kv_heads; }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -419,9 +430,10 @@ bool tensor_map_for(sparrow_ctx* c, const void* base, int tag, CUtensorMap* out)
                       estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     } else {
-        const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)kGroup, (cuuint64_t)L.n_kv_heads, (cuuint64_t)tag};
-        const cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)kGroup * kD * 2, (cuuint64_t)L.n_q_heads * kD * 2};
-        const cuuint32_t box[4] = {64, (cuuint32_t)kGroup, 1, (cuuint32_t)kTokPerBlock};
+        const int group = L.n_q_heads / L.n_kv_heads;
+        const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)group, (cuuint64_t)L.n_kv_heads, (cuuint64_t)tag};
+        const cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)group * kD * 2, (cuuint64_t)L.n_q_heads * kD * 2};
+        const cuuint32_t box[4] = {64, (cuuint32_t)group, 1, (cuuint32_t)tokens_per_block(group)};
         r = c->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
                       estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -549,8 +561,9 @@ sparrow_status verify_call(sparrow_ctx* c, const void* q, const void* k, const v
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool overlaps = call_overlaps(c, st, true);
     SplitPlan plan;
-    sparrow_status s = make_plan(plan_target(c, overlaps), c->layout.batch, c->layout.n_kv_heads, n_keys, T,
-                                 blocks_per_group_tc(T), &plan, kMinPieceKeys, key0);
+    const int group = layout_group(c->layout);
+    sparrow_status s = make_plan(plan_target(c, overlaps), c->layout.batch, c->layout.n_kv_heads, group, n_keys, T,
+                                 blocks_per_group_tc(T, group), &plan, kMinPieceKeys, key0);
     if (s != SPARROW_OK) return s;
     plan.T_tree = T_tree;
     for (int b = 0; b < c->layout.batch; ++b) plan.seq[b].kv_len = kv_len[b];
@@ -595,7 +608,7 @@ sparrow_status sparrow_create(sparrow_ctx** out, const sparrow_layout* L, int de
     if (!out || !L) return SPARROW_ERR_NULL;
     *out = nullptr;
     if (L->batch < 1 || L->batch > kMaxBatch || L->head_dim != kD || L->n_kv_heads < 1 ||
-        L->n_q_heads != kGroup * L->n_kv_heads || L->kv_capacity < 1 ||
+        !layout_heads_ok(*L) || L->kv_capacity < 1 ||
         !(L->softmax_scale > 0.f) || !std::isfinite(L->softmax_scale) ||
         L->kv_stride_head < (int64_t)L->kv_capacity * kD || (L->kv_stride_head % 8) != 0 ||
         (L->kv_stride_batch % 8) != 0 ||
@@ -662,8 +675,9 @@ size_t sparrow_workspace_bytes(const sparrow_ctx* c, int32_t max_T)
 {
     if (!c || max_T < 1 || max_T > kMaxT) return 0;
     size_t worst = 0;
-    for (int nb : {1, blocks_per_group_tc(max_T)}) {         // the gathered pass uses single blocks
-        const int groups = (max_T + kTokPerBlock * nb - 1) / (kTokPerBlock * nb);
+    const int tpb = tokens_per_block(layout_group(c->layout));
+    for (int nb : {1, blocks_per_group_tc(max_T, layout_group(c->layout))}) {         // the gathered pass uses single blocks
+        const int groups = (max_T + tpb * nb - 1) / (tpb * nb);
         const size_t rows = (size_t)max_items(c->n_sm, c->layout.batch, c->layout.n_kv_heads, groups) * (nb * kBlockRows + 1);
         const size_t need = part_bytes(rows);
         if (need > worst) worst = need;
@@ -690,13 +704,13 @@ sparrow_status sparrow_set_workspace(sparrow_ctx* c, void* p, size_t bytes)
     return SPARROW_OK;
 }
 
-sparrow_status sparrow_plan_splits(int32_t n_sm, int32_t batch, int32_t n_kv_heads, const int32_t* n_keys,
+sparrow_status sparrow_plan_splits(int32_t n_sm, int32_t batch, int32_t n_kv_heads, int32_t gqa_group, const int32_t* n_keys,
                                    int32_t T, int32_t* splits_out, int32_t* n_items_out)
 {
     if (!n_keys || !splits_out || !n_items_out) return SPARROW_ERR_NULL;
     SplitPlan p;
-    if (T < 1 || T > kMaxT) return SPARROW_ERR_SHAPE;
-    const sparrow_status s = make_plan(n_sm, batch, n_kv_heads, n_keys, T, blocks_per_group_tc(T), &p);
+    if (T < 1 || T > kMaxT || gqa_group < 1 || gqa_group > kMaxGroup) return SPARROW_ERR_SHAPE;
+    const sparrow_status s = make_plan(n_sm, batch, n_kv_heads, gqa_group, n_keys, T, blocks_per_group_tc(T, gqa_group), &p);
     if (s != SPARROW_OK) return s;
     for (int b = 0; b < batch; ++b) splits_out[b] = p.seq[b].n_splits;
     *n_items_out = p.n_items;
@@ -762,7 +776,7 @@ sparrow_status sparrow_verify_attn_static(const sparrow_layout* L, const void* q
     // every argument check comes first: a refused call has not touched the GPU
     if (!L || !q || !k || !v || !kv_len || !parents || !out || !lse) return SPARROW_ERR_NULL;
     if (L->batch < 1 || L->batch > kMaxBatch || L->head_dim != kD || L->n_kv_heads < 1 ||
-        L->n_q_heads != kGroup * L->n_kv_heads || L->kv_capacity < 1 ||
+        !layout_heads_ok(*L) || L->kv_capacity < 1 ||
         !(L->softmax_scale > 0.f) || !std::isfinite(L->softmax_scale) ||
         L->kv_stride_head < (int64_t)L->kv_capacity * kD || (L->kv_stride_head % 8) != 0 ||
         (L->kv_stride_batch % 8) != 0 ||
@@ -830,7 +844,8 @@ sparrow_status sparrow_verify_attn_static(const sparrow_layout* L, const void* q
     }
     // refuse what does not fit the array before anything is enqueued
     SplitPlan plan;
-    if (make_plan(c->n_sm, L->batch, L->n_kv_heads, n_keys, T, blocks_per_group_tc(T), &plan) != SPARROW_OK) return SPARROW_ERR_SHAPE;
+    if (make_plan(c->n_sm, L->batch, L->n_kv_heads, layout_group(*L), n_keys, T, blocks_per_group_tc(T, layout_group(*L)), &plan) != SPARROW_OK)
+        return SPARROW_ERR_SHAPE;
     if (check_ws(c, plan) != SPARROW_OK) return SPARROW_ERR_WORKSPACE;
     // the status word is the one thing that must start clean
     // the status word must start clean, and so must the two words of the serial merge (an earlier call that gave up
@@ -869,7 +884,7 @@ sparrow_status anchor_call(sparrow_ctx* c, const void* q, const void* k, const v
     int32_t n_keys[kMaxBatch];
     for (int b = 0; b < c->layout.batch; ++b) n_keys[b] = n_anchor;
     SplitPlan plan;
-    sparrow_status s = make_plan(c->n_sm, c->layout.batch, c->layout.n_kv_heads, n_keys, T, 1, &plan, kMinGatherPieceKeys);
+    sparrow_status s = make_plan(c->n_sm, c->layout.batch, c->layout.n_kv_heads, layout_group(c->layout), n_keys, T, 1, &plan, kMinGatherPieceKeys);
     if (s != SPARROW_OK) return s;
     if ((s = check_ws(c, plan)) != SPARROW_OK) return s;
     DeviceGuard guard(c->device);

@@ -46,9 +46,9 @@ __device__ __forceinline__ void fma8(float (&acc)[16], int base, float w, const 
 // by all 32 lanes of a warp.
 __device__ __forceinline__ void combine_row(const SplitPlan& plan, const CombineArgs& args, int b, int kvh, int t, int g, int lane)
 {
-    const int block = t / kTokPerBlock;               // 128-row block holding this token
+    const int block = t / plan.tok_per_block;               // 128-row block holding this token
     const int group = block / plan.blocks_per_group;
-    const int lr = (block - group * plan.blocks_per_group) * kBlockRows + (t - block * kTokPerBlock) * kGroup + g;
+    const int lr = (block - group * plan.blocks_per_group) * kBlockRows + (t - block * plan.tok_per_block) * plan.group + g;
     const int ns = plan.seq[b].n_splits;
     if (ns == 1) return;                              // the split pass wrote this row's result itself
     const int item0 = plan.seq[b].item_begin + (kvh * plan.n_groups + group) * ns;
@@ -125,7 +125,7 @@ __device__ __forceinline__ void combine_row(const SplitPlan& plan, const Combine
         acc[i] += __shfl_xor_sync(0xffffffffu, acc[i], 16);
     }
     if (quarter == 0) {
-        const int h = kvh * kGroup + g;
+        const int h = kvh * plan.group + g;
         __nv_bfloat16* dst = args.out + (((size_t)b * plan.T + t) * args.n_q_heads + h) * kD + sub * 16;
         uint4 pk[2];
         uint32_t* w32 = reinterpret_cast<uint32_t*>(pk);
@@ -152,7 +152,7 @@ combine_kernel(const __grid_constant__ SplitPlan plan, const __grid_constant__ C
     const int rows_total = plan.batch * plan.n_kv_heads * plan.M;
     for (int row_id = blockIdx.x * kWarps + warp; row_id < rows_total; row_id += gridDim.x * kWarps) {
         const int R = row_id % plan.M, unit_bh = row_id / plan.M;
-        combine_row(plan, args, unit_bh / plan.n_kv_heads, unit_bh % plan.n_kv_heads, R / kGroup, R % kGroup, lane);
+        combine_row(plan, args, unit_bh / plan.n_kv_heads, unit_bh % plan.n_kv_heads, R / plan.group, R % plan.group, lane);
     }
 }
 

@@ -8,10 +8,11 @@
 namespace sparrow {
 
 constexpr int kD = 128;           // head_dim
-constexpr int kGroup = 7;         // query heads per KV head
+constexpr int kMaxGroup = 16;      // query heads per KV head: 1 .. 16 (7 for the Qwen2-7B-shaped models of the paper)
 constexpr int kMaxT = 64;
 constexpr int kMaxBatch = 64;
-constexpr int kTokPerBlock = 18;  // draft tokens per 128-row block: 18 x 7 = 126 rows, 2 rows of padding
+// draft tokens per 128-row block for a group of g query heads: 18 for g = 7 (126 rows, 2 rows of padding)
+__host__ __device__ constexpr int tokens_per_block(int g) { return 128 / g < 64 ? 128 / g : 64; }
 constexpr int kBlockRows = 128;
 constexpr int kKeyTile = 128;      // keys per tile of the tensor-core kernel; pieces of the key range are whole tiles
 
@@ -24,9 +25,10 @@ __host__ __device__ constexpr unsigned timeout_bits(int site) { return kStatTime
 enum WaitSite { kSiteProducer = 0, kSiteMma = 1, kSiteSoftmax = 2, kSiteWriteSame = 3, kSiteWriteOther = 4,
                 kSiteArrivals = 5, kSiteFinOther = 6, kSiteFinCopies = 7, kSiteDebug = 8 };
 
-// The GQA group's 7 query heads x T draft tokens are packed into 128-row blocks: block i holds
-// tokens [18 i, 18 i + 18), row r of a block is (token 18 i + r / 7, head r % 7), rows 126 and 127
-// are padding.  A row group is 1 or 2 consecutive blocks, handled by one work item.
+// The GQA group's g query heads x T draft tokens are packed into 128-row blocks of p = 128 / g
+// tokens: block i holds tokens [p i, p i + p), row r of a block is (token p i + r / g, head r % g),
+// rows from g p on are padding (g = 7: 18 tokens, rows 126 and 127).  A row group is 1 or 2
+// consecutive blocks, handled by one work item.
 //
 // One work item = (sequence b, KV head, row group, key-range piece).  Items of sequence b occupy
 // [seq[b].item_begin, seq[b+1].item_begin); inside, the index runs (kv head, row group, piece) with the
@@ -45,7 +47,9 @@ struct SplitPlan {
     int32_t batch;
     int32_t T;                    // query tokens
     int32_t T_tree;               // nodes of the draft tree = rows of the draft block; the queries are its last T nodes
-    int32_t M;                    // query rows per KV head = 7*T
+    int32_t group;                // g: query heads per KV head
+    int32_t tok_per_block;        // p = tokens_per_block(g)
+    int32_t M;                    // query rows per KV head = g*T
     int32_t blocks_per_group;     // 128-row blocks one work item handles (1 or 2)
     int32_t n_groups;             // ceil(T / (18 * blocks_per_group))
     int32_t n_kv_heads;
@@ -55,13 +59,13 @@ struct SplitPlan {
 };
 
 constexpr int kFinisherCtas = 32;  // CTAs of a call that share its combine step
-constexpr int kMaxGroups = 4;      // row groups per (sequence, KV head): ceil(64 / 18) blocks, 1 or 2 per group
+constexpr int kMaxGroups = 4;      // row groups per (sequence, KV head): at most 8 blocks (g = 16), 2 per group
 constexpr int kArrivalSlots = 4;   // arrival words rotate over the call number modulo 4
 // A partial row in the workspace: 128 fp16 outputs, then the row's fp32 LSE, padded to 16 bytes,
 // so that one bulk copy brings a run of rows with everything needed to merge them.
 constexpr int kPartRowHalves = 136;
 
-// Fused mode: ordering between the CTAs of one call and between consecutive calls.
+// Overlapped mode: ordering between the CTAs of one call and between consecutive calls.
 //
 // The split-KV kernel is launched with programmatic stream serialisation and never waits for the
 // previous grid as a whole, so the next call's CTAs start (and read their inputs) while the
@@ -72,7 +76,8 @@ constexpr int kPartRowHalves = 136;
 //   fin_done[n % 2]   final-result writers of calls with this parity that are done, cumulative
 // An item whose unit (sequence, KV head, row group) has several key-range pieces stores a partial
 // and arrives; an item that is its unit's only piece writes final results itself.  The last
-// n_fin CTAs of the grid are the call's finishers -- they are the last to start, so by the time
+// n_fin CTAs of the grid are the call's finishers (all of them where the call has the GPU to
+// itself anyway) -- they are the last to start, so by the time
 // they are through with their own items little is left to wait for: they wait until every
 // partial of the call has arrived, then each merges a contiguous share of the call's rows by
 // log-sum-exp and writes the final out / lse.  Every final-result writer (finisher or single
@@ -83,8 +88,13 @@ constexpr int kPartRowHalves = 136;
 // results land in call order.  CTA 0 then clears the arrival word of slot (n + 2) % 4: its last
 // user was call n-2, and the items of call n+2 cannot arrive before the finishers of call n are
 // done, which in turn have seen CTA 0's arrival (or, if it had none, follow it in the stream).
-// With enabled == 0 the kernels are ordered by the stream alone: they touch no counter, never let
-// dependents launch early, and a separate combine kernel follows the split-KV kernel.
+//
+// Serial mode (enabled == 0, serial == 1): the call is an ordinary launch that runs alone between
+// its neighbours in the stream (stream capture, programmatic launch switched off, the entry point
+// without a workspace).  It touches none of the counters above and never lets dependents launch
+// early; its CTAs arrive on serial_words[0], every CTA is a finisher, and the CTA that leaves last
+// (serial_words[1] counts them) puts both words back to zero -- so the same launch can be replayed
+// from a graph.  With both flags zero (the gathered kernel) a separate combine kernel follows.
 struct SyncArgs {
     unsigned* arrivals;      // [4]
     unsigned* fin_done;      // [2]

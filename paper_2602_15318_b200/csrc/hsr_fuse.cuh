@@ -10,10 +10,10 @@
 // Work item = (tile of 128 output features, slice of the K range); about one item per SM.  The
 // weights are the M-side operand (128 features), the tokens the N side (64 columns, rows past M
 // read as zero):  D[128 features x 64 tokens] += W_tile[128 x 16] X_tile[64 x 16]^T  on tcgen05,
-// operands staged by TMA through a 6-stage mbarrier ring, accumulator in TMEM.  Each item stores
-// its fp32 partial tile; the item that arrives last on its feature tile's counter adds the slices
-// in fixed order (deterministic), adds the bias and writes z (bf16); it also puts the counter back
-// to zero.  Every wait is bounded.
+// operands staged by TMA through a 6-stage mbarrier ring (16 KB of weights + 8 KB of activations per
+// stage), accumulator in TMEM.  Each item stores its fp32 partial tile; the item that arrives last on
+// its feature tile's counter adds the slices in fixed order (deterministic), adds the bias and
+// writes z (bf16); it also puts the counter back to zero.  Every wait is bounded.
 #pragma once
 #include <cuda.h>
 
@@ -23,7 +23,7 @@ namespace sparrow {
 
 struct HsrArgs {
     const __nv_bfloat16* bias;   // [d_out] or nullptr
-    float* partial;              // [n_slices][d_out][64] fp32
+    float* partial;              // [n_slices][64][d_out] fp32 (token rows past M are never touched)
     __nv_bfloat16* z;            // [M][d_out]
     unsigned* counters;          // [d_out / 128], zero between calls
     unsigned* status;
@@ -39,11 +39,13 @@ using namespace tc;
 constexpr int kThreadsHsr = 192;                 // 4 epilogue warps, producer, MMA issuer
 constexpr int kFeat = 128;                       // output features per item
 constexpr int kTok = 64;                         // token columns (M <= 64)
-constexpr int kKTile = 64;                       // K elements per stage
-constexpr int kWBytes = kFeat * kKTile * 2;      // 16 KB
-constexpr int kXBytes = kTok * kKTile * 2;       // 8 KB
+constexpr int kKTile = 64;                       // K elements per TMA box (one 128-byte swizzled row)
+constexpr int kBoxes = 1;                        // boxes per stage (wider stages were measured: no difference)
+constexpr int kWBytes = kFeat * kKTile * 2;      // one weight box: 16 KB
+constexpr int kXBytes = kTok * kKTile * 2;       // one activation box: 8 KB
+constexpr int kStageBytes = kBoxes * (kWBytes + kXBytes);
 constexpr int kStages = 6;
-constexpr int kSmemBytes = 1024 + kStages * (kWBytes + kXBytes) + 256;
+constexpr int kSmemBytes = 1024 + kStages * kStageBytes + 256;
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar)
 {
@@ -59,7 +61,7 @@ hsr_fuse_kernel(const __grid_constant__ HsrArgs args, const __grid_constant__ CU
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     unsigned char* sm = smem_raw + ((1024u - (raw & 1023u)) & 1023u);
-    unsigned char* misc = sm + kStages * (kWBytes + kXBytes);
+    unsigned char* misc = sm + kStages * kStageBytes;
     const uint32_t bar0 = smem_u32(misc);                               // full[6], empty[6], done
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 128);
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(misc + 132);
@@ -74,15 +76,21 @@ hsr_fuse_kernel(const __grid_constant__ HsrArgs args, const __grid_constant__ CU
     const int kt_begin = (int)((long long)args.k_tiles * slice / args.n_slices);
     const int kt_end = (int)((long long)args.k_tiles * (slice + 1) / args.n_slices);
     const int n_kt = kt_end - kt_begin;
+    const int n_st = (n_kt + kBoxes - 1) / kBoxes;                      // ring fills of this item (the last may be short)
     const int d_tiles = args.d / kKTile;                                // K tiles that belong to e
 
+    // Stage layout: kBoxes weight boxes, then kBoxes activation boxes.
     auto issue = [&](int i) {                                           // producer thread only
-        const int st = i % kStages, kt = kt_begin + i;
-        const uint32_t dst = smem_u32(sm + st * (kWBytes + kXBytes));
-        mbar_expect_tx(full(st), kWBytes + kXBytes);
-        tma_load_2d(dst, &tmap_w, kt * kKTile, f_tile * kFeat, full(st));
-        if (kt < d_tiles) tma_load_2d(dst + kWBytes, &tmap_e, kt * kKTile, 0, full(st));
-        else tma_load_2d(dst + kWBytes, &tmap_h, (kt - d_tiles) * kKTile, 0, full(st));
+        const int st = i % kStages;
+        const int boxes = min(kBoxes, n_kt - i * kBoxes);
+        const uint32_t dst = smem_u32(sm + st * kStageBytes);
+        mbar_expect_tx(full(st), boxes * (kWBytes + kXBytes));
+        for (int bx = 0; bx < boxes; ++bx) {
+            const int kt = kt_begin + i * kBoxes + bx;
+            tma_load_2d(dst + bx * kWBytes, &tmap_w, kt * kKTile, f_tile * kFeat, full(st));
+            if (kt < d_tiles) tma_load_2d(dst + kBoxes * kWBytes + bx * kXBytes, &tmap_e, kt * kKTile, 0, full(st));
+            else tma_load_2d(dst + kBoxes * kWBytes + bx * kXBytes, &tmap_h, (kt - d_tiles) * kKTile, 0, full(st));
+        }
     };
 
     if (warp == 4 && lane == 0) {
@@ -93,7 +101,7 @@ hsr_fuse_kernel(const __grid_constant__ HsrArgs args, const __grid_constant__ CU
         mbar_init(done, 1);
         *abort_flag = 0;
         fence_barrier_init();
-        for (int i = 0; i < n_kt && i < kStages; ++i) issue(i);
+        for (int i = 0; i < n_st && i < kStages; ++i) issue(i);
     }
     if (warp == 5) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(64u) : "memory");
@@ -107,7 +115,7 @@ hsr_fuse_kernel(const __grid_constant__ HsrArgs args, const __grid_constant__ CU
     if (warp == 4) {
         if (lane == 0) {                                                // ---- TMA producer: refill freed stages
             #pragma unroll 1
-            for (int i = kStages; i < n_kt; ++i) {
+            for (int i = kStages; i < n_st; ++i) {
                 if (!mbar_wait(empty(i % kStages), (i / kStages - 1) & 1)) {
                     atomicOr(args.status, timeout_bits(kSiteProducer)); *abort_flag = 1; break;
                 }
@@ -119,15 +127,20 @@ hsr_fuse_kernel(const __grid_constant__ HsrArgs args, const __grid_constant__ CU
             constexpr uint32_t idesc = idesc_bf16(false, kTok);
             bool ok = true;
             #pragma unroll 1
-            for (int i = 0; i < n_kt && ok; ++i) {
+            for (int i = 0; i < n_st && ok; ++i) {
                 const int st = i % kStages;
                 if (!mbar_wait(full(st), (i / kStages) & 1)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t base = smem_u32(sm + st * (kWBytes + kXBytes));
-                const uint64_t wd = smem_desc(base, 16, 1024), xd = smem_desc(base + kWBytes, 16, 1024);
-                #pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                    mma_ss(tmem, wd + (uint64_t)((ks * 32) >> 4), xd + (uint64_t)((ks * 32) >> 4), idesc, (i > 0 || ks > 0) ? 1u : 0u);
+                const int boxes = min(kBoxes, n_kt - i * kBoxes);
+                const uint32_t base = smem_u32(sm + st * kStageBytes);
+                for (int bx = 0; bx < boxes; ++bx) {
+                    const uint64_t wd = smem_desc(base + bx * kWBytes, 16, 1024);
+                    const uint64_t xd = smem_desc(base + kBoxes * kWBytes + bx * kXBytes, 16, 1024);
+                    #pragma unroll
+                    for (int ks = 0; ks < 4; ++ks)
+                        mma_ss(tmem, wd + (uint64_t)((ks * 32) >> 4), xd + (uint64_t)((ks * 32) >> 4), idesc,
+                               (i > 0 || bx > 0 || ks > 0) ? 1u : 0u);
+                }
                 tc_commit(empty(st));
             }
             tc_commit(done);
@@ -154,12 +167,14 @@ hsr_fuse_kernel(const __grid_constant__ HsrArgs args, const __grid_constant__ CU
             for (int t = 0; t < 64; ++t)
                 if (t < args.M) args.z[(size_t)t * args.d_out + feat] = __float2bfloat16(acc[t] + b);
         } else {
-            float4* dst = reinterpret_cast<float4*>(args.partial + ((size_t)slice * args.d_out + feat) * kTok);
+            // partial sums as [slice][token][feature]: the 32 features of a warp are 128 contiguous bytes
+            float* mine = args.partial + (size_t)slice * kTok * args.d_out + feat;
             #pragma unroll
-            for (int t = 0; t < 16; ++t) dst[t] = make_float4(acc[4 * t], acc[4 * t + 1], acc[4 * t + 2], acc[4 * t + 3]);
-            __threadfence();
-            asm volatile("bar.sync 1, 128;" ::: "memory");
+            for (int t = 0; t < 64; ++t)
+                if (t < args.M) mine[(size_t)t * args.d_out] = acc[t];
+            asm volatile("bar.sync 1, 128;" ::: "memory");             // every store of this item has been issued
             if (tid == 0) {
+                // release (cumulative over the stores the barrier ordered before it) and acquire in one
                 unsigned old;
                 asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(args.counters + f_tile) : "memory");
                 *is_last = old == (unsigned)args.n_slices - 1u ? 1 : 0;
@@ -167,16 +182,24 @@ hsr_fuse_kernel(const __grid_constant__ HsrArgs args, const __grid_constant__ CU
             }
             asm volatile("bar.sync 1, 128;" ::: "memory");
             if (*is_last) {
-                // the slices in fixed order, whoever arrived last
+                // The slices in fixed order, whoever arrived last (its own slice comes from its
+                // registers: the same values it stored); all loads of a slice in flight at once.
+                // (Two slices in flight, or a sum shared among the tile's items, measured slower.)
                 float sum[64];
                 #pragma unroll
                 for (int t = 0; t < 64; ++t) sum[t] = 0.f;
-                for (int s = 0; s < args.n_slices; ++s) {
-                    const float4* src = reinterpret_cast<const float4*>(args.partial + ((size_t)s * args.d_out + feat) * kTok);
-                    #pragma unroll
-                    for (int t = 0; t < 16; ++t) {
-                        const float4 v = __ldcg(src + t);
-                        sum[4 * t] += v.x; sum[4 * t + 1] += v.y; sum[4 * t + 2] += v.z; sum[4 * t + 3] += v.w;
+                #pragma unroll 1
+                for (int s2 = 0; s2 < args.n_slices; ++s2) {
+                    if (s2 == slice) {
+                        #pragma unroll
+                        for (int t = 0; t < 64; ++t) sum[t] += acc[t];
+                    } else {
+                        const float* src = args.partial + (size_t)s2 * kTok * args.d_out + feat;
+                        float v[64];
+                        #pragma unroll
+                        for (int t = 0; t < 64; ++t) v[t] = t < args.M ? __ldcg(src + (size_t)t * args.d_out) : 0.f;
+                        #pragma unroll
+                        for (int t = 0; t < 64; ++t) sum[t] += v[t];
                     }
                 }
                 #pragma unroll

@@ -2,8 +2,8 @@
 // (Eq. 2: keys/values restricted to the anchor list) and a general path for any key layout.
 //
 // One CTA = one work item (sequence, KV head, one 128-row block of packed query rows, key-range
-// piece).  The 7 query heads of the GQA group times 18 draft tokens form one block (row
-// r = (t % 18)*7 + g, two rows of padding), so every gathered K/V row is loaded once per KV head
+// piece).  The g query heads of the GQA group times p = 128 / g draft tokens form one block (row
+// r = (t % p) g + head; g = 7: 18 tokens, two rows of padding), so every gathered K/V row is loaded once per KV head
 // and block.  K/V rows are fetched
 // with 16-byte cp.async (row index = key index, or anchor_idx[key] when gathering) into a
 // two-stage XOR-swizzled shared-memory ring; S = QK^T and O += PV run on mma.sync m16n8k16 bf16
@@ -176,11 +176,11 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
         for (int u = 0; u < kChunksPerThread; ++u) {
             const int i = tid + u * kThreads;
             const int r = i >> 4, c = i & 15;
-            const int t = it.group * kTokPerBlock + r / kGroup, g = r % kGroup;
+            const int t = it.group * plan.tok_per_block + r / plan.group, g = r % plan.group;
             val[u] = make_uint4(0, 0, 0, 0);
-            if (r < kTokPerBlock * kGroup && t < T) {
+            if (r < plan.tok_per_block * plan.group && t < T) {
                 val[u] = __ldg(reinterpret_cast<const uint4*>(
-                    args.q + (((size_t)it.b * T + t) * args.n_q_heads + it.kvh * kGroup + g) * kD + c * 8));
+                    args.q + (((size_t)it.b * T + t) * args.n_q_heads + it.kvh * plan.group + g) * kD + c * 8));
             }
         }
         #pragma unroll
@@ -202,8 +202,8 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
     #pragma unroll
     for (int rr = 0; rr < 2; ++rr) {
         const int lr = warp * 16 + g4 + rr * 8;
-        row_t[rr] = it.group * kTokPerBlock + lr / kGroup;
-        row_ok[rr] = lr < kTokPerBlock * kGroup && row_t[rr] < T;
+        row_t[rr] = it.group * plan.tok_per_block + lr / plan.group;
+        row_ok[rr] = lr < plan.tok_per_block * plan.group && row_t[rr] < T;
         const int t = row_ok[rr] ? row_t[rr] : 0;
         row_anc[rr] = anchored ? (tree_nodes > 0 ? anc_s[tree_nodes - T + t] : 0ull) : anc_s[t];
         row_qpos[rr] = anchored ? qpos_s[t] : 0;
@@ -338,7 +338,7 @@ split_gather_kernel(const __grid_constant__ SplitPlan plan, const __grid_constan
         const float inv = l > 0.f ? 1.f / l : 0.f;
         const float lse_val = l > 0.f ? (m_run[rr] * c2 + log2f(l)) * 0.6931471805599453f : -INFINITY;
         if (plan.seq[it.b].n_splits == 1) {                 // the only piece: write the final result
-            const int t = row_t[rr], h = it.kvh * kGroup + lr % kGroup;
+            const int t = row_t[rr], h = it.kvh * plan.group + lr % plan.group;
             __nv_bfloat16* dst = args.out + (((size_t)it.b * T + t) * args.n_q_heads + h) * kD;
             #pragma unroll
             for (int nt = 0; nt < 16; ++nt)

@@ -1,10 +1,10 @@
 // Split-KV pass of the verification mode on the sm_100a tensor path.
 //
 // One CTA per SM-sized work item (sequence, KV head, row group of 1 or 2 128-row blocks, piece of
-// the key range).  A block packs the GQA group's 7 heads x 18 draft tokens (row r = (t % 18)*7 + g,
-// 2 rows of padding), so each K/V byte crosses HBM -> SM once per KV head and row group.
+// the key range).  A block packs the GQA group's g heads x p = 128 / g draft tokens (row r = (t % p) g + head;
+// g = 7: 18 tokens, 2 rows of padding), so each K/V byte crosses HBM -> SM once per KV head and row group.
 //
-//   warp 8, one thread   TMA producer: the Q block(s) (two boxes of 64 dims x 7 heads x 18 tokens
+//   warp 8, one thread   TMA producer: the Q block(s) (two boxes of 64 dims x g heads x p tokens
 //                        each, which land exactly in the K-major 128-byte-swizzled operand
 //                        layout), then K and V tiles of 128 keys x 128 dims (4 boxes of 128 x 64)
 //                        into a 2- or 3-stage shared-memory ring, mbarrier full / empty handshakes.
@@ -13,27 +13,34 @@
 //                        block; O += P V with P read from TMEM (bf16, aliasing the S block) and V
 //                        from shared memory as an MN-major operand.  The scores of up to three
 //                        jobs are kept ahead of the softmax.
-//   warps 0-3, 4-7       softmax: the two threads with the same TMEM lane (warps w and w + 4)
-//                        share one query row, warpgroup g taking key columns [64 g, 64 g + 64) of
-//                        every job: tcgen05.ld, ancestor / range masking, fp32 online softmax
-//                        with a lazy maximum, P packed to bf16 and stored back with tcgen05.st.
-//                        The two threads keep the same reference maximum: one barrier with an OR
-//                        reduction per job tells whether any row's maximum grew by more than 2^8;
-//                        only then the halves' maxima meet in shared memory and O is rescaled in
-//                        TMEM.  Each thread sums its own columns; the halves' sums meet once, in
-//                        the epilogue.
+//   warps 0-7            softmax, TMEM lane = query row: tcgen05.ld, ancestor / range / window
+//                        masking, fp32 online softmax with a lazy maximum, P packed to bf16 and
+//                        stored back with tcgen05.st.
+//                        One row block (T <= 18): the two threads with the same lane (warps w and
+//                        w + 4) share a row, warpgroup g taking key columns [64 g, 64 g + 64) of every
+//                        job.  They keep the same reference maximum: one barrier with an OR reduction
+//                        per job tells whether any row's maximum grew by more than 2^8; only then the
+//                        halves' maxima meet in shared memory and O is rescaled in TMEM.  Each
+//                        thread sums its own columns; the halves' sums meet once, in the epilogue.
+//                        Two row blocks: warpgroup g owns block g, one thread per row and all 128
+//                        keys of a tile, and works through its block's tiles on its own (no
+//                        barrier between the warpgroups); per block the chain is scores -> softmax
+//                        -> O += P V -> next scores, and the two chains interleave on the tensor
+//                        pipe and the exponential unit.
+//   warp 10, one thread  gatekeeper (overlapped mode): waits, beside the main loop, for the counters
+//                        that allow this CTA's first global write.
 //
-// With one row block (T <= 18) there are three S blocks and one O accumulator, with two row
-// blocks two S blocks and two accumulators (jobs alternate between the blocks).
+// With one row block there are three S blocks and one O accumulator, with two row blocks one S
+// block and one accumulator per block.
 //
-// Ordering against neighbouring kernels in the stream (fused mode, see SyncArgs): the kernel is
-// launched with programmatic stream serialisation and never waits for the previous grid as a
+// Ordering against neighbouring kernels in the stream (see SyncArgs).  Overlapped mode: the kernel
+// is launched with programmatic stream serialisation and never waits for the previous grid as a
 // whole.  All reads of q / k / v / parents are issued as soon as the CTA starts, so the K/V stream
 // of this call overlaps the tail of the previous one; in front of its first global write a CTA
-// waits on the finisher counters.  After storing its partials a CTA publishes its item; the last
-// CTAs of the grid (the finishers) wait for the call's arrivals, share the call's rows among them,
-// merge each row's pieces by log-sum-exp and write out / lse; the others exit at once.  In
-// stream-ordered mode the kernel only writes partials and a separate combine kernel follows.
+// waits on the finisher counters.  Serial mode: the call runs alone between its neighbours in the
+// stream.  In both, a CTA publishes its item after storing its partials, and the call's finisher
+// CTAs wait for the arrivals, share the call's rows among them, merge each row's pieces by
+// log-sum-exp and write out / lse.
 //
 // Every wait is bounded; a wait that gives up sets the timeout status bit and the CTA drains and
 // exits.  TMEM is always released.
@@ -66,7 +73,6 @@ constexpr int kProducerWarp = 8, kMmaWarp = 9, kGateWarp = 10;
 constexpr int kTile = 128;                       // keys per stage and per job
 constexpr int kSubTileBytes = 128 * 64 * 2;      // one 128 x 64 bf16 box: 16 KB
 constexpr int kQBlockBytes = 2 * kSubTileBytes;  // 128 rows x 128 dims: 32 KB
-constexpr int kQBoxBytes = 64 * kGroup * kTokPerBlock * 2;   // one Q box: 64 dims x 7 heads x 18 tokens
 constexpr int kStageBytes = 4 * kSubTileBytes;   // K (32 KB) + V (32 KB)
 constexpr int kMiscBytes = 2048;                 // barriers, flags, ancestor words, maxima exchange
 constexpr uint32_t kSpinLimit = 1u << 22;        // polls before a wait gives up
@@ -158,8 +164,6 @@ __device__ __forceinline__ void tc_commit(uint32_t bar)
 }
 // barrier among the 256 softmax threads only (id 1; id 0 is __syncthreads)
 __device__ __forceinline__ void softmax_bar_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
-// barrier among the 128 threads of one softmax warpgroup (ids 3 and 4)
-__device__ __forceinline__ void warpgroup_bar_sync(int wg) { asm volatile("bar.sync %0, 128;" ::"r"(3 + wg) : "memory"); }
 // D[tmem] (+)= A[smem] * B[smem]
 __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
 {
@@ -370,6 +374,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const Item it = decode_item(plan, blockIdx.x);
     const int T = plan.T;
+    const int qg = plan.group, tpb = plan.tok_per_block;   // query heads per KV head, tokens per 128-row block
     const int kv_len = plan.seq[it.b].kv_len;
     const int n_keys_seq = plan.seq[it.b].n_keys;
     const int n_tiles = (it.key_end - it.key_begin + kTile - 1) / kTile;
@@ -410,11 +415,11 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
         fence_barrier_init();
         // Q first (the first S = Q K^T needs it and it is small), then K and V tiles in the order
         // they are consumed.  Nothing here depends on the previous kernel in the stream.
-        mbar_expect_tx(B.q_full(), NB * 2 * kQBoxBytes);
+        mbar_expect_tx(B.q_full(), (uint32_t)(NB * 2 * 64 * qg * tpb * 2));   // two boxes of 64 dims x g heads x p tokens per block
         #pragma unroll
         for (int blk = 0; blk < NB; ++blk) {
             const uint32_t dst = smem_u32(q_sm + blk * kQBlockBytes);
-            const int tok = it.b * T + (block0 + blk) * kTokPerBlock;
+            const int tok = it.b * T + (block0 + blk) * tpb;
             tma_load_4d(dst, &tmap_q, 0, 0, it.kvh, tok, B.q_full());
             tma_load_4d(dst + kSubTileBytes, &tmap_q, 64, 0, it.kvh, tok, B.q_full());
         }
@@ -579,15 +584,15 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
         const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
         const float c2 = args.scale_log2e;
         const float thr = kRescaleLog2 / c2;             // threshold in raw score units
-        const int g_row = row_local % kGroup;
+        const int g_row = row_local % qg;
         int t_row[NB], lo_row[NB];
         bool row_ok[NB];
         unsigned long long anc[NB];
         float m_ref[NB], l_run[NB];
         #pragma unroll
         for (int blk = 0; blk < NB; ++blk) {
-            t_row[blk] = (block0 + blk) * kTokPerBlock + row_local / kGroup;
-            row_ok[blk] = row_local < kTokPerBlock * kGroup && t_row[blk] < T;
+            t_row[blk] = (block0 + blk) * tpb + row_local / qg;
+            row_ok[blk] = row_local < tpb * qg && t_row[blk] < T;
             // the queries are the last T nodes of the tree
             anc[blk] = (row_ok[blk] && it.key_end > kv_len) ? anc_s[plan.T_tree - T + t_row[blk]] : 0ull;
             lo_row[blk] = row_ok[blk] ? par_s[t_row[blk]] : 0;
@@ -858,7 +863,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                 lse_val = l_all > 0.f ? (m_ref[blk] * c2 + log2f(l_all)) * 0.6931471805599453f : -INFINITY;
             }
             ok = ok && *write_ok == 1u;                                // (thread 0 settled it before the barriers above)
-            const int h_row = it.kvh * kGroup + g_row;
+            const int h_row = it.kvh * qg + g_row;
             // Staging area for coalesced stores: the Q block (every MMA has completed by now).  Row r
             // holds 16 chunks of 16 bytes (128 halves), chunk c stored at position c ^ (r & 15).
             unsigned char* stage = q_sm + blk * kQBlockBytes;
@@ -897,8 +902,8 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
             softmax_bar_sync();                                        // both halves of every staged row are in place
             if (ok && !direct) {
                 // warp w copies rows [16 w, 16 w + 16), two rows (512 contiguous bytes) per instruction
-                const int tok_here = min(kTokPerBlock, max(0, T - (block0 + blk) * kTokPerBlock));
-                const int rows_here = tok_here * kGroup;
+                const int tok_here = min(tpb, max(0, T - (block0 + blk) * tpb));
+                const int rows_here = tok_here * qg;
                 #pragma unroll 4
                 for (int i = 0; i < 8; ++i) {
                     const int r = warp * 16 + 2 * i + (lane >> 4), c = lane & 15;
@@ -916,17 +921,19 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
         // arrival word and one exit word that start at zero; the CTA that exits last puts both back.
         if (sync.enabled || sync.serial) {
             const int fin_idx = (int)blockIdx.x - (plan.n_items - sync.n_fin);     // >= 0: this CTA is a finisher
-            constexpr int kRowsPerBlock = kTokPerBlock * kGroup;       // 126
+            const int kRowsPerBlock = tpb * qg;                        // 126 for 7 heads x 18 tokens
             // The call's row list: for every unit (sequence, KV head, row group) with several pieces,
             // its valid query rows (7 per draft token).  Finisher f takes rows [f chunk, (f + 1) chunk).
             int total = 0;
             for (int b = 0; b < plan.batch; ++b)
-                if (plan.seq[b].n_splits > 1) total += plan.n_kv_heads * kGroup * T;
+                if (plan.seq[b].n_splits > 1) total += plan.n_kv_heads * qg * T;
             const int chunk = sync.n_fin > 0 ? (total + sync.n_fin - 1) / sync.n_fin : 0;
             const int my_begin = fin_idx >= 0 ? min(total, fin_idx * chunk) : 0;
             const int my_end = fin_idx >= 0 ? min(total, my_begin + chunk) : 0;
             const bool merges = my_begin < my_end;
             unsigned* arrive_word = sync.enabled ? sync.arrivals + sync.slot : sync.serial_words;
+            // the pieces are read by the finishers' bulk copies (async proxy): order this thread's stores ahead of them
+            if (!direct) fence_proxy_async_global();
             softmax_bar_sync();                                        // every global store of this CTA has been issued
             if (tid == 0) {
                 if (!direct) publish_counter(arrive_word);
@@ -948,73 +955,82 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
             if (merges) {
                 softmax_bar_sync();
                 if (*fin_go) {
-                    // 16 R G threads merge R rows at a time: thread (row i, 16-byte chunk c, piece group
-                    // g) takes pieces g, g + G, ... of its row, read straight from the workspace (L2;
-                    // thread 0's acquire and the barrier above order these loads behind the pieces'
-                    // stores), ten pieces in flight at a time (one round trip to L2 for a one-wave call), folding them into a running
-                    // (max, sum, weighted output); the groups' results meet in shared memory (the Q
-                    // blocks, idle by now).
-                    constexpr int kFold = 10;                                   // pieces a thread has in flight
+                    // 16 R G threads merge R rows at a time.  The rows' pieces are first brought into the
+                    // (idle) K/V ring by bulk copies, [piece][row][272 bytes], one copy per piece and
+                    // block touched -- far fewer and larger requests than per-thread loads.  (The pieces
+                    // were written with ordinary stores and the copies read through the async proxy: the
+                    // writers issued the proxy fence, before they published their piece.)
+                    // Thread (row i, 16-byte chunk c, piece group g) then folds pieces g, g + G, ... of its
+                    // row into a running (max, sum, weighted output); the groups' results meet in shared
+                    // memory (the Q blocks, idle by now).
+                    constexpr int kRowBytes = kPartRowHalves * 2;               // 272
                     float* red = reinterpret_cast<float*>(q_sm);                // [256][10]: 8 outputs, sum, max
-                    int ubase = 0;
+                    int ubase = 0, phase = 0;
+                    bool fin_ok = true;
                     #pragma unroll 1
                     for (int b = 0; b < plan.batch; ++b) {
                         const int ns = plan.seq[b].n_splits;
                         if (ns == 1) continue;
-                        // rows per pass: a power of two, no more than this finisher has, or than 16
+                        // rows per pass: a power of two, no more than this finisher has, than fit the ring
+                        // with all their pieces, or than 16
                         int R = 1;
                         while (R < 16 && R < chunk) R <<= 1;
+                        while (R > 1 && R * ns * kRowBytes > NS * kStageBytes) R >>= 1;
                         const int G = 16 / R;                                   // piece groups
                         const int c16 = tid & 15, grp_p = (tid >> 4) % G, row_i = tid / (16 * G);
                         const size_t piece_pitch = (size_t)plan.part_rows * kPartRowHalves;      // halves between pieces
                         #pragma unroll 1
                         for (int u = 0; u < plan.n_kv_heads * plan.n_groups; ++u) {
                             const int kvh = u / plan.n_groups, grp = u - kvh * plan.n_groups;
-                            const int tok0 = grp * NB * kTokPerBlock;                        // first token of this row group
-                            const int list_len = kGroup * min(NB * kTokPerBlock, T - tok0);  // its valid rows
+                            const int tok0 = grp * NB * tpb;                        // first token of this row group
+                            const int list_len = qg * min(NB * tpb, T - tok0);  // its valid rows
                             const int row_begin = max(my_begin, ubase) - ubase, row_end = min(my_end, ubase + list_len) - ubase;
                             ubase += list_len;
                             if (row_begin >= row_end) continue;                    // (the same in every thread of the CTA)
                             const size_t item0 = (size_t)plan.seq[b].item_begin + (size_t)u * ns;
                             #pragma unroll 1
-                            for (int r0 = row_begin; r0 < row_end; r0 += R) {
+                            for (int r0 = row_begin; r0 < row_end; r0 += R, phase ^= 1) {
+                                const int n_here = min(R, row_end - r0);
+                                // the rows may straddle the unit's two blocks: rows [r0, split) and [split, r0 + n_here)
+                                const int split = (r0 < kRowsPerBlock && r0 + n_here > kRowsPerBlock) ? kRowsPerBlock : r0 + n_here;
+                                if (tid == 0) mbar_expect_tx(B.fin(), (uint32_t)(n_here * ns * kRowBytes));
+                                softmax_bar_sync();                                // the ring's previous contents have been read, the byte count is posted
+                                {
+                                    const int bk0 = r0 / kRowsPerBlock;
+                                    const __half* first = args.o_part + (item0 * plan.part_rows + (size_t)(bk0 * kBlockRows + r0 - bk0 * kRowsPerBlock)) * kPartRowHalves;
+                                    const __half* second = args.o_part + (item0 * plan.part_rows + (size_t)kBlockRows) * kPartRowHalves;
+                                    for (int sp = tid; sp < ns; sp += 256) {           // thread sp brings piece sp
+                                        const uint32_t dst = smem_u32(kv_sm) + (uint32_t)(sp * n_here * kRowBytes);
+                                        bulk_load(dst, first + (size_t)sp * piece_pitch, (uint32_t)(split - r0) * kRowBytes, B.fin());
+                                        if (split < r0 + n_here)
+                                            bulk_load(dst + (uint32_t)(split - r0) * kRowBytes, second + (size_t)sp * piece_pitch,
+                                                      (uint32_t)(r0 + n_here - split) * kRowBytes, B.fin());
+                                    }
+                                }
+                                fin_ok = fin_ok && mbar_wait_warp(B.fin(), phase);
                                 const int idx = r0 + row_i;                            // row of the unit's list: token idx / 7, head idx % 7
-                                const bool active = idx < row_end;
-                                const int bk = idx / kRowsPerBlock;
-                                const __half* row0 = args.o_part + (item0 * plan.part_rows + (size_t)(bk * kBlockRows + idx - bk * kRowsPerBlock)) * kPartRowHalves;
+                                const bool active = fin_ok && row_i < n_here;
+                                const uint32_t pstride = (uint32_t)n_here * kRowBytes;     // bytes between pieces in the ring
+                                const uint32_t row_sm = smem_u32(kv_sm) + (uint32_t)row_i * kRowBytes;
                                 float m_run = -INFINITY, s_run = 0.f;                  // natural-log units
                                 float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
                                 if (active) {
-                                    #pragma unroll 1
-                                    for (int sp0 = grp_p; sp0 < ns; sp0 += kFold * G) {
-                                        float l4[kFold];
-                                        uint4 o4[kFold];
+                                    #pragma unroll 2
+                                    for (uint32_t sp = grp_p, a_o = row_sm + grp_p * pstride; sp < (uint32_t)ns; sp += G, a_o += G * pstride) {
+                                        const float l = lds_f32(a_o + 2 * kD);
+                                        uint32_t raw[4];
+                                        lds_v4(a_o + c16 * 16, raw);
+                                        if (l == -INFINITY) continue;                  // a piece that saw no visible key
+                                        const float m_new = fmaxf(m_run, l);
+                                        const float a = ex2((m_run - m_new) * 1.4426950408889634f);   // 0 for the first piece
+                                        const float w = ex2((l - m_new) * 1.4426950408889634f);
+                                        s_run = fmaf(s_run, a, w);
                                         #pragma unroll
-                                        for (int k = 0; k < kFold; ++k) {
-                                            const int sp = sp0 + k * G;
-                                            l4[k] = -INFINITY;
-                                            o4[k] = make_uint4(0, 0, 0, 0);
-                                            if (sp < ns) {
-                                                const __half* pr = row0 + (size_t)sp * piece_pitch;
-                                                l4[k] = __ldcg(reinterpret_cast<const float*>(pr + kD));
-                                                o4[k] = __ldcg(reinterpret_cast<const uint4*>(pr) + c16);
-                                            }
+                                        for (int q = 0; q < 4; ++q) {
+                                            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&raw[q]));
+                                            acc[2 * q] = fmaf(acc[2 * q], a, w * f.x); acc[2 * q + 1] = fmaf(acc[2 * q + 1], a, w * f.y);
                                         }
-                                        #pragma unroll
-                                        for (int k = 0; k < kFold; ++k) {
-                                            if (l4[k] == -INFINITY) continue;          // a piece that saw no visible key (or none at all)
-                                            const float m_new = fmaxf(m_run, l4[k]);
-                                            const float a = ex2((m_run - m_new) * 1.4426950408889634f);   // 0 for the first piece
-                                            const float w = ex2((l4[k] - m_new) * 1.4426950408889634f);
-                                            const uint32_t* raw = reinterpret_cast<const uint32_t*>(&o4[k]);
-                                            s_run = fmaf(s_run, a, w);
-                                            #pragma unroll
-                                            for (int q = 0; q < 4; ++q) {
-                                                const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&raw[q]));
-                                                acc[2 * q] = fmaf(acc[2 * q], a, w * f.x); acc[2 * q + 1] = fmaf(acc[2 * q + 1], a, w * f.y);
-                                            }
-                                            m_run = m_new;
-                                        }
+                                        m_run = m_new;
                                     }
                                 }
                                 if (G > 1) {                                           // (G is the same in every thread)
@@ -1044,8 +1060,8 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                                     }
                                 }
                                 if (active && grp_p == 0) {
-                                    const int t = tok0 + idx / kGroup;
-                                    const int h = kvh * kGroup + idx % kGroup;
+                                    const int t = tok0 + idx / qg;
+                                    const int h = kvh * qg + idx % qg;
                                     const float inv = s_run > 0.f ? __fdividef(1.f, s_run) : 0.f;
                                     uint4 pk;
                                     pk.x = pack_bf16x2(acc[0] * inv, acc[1] * inv); pk.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
@@ -1056,6 +1072,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                             }
                         }
                     }
+                    if (!fin_ok) atomicOr(args.status, timeout_bits(kSiteFinCopies));
                 }
                 softmax_bar_sync();
             }

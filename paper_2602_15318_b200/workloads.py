@@ -199,14 +199,15 @@ class AnchorCase:
 
 def make_verify_case(seed: int, kv_len: List[int], T: int, tree: str = "chain", device="cpu",
                      capacity: Optional[int] = None, heavy_frac: float = 0.0,
-                     n_visual: Optional[List[int]] = None, name: str = "") -> VerifyCase:
-    """tree: "chain", "random" (seeded, depth <= 8, <= 4 children) or "forest" (all roots)."""
+                     n_visual: Optional[List[int]] = None, name: str = "", hq: int = HQ, hkv: int = HKV) -> VerifyCase:
+    """tree: "chain", "random" (seeded, depth <= 8, <= 4 children) or "forest" (all roots).
+    hq / hkv: query and KV heads (28 / 4 unless a test asks for another GQA ratio)."""
     B = len(kv_len)
     cap = capacity if capacity is not None else max(kv_len) + T
     assert cap >= max(kv_len) + T
-    q = normal_bf16(seed, _TID_Q, (B, T, HQ, D), device)
-    k = normal_bf16(seed, _TID_K, (B, HKV, cap, D), device)
-    v = normal_bf16(seed, _TID_V, (B, HKV, cap, D), device)
+    q = normal_bf16(seed, _TID_Q, (B, T, hq, D), device)
+    k = normal_bf16(seed, _TID_K, (B, hkv, cap, D), device)
+    v = normal_bf16(seed, _TID_V, (B, hkv, cap, D), device)
     par = []
     for b in range(B):
         if tree == "chain":
@@ -223,8 +224,8 @@ def make_verify_case(seed: int, kv_len: List[int], T: int, tree: str = "chain", 
         for b in range(B):
             nv = n_visual[b] if n_visual is not None else kv_len[b]
             n_heavy = int(math.floor(heavy_frac * nv))
-            for h in range(HKV):
-                qbar = q[b, :, h * GROUP:(h + 1) * GROUP, :].float().mean(dim=(0, 1))
+            for h in range(hkv):
+                qbar = q[b, :, h * (hq // hkv):(h + 1) * (hq // hkv), :].float().mean(dim=(0, 1))
                 rows = sample_without_replacement(seed + 104729 * b + h, _TID_HEAVY, nv, n_heavy)
                 ridx = torch.tensor(rows, dtype=torch.long, device=device)
                 k[b, h, ridx, :] = (k[b, h, ridx, :].float() + 2.0 * qbar).to(torch.bfloat16)

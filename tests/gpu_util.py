@@ -12,11 +12,11 @@ TOL_LSE = 1e-3      # max |lse_gpu - lse_oracle|
 
 
 def run_verify(case: W.VerifyCase, ctx=None, policy=None):
-    ctx = ctx or B.Context.for_cache(case.k, W.SCALE)
+    ctx = ctx or B.Context.for_cache(case.k, W.SCALE, n_q_heads=case.q.shape[2])
     if policy is not None:
         ctx.set_plan_policy(policy)
     out = torch.full_like(case.q, float("nan"))
-    lse = torch.full((case.B, W.HQ, case.T), float("nan"), dtype=torch.float32, device=case.q.device)
+    lse = torch.full((case.B, case.q.shape[2], case.T), float("nan"), dtype=torch.float32, device=case.q.device)
     B.sparrow_verify_attn(ctx, case.q, case.k, case.v, case.kv_len, case.parents, case.T, out, lse)
     torch.cuda.synchronize()
     assert ctx.last_device_status() == 0

@@ -121,6 +121,56 @@ def test_verify_on_side_stream():
     check(out, lse, ref_out, ref_lse)
 
 
+# ---- other head geometries (query heads per KV head from 1 to 16) ----------------------------------
+
+@pytest.mark.parametrize("hq,hkv,kv_len,T,tree,policy", [
+    (32, 8, [3000, 700], 12, "random", B.PLAN_LATENCY),        # group 4: 32 tokens per row block
+    (32, 8, [2000], 40, "random", B.PLAN_THROUGHPUT),          # group 4, two row blocks
+    (32, 4, [2500], 16, "chain", B.PLAN_BALANCED),             # group 8: 16 tokens per block, no padding rows
+    (32, 4, [1500, 90], 33, "random", B.PLAN_LATENCY),         # group 8: three blocks -> two row groups
+    (8, 8, [1800], 64, "random", B.PLAN_LATENCY),              # multi-head attention: one head per KV head
+    (16, 1, [4000], 9, "random", B.PLAN_THROUGHPUT),           # multi-query attention, group 16: 8 tokens per block
+    (16, 1, [600], 64, "random", B.PLAN_LATENCY),              # group 16: eight blocks, four row groups
+    (12, 4, [1000, 1000, 5], 50, "random", B.PLAN_BALANCED),   # group 3: 42 tokens per block
+    (10, 2, [777], 26, "chain", B.PLAN_LATENCY),               # group 5: 25 tokens per block, 3 rows of padding
+])
+def test_verify_other_gqa_ratios(hq, hkv, kv_len, T, tree, policy):
+    case = W.make_verify_case(3300 + hq + T, kv_len, T, tree, DEV, hq=hq, hkv=hkv)
+    out, lse, _ = run_verify(case, policy=policy)
+    ref_out, ref_lse = oracle_verify(case)
+    check(out, lse, ref_out, ref_lse)
+
+
+def test_anchored_modes_with_another_gqa_ratio():
+    """Group 4 (32 / 8 heads): the gather kernel, and the compacted cache with a cutting window."""
+    hq, hkv, T = 32, 8, 10
+    idx = oracle.anchor_idx(6000, [[50, 4000]], 1200, T).tolist()
+    base = W.make_verify_case(3400, [idx[-1] + 1 - T], T, "chain", DEV, hq=hq, hkv=hkv)       # tensors only
+    anchor = torch.tensor([idx], dtype=torch.int32, device=DEV)
+    parents = torch.tensor([W.random_tree_parents(3401, 99, T)], dtype=torch.int32, device=DEV)
+    ctx = B.Context.for_cache(base.k, W.SCALE, n_q_heads=hq)
+    ref = oracle.anchor_attn_tree(W.bf16_bits(base.q), W.bf16_bits(base.k), W.bf16_bits(base.v), anchor.cpu().numpy(), 1200,
+                                  parents.cpu().numpy(), W.SCALE)
+    out = torch.full_like(base.q, float("nan"))
+    lse = torch.full((1, hq, T), float("nan"), dtype=torch.float32, device=DEV)
+    B.sparrow_anchor_attn_tree(ctx, base.q, base.k, base.v, anchor, len(idx), 1200, parents, T, T, out, lse)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == 0
+    check(out, lse, *ref)
+    kc = torch.zeros((1, hkv, len(idx), W.D), dtype=torch.bfloat16, device=DEV)
+    vc = torch.zeros_like(kc)
+    B.sparrow_compact_anchors(ctx, base.k, base.v, anchor, len(idx), kc, vc, len(idx), 0)
+    first = torch.empty((1, T), dtype=torch.int32, device=DEV)
+    B.sparrow_window_first_visible_device(ctx, anchor, len(idx), 1200, T, T, first)
+    cctx = B.Context.for_cache(kc, W.SCALE, n_q_heads=hq)
+    out2 = torch.full_like(base.q, float("nan"))
+    lse2 = torch.full((1, hq, T), float("nan"), dtype=torch.float32, device=DEV)
+    B.sparrow_verify_attn_window(cctx, base.q, kc, vc, [len(idx) - T], parents, T, T, first, None, out2, lse2)
+    torch.cuda.synchronize()
+    assert cctx.last_device_status() == 0
+    check(out2, lse2, *ref)
+
+
 # ---- masks and indices: bit-exact -----------------------------------------------------------
 
 def test_device_ancestor_masks_bit_exact():
@@ -315,7 +365,9 @@ def test_argument_errors_launch_nothing():
         B.sparrow_verify_attn(bare, case.q, case.k, case.v, case.kv_len, case.parents, 4, out, lse)
     assert e.value.status == 5
     with pytest.raises(B.SparrowError):
-        B.Context(1, 100, 51200, 12800, W.SCALE, n_q_heads=32)       # not 7:1
+        B.Context(1, 100, 51200, 12800, W.SCALE, n_q_heads=30)       # not a multiple of the 4 KV heads
+    with pytest.raises(B.SparrowError):
+        B.Context(1, 100, 51200, 12800, W.SCALE, n_q_heads=68)       # 17 query heads per KV head: more than 16
     with pytest.raises(B.SparrowError):
         B.Context(1, 100, 51200, 12800, W.SCALE, head_dim=64, n_q_heads=28)
     assert ctx.launch_count() == n0
