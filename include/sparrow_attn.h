@@ -90,8 +90,8 @@ sparrow_status sparrow_destroy(sparrow_ctx* ctx);
  *   THROUGHPUT  about n_sm / 7 items: longest pieces, several calls resident at once; best when
  *               many independent calls are queued back to back (one per layer or per request).
  * Results differ between policies only by the rounding order of the split-KV merge.  Calls that
- * cannot overlap (stream-ordered mode, graph capture, sparrow_anchor_attn,
- * sparrow_verify_attn_static) always use one wave over all SMs. */
+ * cannot overlap (graph capture, SPARROW_NO_PDL, sparrow_anchor_attn, sparrow_verify_attn_static)
+ * always use one wave over all SMs. */
 typedef enum {
     SPARROW_PLAN_LATENCY    = 0,
     SPARROW_PLAN_BALANCED   = 1,
@@ -151,8 +151,8 @@ sparrow_status sparrow_set_workspace(sparrow_ctx* ctx, void* dev_ptr, size_t byt
  * through counters in its workspace.  All calls of a context belong on one stream (or must be kept
  * from running concurrently by events): the counters assume that calls run in the order they were
  * enqueued.  While a stream is being captured into a graph, or with SPARROW_NO_PDL=1 in the
- * environment when the context is created, a call is two ordinary launches (split-KV pass,
- * combine) ordered by the stream alone.
+ * environment when the context is created, a call is two ordinary launches (split-KV pass over
+ * one wave of pieces, combine kernel) ordered by the stream alone and touches no counter.
  * Results are deterministic for fixed arguments. */
 sparrow_status sparrow_verify_attn(sparrow_ctx* ctx, const void* q, const void* k_cache,
                                    const void* v_cache, const int32_t* kv_len,
@@ -391,7 +391,8 @@ sparrow_status sparrow_verify_step_host(sparrow_ctx* ctx, const void* q_host,
  *     1 KiB header: a call has max(SM count, batch x KV heads x row groups) work items of at most
  *     70 KB each, so on a 148-SM part everything fits except very large batches of draft blocks
  *     longer than 18 tokens (e.g. 32 sequences x 64 tokens); nothing is enqueued then either.
- *   - The call always runs in the stream-ordered mode: two ordinary kernel launches on `stream`.
+ *   - The call always runs in the stream-ordered mode: two ordinary kernel launches on `stream`
+ *     (one when no sequence needs more than one piece).
  *   - All calls on a device share the one array, which keeps the previous call's contents.  What
  *     must start clean (the status word) is cleared on `stream` at the start of every call;
  *     partials are always written before they are read.  Calls that overlap on the GPU (two

@@ -85,7 +85,6 @@ constexpr size_t kFinDoneOffset = 64;
 constexpr size_t kArrivalsOffset = 128;     // words 32..35: arrival words of the four call slots
 constexpr size_t kHsrCountersOffset = 256;  // words 64..255: one arrival counter per 128-feature tile of sparrow_hsr_fuse()
 constexpr int kHsrMaxFeatureTiles = 192;
-constexpr size_t kSerialOffset = 192;       // words 48, 49: arrival / exit words of a call that runs alone (serial mode)
 constexpr int kMinPieceKeys = 128;
 // The gathered kernel works on 64-key tiles and pays two dependent memory round trips per tile
 // (anchor indices, then the rows), which a CTA with several tiles takes one after the other: short
@@ -306,15 +305,12 @@ void note_fused_launch(sparrow_ctx* c, const CallRanges& cr, bool launched_early
 
 // `after_previous`: the call's final results must wait for the previous fused call as a whole (its
 // outputs overlap that call's memory); otherwise they only wait for the calls before that one.
-// `self_merging`: the kernel merges its own partials (the tensor-core kernel); a call of it that
-// cannot overlap its neighbours runs in serial mode.
-SyncArgs next_sync(const sparrow_ctx* c, const SplitPlan& p, bool overlaps, bool after_previous, bool self_merging)
+SyncArgs next_sync(const sparrow_ctx* c, const SplitPlan& p, bool overlaps, bool after_previous)
 {
     SyncArgs sy;
     const int parity = (int)(c->seq & 1u);
     sy.arrivals = reinterpret_cast<unsigned*>(c->ws + kArrivalsOffset);
     sy.fin_done = reinterpret_cast<unsigned*>(c->ws + kFinDoneOffset);
-    sy.serial_words = reinterpret_cast<unsigned*>(c->ws + kSerialOffset);
     sy.enabled = overlaps ? 1 : 0;
     sy.parity = parity;
     sy.slot = (int)(c->seq & 3u);
@@ -322,11 +318,9 @@ SyncArgs next_sync(const sparrow_ctx* c, const SplitPlan& p, bool overlaps, bool
     for (int b = 0; b < p.batch; ++b)
         if (p.seq[b].n_splits > 1) n_arrive += p.n_kv_heads * p.n_groups * p.seq[b].n_splits;
     sy.n_arrive = n_arrive;
-    sy.serial = (!overlaps && self_merging && n_arrive > 0) ? 1 : 0;
     // Finishers wait, holding their SM, until the call's last piece is in: few of them where later
-    // calls should move in beside this one, all CTAs where the call has the GPU to itself anyway
-    // (serial mode, and the one-wave latency policy).
-    const bool all_finish = sy.serial || (overlaps && c->plan_policy == SPARROW_PLAN_LATENCY);
+    // calls should move in beside this one, all CTAs under the one-wave latency policy.
+    const bool all_finish = overlaps && c->plan_policy == SPARROW_PLAN_LATENCY;
     sy.n_fin = n_arrive == 0 ? 0 : ((all_finish || p.n_items < kFinisherCtas) ? p.n_items : kFinisherCtas);
     sy.fin_wait_same = c->fin_total[parity];
     sy.fin_wait_other = after_previous ? c->fin_total[parity ^ 1] : c->fin_before_last[parity ^ 1];
@@ -453,7 +447,7 @@ void clear_tensor_maps(sparrow_ctx* c)
 
 sparrow_status launch_verify_tc(sparrow_ctx* c, const SplitPlan& plan, const SyncArgs& sy, const void* q, const void* k, const void* v,
                                 const int32_t* parents, const int32_t* first_visible, void* out, float* lse, cudaStream_t st,
-                                bool may_start_early, bool* started_early)
+                                bool start_early)
 {
     CUtensorMap mq, mk, mv;
     if (!tensor_map_for(c, q, plan.batch * plan.T, &mq) || !tensor_map_for(c, k, 0, &mk) || !tensor_map_for(c, v, 0, &mv))
@@ -478,16 +472,10 @@ sparrow_status launch_verify_tc(sparrow_ctx* c, const SplitPlan& plan, const Syn
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    // The early start reaches back to the kernel launched directly before this one in the stream,
-    // whatever it is, so it is only taken where that kernel is known: this context's previous
-    // fused call (the counters order this context's own calls and know nothing about another
-    // context's writes), with nothing enqueued in between as far as the library can tell -- the
-    // calls after the first of sparrow_verify_attn_batch(), or any call once the caller has vouched
-    // for the stream with sparrow_set_call_overlap().  Every other launch takes plain stream order.
-    const bool same_ctx_before = g_last_fused_ctx.exchange(c) == c;
-    const bool early = sy.enabled && same_ctx_before && may_start_early;
-    cfg.numAttrs = early ? 1 : 0;
-    if (started_early) *started_early = early;
+    // A call may start early behind the kernel launched directly before it in the stream only
+    // where the caller of this function has made sure that that kernel is this context's previous
+    // call; every other launch takes plain stream order.
+    cfg.numAttrs = start_early ? 1 : 0;
     const cudaError_t e = nb == 1 ? cudaLaunchKernelEx(&cfg, tc::verify_tc_kernel<1>, a, sy, plan, mq, mk, mv)
                                   : cudaLaunchKernelEx(&cfg, tc::verify_tc_kernel<2>, a, sy, plan, mq, mk, mv);
     if (e != cudaSuccess) return SPARROW_ERR_CUDA;
@@ -559,28 +547,40 @@ sparrow_status verify_call(sparrow_ctx* c, const void* q, const void* k, const v
     DeviceGuard guard(c->device);
     if (!guard.ok) return SPARROW_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const bool overlaps = call_overlaps(c, st, true);
+    // Outside stream capture (and with programmatic launch on) a call takes part in the counter
+    // protocol and merges its own pieces.  Whether it also STARTS EARLY, overlapping the previous
+    // call, is a separate decision: only where the kernel directly before it in the stream is known
+    // to be this context's previous call (the counters order this context's own calls and know
+    // nothing about another context's writes; nothing else can sit in between for the calls after
+    // the first of sparrow_verify_attn_batch(), or once the caller has vouched for the stream with
+    // sparrow_set_call_overlap()), and where it reads nothing that a call which may still be
+    // running writes.  Every other launch takes plain stream order.  A captured call is two plain
+    // launches: the split-KV pass and the combine kernel.
+    const CallRanges cr = call_ranges(c, q, k, v, parents, T_tree, T, first_visible, out, lse);
+    const bool protocol = call_overlaps(c, st, true);                // not capturing, programmatic launch on
+    const bool same_ctx_before = g_last_fused_ctx.exchange(c) == c;
+    const bool early = protocol && same_ctx_before && (c->chain_next || c->overlap_single_calls) &&
+                       !inputs_touch_recent_outputs(c, cr);
     SplitPlan plan;
     const int group = layout_group(c->layout);
-    sparrow_status s = make_plan(plan_target(c, overlaps), c->layout.batch, c->layout.n_kv_heads, group, n_keys, T,
+    sparrow_status s = make_plan(plan_target(c, protocol), c->layout.batch, c->layout.n_kv_heads, group, n_keys, T,
                                  blocks_per_group_tc(T, group), &plan, kMinPieceKeys, key0);
     if (s != SPARROW_OK) return s;
     plan.T_tree = T_tree;
     for (int b = 0; b < c->layout.batch; ++b) plan.seq[b].kv_len = kv_len[b];
     if ((s = check_ws(c, plan)) != SPARROW_OK) return s;
-    const CallRanges cr = call_ranges(c, q, k, v, parents, T_tree, T, first_visible, out, lse);
-    const SyncArgs sy = next_sync(c, plan, overlaps, outputs_touch_previous(c, cr), true);
-    const bool may_start_early = overlaps && (c->chain_next || c->overlap_single_calls) && !inputs_touch_recent_outputs(c, cr);
-    bool started_early = false;
-    if ((s = launch_verify_tc(c, plan, sy, q, k, v, parents, first_visible, out, lse, st, may_start_early, &started_early)) != SPARROW_OK)
-        return s;
-    advance_sync(c, plan, sy);
-    if (sy.enabled) {
+    const SyncArgs sy = next_sync(c, plan, protocol, outputs_touch_previous(c, cr));
+    if ((s = launch_verify_tc(c, plan, sy, q, k, v, parents, first_visible, out, lse, st, early)) != SPARROW_OK) return s;
+    if (protocol) {
+        advance_sync(c, plan, sy);
         std::memcpy(c->prev_ranges, cr.r, sizeof(cr.r));
         c->prev_valid = true;
-        note_fused_launch(c, cr, started_early);
+        note_fused_launch(c, cr, early);
+        return SPARROW_OK;                                   // the kernel merges its own partials
     }
-    return SPARROW_OK;                                       // the kernel merges its own partials in either mode
+    bool needs_combine = false;
+    for (int b = 0; b < plan.batch; ++b) needs_combine = needs_combine || plan.seq[b].n_splits > 1;
+    return needs_combine ? launch_combine(c, plan, sy, out, lse, st) : SPARROW_OK;
 }
 
 }  // namespace
@@ -848,9 +848,8 @@ sparrow_status sparrow_verify_attn_static(const sparrow_layout* L, const void* q
         return SPARROW_ERR_SHAPE;
     if (check_ws(c, plan) != SPARROW_OK) return SPARROW_ERR_WORKSPACE;
     // the status word is the one thing that must start clean
-    // the status word must start clean, and so must the two words of the serial merge (an earlier call that gave up
-    // on a wait may have left them behind)
-    if (cudaMemsetAsync(c->ws, 0, 256, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SPARROW_ERR_CUDA;
+    // the status word is the one thing that must start clean
+    if (cudaMemsetAsync(c->ws, 0, sizeof(unsigned), static_cast<cudaStream_t>(stream)) != cudaSuccess) return SPARROW_ERR_CUDA;
     return sparrow_verify_attn(c, q, k, v, kv_len, parents, T, out, lse, stream);
 }
 
@@ -890,7 +889,7 @@ sparrow_status anchor_call(sparrow_ctx* c, const void* q, const void* k, const v
     DeviceGuard guard(c->device);
     if (!guard.ok) return SPARROW_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const SyncArgs sy = next_sync(c, plan, false, true, false);
+    const SyncArgs sy = next_sync(c, plan, false, true);
     // the two kernels of the call are chained programmatically unless the stream is being captured
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
     if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) { cudaGetLastError(); cap = cudaStreamCaptureStatusActive; }

@@ -88,19 +88,12 @@ constexpr int kPartRowHalves = 136;
 // results land in call order.  CTA 0 then clears the arrival word of slot (n + 2) % 4: its last
 // user was call n-2, and the items of call n+2 cannot arrive before the finishers of call n are
 // done, which in turn have seen CTA 0's arrival (or, if it had none, follow it in the stream).
-//
-// Serial mode (enabled == 0, serial == 1): the call is an ordinary launch that runs alone between
-// its neighbours in the stream (stream capture, programmatic launch switched off, the entry point
-// without a workspace).  It touches none of the counters above and never lets dependents launch
-// early; its CTAs arrive on serial_words[0], every CTA is a finisher, and the CTA that leaves last
-// (serial_words[1] counts them) puts both words back to zero -- so the same launch can be replayed
-// from a graph.  With both flags zero (the gathered kernel) a separate combine kernel follows.
+// With enabled == 0 the kernels are ordered by the stream alone: they touch no counter, and a
+// separate combine kernel follows the split-KV kernel.
 struct SyncArgs {
     unsigned* arrivals;      // [4]
     unsigned* fin_done;      // [2]
-    unsigned* serial_words;  // [2] serial mode: arrivals of the running call, CTAs that have left it
     int32_t enabled;         // overlapped mode
-    int32_t serial;          // serial mode: the call runs alone between its neighbours in the stream, and merges its own partials
     int32_t parity;          // n % 2
     int32_t slot;            // n % 4
     int32_t n_arrive;        // items of this call that store partials

@@ -37,10 +37,11 @@
 // is launched with programmatic stream serialisation and never waits for the previous grid as a
 // whole.  All reads of q / k / v / parents are issued as soon as the CTA starts, so the K/V stream
 // of this call overlaps the tail of the previous one; in front of its first global write a CTA
-// waits on the finisher counters.  Serial mode: the call runs alone between its neighbours in the
-// stream.  In both, a CTA publishes its item after storing its partials, and the call's finisher
-// CTAs wait for the arrivals, share the call's rows among them, merge each row's pieces by
-// log-sum-exp and write out / lse.
+// waits on the finisher counters.  A CTA publishes its item after storing its partials, and the
+// call's finisher CTAs wait for the arrivals, share the call's rows among them, merge each row's
+// pieces by log-sum-exp and write out / lse.  Stream-ordered mode (a call captured into a graph, or
+// with programmatic launch switched off): the kernel touches no counter, only stores partials and
+// direct results, and the combine kernel follows.
 //
 // Every wait is bounded; a wait that gives up sets the timeout status bit and the CTA drains and
 // exits.  TMEM is always released.
@@ -916,10 +917,9 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
         }
 
         // ---- publish this item; the call's finisher CTAs merge its partials ---------------------------
-        // Overlapped mode (sync.enabled): arrival words and finisher counters as described at SyncArgs.
-        // Serial mode (sync.serial; the call runs alone between its neighbours in the stream): one
-        // arrival word and one exit word that start at zero; the CTA that exits last puts both back.
-        if (sync.enabled || sync.serial) {
+        // (overlapped mode: arrival words and finisher counters as described at SyncArgs; a
+        // stream-ordered call only stores its partials, and a combine kernel follows)
+        if (sync.enabled) {
             const int fin_idx = (int)blockIdx.x - (plan.n_items - sync.n_fin);     // >= 0: this CTA is a finisher
             const int kRowsPerBlock = tpb * qg;                        // 126 for 7 heads x 18 tokens
             // The call's row list: for every unit (sequence, KV head, row group) with several pieces,
@@ -931,7 +931,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
             const int my_begin = fin_idx >= 0 ? min(total, fin_idx * chunk) : 0;
             const int my_end = fin_idx >= 0 ? min(total, my_begin + chunk) : 0;
             const bool merges = my_begin < my_end;
-            unsigned* arrive_word = sync.enabled ? sync.arrivals + sync.slot : sync.serial_words;
+            unsigned* arrive_word = sync.arrivals + sync.slot;
             // the pieces are read by the finishers' bulk copies (async proxy): order this thread's stores ahead of them
             if (!direct) fence_proxy_async_global();
             softmax_bar_sync();                                        // every global store of this CTA has been issued
@@ -940,7 +940,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                 if (merges) {
                     // every partial of the call in place, and (overlapped mode) the previous call's final results written
                     // (both words are polled in one loop: the second is usually there already)
-                    bool have_all = false, prev_done = !sync.enabled;
+                    bool have_all = false, prev_done = false;
                     #pragma unroll 1
                     for (uint32_t i = 0; i < kCounterPolls && !(have_all && prev_done); ++i) {
                         if (!have_all) have_all = ld_acquire(arrive_word) == (unsigned)sync.n_arrive;
@@ -1077,17 +1077,8 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                 softmax_bar_sync();
             }
             if (tid == 0) {
-                if (sync.enabled) {
-                    if (direct) publish_counter(sync.fin_done + sync.parity);
-                    if (fin_idx >= 0) publish_counter(sync.fin_done + sync.parity);
-                } else {
-                    // serial mode: the last CTA to leave puts the two words back to zero for the next call
-                    __threadfence();
-                    if (atomicAdd(sync.serial_words + 1, 1u) == (unsigned)plan.n_items - 1u) {
-                        sync.serial_words[0] = 0u;
-                        sync.serial_words[1] = 0u;
-                    }
-                }
+                if (direct) publish_counter(sync.fin_done + sync.parity);
+                if (fin_idx >= 0) publish_counter(sync.fin_done + sync.parity);
             }
         }
         if (!ok) { atomicOr(args.status, timeout_bits(kSiteSoftmax)); *abort_flag = 1; }

@@ -90,15 +90,15 @@ def test_anchor_and_verify_calls_interleave():
 
 
 def test_stream_ordered_mode(monkeypatch):
-    """SPARROW_NO_PDL=1 at context creation: every call is one ordinary launch that merges its own
-    pieces (serial mode), ordered by the stream alone."""
+    """SPARROW_NO_PDL=1 at context creation: every call is ordered by the stream alone and touches no
+    counter -- the split-KV pass and, where a sequence has several pieces, the combine kernel."""
     monkeypatch.setenv("SPARROW_NO_PDL", "1")
     for kv, T, tree in [([3000, 1500], 12, "random"), ([129], 19, "random"), ([64], 8, "chain")]:
         case = W.make_verify_case(610 + T, kv, T, tree, DEV)
         ctx = _overlapping_ctx(case.k)
         n0 = ctx.launch_count()
         out, lse, _ = run_verify(case, ctx)
-        assert ctx.launch_count() - n0 == 1
+        assert ctx.launch_count() - n0 == (2 if max(kv) + T > 128 else 1)
         check(out, lse, *oracle_verify(case))
 
 
@@ -182,7 +182,7 @@ def test_long_stream_is_bitwise_reproducible(policy):
     ctx = _overlapping_ctx(cases[0].k)
     ctx.set_plan_policy(policy)
     alone = []
-    for c in cases:
+    for c in cases:                                # (each call alone on the GPU: the stream is drained after it)
         out, lse = _new(c)
         B.sparrow_verify_attn(ctx, c.q, c.k, c.v, c.kv_len, c.parents, c.T, out, lse)
         torch.cuda.synchronize()
