@@ -68,6 +68,7 @@ def compare(out, lse, ref_out, ref_lse, rows=None):
 
 def check(out, lse, ref_out, ref_lse, rows=None):
     d_out, d_lse = compare(out, lse, ref_out, ref_lse, rows)
+    print(f"[parity] max|d out| = {d_out:.3e}  max|d lse| = {d_lse:.3e}  ({ref_lse.size} rows)")     # shown by pytest -s
     assert d_out <= TOL_OUT, f"max |d out| = {d_out}"
     assert d_lse <= TOL_LSE, f"max |d lse| = {d_lse}"
     return d_out, d_lse
