@@ -76,7 +76,9 @@ typedef struct {
 
 typedef struct sparrow_ctx sparrow_ctx;
 
-/* Creates a context on CUDA device `device` (queries the SM count, loads the kernels).
+/* Creates a context on CUDA device `device` (queries the SM count, loads the kernels).  With
+ * SPARROW_LOG=1 in the environment the context prints one line per verification call on stderr
+ * (the split plan and how the call is launched); SPARROW_NO_PDL=1 switches programmatic launch off.
  * SPARROW_ERR_ARCH unless the device is sm_100; SPARROW_ERR_CUDA when no usable device exists. */
 sparrow_status sparrow_create(sparrow_ctx** ctx, const sparrow_layout* layout, int device);
 sparrow_status sparrow_destroy(sparrow_ctx* ctx);

@@ -61,6 +61,7 @@ struct sparrow_ctx {
     int part_buffers;                        // 2: alternate by call parity (fused mode); 1: stream-ordered calls only
     std::atomic<long long> launches;
     bool use_pdl;
+    bool log_plans;                          // SPARROW_LOG=1 when the context was created: one line per call on stderr
     bool overlap_single_calls;               // sparrow_set_call_overlap()
     bool chain_next;                         // the call being enqueued directly follows this context's previous fused call
     // Host mirror of the ordering counters in the workspace (see SyncArgs): call sequence number
@@ -570,6 +571,14 @@ sparrow_status verify_call(sparrow_ctx* c, const void* q, const void* k, const v
     for (int b = 0; b < c->layout.batch; ++b) plan.seq[b].kv_len = kv_len[b];
     if ((s = check_ws(c, plan)) != SPARROW_OK) return s;
     const SyncArgs sy = next_sync(c, plan, protocol, outputs_touch_previous(c, cr));
+    if (c->log_plans) {
+        std::fprintf(stderr, "[sparrow] verify call %u: T %d of %d nodes, %d row block(s) x %d group(s), %d items (target %d), %s, %s;",
+                     c->seq, T, T_tree, plan.blocks_per_group, plan.n_groups, plan.n_items, plan_target(c, protocol),
+                     protocol ? "counter protocol" : "stream-ordered", early ? "starts early" : "plain launch");
+        for (int b = 0; b < plan.batch; ++b)
+            std::fprintf(stderr, " seq %d: keys [%d, %d) in %d piece(s)", b, plan.seq[b].key0, plan.seq[b].n_keys, plan.seq[b].n_splits);
+        std::fprintf(stderr, "; %d finisher(s)\n", sy.n_fin);
+    }
     if ((s = launch_verify_tc(c, plan, sy, q, k, v, parents, first_visible, out, lse, st, early)) != SPARROW_OK) return s;
     if (protocol) {
         advance_sync(c, plan, sy);
@@ -651,6 +660,8 @@ sparrow_status sparrow_create(sparrow_ctx** out, const sparrow_layout* L, int de
     // more SMs than the list of possibly-resident calls can hold: calls never start early
     c->use_pdl = !(e && e[0] == '1') && c->n_sm < kRecentCalls;
     c->overlap_single_calls = false;
+    const char* lg = std::getenv("SPARROW_LOG");
+    c->log_plans = lg && lg[0] == '1';
     c->chain_next = false;
     c->n_recent = c->recent_head = 0;
     c->seq = 0;

@@ -364,3 +364,13 @@ def test_many_caches_through_one_context():
         B.sparrow_verify_attn(ctx, qs[i:i + 1], ks[i:i + 1], vs[i:i + 1], [kv], base.parents, T, outs[i:i + 1], lses[i:i + 1])
     torch.cuda.synchronize()
     assert torch.equal(first, outs)
+
+
+def test_plan_log_line(monkeypatch, capfd):
+    """SPARROW_LOG=1 at context creation: one line per verification call on stderr."""
+    monkeypatch.setenv("SPARROW_LOG", "1")
+    case = W.make_verify_case(990, [3000], 20, "random", DEV)
+    out, lse, ctx = run_verify(case)
+    check(out, lse, *oracle_verify(case))
+    err = capfd.readouterr().err
+    assert "[sparrow] verify call" in err and "2 row block(s)" in err and "keys [0, 3020)" in err
