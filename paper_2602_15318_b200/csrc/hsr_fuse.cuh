@@ -147,38 +147,31 @@ hsr_fuse_kernel(const __grid_constant__ HsrArgs args, const __grid_constant__ CU
             if (!ok) { atomicOr(args.status, timeout_bits(kSiteMma)); *abort_flag = 1; }
         }
     } else {
-        // ---- epilogue warps: thread = one output feature (TMEM lane), 64 token columns, handled 16
-        // at a time in rolled loops: this code runs once per CTA, from a cold instruction cache, so
-        // its size is what it costs
+        // ---- epilogue warps: thread = one output feature (TMEM lane), 64 token columns
         bool ok = n_kt == 0 || mbar_wait_warp(done, 0);
         tc_fence_after();
-        if (!ok) { atomicOr(args.status, timeout_bits(kSiteSoftmax)); *abort_flag = 1; }
         const int feat = f_tile * kFeat + warp * 32 + lane;
-        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+        float acc[64];
+        if (ok && n_kt > 0) {
+            tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16), acc);
+            tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + 32, acc + 32);
+            tmem_wait_ld();
+        } else {
+            #pragma unroll
+            for (int t = 0; t < 64; ++t) acc[t] = 0.f;
+        }
+        if (!ok) { atomicOr(args.status, timeout_bits(kSiteSoftmax)); *abort_flag = 1; }
         const float b = args.bias ? __bfloat162float(args.bias[feat]) : 0.f;
-        const bool have_acc = ok && n_kt > 0;
         if (args.n_slices == 1) {
-            #pragma unroll 1
-            for (int t0 = 0; t0 < args.M; t0 += 16) {
-                float acc[16];
-                tmem_ld16(lane_addr + t0, acc);
-                tmem_wait_ld();
-                #pragma unroll
-                for (int t = 0; t < 16; ++t)
-                    if (t0 + t < args.M) args.z[(size_t)(t0 + t) * args.d_out + feat] = __float2bfloat16((have_acc ? acc[t] : 0.f) + b);
-            }
+            #pragma unroll
+            for (int t = 0; t < 64; ++t)
+                if (t < args.M) args.z[(size_t)t * args.d_out + feat] = __float2bfloat16(acc[t] + b);
         } else {
             // partial sums as [slice][token][feature]: the 32 features of a warp are 128 contiguous bytes
             float* mine = args.partial + (size_t)slice * kTok * args.d_out + feat;
-            #pragma unroll 1
-            for (int t0 = 0; t0 < args.M; t0 += 16) {
-                float acc[16];
-                tmem_ld16(lane_addr + t0, acc);
-                tmem_wait_ld();
-                #pragma unroll
-                for (int t = 0; t < 16; ++t)
-                    if (t0 + t < args.M) mine[(size_t)(t0 + t) * args.d_out] = have_acc ? acc[t] : 0.f;
-            }
+            #pragma unroll
+            for (int t = 0; t < 64; ++t)
+                if (t < args.M) mine[(size_t)t * args.d_out] = acc[t];
             asm volatile("bar.sync 1, 128;" ::: "memory");             // every store of this item has been issued
             if (tid == 0) {
                 // release (cumulative over the stores the barrier ordered before it) and acquire in one
@@ -189,34 +182,29 @@ hsr_fuse_kernel(const __grid_constant__ HsrArgs args, const __grid_constant__ CU
             }
             asm volatile("bar.sync 1, 128;" ::: "memory");
             if (*is_last) {
-                // The slices in fixed order, whoever arrived last (every slice, its own included, is
-                // read back: the sum must not depend on who is last); 16 tokens of up to 4 slices in
-                // flight at a time.
+                // The slices in fixed order, whoever arrived last (its own slice comes from its
+                // registers: the same values it stored); all loads of a slice in flight at once.
+                // (Two slices in flight, or a sum shared among the tile's items, measured slower.)
+                float sum[64];
+                #pragma unroll
+                for (int t = 0; t < 64; ++t) sum[t] = 0.f;
                 #pragma unroll 1
-                for (int t0 = 0; t0 < args.M; t0 += 16) {
-                    float sum[16];
-                    #pragma unroll
-                    for (int t = 0; t < 16; ++t) sum[t] = 0.f;
-                    #pragma unroll 1
-                    for (int s0 = 0; s0 < args.n_slices; s0 += 4) {
-                        float v[4][16];
+                for (int s2 = 0; s2 < args.n_slices; ++s2) {
+                    if (s2 == slice) {
                         #pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            const float* src = args.partial + ((size_t)(s0 + k) * kTok + t0) * args.d_out + feat;
-                            #pragma unroll
-                            for (int t = 0; t < 16; ++t)
-                                v[k][t] = (s0 + k < args.n_slices && t0 + t < args.M) ? __ldcg(src + (size_t)t * args.d_out) : 0.f;
-                        }
+                        for (int t = 0; t < 64; ++t) sum[t] += acc[t];
+                    } else {
+                        const float* src = args.partial + (size_t)s2 * kTok * args.d_out + feat;
+                        float v[64];
                         #pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            #pragma unroll
-                            for (int t = 0; t < 16; ++t) sum[t] += v[k][t];
-                        }
+                        for (int t = 0; t < 64; ++t) v[t] = t < args.M ? __ldcg(src + (size_t)t * args.d_out) : 0.f;
+                        #pragma unroll
+                        for (int t = 0; t < 64; ++t) sum[t] += v[t];
                     }
-                    #pragma unroll
-                    for (int t = 0; t < 16; ++t)
-                        if (t0 + t < args.M) args.z[(size_t)(t0 + t) * args.d_out + feat] = __float2bfloat16(sum[t] + b);
                 }
+                #pragma unroll
+                for (int t = 0; t < 64; ++t)
+                    if (t < args.M) args.z[(size_t)t * args.d_out + feat] = __float2bfloat16(sum[t] + b);
             }
         }
     }
