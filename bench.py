@@ -435,8 +435,9 @@ def main():
         "clocks": clocks,
         "e2e": {"value": us_e2e, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": e2e_steps,
-                "what": "sparrow_verify_step_host: pinned host q / new K,V rows / parents in, out + lse back, "
-                        "stream synchronised every step (latency policy); the committed KV prefix stays resident"},
+                "what": "sparrow_verify_step_host: pinned host q / new K,V rows / parents read over the host link "
+                        "by the ingest kernel every step, out + lse stored into pinned host memory by the attention "
+                        "kernel, stream synchronised every step (latency policy); the committed KV prefix stays resident"},
         "gpu_launches": launches_timed,
     }
     if rank == 0 and not args.no_cpu_baseline and world == 1:

@@ -362,7 +362,12 @@ sparrow_status sparrow_kv_keep_accepted(sparrow_ctx* ctx, void* k_cache, void* v
  *   v_new_host   HOST bf16 [batch][n_kv_heads][T][128]
  *   parents_host HOST int32 [batch][T]  (validated on the host: SPARROW_ERR_TREE)
  *   out_host     HOST bf16 [batch][T][n_q_heads][128];  lse_host HOST fp32 [batch][n_q_heads][T]
- * Device staging comes from the registered workspace; nothing is allocated. */
+ * Device staging comes from the registered workspace; nothing is allocated.
+ * When all six host buffers are page-locked (cudaHostAlloc / cudaHostRegister) and 16-byte
+ * aligned, no copy engine is involved: one kernel reads q, parents and the new rows from host
+ * memory (q and parents into staging, the rows into the cache) and the attention kernel stores
+ * out / lse into the host buffers; otherwise every buffer goes through cudaMemcpyAsync.  The
+ * results are the same bits either way; the host buffers must not change until the call returns. */
 sparrow_status sparrow_verify_step_host(sparrow_ctx* ctx, const void* q_host,
                                         const void* k_new_host, const void* v_new_host,
                                         void* k_cache, void* v_cache, const int32_t* kv_len,

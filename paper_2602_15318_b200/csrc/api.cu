@@ -95,7 +95,7 @@ constexpr int kMinGatherPieceKeys = 64;
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Staging {
-    size_t q, out, lse, parents, total;
+    size_t q, out, lse, parents, k_new, v_new, total;
 };
 
 Staging staging_layout(const sparrow_layout& L)
@@ -106,7 +106,9 @@ Staging staging_layout(const sparrow_layout& L)
     s.out = s.q + align_up(B * kMaxT * L.n_q_heads * kD * 2, 256);
     s.lse = s.out + align_up(B * kMaxT * L.n_q_heads * kD * 2, 256);
     s.parents = s.lse + align_up(B * kMaxT * L.n_q_heads * 4, 256);
-    s.total = s.parents + align_up(B * kMaxT * 4, 256);
+    s.k_new = s.parents + align_up(B * kMaxT * 4, 256);
+    s.v_new = s.k_new + align_up(B * L.n_kv_heads * kMaxT * kD * 2, 256);
+    s.total = s.v_new + align_up(B * L.n_kv_heads * kMaxT * kD * 2, 256);
     return s;
 }
 
@@ -180,6 +182,19 @@ bool layout_heads_ok(const sparrow_layout& L)
 int layout_group(const sparrow_layout& L) { return L.n_q_heads / L.n_kv_heads; }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Device-side address of a host buffer that kernels can reach themselves (page-locked memory,
+// which unified addressing maps into every device; 16-byte aligned), else nullptr: the caller
+// then goes through copies.
+template <class P>
+P* device_view(P* host)
+{
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, host) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    if (at.type != cudaMemoryTypeHost || !at.devicePointer || !aligned16(at.devicePointer)) return nullptr;
+    return static_cast<P*>(at.devicePointer);
+}
+
 
 size_t fixed_bytes(const sparrow_layout& L) { return kStatusBytes + staging_layout(L).total; }
 size_t part_bytes(size_t rows) { return align_up(rows * kPartRowHalves * sizeof(__half), 256); }
@@ -338,6 +353,9 @@ void advance_sync(sparrow_ctx* c, const SplitPlan& p, const SyncArgs& sy)
 
 // Context of the most recent fused launch in this process (any stream): see launch_verify_tc().
 std::atomic<sparrow_ctx*> g_last_fused_ctx{nullptr};
+// Any other kernel this library enqueues breaks the "directly before" knowledge: the next
+// verification call takes a plain launch behind it.
+inline void other_kernel_enqueued() { g_last_fused_ctx.store(nullptr); }
 
 sparrow_status launch_combine(sparrow_ctx* c, const SplitPlan& plan, const SyncArgs& sy, void* out, float* lse, cudaStream_t st,
                               bool programmatic = false)
@@ -388,6 +406,7 @@ sparrow_status launch_split_gather(sparrow_ctx* c, const SplitPlan& plan, const 
     a.lse = lse;
     a.status = reinterpret_cast<unsigned*>(c->ws);
     a.early_dependents = early_dependents ? 1 : 0;
+    other_kernel_enqueued();
     gather::split_gather_kernel<<<plan.n_items, gather::kThreads, gather::kSmemBytes, st>>>(plan, a);
     if (cudaGetLastError() != cudaSuccess) return SPARROW_ERR_CUDA;
     c->launches.fetch_add(1);
@@ -963,6 +982,7 @@ sparrow_status sparrow_kv_append(sparrow_ctx* c, const void* k_new, const void* 
     DeviceGuard guard(c->device);
     if (!guard.ok) return SPARROW_ERR_CUDA;
     const long long threads = (long long)L.batch * L.n_kv_heads * T * 16;
+    other_kernel_enqueued();
     move_rows_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(a);
     if (cudaGetLastError() != cudaSuccess) return SPARROW_ERR_CUDA;
     c->launches.fetch_add(1);
@@ -1001,6 +1021,7 @@ sparrow_status sparrow_compact_anchors(sparrow_ctx* c, const void* k, const void
     const long long threads = (long long)L.batch * L.n_kv_heads * n_anchor * 16;
     long long blocks = (threads + 255) / 256;
     if (blocks > 8LL * c->n_sm) blocks = 8LL * c->n_sm;
+    other_kernel_enqueued();
     move_rows_kernel<<<(unsigned)blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(a);
     if (cudaGetLastError() != cudaSuccess) return SPARROW_ERR_CUDA;
     c->launches.fetch_add(1);
@@ -1036,6 +1057,7 @@ sparrow_status sparrow_window_first_visible_device(sparrow_ctx* c, const int32_t
     DeviceGuard guard(c->device);
     if (!guard.ok) return SPARROW_ERR_CUDA;
     const int n = c->layout.batch * T_new;
+    other_kernel_enqueued();
     window_bounds_kernel<<<(n + 127) / 128, 128, 0, static_cast<cudaStream_t>(stream)>>>(anchor_idx, n_anchor, window, T_tree, T_new,
                                                                                          c->layout.batch, first_visible);
     if (cudaGetLastError() != cudaSuccess) return SPARROW_ERR_CUDA;
@@ -1102,6 +1124,7 @@ sparrow_status sparrow_hsr_fuse(sparrow_ctx* c, const void* e, const void* h, co
     a.M = M; a.d = d; a.d_out = d_out;
     a.n_slices = n_slices;
     a.k_tiles = 2 * d / hsr::kKTile;
+    other_kernel_enqueued();
     hsr::hsr_fuse_kernel<<<(d_out / hsr::kFeat) * n_slices, hsr::kThreadsHsr, hsr::kSmemBytes, static_cast<cudaStream_t>(stream)>>>(a, mw, me, mh);
     if (cudaGetLastError() != cudaSuccess) return SPARROW_ERR_CUDA;
     c->launches.fetch_add(1);
@@ -1117,6 +1140,7 @@ sparrow_status sparrow_accept_greedy(sparrow_ctx* c, const int32_t* draft_tokens
     if (!c->ws) return SPARROW_ERR_WORKSPACE;
     DeviceGuard guard(c->device);
     if (!guard.ok) return SPARROW_ERR_CUDA;
+    other_kernel_enqueued();
     accept_greedy_kernel<<<1, kMaxBatch, 0, static_cast<cudaStream_t>(stream)>>>(
         draft_tokens, parents, target_next, c->layout.batch, T, path_out, n_accept_out, bonus_out,
         reinterpret_cast<unsigned*>(c->ws));
@@ -1135,6 +1159,7 @@ sparrow_status sparrow_accept_sample(sparrow_ctx* c, const int32_t* draft_tokens
     if (!c->ws) return SPARROW_ERR_WORKSPACE;
     DeviceGuard guard(c->device);
     if (!guard.ok) return SPARROW_ERR_CUDA;
+    other_kernel_enqueued();
     sample::accept_sample_kernel<<<c->layout.batch, sample::kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
         draft_tokens, parents, p_target, p_draft, u_node, u_bonus, T, vocab, path_out, n_accept_out, bonus_out,
         reinterpret_cast<unsigned*>(c->ws));
@@ -1166,6 +1191,7 @@ sparrow_status sparrow_kv_keep_accepted(sparrow_ctx* c, void* k_cache, void* v_c
     a.stride_head = L.kv_stride_head;
     DeviceGuard guard(c->device);
     if (!guard.ok) return SPARROW_ERR_CUDA;
+    other_kernel_enqueued();
     keep_accepted_rows_kernel<<<L.batch * L.n_kv_heads, 256, (size_t)2 * T * 256, static_cast<cudaStream_t>(stream)>>>(a);
     if (cudaGetLastError() != cudaSuccess) return SPARROW_ERR_CUDA;
     c->launches.fetch_add(1);
@@ -1199,22 +1225,60 @@ sparrow_status sparrow_verify_step_host(sparrow_ctx* c, const void* q_host, cons
     int32_t* par_dev = reinterpret_cast<int32_t*>(base + sl.parents);
     const size_t q_bytes = (size_t)L.batch * T * L.n_q_heads * kD * 2;
     const size_t lse_bytes = (size_t)L.batch * L.n_q_heads * T * 4;
+    const size_t new_bytes = (size_t)L.batch * L.n_kv_heads * T * kD * 2;
+    // Host buffers the GPU can address itself (pinned or registered memory) are not copied by the
+    // copy engine at all: one kernel reads q, the tree and the new K/V rows over the host link,
+    // and the attention kernel writes out / lse straight into the host buffers.
+    const void* q_view = device_view(q_host);
+    const void* kn_view = device_view(k_new_host);
+    const void* vn_view = device_view(v_new_host);
+    const void* par_view = device_view(parents_host);
+    void* out_view = device_view(out_host);
+    void* lse_view = device_view(lse_host);
+    if (q_view && kn_view && vn_view && par_view && out_view && lse_view) {
+        IngestArgs ia;
+        std::memset(&ia, 0, sizeof ia);
+        for (int b = 0; b < L.batch; ++b) ia.rows.dst_row0[b] = kv_len[b];
+        ia.rows.k_src = static_cast<const __nv_bfloat16*>(kn_view);
+        ia.rows.v_src = static_cast<const __nv_bfloat16*>(vn_view);
+        ia.rows.k_dst = static_cast<__nv_bfloat16*>(k_cache);
+        ia.rows.v_dst = static_cast<__nv_bfloat16*>(v_cache);
+        ia.rows.n_rows = T;
+        ia.rows.batch = L.batch;
+        ia.rows.n_kv_heads = L.n_kv_heads;
+        ia.rows.src_capacity = T;
+        ia.rows.src_stride_head = (int64_t)T * kD;
+        ia.rows.src_stride_batch = ia.rows.src_stride_head * L.n_kv_heads;
+        ia.rows.dst_stride_batch = L.kv_stride_batch;
+        ia.rows.dst_stride_head = L.kv_stride_head;
+        ia.rows.status = reinterpret_cast<unsigned*>(c->ws);
+        ia.q_src = static_cast<const uint4*>(q_view);
+        ia.q_dst = static_cast<uint4*>(q_dev);
+        ia.q_chunks = (int32_t)(q_bytes / 16);
+        ia.parents_src = static_cast<const int32_t*>(par_view);
+        ia.parents_dst = par_dev;
+        ia.n_parents = L.batch * T;
+        const long long work = (long long)(new_bytes / 16) + ia.q_chunks + ia.n_parents;
+        other_kernel_enqueued();
+        ingest_step_kernel<<<(unsigned)((work + 255) / 256), 256, 0, st>>>(ia);
+        if (cudaGetLastError() != cudaSuccess) return SPARROW_ERR_CUDA;
+        c->launches.fetch_add(1);
+        const sparrow_status s = sparrow_verify_attn(c, q_dev, k_cache, v_cache, kv_len, par_dev, T, out_view,
+                                                     static_cast<float*>(lse_view), stream);
+        if (s != SPARROW_OK) return s;
+        return cudaStreamSynchronize(st) == cudaSuccess ? SPARROW_OK : SPARROW_ERR_CUDA;
+    }
     if (cudaMemcpyAsync(q_dev, q_host, q_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return SPARROW_ERR_CUDA;
     if (cudaMemcpyAsync(par_dev, parents_host, (size_t)L.batch * T * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return SPARROW_ERR_CUDA;
-    const size_t row_block = (size_t)T * kD * 2;             // T new rows of one (batch, KV head)
-    for (int b = 0; b < L.batch; ++b) {
-        const size_t dst_off = ((size_t)b * L.kv_stride_batch + (size_t)kv_len[b] * kD) * 2;
-        const size_t src_off = (size_t)b * L.n_kv_heads * row_block;
-        if (cudaMemcpy2DAsync(static_cast<unsigned char*>(k_cache) + dst_off, (size_t)L.kv_stride_head * 2,
-                              static_cast<const unsigned char*>(k_new_host) + src_off, row_block, row_block,
-                              L.n_kv_heads, cudaMemcpyHostToDevice, st) != cudaSuccess)
-            return SPARROW_ERR_CUDA;
-        if (cudaMemcpy2DAsync(static_cast<unsigned char*>(v_cache) + dst_off, (size_t)L.kv_stride_head * 2,
-                              static_cast<const unsigned char*>(v_new_host) + src_off, row_block, row_block,
-                              L.n_kv_heads, cudaMemcpyHostToDevice, st) != cudaSuccess)
-            return SPARROW_ERR_CUDA;
-    }
+    // the new rows: one contiguous copy each into the staging area, then the append kernel puts them
+    // into the cache rows
+    void* k_new_dev = base + sl.k_new;
+    void* v_new_dev = base + sl.v_new;
+    if (cudaMemcpyAsync(k_new_dev, k_new_host, new_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return SPARROW_ERR_CUDA;
+    if (cudaMemcpyAsync(v_new_dev, v_new_host, new_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return SPARROW_ERR_CUDA;
+    const sparrow_status as = sparrow_kv_append(c, k_new_dev, v_new_dev, k_cache, v_cache, kv_len, T, stream);
+    if (as != SPARROW_OK) return as;
     const sparrow_status s = sparrow_verify_attn(c, q_dev, k_cache, v_cache, kv_len, par_dev, T, out_dev, lse_dev, stream);
     if (s != SPARROW_OK) return s;
     if (cudaMemcpyAsync(out_host, out_dev, q_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return SPARROW_ERR_CUDA;
@@ -1264,6 +1328,7 @@ sparrow_status sparrow_debug_ancestor_masks_device(sparrow_ctx* c, const int32_t
     if (!c->ws) return SPARROW_ERR_WORKSPACE;
     DeviceGuard guard(c->device);
     if (!guard.ok) return SPARROW_ERR_CUDA;
+    other_kernel_enqueued();
     ancestor_masks_kernel<<<1, kMaxT, 0, static_cast<cudaStream_t>(stream)>>>(
         parents_dev, T, reinterpret_cast<unsigned long long*>(masks_dev), reinterpret_cast<unsigned*>(c->ws));
     if (cudaGetLastError() != cudaSuccess) return SPARROW_ERR_CUDA;

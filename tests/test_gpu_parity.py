@@ -343,6 +343,42 @@ def test_verify_step_host_matches_device_call():
     check(out_h, lse_h, ref_out, ref_lse)
 
 
+def test_verify_step_host_pinned_buffers_twice():
+    """All six host buffers page-locked: the kernels read and write them over the host link.  The
+    second step reuses the same host buffers with other contents, so a stale cached line would show."""
+    ctx = None
+    bufs = None
+    for seed, lens in [(93, [1500, 700]), (94, [1490, 333])]:
+        case = W.make_verify_case(seed, lens, 12, "random", DEV, capacity=2048)
+        ref_out, ref_lse = oracle_verify(case)
+        T = case.T
+        if ctx is None:
+            ctx = B.Context.for_cache(case.k, W.SCALE)
+            bufs = dict(q=torch.empty(case.q.shape, dtype=case.q.dtype).pin_memory(),
+                        k=torch.empty((2, W.HKV, T, W.D), dtype=case.k.dtype).pin_memory(),
+                        v=torch.empty((2, W.HKV, T, W.D), dtype=case.k.dtype).pin_memory(),
+                        par=torch.empty((2, T), dtype=torch.int32).pin_memory(),
+                        out=torch.empty(case.q.shape, dtype=case.q.dtype).pin_memory(),
+                        lse=torch.empty((2, W.HQ, T), dtype=torch.float32).pin_memory())
+        bufs["q"].copy_(case.q)
+        bufs["k"].copy_(torch.stack([case.k[b, :, n:n + T, :] for b, n in enumerate(case.kv_len)]))
+        bufs["v"].copy_(torch.stack([case.v[b, :, n:n + T, :] for b, n in enumerate(case.kv_len)]))
+        bufs["par"].copy_(case.parents)
+        bufs["out"].zero_(); bufs["lse"].zero_()
+        torch.cuda.synchronize()
+        for b, n in enumerate(case.kv_len):
+            case.k[b, :, n:n + T, :] = 0
+            case.v[b, :, n:n + T, :] = 0
+        n0 = ctx.launch_count()
+        B.sparrow_verify_step_host(ctx, bufs["q"], bufs["k"], bufs["v"], case.k, case.v, case.kv_len,
+                                   bufs["par"], T, bufs["out"], bufs["lse"])
+        assert ctx.launch_count() - n0 == 2          # the ingest kernel and the attention kernel
+        check(bufs["out"], bufs["lse"], ref_out, ref_lse)
+        for b, n in enumerate(case.kv_len):          # the new rows reached the cache bit for bit
+            assert torch.equal(case.k[b, :, n:n + T, :].cpu(), bufs["k"][b])
+            assert torch.equal(case.v[b, :, n:n + T, :].cpu(), bufs["v"][b])
+
+
 def test_argument_errors_launch_nothing():
     case = W.make_verify_case(92, [100], 4, "chain", DEV)
     ctx = B.Context.for_cache(case.k, W.SCALE)
