@@ -469,13 +469,12 @@ def run_only(args, W, B, torch, dev, l2, steps, warmup):
         h_ = W.normal_bf16(W.config_seed(5), 62, (m_tok, d_model), dev)
         z_ = torch.empty((m_tok, d_model), dtype=torch.bfloat16, device=dev)
         hctx = B.Context.for_cache(torch.empty((1, W.HKV, 128, W.D), dtype=torch.bfloat16, device=dev), W.SCALE)
-        scratch = torch.empty(max(16, B.sparrow_hsr_scratch_bytes(hctx, d_model, d_model)), dtype=torch.uint8, device=dev)
 
         def run(n):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             torch.cuda.synchronize(); e0.record()
             for i in range(n):
-                B.sparrow_hsr_fuse(hctx, e_, h_, ws_[i % n_w], None, z_, scratch)
+                B.sparrow_hsr_fuse(hctx, e_, h_, ws_[i % n_w], None, z_)
             e1.record(); torch.cuda.synchronize()
             return e0.elapsed_time(e1) * 1e3 / n
         run(warmup)
@@ -633,16 +632,15 @@ def extra_configs(W, B, torch, dev, l2, peak, peaks, anchored_variants):
     z_ = torch.empty((m_tok, d_model), dtype=torch.bfloat16, device=dev)
     hk = torch.empty((1, W.HKV, 128, W.D), dtype=torch.bfloat16, device=dev)
     hctx = B.Context.for_cache(hk, W.SCALE)
-    scratch = torch.empty(max(16, B.sparrow_hsr_scratch_bytes(hctx, d_model, d_model)), dtype=torch.uint8, device=dev)
     side = torch.cuda.Stream()
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.stream(side):
         for w_ in ws_:
-            B.sparrow_hsr_fuse(hctx, e_, h_, w_, b_, z_, scratch, stream=side)
+            B.sparrow_hsr_fuse(hctx, e_, h_, w_, b_, z_, stream=side)
         side.synchronize()
         with torch.cuda.graph(graph, stream=side):
             for w_ in ws_:
-                B.sparrow_hsr_fuse(hctx, e_, h_, w_, b_, z_, scratch, stream=side)
+                B.sparrow_hsr_fuse(hctx, e_, h_, w_, b_, z_, stream=side)
         graph.replay(); side.synchronize()
         g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         g0.record(side)

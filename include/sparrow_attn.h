@@ -285,17 +285,14 @@ sparrow_status sparrow_compact_anchors(sparrow_ctx* ctx, const void* k, const vo
  * has a bias, so `bias` may be NULL.  The concatenation is never materialised.
  *   e, h     DEV bf16 [M][d], dense          w  DEV bf16 [d_out][2 d], dense (torch.nn.Linear layout)
  *   bias     DEV bf16 [d_out] or NULL        z  DEV bf16 [M][d_out]
- *   scratch  DEV, 16-byte aligned, >= sparrow_hsr_scratch_bytes(ctx, d, d_out) bytes (split-K
- *            partial sums; may be NULL when that is 0); caller-owned, free again when the call has run
- * One kernel, ordered by the stream; fp32 accumulation in a fixed order (results are
- * deterministic).  The context provides the status word and per-tile counters (its workspace must
- * be registered) -- its layout is not used.
- * SPARROW_ERR_SHAPE unless 1 <= M <= 64, d a multiple of 64, d_out a multiple of 128 (at most
- * 24,576) and the pointers 16-byte aligned; SPARROW_ERR_WORKSPACE when scratch is too small. */
-size_t sparrow_hsr_scratch_bytes(const sparrow_ctx* ctx, int32_t d, int32_t d_out);
+ * One kernel, ordered by the stream: a split-K pass whose slices meet inside a thread-block
+ * cluster (no scratch memory, no counters); fp32 accumulation in a fixed order (results are
+ * deterministic).  The context provides the status word (its workspace must be registered) -- its
+ * layout is not used.
+ * SPARROW_ERR_SHAPE unless 1 <= M <= 64, d a multiple of 64, d_out a multiple of 128 and the
+ * pointers 16-byte aligned. */
 sparrow_status sparrow_hsr_fuse(sparrow_ctx* ctx, const void* e, const void* h, const void* w, const void* bias,
-                                int32_t M, int32_t d, int32_t d_out, void* scratch, size_t scratch_bytes,
-                                void* z, void* stream);
+                                int32_t M, int32_t d, int32_t d_out, void* z, void* stream);
 
 /* After the verification pass (Appendix A, "Speculative Decoding": the target keeps exactly what it
  * would have produced itself; the paper relies on the standard procedure and does not restate it).

@@ -28,7 +28,7 @@ EXPORTS = ["sparrow_create", "sparrow_destroy", "sparrow_workspace_bytes", "spar
            "sparrow_set_plan_policy", "sparrow_set_call_overlap", "sparrow_debug_early_trigger_copy",
            "sparrow_verify_attn_window", "sparrow_window_first_visible", "sparrow_window_first_visible_device",
            "sparrow_plan_target_items", "sparrow_anchor_attn_tree", "sparrow_kv_append", "sparrow_compact_anchors",
-           "sparrow_hsr_scratch_bytes", "sparrow_hsr_fuse", "sparrow_accept_greedy", "sparrow_accept_sample", "sparrow_kv_keep_accepted", "sparrow_plan_piece_range",
+           "sparrow_hsr_fuse", "sparrow_accept_greedy", "sparrow_accept_sample", "sparrow_kv_keep_accepted", "sparrow_plan_piece_range",
            "sparrow_status_string"]
 
 
@@ -74,9 +74,7 @@ def lib():
         L.sparrow_anchor_attn.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp]
         L.sparrow_plan_piece_range.argtypes = [i32, i32, i32, vp, vp]
         L.sparrow_accept_greedy.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp]
-        L.sparrow_hsr_scratch_bytes.argtypes = [vp, i32, i32]
-        L.sparrow_hsr_scratch_bytes.restype = ctypes.c_size_t
-        L.sparrow_hsr_fuse.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp, ctypes.c_size_t, vp, vp]
+        L.sparrow_hsr_fuse.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp, vp]
         L.sparrow_accept_sample.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp]
         L.sparrow_kv_keep_accepted.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp]
         L.sparrow_kv_append.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp]
@@ -101,7 +99,7 @@ def lib():
         L.sparrow_status_string.argtypes = [ctypes.c_int]
         L.sparrow_status_string.restype = ctypes.c_char_p
         for name in EXPORTS:
-            if name not in ("sparrow_workspace_bytes", "sparrow_hsr_scratch_bytes", "sparrow_launch_count", "sparrow_status_string",
+            if name not in ("sparrow_workspace_bytes", "sparrow_launch_count", "sparrow_status_string",
                             "sparrow_debug_status_word", "sparrow_plan_target_items"):
                 getattr(L, name).restype = ctypes.c_int
         _lib = L
@@ -307,17 +305,13 @@ def sparrow_accept_greedy(ctx: Context, draft_tokens, parents, target_next, T: i
          "sparrow_accept_greedy")
 
 
-def sparrow_hsr_scratch_bytes(ctx: Context, d: int, d_out: int) -> int:
-    return int(lib().sparrow_hsr_scratch_bytes(ctx.handle, d, d_out))
-
-
-def sparrow_hsr_fuse(ctx: Context, e, h, w, bias, z, scratch=None, stream=None):
+def sparrow_hsr_fuse(ctx: Context, e, h, w, bias, z, stream=None):
     """z = [e | h] @ w.T (+ bias).  e, h: CUDA bf16 [M, d]; w: CUDA bf16 [d_out, 2d]; bias: CUDA bf16
-    [d_out] or None; z: CUDA bf16 [M, d_out]; scratch: CUDA uint8 tensor of sparrow_hsr_scratch_bytes."""
+    [d_out] or None; z: CUDA bf16 [M, d_out]."""
     M, d = e.shape
     d_out = w.shape[0]
-    _chk(lib().sparrow_hsr_fuse(ctx.handle, _ptr(e), _ptr(h), _ptr(w), _ptr(bias), M, d, d_out, _ptr(scratch),
-                                scratch.numel() if scratch is not None else 0, _ptr(z), _stream_handle(stream)),
+    _chk(lib().sparrow_hsr_fuse(ctx.handle, _ptr(e), _ptr(h), _ptr(w), _ptr(bias), M, d, d_out, _ptr(z),
+                                _stream_handle(stream)),
          "sparrow_hsr_fuse")
 
 

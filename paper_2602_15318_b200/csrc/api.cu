@@ -84,8 +84,6 @@ namespace {
 constexpr size_t kStatusBytes = 1024;      // word 0: sticky status; words 16, 17: finisher counters
 constexpr size_t kFinDoneOffset = 64;
 constexpr size_t kArrivalsOffset = 128;     // words 32..35: arrival words of the four call slots
-constexpr size_t kHsrCountersOffset = 256;  // words 64..255: one arrival counter per 128-feature tile of sparrow_hsr_fuse()
-constexpr int kHsrMaxFeatureTiles = 192;
 constexpr int kMinPieceKeys = 128;
 // The gathered kernel works on 64-key tiles and pays two dependent memory round trips per tile
 // (anchor indices, then the rows), which a CTA with several tiles takes one after the other: short
@@ -1068,30 +1066,23 @@ sparrow_status sparrow_window_first_visible_device(sparrow_ctx* c, const int32_t
 // K-range slices per feature tile: about one work item per SM, never more slices than K tiles.
 static int hsr_slices(int n_sm, int d, int d_out)
 {
+    // slices of one feature tile = CTAs of one cluster: a power of two up to the portable limit of
+    // 8, at most one wave over the SMs (clusters of 5 x 28 tiles did not all fit at once: slower)
     const int f_tiles = d_out / hsr::kFeat, k_tiles = 2 * d / hsr::kKTile;
-    int s = n_sm / f_tiles;
-    if (s < 1) s = 1;
-    if (s > k_tiles) s = k_tiles;
+    int s = 1;
+    while (s < 8 && 2 * s * f_tiles <= n_sm && 2 * s <= k_tiles) s *= 2;
     return s;
 }
 
-size_t sparrow_hsr_scratch_bytes(const sparrow_ctx* c, int32_t d, int32_t d_out)
-{
-    if (!c || d < 64 || (d % 64) != 0 || d_out < 128 || (d_out % 128) != 0) return 0;
-    return (size_t)hsr_slices(c->n_sm, d, d_out) * d_out * hsr::kTok * sizeof(float);
-}
-
 sparrow_status sparrow_hsr_fuse(sparrow_ctx* c, const void* e, const void* h, const void* w, const void* bias, int32_t M,
-                                int32_t d, int32_t d_out, void* scratch, size_t scratch_bytes, void* z, void* stream)
+                                int32_t d, int32_t d_out, void* z, void* stream)
 {
     if (!c || !e || !h || !w || !z) return SPARROW_ERR_NULL;
-    if (M < 1 || M > hsr::kTok || d < 64 || (d % 64) != 0 || d_out < 128 || (d_out % 128) != 0 ||
-        d_out / hsr::kFeat > kHsrMaxFeatureTiles)
+    if (M < 1 || M > hsr::kTok || d < 64 || (d % 64) != 0 || d_out < 128 || (d_out % 128) != 0)
         return SPARROW_ERR_SHAPE;
-    if (!aligned16(e) || !aligned16(h) || !aligned16(w) || !aligned16(z) || (scratch && !aligned16(scratch))) return SPARROW_ERR_SHAPE;
-    if (!c->ws) return SPARROW_ERR_WORKSPACE;                       // status word and the tiles' arrival counters live there
+    if (!aligned16(e) || !aligned16(h) || !aligned16(w) || !aligned16(z)) return SPARROW_ERR_SHAPE;
+    if (!c->ws) return SPARROW_ERR_WORKSPACE;                       // the status word lives there
     const int n_slices = hsr_slices(c->n_sm, d, d_out);
-    if (n_slices > 1 && (!scratch || scratch_bytes < (size_t)n_slices * d_out * hsr::kTok * sizeof(float))) return SPARROW_ERR_WORKSPACE;
     if (!c->encode) return SPARROW_ERR_CUDA;
     DeviceGuard guard(c->device);
     if (!guard.ok) return SPARROW_ERR_CUDA;
@@ -1117,16 +1108,25 @@ sparrow_status sparrow_hsr_fuse(sparrow_ctx* c, const void* e, const void* h, co
         return SPARROW_ERR_CUDA;
     HsrArgs a;
     a.bias = static_cast<const __nv_bfloat16*>(bias);
-    a.partial = static_cast<float*>(scratch);
     a.z = static_cast<__nv_bfloat16*>(z);
-    a.counters = reinterpret_cast<unsigned*>(c->ws + kHsrCountersOffset);
     a.status = reinterpret_cast<unsigned*>(c->ws);
     a.M = M; a.d = d; a.d_out = d_out;
     a.n_slices = n_slices;
     a.k_tiles = 2 * d / hsr::kKTile;
     other_kernel_enqueued();
-    hsr::hsr_fuse_kernel<<<(d_out / hsr::kFeat) * n_slices, hsr::kThreadsHsr, hsr::kSmemBytes, static_cast<cudaStream_t>(stream)>>>(a, mw, me, mh);
-    if (cudaGetLastError() != cudaSuccess) return SPARROW_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((d_out / hsr::kFeat) * n_slices));
+    cfg.blockDim = dim3(hsr::kThreadsHsr);
+    cfg.dynamicSmemBytes = hsr::kSmemBytes;
+    cfg.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;              // the slices of a feature tile share a cluster
+    attr[0].val.clusterDim.x = (unsigned)n_slices;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, hsr::hsr_fuse_kernel, a, mw, me, mh) != cudaSuccess) { cudaGetLastError(); return SPARROW_ERR_CUDA; }
     c->launches.fetch_add(1);
     return SPARROW_OK;
 }

@@ -11,9 +11,12 @@
 // weights are the M-side operand (128 features), the tokens the N side (64 columns, rows past M
 // read as zero):  D[128 features x 64 tokens] += W_tile[128 x 16] X_tile[64 x 16]^T  on tcgen05,
 // operands staged by TMA through a 6-stage mbarrier ring (16 KB of weights + 8 KB of activations per
-// stage), accumulator in TMEM.  Each item stores its fp32 partial tile; the item that arrives last on
-// its feature tile's counter adds the slices in fixed order (deterministic), adds the bias and
-// writes z (bf16); it also puts the counter back to zero.  Every wait is bounded.
+// stage), accumulator in TMEM.  The slices of one feature tile form a thread-block cluster (2, 4 or
+// 8 CTAs).  The CTA of rank r finishes tokens [r 64/n, (r + 1) 64/n): every CTA pushes its fp32
+// partial sums for those tokens into that CTA's shared memory, and after one cluster barrier each
+// CTA adds the slices in fixed order (deterministic), adds the bias and writes z (bf16).  Nothing
+// goes through global scratch and no counter is needed.  Every mbarrier wait is bounded; a CTA
+// whose wait ran out still takes part in the cluster barrier.
 #pragma once
 #include <cuda.h>
 
@@ -23,12 +26,10 @@ namespace sparrow {
 
 struct HsrArgs {
     const __nv_bfloat16* bias;   // [d_out] or nullptr
-    float* partial;              // [n_slices][64][d_out] fp32 (token rows past M are never touched)
     __nv_bfloat16* z;            // [M][d_out]
-    unsigned* counters;          // [d_out / 128], zero between calls
     unsigned* status;
     int32_t M, d, d_out;
-    int32_t n_slices;            // K-range slices per feature tile
+    int32_t n_slices;            // K-range slices per feature tile = CTAs per cluster (1 .. 8)
     int32_t k_tiles;             // 2 d / 64
 };
 
@@ -45,13 +46,46 @@ constexpr int kWBytes = kFeat * kKTile * 2;      // one weight box: 16 KB
 constexpr int kXBytes = kTok * kKTile * 2;       // one activation box: 8 KB
 constexpr int kStageBytes = kBoxes * (kWBytes + kXBytes);
 constexpr int kStages = 6;
-constexpr int kSmemBytes = 1024 + kStages * kStageBytes + 256;
+constexpr int kRecvBytes = (kTok + 4 * 8) * kFeat * 4;   // partial sums pushed by the cluster's CTAs: [slice][feature][share + 4] fp32
+constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kRecvBytes + 256;
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar)
 {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float (&v)[8])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7])
+                 : "r"(taddr) : "memory");
+}
+
+__device__ __forceinline__ void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait_acquire() { asm volatile("barrier.cluster.wait.acquire;" ::: "memory"); }
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void st_cluster_v4(uint32_t addr, float a, float b, float c, float d)
+{
+    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+
+// eight token columns of this thread's feature row (zeros when the item has no accumulator)
+__device__ __forceinline__ void load8(bool have, uint32_t taddr, float (&v)[8])
+{
+    if (have) {
+        tmem_ld8(taddr, v);
+        tmem_wait_ld();
+    } else {
+        #pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = 0.f;
+    }
 }
 
 __global__ void __launch_bounds__(kThreadsHsr, 1)
@@ -61,11 +95,11 @@ hsr_fuse_kernel(const __grid_constant__ HsrArgs args, const __grid_constant__ CU
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     unsigned char* sm = smem_raw + ((1024u - (raw & 1023u)) & 1023u);
-    unsigned char* misc = sm + kStages * kStageBytes;
+    unsigned char* recv = sm + kStages * kStageBytes;                    // [n_slices][128][share + 4] fp32 (rows padded against bank conflicts)
+    unsigned char* misc = recv + kRecvBytes;
     const uint32_t bar0 = smem_u32(misc);                               // full[6], empty[6], done
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 128);
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(misc + 132);
-    volatile int32_t* is_last = reinterpret_cast<volatile int32_t*>(misc + 136);
     auto full = [&](int i) { return bar0 + 8u * (uint32_t)i; };
     auto empty = [&](int i) { return bar0 + 48u + 8u * (uint32_t)i; };
     const uint32_t done = bar0 + 96u;
@@ -112,6 +146,9 @@ hsr_fuse_kernel(const __grid_constant__ HsrArgs args, const __grid_constant__ CU
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
+    const int feat_local = (warp & 3) * 32 + lane;
+    // n_slices is a power of two: each CTA of the cluster finishes `share` of the 64 token columns
+    const int share = kTok / args.n_slices, lg_share = 31 - __clz(share), row_floats = share + 4;
     if (warp == 4) {
         if (lane == 0) {                                                // ---- TMA producer: refill freed stages
             #pragma unroll 1
@@ -147,64 +184,62 @@ hsr_fuse_kernel(const __grid_constant__ HsrArgs args, const __grid_constant__ CU
             if (!ok) { atomicOr(args.status, timeout_bits(kSiteMma)); *abort_flag = 1; }
         }
     } else {
-        // ---- epilogue warps: thread = one output feature (TMEM lane), 64 token columns
+        // ---- epilogue warps, part 1: thread = one output feature (TMEM lane), 64 token columns.
+        // Everything from here on runs once per CTA, i.e. from a cold instruction cache: the loops
+        // are kept rolled (8 token columns per trip) so that few distinct instructions are fetched.
         bool ok = n_kt == 0 || mbar_wait_warp(done, 0);
         tc_fence_after();
-        const int feat = f_tile * kFeat + warp * 32 + lane;
-        float acc[64];
-        if (ok && n_kt > 0) {
-            tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16), acc);
-            tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + 32, acc + 32);
-            tmem_wait_ld();
-        } else {
-            #pragma unroll
-            for (int t = 0; t < 64; ++t) acc[t] = 0.f;
-        }
         if (!ok) { atomicOr(args.status, timeout_bits(kSiteSoftmax)); *abort_flag = 1; }
-        const float b = args.bias ? __bfloat162float(args.bias[feat]) : 0.f;
-        if (args.n_slices == 1) {
-            #pragma unroll
-            for (int t = 0; t < 64; ++t)
-                if (t < args.M) args.z[(size_t)t * args.d_out + feat] = __float2bfloat16(acc[t] + b);
-        } else {
-            // partial sums as [slice][token][feature]: the 32 features of a warp are 128 contiguous bytes
-            float* mine = args.partial + (size_t)slice * kTok * args.d_out + feat;
-            #pragma unroll
-            for (int t = 0; t < 64; ++t)
-                if (t < args.M) mine[(size_t)t * args.d_out] = acc[t];
-            asm volatile("bar.sync 1, 128;" ::: "memory");             // every store of this item has been issued
-            if (tid == 0) {
-                // release (cumulative over the stores the barrier ordered before it) and acquire in one
-                unsigned old;
-                asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(args.counters + f_tile) : "memory");
-                *is_last = old == (unsigned)args.n_slices - 1u ? 1 : 0;
-                if (*is_last) args.counters[f_tile] = 0u;              // back to zero for the next call
-            }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (*is_last) {
-                // The slices in fixed order, whoever arrived last (its own slice comes from its
-                // registers: the same values it stored); all loads of a slice in flight at once.
-                // (Two slices in flight, or a sum shared among the tile's items, measured slower.)
-                float sum[64];
+        const bool have = ok && n_kt > 0;
+        if (args.n_slices == 1) {                                       // a single slice writes z itself
+            const float b = args.bias ? __bfloat162float(args.bias[f_tile * kFeat + feat_local]) : 0.f;
+            #pragma unroll 1
+            for (int c = 0; c < args.M; c += 8) {
+                float v[8];
+                load8(have, tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c, v);
                 #pragma unroll
-                for (int t = 0; t < 64; ++t) sum[t] = 0.f;
+                for (int i = 0; i < 8; ++i)
+                    if (c + i < args.M) args.z[(size_t)(c + i) * args.d_out + f_tile * kFeat + feat_local] = __float2bfloat16(v[i] + b);
+            }
+        } else {
+            // The CTA of rank r finishes tokens [r share, (r + 1) share): this slice's partial sums
+            // for them are pushed into that CTA's receive buffer, laid out [slice][feature][token in
+            // share] with padded rows.  Remote stores are not waited for.  Columns past M hold
+            // zeros (TMA fills the token rows past M with zeros), so whole chunks are pushed.
+            const uint32_t row0 = smem_u32(recv) + (uint32_t)((slice * kFeat + feat_local) * row_floats) * 4u;
+            #pragma unroll 1
+            for (int c = 0; c < args.M; c += 8) {
+                float v[8];
+                load8(have, tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c, v);
+                const uint32_t dst = map_to_rank(row0 + (uint32_t)(c & (share - 1)) * 4u, (uint32_t)(c >> lg_share));
+                st_cluster_v4(dst, v[0], v[1], v[2], v[3]);
+                st_cluster_v4(dst + 16u, v[4], v[5], v[6], v[7]);
+            }
+        }
+    }
+    if (args.n_slices > 1) {
+        // one cluster barrier: every slice's pushes have landed; after it nobody touches a peer
+        cluster_arrive_release();
+        cluster_wait_acquire();
+        if (warp < 4) {
+            // part 2: the slices in fixed order (results do not depend on timing), bias, bf16 z
+            const float b = args.bias ? __bfloat162float(args.bias[f_tile * kFeat + feat_local]) : 0.f;
+            const float* mine = reinterpret_cast<const float*>(recv) + feat_local * row_floats;
+            const int t0 = slice * share;
+            const int n_mine = min(share, args.M - t0);                 // may be <= 0: nothing to finish
+            #pragma unroll 1
+            for (int j0 = 0; j0 < n_mine; j0 += 4) {
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
                 #pragma unroll 1
                 for (int s2 = 0; s2 < args.n_slices; ++s2) {
-                    if (s2 == slice) {
-                        #pragma unroll
-                        for (int t = 0; t < 64; ++t) sum[t] += acc[t];
-                    } else {
-                        const float* src = args.partial + (size_t)s2 * kTok * args.d_out + feat;
-                        float v[64];
-                        #pragma unroll
-                        for (int t = 0; t < 64; ++t) v[t] = t < args.M ? __ldcg(src + (size_t)t * args.d_out) : 0.f;
-                        #pragma unroll
-                        for (int t = 0; t < 64; ++t) sum[t] += v[t];
-                    }
+                    const float4 p = *reinterpret_cast<const float4*>(mine + s2 * kFeat * row_floats + j0);
+                    acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
                 }
-                #pragma unroll
-                for (int t = 0; t < 64; ++t)
-                    if (t < args.M) args.z[(size_t)t * args.d_out + feat] = __float2bfloat16(sum[t] + b);
+                __nv_bfloat16* zp = args.z + (size_t)(t0 + j0) * args.d_out + f_tile * kFeat + feat_local;
+                zp[0] = __float2bfloat16(acc.x + b);
+                if (j0 + 1 < n_mine) zp[args.d_out] = __float2bfloat16(acc.y + b);
+                if (j0 + 2 < n_mine) zp[2 * (size_t)args.d_out] = __float2bfloat16(acc.z + b);
+                if (j0 + 3 < n_mine) zp[3 * (size_t)args.d_out] = __float2bfloat16(acc.w + b);
             }
         }
     }

@@ -31,10 +31,8 @@ def _ctx():
 def _run(ctx, e, h, w, b):
     M, d = e.shape
     d_out = w.shape[0]
-    n = B.sparrow_hsr_scratch_bytes(ctx, d, d_out)
-    scratch = torch.empty(max(n, 16), dtype=torch.uint8, device=DEV)
     z = torch.full((M, d_out), float("nan"), dtype=torch.bfloat16, device=DEV)
-    B.sparrow_hsr_fuse(ctx, e, h, w, b, z, scratch)
+    B.sparrow_hsr_fuse(ctx, e, h, w, b, z)
     torch.cuda.synchronize()
     assert ctx.last_device_status() == 0
     return z
@@ -51,11 +49,13 @@ def _check(z, e, h, w, b):
 
 @pytest.mark.parametrize("M,d,d_out,bias", [
     (1, 64, 128, True),            # smallest shape: one feature tile, two K tiles
-    (8, 3584, 3584, True),         # one drafting step of a Qwen2-7B-shaped model (28 feature tiles x 5 K slices)
+    (8, 3584, 3584, True),         # one drafting step of a Qwen2-7B-shaped model (28 feature tiles x clusters of 4 K slices)
     (48, 3584, 3584, False),       # a 48-node tree, no bias
     (64, 3584, 3584, True),
-    (30, 1536, 1536, True),        # a smaller model: 12 feature tiles, 12 slices
-    (5, 128, 24576, True),         # more feature tiles than SMs: one slice each, no partial sums
+    (30, 1536, 1536, True),        # a smaller model: 12 feature tiles, clusters of 8
+    (5, 128, 24576, True),         # more feature tiles than SMs: one slice each, no cluster
+    (33, 512, 8192, False),        # 64 feature tiles: clusters of 2, 32 tokens each (the second CTA finishes one)
+    (9, 1024, 3584, True),         # clusters of 4 of which only the first has tokens to finish
     (17, 4096, 512, True),         # few feature tiles, long K slices
 ])
 def test_hsr_fuse_matches_the_oracle(M, d, d_out, bias):
@@ -64,7 +64,7 @@ def test_hsr_fuse_matches_the_oracle(M, d, d_out, bias):
     _check(_run(ctx, e, h, w, b), e, h, w, b)
 
 
-def test_hsr_fuse_repeats_bit_for_bit_and_keeps_its_counters_clean():
+def test_hsr_fuse_repeats_bit_for_bit():
     e, h, w, b = _case(7100, 25, 3584, 3584)
     ctx = _ctx()
     first = _run(ctx, e, h, w, b)
@@ -94,11 +94,7 @@ def test_hsr_fuse_argument_errors():
     n0 = ctx.launch_count()
     L = B.lib()
     for M, d, d_out, status in ((0, 128, 256, 2), (65, 128, 256, 2), (4, 100, 256, 2), (4, 128, 200, 2)):
-        assert L.sparrow_hsr_fuse(ctx.handle, e.data_ptr(), h.data_ptr(), w.data_ptr(), None, M, d, d_out, None, 0,
-                                  z.data_ptr(), None) == status
-    assert L.sparrow_hsr_fuse(ctx.handle, None, h.data_ptr(), w.data_ptr(), None, 4, 128, 256, None, 0, z.data_ptr(), None) == 1
-    e2, h2, w2, b2 = _case(7301, 4, 3584, 3584)
-    z2 = torch.empty((4, 3584), dtype=torch.bfloat16, device=DEV)
-    assert L.sparrow_hsr_fuse(ctx.handle, e2.data_ptr(), h2.data_ptr(), w2.data_ptr(), None, 4, 3584, 3584, None, 0,
-                              z2.data_ptr(), None) == 5          # split-K partials need scratch
+        assert L.sparrow_hsr_fuse(ctx.handle, e.data_ptr(), h.data_ptr(), w.data_ptr(), None, M, d, d_out, z.data_ptr(), None) == status
+    assert L.sparrow_hsr_fuse(ctx.handle, None, h.data_ptr(), w.data_ptr(), None, 4, 128, 256, z.data_ptr(), None) == 1
+    assert L.sparrow_hsr_fuse(ctx.handle, e.data_ptr() + 2, h.data_ptr(), w.data_ptr(), None, 4, 128, 256, z.data_ptr(), None) == 2
     assert ctx.launch_count() == n0
