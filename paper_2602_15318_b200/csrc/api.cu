@@ -1413,4 +1413,27 @@ uint32_t sparrow_debug_status_word(const sparrow_ctx* c) { return c ? c->last_st
 
 int64_t sparrow_launch_count(const sparrow_ctx* c) { return c ? (int64_t)c->launches.load() : 0; }
 
+#ifdef SPARROW_TIMELINE
+// Timeline build only (see common.cuh): read / clear the stamp table, and a one-thread kernel that
+// stamps the stream position (so that a call's launch gap can be seen).
+namespace {
+__global__ void timeline_mark_kernel(unsigned long long* dst) { *dst = sparrow::global_timer_ns(); }
+}
+int sparrow_timeline_read(void* host_dst)
+{
+    return (int)cudaMemcpyFromSymbol(host_dst, sparrow::g_timeline, sizeof(sparrow::g_timeline));
+}
+int sparrow_timeline_clear()
+{
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, sparrow::g_timeline) != cudaSuccess) return 1;
+    return (int)cudaMemset(p, 0, sizeof(sparrow::g_timeline));
+}
+int sparrow_timeline_mark(void* dev_dst, void* stream)
+{
+    timeline_mark_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<unsigned long long*>(dev_dst));
+    return (int)cudaGetLastError();
+}
+#endif
+
 }  // extern "C"

@@ -5,6 +5,29 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+// Timeline build (-DSPARROW_TIMELINE, made by `python -m paper_2602_15318_b200.timeline`; never
+// the shipped library): SPARROW_STAMP(slot) records %globaltimer for (CTA, slot), and three extra
+// exported calls read the table back.  In the ordinary build the macro expands to nothing.
+#ifdef SPARROW_TIMELINE
+namespace sparrow {
+constexpr int kTimelineCtas = 256, kTimelineSlots = 16;
+__device__ unsigned long long g_timeline[kTimelineCtas * kTimelineSlots];
+__device__ __forceinline__ unsigned long long global_timer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+}  // namespace sparrow
+#define SPARROW_STAMP(slot)                                                                        \
+    do {                                                                                           \
+        if (blockIdx.x < ::sparrow::kTimelineCtas)                                                 \
+            ::sparrow::g_timeline[blockIdx.x * ::sparrow::kTimelineSlots + (slot)] = ::sparrow::global_timer_ns(); \
+    } while (0)
+#else
+#define SPARROW_STAMP(slot) ((void)0)
+#endif
+
 namespace sparrow {
 
 constexpr int kD = 128;           // head_dim

@@ -105,6 +105,7 @@ hsr_fuse_kernel(const __grid_constant__ HsrArgs args, const __grid_constant__ CU
     const uint32_t done = bar0 + 96u;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) SPARROW_STAMP(0);                                     // entry
     const int f_tile = blockIdx.x / args.n_slices, slice = blockIdx.x - f_tile * args.n_slices;
     // K tiles of this slice: as even as whole tiles allow
     const int kt_begin = (int)((long long)args.k_tiles * slice / args.n_slices);
@@ -145,6 +146,7 @@ hsr_fuse_kernel(const __grid_constant__ HsrArgs args, const __grid_constant__ CU
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    if (tid == 0) SPARROW_STAMP(1);                                     // set-up done
 
     const int feat_local = (warp & 3) * 32 + lane;
     // n_slices is a power of two: each CTA of the cluster finishes `share` of the 64 token columns
@@ -168,6 +170,7 @@ hsr_fuse_kernel(const __grid_constant__ HsrArgs args, const __grid_constant__ CU
                 const int st = i % kStages;
                 if (!mbar_wait(full(st), (i / kStages) & 1)) { ok = false; break; }
                 tc_fence_after();
+                if (i == 0) SPARROW_STAMP(2);                           // first tile landed
                 const int boxes = min(kBoxes, n_kt - i * kBoxes);
                 const uint32_t base = smem_u32(sm + st * kStageBytes);
                 for (int bx = 0; bx < boxes; ++bx) {
@@ -181,6 +184,7 @@ hsr_fuse_kernel(const __grid_constant__ HsrArgs args, const __grid_constant__ CU
                 tc_commit(empty(st));
             }
             tc_commit(done);
+            SPARROW_STAMP(3);                                           // last MMA issued
             if (!ok) { atomicOr(args.status, timeout_bits(kSiteMma)); *abort_flag = 1; }
         }
     } else {
@@ -191,6 +195,7 @@ hsr_fuse_kernel(const __grid_constant__ HsrArgs args, const __grid_constant__ CU
         tc_fence_after();
         if (!ok) { atomicOr(args.status, timeout_bits(kSiteSoftmax)); *abort_flag = 1; }
         const bool have = ok && n_kt > 0;
+        if (tid == 0) SPARROW_STAMP(4);                                 // accumulator complete
         if (args.n_slices == 1) {                                       // a single slice writes z itself
             const float b = args.bias ? __bfloat162float(args.bias[f_tile * kFeat + feat_local]) : 0.f;
             #pragma unroll 1
@@ -219,8 +224,10 @@ hsr_fuse_kernel(const __grid_constant__ HsrArgs args, const __grid_constant__ CU
     }
     if (args.n_slices > 1) {
         // one cluster barrier: every slice's pushes have landed; after it nobody touches a peer
+        if (tid == 0) SPARROW_STAMP(5);                                 // partial sums pushed
         cluster_arrive_release();
         cluster_wait_acquire();
+        if (tid == 0) SPARROW_STAMP(6);                                 // cluster barrier passed
         if (warp < 4) {
             // part 2: the slices in fixed order (results do not depend on timing), bias, bf16 z
             const float b = args.bias ? __bfloat162float(args.bias[f_tile * kFeat + feat_local]) : 0.f;
@@ -243,6 +250,7 @@ hsr_fuse_kernel(const __grid_constant__ HsrArgs args, const __grid_constant__ CU
             }
         }
     }
+    if (tid == 0) SPARROW_STAMP(7);                                     // z written, leaving
     tc_fence_before();
     __syncthreads();
     if (*abort_flag) {

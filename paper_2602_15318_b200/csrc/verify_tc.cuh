@@ -370,6 +370,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
     float* xch = reinterpret_cast<float*>(misc + 1024);                               // [2][128] maxima / sums exchange
 
     Bars B;
+    if (threadIdx.x == 0) SPARROW_STAMP(0);                             // entry
     B.base = smem_u32(bar_mem);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -456,6 +457,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    if (threadIdx.x == 0) SPARROW_STAMP(1);                             // set-up done
     if (sync.enabled) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == kProducerWarp) {
@@ -481,6 +483,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
             const uint64_t k_desc0 = smem_desc(smem_u32(kv_sm), 16, 1024);
             const uint64_t v_desc0 = smem_desc(smem_u32(kv_sm) + 2 * kSubTileBytes, kSubTileBytes, 1024);
             bool ok = mbar_wait(B.q_full(), 0);
+            SPARROW_STAMP(2);                                           // Q landed
             if constexpr (NB == 2) {
                 // Two row blocks, each with its own softmax warpgroup.  Job n = (key tile j = n / 2,
                 // block b = n % 2).  Block b owns TMEM columns [128 b, 128 b + 128) for its scores,
@@ -495,6 +498,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                     if (b == 0) {                                             // first use of this K tile
                         if (!mbar_wait(B.k_full(st), (j / NS) & 1)) return false;
                         tc_fence_after();
+                        if (j == 0) SPARROW_STAMP(3);                   // first K tile landed
                     }
                     const uint64_t qd = q_desc0 + (uint64_t)((b * kQBlockBytes) >> 4);
                     const uint64_t kd = k_desc0 + (uint64_t)((st * kStageBytes) >> 4);
@@ -532,6 +536,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                 if (blk == 0) {                                           // first use of this K tile
                     if (!mbar_wait(B.k_full(st), (j / NS) & 1)) return false;
                     tc_fence_after();
+                    if (j == 0) SPARROW_STAMP(3);                       // first K tile landed
                 }
                 const uint64_t qd = q_desc0 + (uint64_t)((blk * kQBlockBytes) >> 4);
                 const uint64_t kd = k_desc0 + (uint64_t)((st * kStageBytes) >> 4);
@@ -561,6 +566,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                 if (n + NSB < n_jobs) ok = issue_qk(n + NSB);             // its S block was job n's
             }
             }
+            SPARROW_STAMP(4);                                           // last product issued
             if (!ok) { atomicOr(args.status, timeout_bits(kSiteMma)); *abort_flag = 1; }
         }
     } else if (warp == kGateWarp) {
@@ -828,6 +834,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
 
         }
         // ---- epilogue: normalised partial output + natural-log LSE -------------------------------
+        if (tid == 0) SPARROW_STAMP(5);                                 // softmax loop left
         const bool direct = plan.seq[it.b].n_splits == 1;                  // the only piece: write the final result
         if (tid == 0) {
             // Global writes start below.  In overlapped mode a lane of the MMA warp has been waiting,
@@ -850,6 +857,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
             const int last_product = n_tiles - 1;
             if (ok) ok = mbar_wait_warp(B.o_done(blk, last_product), (last_product >> 2) & 1);    // the last product is in
             tc_fence_after();
+            if (tid == 0 && blk == 0) SPARROW_STAMP(6);                // last product complete
             float inv, lse_val;
             if constexpr (NB == 2) {
                 inv = xch[blk * 128 + row_local];
@@ -935,6 +943,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
             // the pieces are read by the finishers' bulk copies (async proxy): order this thread's stores ahead of them
             if (!direct) fence_proxy_async_global();
             softmax_bar_sync();                                        // every global store of this CTA has been issued
+            if (tid == 0) SPARROW_STAMP(7);                            // partial rows stored
             if (tid == 0) {
                 if (!direct) publish_counter(arrive_word);
                 if (merges) {
@@ -947,8 +956,10 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                         if (!prev_done) prev_done = (int32_t)(ld_acquire(sync.fin_done + (sync.parity ^ 1)) - sync.fin_wait_other) >= 0;
                         if (!(have_all && prev_done)) __nanosleep(i < 256 ? 20 : 200);
                     }
+                    SPARROW_STAMP(8);                                   // all arrivals seen
                     if (!have_all) atomicOr(args.status, timeout_bits(kSiteArrivals));
                     else if (!prev_done) atomicOr(args.status, timeout_bits(kSiteFinOther));
+                    SPARROW_STAMP(9);                                   // previous call's finishers seen
                     *fin_go = (have_all && prev_done) ? 1 : 0;
                 }
             }
@@ -1007,7 +1018,9 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                                                       (uint32_t)(r0 + n_here - split) * kRowBytes, B.fin());
                                     }
                                 }
+                                if (tid == 0) SPARROW_STAMP(12);        // bulk copies issued
                                 fin_ok = fin_ok && mbar_wait_warp(B.fin(), phase);
+                                if (tid == 0) SPARROW_STAMP(15);        // bulk copies landed
                                 const int idx = r0 + row_i;                            // row of the unit's list: token idx / 7, head idx % 7
                                 const bool active = fin_ok && row_i < n_here;
                                 const uint32_t pstride = (uint32_t)n_here * kRowBytes;     // bytes between pieces in the ring
@@ -1033,6 +1046,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                                         m_run = m_new;
                                     }
                                 }
+                                if (tid == 0) SPARROW_STAMP(13);        // pieces folded
                                 if (G > 1) {                                           // (G is the same in every thread)
                                     softmax_bar_sync();                                // the pass before has been read
                                     #pragma unroll
@@ -1059,6 +1073,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                                         m_run = m_all;
                                     }
                                 }
+                                if (tid == 0) SPARROW_STAMP(14);        // groups reduced
                                 if (active && grp_p == 0) {
                                     const int t = tok0 + idx / qg;
                                     const int h = kvh * qg + idx % qg;
@@ -1074,6 +1089,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
                     }
                     if (!fin_ok) atomicOr(args.status, timeout_bits(kSiteFinCopies));
                 }
+                if (tid == 0) SPARROW_STAMP(10);                        // merged rows written
                 softmax_bar_sync();
             }
             if (tid == 0) {
@@ -1093,6 +1109,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
         for (int i = 0; i < 2000; ++i) __nanosleep(1000);
         __syncthreads();
     }
+    if (threadIdx.x == 0) SPARROW_STAMP(11);                            // leaving
     if (warp == kMmaWarp) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
