@@ -28,6 +28,17 @@ def test_library_exports_every_declared_symbol():
         assert hasattr(L, name), name
 
 
+def test_timeline_build_compiles_and_exports_its_calls():
+    """The stamped variant of the library (-DSPARROW_TIMELINE) still builds and carries the three
+    extra calls the timeline tool uses, beside everything the header declares."""
+    import ctypes
+    from paper_2602_15318_b200 import timeline
+    L = ctypes.CDLL(timeline.build_timeline_library())
+    for name in list(B.EXPORTS) + ["sparrow_timeline_read", "sparrow_timeline_clear", "sparrow_timeline_mark"]:
+        assert hasattr(L, name), name
+    assert not hasattr(B.lib(), "sparrow_timeline_read")         # the shipped library has no stamps
+
+
 def test_ancestor_masks_match_oracle_all_small_trees():
     for T in range(1, 7):
         for par in itertools.product(*[range(-1, i) for i in range(T)]):
