@@ -374,3 +374,17 @@ def test_plan_log_line(monkeypatch, capfd):
     check(out, lse, *oracle_verify(case))
     err = capfd.readouterr().err
     assert "[sparrow] verify call" in err and "2 row block(s)" in err and "keys [0, 3020)" in err
+
+
+def test_timeline_tool_runs_and_sees_every_cta():
+    """The stamped build runs the same kernels: a short C1 timeline reports one row per phase and
+    the CTA count of the latency policy's plan."""
+    import subprocess, sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-m", "paper_2602_15318_b200.timeline", "--config", "C1", "--calls", "8"],
+                       cwd=root, capture_output=True, text=True, timeout=900)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = r.stdout.strip().splitlines()
+    assert "CTAs" in lines[0] and int(lines[0].split(":")[1].split("CTAs")[0]) > 1
+    for phase in ("kernel entered", "partial rows stored", "finisher: merged rows written", "leaving"):
+        assert any(l.startswith(phase) for l in lines), phase

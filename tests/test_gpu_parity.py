@@ -379,6 +379,28 @@ def test_verify_step_host_pinned_buffers_twice():
             assert torch.equal(case.v[b, :, n:n + T, :].cpu(), bufs["v"][b])
 
 
+def test_verify_step_host_pinned_ragged_batch_tree():
+    """The page-locked route on a ragged batch of 8 with a 32-node tree (two row blocks per tile,
+    results stored straight into host memory by the finishers of every sequence)."""
+    lens = [1900, 37, 1024, 0, 777, 1500, 129, 640]
+    case = W.make_verify_case(95, lens, 32, "random", DEV, capacity=2048)
+    ref_out, ref_lse = oracle_verify(case)
+    ctx = B.Context.for_cache(case.k, W.SCALE)
+    T, nb = case.T, len(lens)
+    q_h = case.q.cpu().pin_memory()
+    k_new = torch.stack([case.k[b, :, n:n + T, :] for b, n in enumerate(case.kv_len)]).cpu().pin_memory()
+    v_new = torch.stack([case.v[b, :, n:n + T, :] for b, n in enumerate(case.kv_len)]).cpu().pin_memory()
+    par_h = case.parents.cpu().pin_memory()
+    for b, n in enumerate(case.kv_len):
+        case.k[b, :, n:n + T, :] = float("nan")
+        case.v[b, :, n:n + T, :] = float("nan")
+    out_h = torch.full(q_h.shape, float("nan"), dtype=q_h.dtype).pin_memory()
+    lse_h = torch.full((nb, W.HQ, T), float("nan"), dtype=torch.float32).pin_memory()
+    B.sparrow_verify_step_host(ctx, q_h, k_new, v_new, case.k, case.v, case.kv_len, par_h, T, out_h, lse_h)
+    assert ctx.last_device_status() == 0
+    check(out_h, lse_h, ref_out, ref_lse)
+
+
 def test_argument_errors_launch_nothing():
     case = W.make_verify_case(92, [100], 4, "chain", DEV)
     ctx = B.Context.for_cache(case.k, W.SCALE)
