@@ -338,6 +338,7 @@ SyncArgs next_sync(const sparrow_ctx* c, const SplitPlan& p, bool overlaps, bool
     sy.n_fin = n_arrive == 0 ? 0 : ((all_finish || p.n_items < kFinisherCtas) ? p.n_items : kFinisherCtas);
     sy.fin_wait_same = c->fin_total[parity];
     sy.fin_wait_other = after_previous ? c->fin_total[parity ^ 1] : c->fin_before_last[parity ^ 1];
+    sy.call = c->seq;
     return sy;
 }
 

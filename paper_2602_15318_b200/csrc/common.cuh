@@ -6,12 +6,13 @@
 #include <stdint.h>
 
 // Timeline build (-DSPARROW_TIMELINE, made by `python -m paper_2602_15318_b200.timeline`; never
-// the shipped library): SPARROW_STAMP(slot) records %globaltimer for (CTA, slot), and three extra
-// exported calls read the table back.  In the ordinary build the macro expands to nothing.
+// the shipped library): SPARROW_STAMP(slot) records %globaltimer for (call, CTA, slot), and three
+// extra exported calls read the table back.  A kernel names the call it belongs to once with
+// SPARROW_TIMELINE_CALL(index) (kept modulo 32).  In the ordinary build both macros expand to nothing.
 #ifdef SPARROW_TIMELINE
 namespace sparrow {
-constexpr int kTimelineCtas = 256, kTimelineSlots = 16;
-__device__ unsigned long long g_timeline[kTimelineCtas * kTimelineSlots];
+constexpr int kTimelineCalls = 32, kTimelineCtas = 256, kTimelineSlots = 16;
+__device__ unsigned long long g_timeline[kTimelineCalls * kTimelineCtas * kTimelineSlots];
 __device__ __forceinline__ unsigned long long global_timer_ns()
 {
     unsigned long long t;
@@ -19,12 +20,15 @@ __device__ __forceinline__ unsigned long long global_timer_ns()
     return t;
 }
 }  // namespace sparrow
+#define SPARROW_TIMELINE_CALL(index) const unsigned sparrow_tl_call = (unsigned)(index) % ::sparrow::kTimelineCalls
 #define SPARROW_STAMP(slot)                                                                        \
     do {                                                                                           \
         if (blockIdx.x < ::sparrow::kTimelineCtas)                                                 \
-            ::sparrow::g_timeline[blockIdx.x * ::sparrow::kTimelineSlots + (slot)] = ::sparrow::global_timer_ns(); \
+            ::sparrow::g_timeline[((size_t)sparrow_tl_call * ::sparrow::kTimelineCtas + blockIdx.x) * ::sparrow::kTimelineSlots + (slot)] = \
+                ::sparrow::global_timer_ns();                                                      \
     } while (0)
 #else
+#define SPARROW_TIMELINE_CALL(index) ((void)0)
 #define SPARROW_STAMP(slot) ((void)0)
 #endif
 
@@ -123,6 +127,7 @@ struct SyncArgs {
     int32_t n_fin;           // finisher CTAs of this call (0 when no unit has several pieces)
     uint32_t fin_wait_same;
     uint32_t fin_wait_other;
+    uint32_t call;           // running number of the context's fused calls (the timeline build files its stamps under it)
 };
 
 __device__ __forceinline__ unsigned ld_acquire(const unsigned* addr)

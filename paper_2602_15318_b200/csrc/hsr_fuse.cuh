@@ -105,6 +105,7 @@ hsr_fuse_kernel(const __grid_constant__ HsrArgs args, const __grid_constant__ CU
     const uint32_t done = bar0 + 96u;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    SPARROW_TIMELINE_CALL(0);
     if (tid == 0) SPARROW_STAMP(0);                                     // entry
     const int f_tile = blockIdx.x / args.n_slices, slice = blockIdx.x - f_tile * args.n_slices;
     // K tiles of this slice: as even as whole tiles allow

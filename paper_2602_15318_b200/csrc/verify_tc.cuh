@@ -370,6 +370,7 @@ verify_tc_kernel(const __grid_constant__ TcArgs args, const __grid_constant__ Sy
     float* xch = reinterpret_cast<float*>(misc + 1024);                               // [2][128] maxima / sums exchange
 
     Bars B;
+    SPARROW_TIMELINE_CALL(sync.call);
     if (threadIdx.x == 0) SPARROW_STAMP(0);                             // entry
     B.base = smem_u32(bar_mem);
 

@@ -4,7 +4,12 @@ first, the median and the last CTA reached it (%globaltimer, microseconds after 
 position just before the call).
 
     python -m paper_2602_15318_b200.timeline --config C2 --policy latency
+    python -m paper_2602_15318_b200.timeline --config C2 --policy throughput --burst 20
     python -m paper_2602_15318_b200.timeline --hsr
+
+With --burst N the N calls are enqueued back to back from C (one sparrow_verify_attn_batch, as the
+bench's timed region does) and one line per call says when its CTAs started, left their main loop,
+stored their partial rows and when its merged rows were written.
 
 Stamping costs a few stores per CTA; the figures are for reading the shape of a call, the bench
 times the shipped library.
@@ -22,7 +27,7 @@ from . import build as _build
 from . import workloads as W
 
 LIB = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libsparrow_attn_timeline.so")
-CTAS, SLOTS = 256, 16
+CALLS, CTAS, SLOTS = 32, 256, 16
 
 VERIFY_SLOTS = ["kernel entered", "set-up done (barriers, TMEM)", "Q landed", "first K tile landed",
                 "last product issued", "softmax loop left", "last product complete", "partial rows stored",
@@ -62,6 +67,7 @@ def main():
     ap.add_argument("--policy", choices=["latency", "balanced", "throughput"], default="latency")
     ap.add_argument("--hsr", action="store_true", help="the Eq. 1 projection (48 tokens, d = 3584) instead of attention")
     ap.add_argument("--calls", type=int, default=40)
+    ap.add_argument("--burst", type=int, default=0, help="enqueue this many calls (at most 32) back to back and print one line per call")
     args = ap.parse_args()
 
     B.LIB_PATH = build_timeline_library()
@@ -95,6 +101,51 @@ def main():
             B.sparrow_verify_attn(ctx, c.q, c.k, c.v, c.kv_len, c.parents, c.T, outs[i % n_rot], lses[i % n_rot])
         names, what = VERIFY_SLOTS, f"sparrow_verify_attn, {args.config}, {args.policy} policy"
 
+    def read_table():
+        buf = np.zeros(CALLS * CTAS * SLOTS, dtype=np.uint64)
+        if L.sparrow_timeline_read(buf.ctypes.data) != 0:
+            raise SystemExit("reading the stamp table failed")
+        return buf.reshape(CALLS, CTAS, SLOTS).astype(np.int64)
+
+    if args.burst:
+        if args.hsr or not 1 <= args.burst <= CALLS:
+            raise SystemExit("--burst: 1 .. 32 attention calls")
+        n = args.burst
+        batch = B.VerifyBatch([(cases[i % n_rot].q, cases[i % n_rot].k, cases[i % n_rot].v, cases[i % n_rot].kv_len,
+                                cases[i % n_rot].parents, cases[i % n_rot].T, outs[i % n_rot], lses[i % n_rot]) for i in range(n)])
+        runs = []
+        for rep in range(8):
+            torch.cuda.synchronize()
+            L.sparrow_timeline_clear()
+            torch.cuda._sleep(400000)
+            L.sparrow_timeline_mark(marks.data_ptr(), stream)
+            B.sparrow_verify_attn_batch(ctx, batch)
+            L.sparrow_timeline_mark(marks.data_ptr() + 8, stream)
+            torch.cuda.synchronize()
+            if ctx.last_device_status() != 0:
+                raise SystemExit("device status set")
+            t = read_table()
+            m0, m1 = int(marks[0]), int(marks[1])
+            used = [c for c in range(CALLS) if (t[c, :, 0] > 0).any()]
+            used.sort(key=lambda c: t[c, :, 0][t[c, :, 0] > 0].min())
+            per_call = []
+            for c in used:
+                tc = t[c][t[c, :, 0] > 0]
+                rel = np.where(tc > 0, tc - m0, -1)
+                col = lambda k, f: (f(rel[:, k][rel[:, k] >= 0]) / 1e3 if (rel[:, k] >= 0).any() else float("nan"))
+                per_call.append((rel.shape[0], col(0, np.min), col(0, np.max), col(5, np.min), col(5, np.max), col(7, np.max),
+                                 col(8, np.min), col(10, np.max), col(11, np.max)))
+            runs.append(((m1 - m0) / 1e3, per_call))
+        runs = runs[2:]
+        print(f"{what}: burst of {n} calls; mark before -> mark after: {np.median([r[0] for r in runs]):.1f} us "
+              f"({np.median([r[0] for r in runs]) / n:.2f} us per call); medians over {len(runs)} bursts, us after the first mark")
+        print(f"{'call':>4s} {'CTAs':>5s} {'first in':>9s} {'last in':>9s} {'loop left: first':>17s} {'last':>8s} {'stored':>8s} "
+              f"{'arrivals seen':>14s} {'merged':>8s} {'last out':>9s}")
+        for i in range(len(runs[0][1])):
+            vals = np.median(np.array([r[1][i] for r in runs if len(r[1]) > i], dtype=np.float64), axis=0)
+            print(f"{i:4d} {int(vals[0]):5d} {vals[1]:9.1f} {vals[2]:9.1f} {vals[3]:17.1f} {vals[4]:8.1f} {vals[5]:8.1f} {vals[6]:14.1f} {vals[7]:8.1f} {vals[8]:9.1f}")
+        return
+
     rows, spans = [], []
     for i in range(args.calls):
         torch.cuda.synchronize()
@@ -106,10 +157,7 @@ def main():
         torch.cuda.synchronize()
         if ctx.last_device_status() != 0:
             raise SystemExit("device status set")
-        buf = np.zeros(CTAS * SLOTS, dtype=np.uint64)
-        if L.sparrow_timeline_read(buf.ctypes.data) != 0:
-            raise SystemExit("reading the stamp table failed")
-        t = buf.reshape(CTAS, SLOTS).astype(np.int64)
+        t = read_table().reshape(CALLS * CTAS, SLOTS)
         t = t[t[:, 0] > 0]
         m0, m1 = int(marks[0]), int(marks[1])
         rows.append(np.where(t > 0, t - m0, -1))
@@ -117,7 +165,6 @@ def main():
     rows, spans = rows[args.calls // 4:], spans[args.calls // 4:]
     print(f"{what}: {rows[0].shape[0]} CTAs; mark before the call -> mark after it: {np.median(spans) / 1e3:.2f} us")
     _table(rows, names)
-
 
 if __name__ == "__main__":
     main()
